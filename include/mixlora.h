@@ -1,0 +1,157 @@
+/*
+ * mixlora.h - C ABI of the MixLoRA feed-forward block for NVIDIA B200 (sm_100a).
+ *
+ * The block is the one defined by Eq. 6-9 and Algorithm 1 of "MixLoRA: Enhancing Large
+ * Language Models Fine-Tuning with LoRA-based Mixture of Experts" (arXiv 2404.15159):
+ * a frozen SwiGLU FFN (W1 = gate, W3 = up, W2 = down; Section 3.3) shared by N LoRA
+ * experts (Eq. 1: W' = W + B A on each of the three projections) under a top-k softmax
+ * router (Eq. 7) with the load-balance auxiliary loss of Eq. 8-9.
+ *
+ * Conventions
+ *   - Every tensor pointer is a DEVICE pointer unless marked "host".  All tensors are
+ *     dense, row-major, 16-byte aligned and owned by the caller, including the workspace.
+ *     The library allocates no device memory in these calls and keeps no state between
+ *     calls other than what it writes into the caller's workspace.
+ *   - Weights are stored [out, in] as in Eq. 1 (W in R^{d1 x d2}).
+ *   - T tokens, d = d_model, f = d_ff, N experts, k = top_k, r = rank, s = lora_alpha / r.
+ *     A slot is one (token, selected expert) pair; slot id = t * k + j, j = 0 for the
+ *     expert with the largest logit.
+ *   - dtype 0: x, dy, y, d_x, frozen weights and LoRA matrices are bfloat16, arithmetic
+ *     accumulates in fp32.  dtype 1: all of them are fp32 (check mode).  Router weight,
+ *     router bias, probabilities, gates and every gradient output are fp32 in both modes.
+ *   - Work is enqueued on `stream` (a cudaStream_t passed as void*); calls return after
+ *     enqueueing and never synchronise the device (mixlora_device_status excepted).
+ *   - Errors: every call validates its arguments on the host and returns a status; nothing
+ *     aborts or throws.  A failed validation enqueues nothing.
+ */
+#ifndef MIXLORA_H_
+#define MIXLORA_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  MIXLORA_OK = 0,
+  MIXLORA_ERR_INVALID_ARG = 1,   /* NULL or misaligned pointer, inconsistent sizes            */
+  MIXLORA_ERR_UNSUPPORTED = 2,   /* a size outside the compiled limits (see mixlora_limits)  */
+  MIXLORA_ERR_WORKSPACE = 3,     /* workspace NULL, misaligned or smaller than required      */
+  MIXLORA_ERR_CUDA = 4,          /* a CUDA runtime or driver call failed                     */
+  MIXLORA_ERR_DEVICE_TIMEOUT = 5 /* a bounded wait inside a kernel ran out (device status)   */
+} mixlora_status_t;
+
+#define MIXLORA_DTYPE_BF16 0
+#define MIXLORA_DTYPE_FP32 1
+
+#define MIXLORA_MAX_EXPERTS 32   /* N <= 32                                              */
+#define MIXLORA_MAX_TOP_K 8      /* k <= min(N, 8)                                       */
+#define MIXLORA_MAX_RANK 128     /* r <= 128; r % 8 == 0 in bf16 mode, r % 4 == 0 in fp32 */
+
+/* Problem shape.  Plain data; set struct_size = sizeof(mixlora_shape_t). */
+typedef struct {
+  uint32_t struct_size;
+  int32_t tokens;       /* T >= 0 (T = 0 is a valid no-op); T * k <= 4,000,000                */
+  int32_t d_model;      /* d, multiple of 8                                                  */
+  int32_t d_ff;         /* f, multiple of 8                                                  */
+  int32_t n_experts;    /* N                                                                 */
+  int32_t top_k;        /* k, 1 <= k <= N                                                    */
+  int32_t rank;         /* r                                                                 */
+  float lora_alpha;     /* scale s = lora_alpha / rank (alpha of Table 3)                    */
+  int32_t dtype;        /* MIXLORA_DTYPE_BF16 or MIXLORA_DTYPE_FP32                          */
+  int32_t renormalize;  /* 1: gates divided by their top-k sum (Norm(.) of Algorithm 1); 0: Eq. 7 as printed */
+  int32_t aux_f_mode;   /* 0: F_i counts the arg-max expert (Eq. 9); 1: all k selections / (T k)            */
+} mixlora_shape_t;
+
+/* Inputs of the block.  `void*` tensors have the element type selected by shape.dtype. */
+typedef struct {
+  const void *x;               /* [T, d]  hidden states (after the layer norm of Eq. 5)      */
+  const void *w_gate;          /* [f, d]  W1, frozen                                         */
+  const void *w_up;            /* [f, d]  W3, frozen                                         */
+  const void *w_down;          /* [d, f]  W2, frozen                                         */
+  const float *w_router;       /* [N, d]  W_r of Eq. 7, fp32                                 */
+  const float *router_bias;    /* [N] fp32 added to the logits, or NULL                      */
+  const void *a_gate, *b_gate; /* [N, r, d], [N, f, r]                                       */
+  const void *a_up, *b_up;     /* [N, r, d], [N, f, r]                                       */
+  const void *a_down, *b_down; /* [N, r, f], [N, d, r]                                       */
+} mixlora_params_t;
+
+/* Gradient outputs, fp32 (d_x in shape.dtype), same shapes as the parameter they belong to.
+ * A NULL pointer skips that gradient.  The frozen weights never get one. */
+typedef struct {
+  float *d_a_gate, *d_b_gate;
+  float *d_a_up, *d_b_up;
+  float *d_a_down, *d_b_down;
+  float *d_w_router;          /* [N, d] */
+  float *d_router_bias;       /* [N]    */
+  void *d_x;                  /* [T, d] or NULL                                               */
+  int32_t accumulate;         /* 0: overwrite the fp32 outputs; 1: add to them (gradient
+                                 accumulation, Table 3).  d_x is always overwritten.          */
+} mixlora_grads_t;
+
+/* Compiled limits, for callers that size things ahead of time. */
+typedef struct {
+  int32_t max_experts, max_top_k, max_rank;
+} mixlora_limits_t;
+void mixlora_limits(mixlora_limits_t *out /* host */);
+
+/* Bytes of workspace that forward (for_backward = 0) or forward followed by backward
+ * (for_backward = 1) need for this shape.  Returns 0 if the shape is invalid. */
+size_t mixlora_workspace_bytes(const mixlora_shape_t *shape /* host */, int for_backward);
+
+/* Forward pass: y = sum_j g_tj * E_{e_tj}(x_t)  (Eq. 6 through Algorithm 1).
+ * Steps, all on the device: router logits, softmax, top-k, gates (Eq. 7); slot histogram,
+ * prefix scan and stable permutation by expert; shared W1/W3 projections once per token
+ * (Section 3.3 (I)); per-expert LoRA deltas; SwiGLU; down projection plus its LoRA; gate-
+ * weighted combine.  `y` is [T, d] in shape.dtype.  The routing, the probabilities and the
+ * activations that the backward pass re-uses are left in `workspace` (256-byte aligned). */
+mixlora_status_t mixlora_ffn_forward(const mixlora_shape_t *shape /* host */,
+                                     const mixlora_params_t *params /* host struct of device ptrs */,
+                                     void *y, void *workspace, size_t workspace_bytes, void *stream);
+
+/* Auxiliary load-balance loss of Eq. 8-9 from the routing that the last forward call left
+ * in `workspace`: loss = coef * N * sum_i F_i * P_i.  `loss` is a device scalar; `F`, `P`
+ * are device arrays of N floats or NULL. */
+mixlora_status_t mixlora_aux_loss(const mixlora_shape_t *shape /* host */, const void *workspace, float coef,
+                                  float *loss, float *F, float *P, void *stream);
+
+/* Backward pass of L = <dy, y> + aux_coef * N * sum_i F_i P_i with respect to the LoRA
+ * matrices, the router and, if grads->d_x is not NULL, x (chain rule on Algorithm 1; the
+ * paper prints no backward).  Needs the workspace exactly as the forward call for the same
+ * shape and params left it (size for_backward = 1).  `dy` is [T, d] in shape.dtype. */
+mixlora_status_t mixlora_ffn_backward(const mixlora_shape_t *shape /* host */,
+                                      const mixlora_params_t *params /* host struct of device ptrs */,
+                                      const void *dy, float aux_coef, void *workspace, size_t workspace_bytes,
+                                      const mixlora_grads_t *grads /* host struct of device ptrs */, void *stream);
+
+/* Device pointers into the workspace, for inspection after a forward call:
+ * expert_idx [T, k] (descending logit), gates [T, k], perm [T*k] (slot id at each position
+ * of the order "expert ascending, token ascending"), seg_off [N+1] (first position of each
+ * expert), low_margin [T] (1 where a logit gap deciding the top-k set or the arg-max is
+ * below 1e-4), probs [T, N].  Any output pointer may be NULL. */
+mixlora_status_t mixlora_routing_view(const mixlora_shape_t *shape /* host */, const void *workspace,
+                                      const int32_t **expert_idx, const float **gates, const int32_t **perm,
+                                      const int32_t **seg_off, const uint8_t **low_margin, const float **probs);
+
+/* Reads the device status word of the workspace (synchronises `stream`).  *code is 0 when
+ * no kernel reported a problem, else the mixlora_status_t the kernel recorded. */
+mixlora_status_t mixlora_device_status(const void *workspace, int32_t *code /* host */, void *stream);
+
+/* Dense product C[M, N] = A[M, K] * op(B) on the tensor-core path used for the frozen
+ * projections (the W1/W3/W2 products of Algorithm 1 and their transposes in the backward
+ * pass), exposed so that it can be tested and timed on its own.  A is [M, K] row-major
+ * bf16.  b_is_kn = 0: B is [N, K] row-major (a weight stored [out, in]); b_is_kn = 1: B is
+ * [K, N] row-major (the same weight used transposed).  C is [M, N] row-major bf16.
+ * K and N must be multiples of 8.  `status_word` is a device int32 that receives a non-zero
+ * code if a bounded wait in the kernel runs out, or NULL. */
+mixlora_status_t mixlora_gemm_bf16(const void *A, const void *B, void *C, int32_t M, int32_t N, int32_t K,
+                                   int32_t b_is_kn, int32_t *status_word, void *stream);
+
+const char *mixlora_status_string(mixlora_status_t status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* MIXLORA_H_ */

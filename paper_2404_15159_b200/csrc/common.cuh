@@ -1,0 +1,154 @@
+// Shared declarations of the MixLoRA FFN library: workspace layout, launch helpers.
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stddef.h>
+#include <stdint.h>
+
+#include "mixlora.h"
+
+namespace mixlora {
+
+typedef __nv_bfloat16 bf16;
+
+// ---------------------------------------------------------------------------------------
+// Workspace layout.  Every region starts on a 256-byte boundary.  "act" regions hold
+// elements of the activation type (bf16 or fp32 according to shape.dtype).
+// The regions up to total_fwd are what a forward call needs; the rest is backward scratch.
+// ---------------------------------------------------------------------------------------
+struct WsLayout {
+  size_t status;      // int32[64]; [0] = device status word
+  size_t probs;       // f32 [T, N]        softmax probabilities (Eq. 7)
+  size_t expert_idx;  // i32 [T, k]
+  size_t gates;       // f32 [T, k]
+  size_t low_margin;  // u8  [T]
+  size_t perm;        // i32 [T*k]         slot id at sorted position
+  size_t inv;         // i32 [T*k]         sorted position of slot id
+  size_t pos_token;   // i32 [T*k]         token of sorted position
+  size_t pos_expert;  // i32 [T*k]         expert of sorted position
+  size_t seg_off;     // i32 [N+1]
+  size_t blk_counts;  // i32 [nblk, N]
+  size_t blk_off;     // i32 [nblk, N]
+  size_t stat_F;      // f32 [N]           F_i of Eq. 9
+  size_t stat_P;      // f32 [N]           P_i of Eq. 9
+  size_t tile_info;   // i32 [max_tiles, 4] (expert, first position, rows, 0) of kSegTile-row segment tiles;
+                      //                    the int after the table holds the tile count
+  size_t G, U;        // act [T, f]        shared W1 / W3 projections (Section 3.3 (I))
+  size_t zga, zua;    // act [T, N*r]      A_g x and A_u x for every expert
+  size_t zd;          // act [T*k, r]      A_d h per sorted slot
+  size_t Zs;          // act [T, N*r]      gate * zd scattered to the slot's expert block
+  size_t bd_cat;      // act [d, N*r]      s * B_d laid out [c][e*r + rr]
+  size_t h_sorted;    // act [T*k, f]
+  size_t hbar;        // act [T, f]        sum_j g_j h_j
+  size_t total_fwd;
+  size_t D;           // act [T, f]        dy W_d
+  size_t spd;         // act [T, N*r]      s * B_d^T dy for every expert
+  size_t da_sorted, db_sorted;  // act [T*k, f]
+  size_t dabar, dbbar;          // act [T, f]
+  size_t zg_sorted, zu_sorted;  // act [T*k, r]
+  size_t dzg_sorted, dzu_sorted, dzd_sorted, gzd_sorted;  // act [T*k, r]
+  size_t dZg, dZu;    // act [T, N*r]      dzg / dzu scattered dense
+  size_t dgate;       // f32 [T*k]         by slot id
+  size_t dlogits;     // f32 [T, N]
+  size_t dl_act;      // act [T, NP]       dlogits in the activation type, NP = N rounded up to 8
+  size_t wr_act;      // act [NP, d]       router weight in the activation type
+  size_t total_bwd;
+};
+
+static inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+static const int kRouteBlockTokens = 256;  // tokens per block in the dispatch kernels
+static const int kSegTile = 128;           // rows of a segment tile
+
+static inline int route_blocks(int T) { return (T + kRouteBlockTokens - 1) / kRouteBlockTokens; }
+static inline int max_seg_tiles(int T, int k, int N) { return (int)(((long long)T * k + kSegTile - 1) / kSegTile) + N; }
+static inline int round_up8(int v) { return (v + 7) / 8 * 8; }
+
+WsLayout ws_layout(const mixlora_shape_t& s);
+
+static inline size_t act_size(const mixlora_shape_t& s) { return s.dtype == MIXLORA_DTYPE_BF16 ? 2 : 4; }
+
+// ---------------------------------------------------------------------------------------
+// Generic SIMT product with fp32 accumulation:
+//   C[g][m, n] (+)= alpha * sum_seg sum_k A_seg(m, k) * B_seg(n, k)
+// Operand element (i, k) of group g sits at p + g*sg + I(i)*si + K(k)*sk, where I / K are
+// optional gather tables.  group_mode 1 takes the row range of group g from
+// seg_off[g..g+1] (rows are absolute positions), group_mode 2 takes the reduction range of
+// the first K-segment from seg_off instead.
+// ---------------------------------------------------------------------------------------
+struct SOperand {
+  const void* p;
+  const int* gi;  // gather on the row / column index, or nullptr
+  const int* gk;  // gather on the reduction index, or nullptr
+  long long si, sk, sg;
+  int is_bf16;
+};
+
+static const int kMaxKSeg = 5;
+
+struct SGemm {
+  SOperand A[kMaxKSeg], B[kMaxKSeg];
+  int K[kMaxKSeg];
+  int nseg;
+  void* C;
+  long long c_sm, c_sn, c_sg;
+  int c_is_bf16;
+  int M, N;            // for group_mode 1, M is the upper bound of rows over all groups
+  const int* seg_off;  // device
+  int group_mode;
+  int groups;
+  float alpha;
+  int accumulate;
+};
+
+cudaError_t launch_simt_gemm(const SGemm& g, cudaStream_t st);
+
+static inline SOperand soperand(const void* p, long long si, long long sk, int is_bf16, long long sg = 0,
+                                const int* gi = nullptr, const int* gk = nullptr) {
+  SOperand o;
+  o.p = p; o.gi = gi; o.gk = gk; o.si = si; o.sk = sk; o.sg = sg; o.is_bf16 = is_bf16;
+  return o;
+}
+
+// ---------------------------------------------------------------------------------------
+// Kernel launchers (router.cu, elementwise.cu, tc_gemm.cu)
+// ---------------------------------------------------------------------------------------
+struct Ctx {
+  mixlora_shape_t s;
+  mixlora_params_t p;
+  WsLayout L;
+  char* ws;
+  cudaStream_t st;
+  int bf16;  // activation type is bf16
+  float scale;
+  template <typename T> T* at(size_t off) const { return reinterpret_cast<T*>(ws + off); }
+};
+
+cudaError_t launch_router(const Ctx& c);              // probs, expert_idx, gates, low_margin, stats
+cudaError_t launch_dispatch(const Ctx& c);            // perm, inv, pos_token, pos_expert, seg_off, tile_info
+cudaError_t launch_aux_loss(const Ctx& c, float coef, float* loss, float* F, float* P);
+cudaError_t launch_bd_cat(const Ctx& c);
+cudaError_t launch_lora_b_swiglu(const Ctx& c);       // h_sorted from G, U, zga, zua, B_g, B_u
+cudaError_t launch_combine_h(const Ctx& c);           // hbar, Zs
+cudaError_t launch_swiglu_bwd(const Ctx& c);          // h_sorted, da_sorted, db_sorted, dgate, z*_sorted
+cudaError_t launch_slot_prep_bwd(const Ctx& c);       // dzd_sorted, gzd_sorted
+cudaError_t launch_combine_bwd(const Ctx& c);         // dabar, dbbar, dZg, dZu
+cudaError_t launch_router_bwd(const Ctx& c, float aux_coef, float* d_bias, int accumulate, int want_dx);
+
+// Tensor-core dense product (tc_gemm.cu).  K-concatenated segments; every operand bf16.
+//   C_o[M, N_o] = sum_seg A_seg[M, K_seg] * op(B_o,seg)
+// B is [N, K_seg] row-major (b_kn = 0) or [K_seg, N] row-major (b_kn = 1).  Several outputs
+// (column blocks with their own B and C) may share one launch when they share A.
+struct TcSeg {
+  const void* A; long long lda; int K;
+  const void* B; long long ldb; int b_kn;
+};
+struct TcOut {
+  void* C; long long ldc; int N;
+  TcSeg seg[kMaxKSeg]; int nseg;
+};
+bool tc_gemm_supported(int M, const TcOut* outs, int nout);
+cudaError_t launch_tc_gemm(int M, const TcOut* outs, int nout, int* status_word, cudaStream_t st);
+
+}  // namespace mixlora
