@@ -1,0 +1,447 @@
+// Memory-bound stages of the block in the order "expert ascending, token ascending":
+// LoRA-B expansion + SwiGLU (forward and backward), combine over a token's slots,
+// small repacks, router backward.
+#include "common.cuh"
+
+namespace mixlora {
+
+namespace {
+
+__device__ __forceinline__ float to_f(float v) { return v; }
+__device__ __forceinline__ float to_f(bf16 v) { return __bfloat162float(v); }
+template <typename T> __device__ __forceinline__ T from_f(float v);
+template <> __device__ __forceinline__ float from_f<float>(float v) { return v; }
+template <> __device__ __forceinline__ bf16 from_f<bf16>(float v) { return __float2bfloat16(v); }
+
+__device__ __forceinline__ float sigmoidf_(float v) { return 1.f / (1.f + expf(-v)); }
+
+constexpr int SL = 8;      // sorted slots per block in the per-slot kernels
+constexpr int ENT = 256;   // threads per block
+
+// bd_cat[c][e*r + rr] = s * B_d[e][c][rr]
+template <typename T>
+__global__ void bd_cat_kernel(const T* __restrict__ b_down, T* __restrict__ bd_cat, int d, int N, int r, float s) {
+  const long long n = (long long)d * N * r;
+  for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < n; i += (long long)gridDim.x * blockDim.x) {
+    int rr = (int)(i % r);
+    int e = (int)((i / r) % N);
+    int c = (int)(i / ((long long)r * N));
+    bd_cat[i] = from_f<T>(s * to_f(b_down[((long long)e * d + c) * r + rr]));
+  }
+}
+
+// Forward, per sorted slot: a = G_t + s B_g[e] zg, b = U_t + s B_u[e] zu, h = SiLU(a) * b
+// (Algorithm 1, the three steps inside the expert loop before the down projection).
+template <typename T>
+__global__ void __launch_bounds__(ENT)
+lora_b_swiglu_kernel(const T* __restrict__ G, const T* __restrict__ U, const T* __restrict__ zga,
+                     const T* __restrict__ zua, const T* __restrict__ b_gate, const T* __restrict__ b_up,
+                     const int* __restrict__ pos_token, const int* __restrict__ pos_expert, T* __restrict__ h_sorted,
+                     int slots, int f, int N, int r, float s) {
+  extern __shared__ float sm[];
+  float* zg = sm;              // [SL][r], already scaled by s
+  float* zu = sm + SL * r;     // [SL][r]
+  __shared__ int tok[SL], ex[SL];
+  const int base = blockIdx.x * SL;
+  const int ns = min(SL, slots - base);
+  if (threadIdx.x < SL) {
+    int i = threadIdx.x;
+    tok[i] = (i < ns) ? pos_token[base + i] : 0;
+    ex[i] = (i < ns) ? pos_expert[base + i] : -1;
+  }
+  __syncthreads();
+  for (int i = threadIdx.x; i < SL * r; i += ENT) {
+    int sl = i / r, rr = i % r;
+    float vg = 0.f, vu = 0.f;
+    if (sl < ns) {
+      size_t o = (size_t)tok[sl] * N * r + (size_t)ex[sl] * r + rr;
+      vg = s * to_f(zga[o]);
+      vu = s * to_f(zua[o]);
+    }
+    zg[i] = vg;
+    zu[i] = vu;
+  }
+  __syncthreads();
+  for (int c = threadIdx.x; c < f; c += ENT) {
+    int i0 = 0;
+    while (i0 < ns) {
+      const int e = ex[i0];
+      int i1 = i0;
+      while (i1 < ns && ex[i1] == e) ++i1;
+      float ea[SL], eb[SL];
+#pragma unroll
+      for (int i = 0; i < SL; ++i) { ea[i] = 0.f; eb[i] = 0.f; }
+      const T* bg = b_gate + ((size_t)e * f + c) * r;
+      const T* bu = b_up + ((size_t)e * f + c) * r;
+      for (int rr = 0; rr < r; ++rr) {
+        const float wg = to_f(bg[rr]), wu = to_f(bu[rr]);
+#pragma unroll
+        for (int i = 0; i < SL; ++i) {
+          ea[i] = fmaf(zg[i * r + rr], wg, ea[i]);
+          eb[i] = fmaf(zu[i * r + rr], wu, eb[i]);
+        }
+      }
+#pragma unroll
+      for (int i = 0; i < SL; ++i) {
+        if (i >= i0 && i < i1) {
+          const size_t go = (size_t)tok[i] * f + c;
+          const float a = to_f(G[go]) + ea[i];
+          const float b = to_f(U[go]) + eb[i];
+          h_sorted[(size_t)(base + i) * f + c] = from_f<T>(a * sigmoidf_(a) * b);
+        }
+      }
+      i0 = i1;
+    }
+  }
+}
+
+// hbar_t = sum_j g_tj h_tj ;  Zs[t, e_j*r + rr] = g_tj * zd_j[rr], zero elsewhere.
+template <typename T>
+__global__ void __launch_bounds__(ENT)
+combine_h_kernel(const T* __restrict__ h_sorted, const T* __restrict__ zd, const float* __restrict__ gates,
+                 const int* __restrict__ inv, const int* __restrict__ expert_idx, T* __restrict__ hbar,
+                 T* __restrict__ Zs, int f, int N, int r, int k) {
+  const int t = blockIdx.x;
+  __shared__ int pos[MIXLORA_MAX_TOP_K], ex[MIXLORA_MAX_TOP_K];
+  __shared__ float g[MIXLORA_MAX_TOP_K];
+  if (threadIdx.x < k) {
+    pos[threadIdx.x] = inv[(size_t)t * k + threadIdx.x];
+    ex[threadIdx.x] = expert_idx[(size_t)t * k + threadIdx.x];
+    g[threadIdx.x] = gates[(size_t)t * k + threadIdx.x];
+  }
+  __syncthreads();
+  for (int c = threadIdx.x; c < f; c += ENT) {
+    float acc = 0.f;
+    for (int j = 0; j < k; ++j) acc = fmaf(g[j], to_f(h_sorted[(size_t)pos[j] * f + c]), acc);
+    hbar[(size_t)t * f + c] = from_f<T>(acc);
+  }
+  const int nr = N * r;
+  for (int q = threadIdx.x; q < nr; q += ENT) {
+    const int e = q / r, rr = q % r;
+    float v = 0.f;
+    for (int j = 0; j < k; ++j)
+      if (ex[j] == e) v = g[j] * to_f(zd[(size_t)pos[j] * r + rr]);
+    Zs[(size_t)t * nr + q] = from_f<T>(v);
+  }
+}
+
+// Backward, per sorted slot.  Re-computes a, b, h from the saved G, U, zg, zu, then
+//   Dt = D_t + A_d[e]^T (s pd)      (gradient of the slot's h before the gate)
+//   dgate = <Dt, h> ;  dh = g Dt ;  da = dh * b * SiLU'(a) ;  db = dh * SiLU(a)
+template <typename T>
+__global__ void __launch_bounds__(ENT)
+swiglu_bwd_kernel(const T* __restrict__ G, const T* __restrict__ U, const T* __restrict__ D,
+                  const T* __restrict__ zga, const T* __restrict__ zua, const T* __restrict__ spd,
+                  const T* __restrict__ b_gate, const T* __restrict__ b_up, const T* __restrict__ a_down,
+                  const float* __restrict__ gates, const int* __restrict__ perm, const int* __restrict__ pos_token,
+                  const int* __restrict__ pos_expert, T* __restrict__ h_sorted, T* __restrict__ da_sorted,
+                  T* __restrict__ db_sorted, T* __restrict__ zg_sorted, T* __restrict__ zu_sorted,
+                  float* __restrict__ dgate, int slots, int f, int N, int r, float s) {
+  extern __shared__ float sm[];
+  float* zg = sm;                 // [SL][r] scaled by s
+  float* zu = sm + SL * r;        // [SL][r] scaled by s
+  float* pd = sm + 2 * SL * r;    // [SL][r] = s * pd
+  __shared__ int tok[SL], ex[SL], slot[SL];
+  __shared__ float gt[SL];
+  __shared__ float red[SL][ENT / 32];
+  const int base = blockIdx.x * SL;
+  const int ns = min(SL, slots - base);
+  if (threadIdx.x < SL) {
+    int i = threadIdx.x;
+    tok[i] = (i < ns) ? pos_token[base + i] : 0;
+    ex[i] = (i < ns) ? pos_expert[base + i] : -1;
+    slot[i] = (i < ns) ? perm[base + i] : 0;
+    gt[i] = (i < ns) ? gates[slot[i]] : 0.f;
+  }
+  __syncthreads();
+  for (int i = threadIdx.x; i < SL * r; i += ENT) {
+    int sl = i / r, rr = i % r;
+    float vg = 0.f, vu = 0.f, vp = 0.f;
+    if (sl < ns) {
+      size_t o = (size_t)tok[sl] * N * r + (size_t)ex[sl] * r + rr;
+      T zgv = zga[o], zuv = zua[o];
+      vg = s * to_f(zgv);
+      vu = s * to_f(zuv);
+      vp = to_f(spd[o]);
+      zg_sorted[(size_t)(base + sl) * r + rr] = zgv;
+      zu_sorted[(size_t)(base + sl) * r + rr] = zuv;
+    }
+    zg[i] = vg; zu[i] = vu; pd[i] = vp;
+  }
+  __syncthreads();
+  float dg_acc[SL];
+#pragma unroll
+  for (int i = 0; i < SL; ++i) dg_acc[i] = 0.f;
+  for (int c = threadIdx.x; c < f; c += ENT) {
+    int i0 = 0;
+    while (i0 < ns) {
+      const int e = ex[i0];
+      int i1 = i0;
+      while (i1 < ns && ex[i1] == e) ++i1;
+      float ea[SL], eb[SL], ed[SL];
+#pragma unroll
+      for (int i = 0; i < SL; ++i) { ea[i] = 0.f; eb[i] = 0.f; ed[i] = 0.f; }
+      const T* bg = b_gate + ((size_t)e * f + c) * r;
+      const T* bu = b_up + ((size_t)e * f + c) * r;
+      const T* ad = a_down + (size_t)e * r * f + c;
+      for (int rr = 0; rr < r; ++rr) {
+        const float wg = to_f(bg[rr]), wu = to_f(bu[rr]), wd = to_f(ad[(size_t)rr * f]);
+#pragma unroll
+        for (int i = 0; i < SL; ++i) {
+          ea[i] = fmaf(zg[i * r + rr], wg, ea[i]);
+          eb[i] = fmaf(zu[i * r + rr], wu, eb[i]);
+          ed[i] = fmaf(pd[i * r + rr], wd, ed[i]);
+        }
+      }
+#pragma unroll
+      for (int i = 0; i < SL; ++i) {
+        if (i >= i0 && i < i1) {
+          const size_t go = (size_t)tok[i] * f + c;
+          const float a = to_f(G[go]) + ea[i];
+          const float b = to_f(U[go]) + eb[i];
+          const float sg = sigmoidf_(a);
+          const float sa = a * sg;
+          const float h = sa * b;
+          const float Dt = to_f(D[go]) + ed[i];
+          dg_acc[i] = fmaf(Dt, h, dg_acc[i]);
+          const float dh = gt[i] * Dt;
+          const size_t so = (size_t)(base + i) * f + c;
+          h_sorted[so] = from_f<T>(h);
+          da_sorted[so] = from_f<T>(dh * b * sg * (1.f + a * (1.f - sg)));
+          db_sorted[so] = from_f<T>(dh * sa);
+        }
+      }
+      i0 = i1;
+    }
+  }
+  // deterministic block reduction of the gate gradients
+  const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+#pragma unroll
+  for (int i = 0; i < SL; ++i) {
+    float v = dg_acc[i];
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    if (lane == 0) red[i][w] = v;
+  }
+  __syncthreads();
+  if (threadIdx.x < ns) {
+    float v = 0.f;
+    for (int ww = 0; ww < ENT / 32; ++ww) v += red[threadIdx.x][ww];
+    dgate[slot[threadIdx.x]] = v;
+  }
+}
+
+// dzd_sorted = g * (s pd) at the slot's expert ; gzd_sorted = g * zd
+template <typename T>
+__global__ void slot_prep_bwd_kernel(const T* __restrict__ spd, const T* __restrict__ zd, const float* __restrict__ gates,
+                                     const int* __restrict__ perm, const int* __restrict__ pos_token,
+                                     const int* __restrict__ pos_expert, T* __restrict__ dzd_sorted,
+                                     T* __restrict__ gzd_sorted, int slots, int N, int r) {
+  const long long n = (long long)slots * r;
+  for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < n; i += (long long)gridDim.x * blockDim.x) {
+    const int pos = (int)(i / r), rr = (int)(i % r);
+    const float g = gates[perm[pos]];
+    const size_t o = (size_t)pos_token[pos] * N * r + (size_t)pos_expert[pos] * r + rr;
+    dzd_sorted[i] = from_f<T>(g * to_f(spd[o]));
+    gzd_sorted[i] = from_f<T>(g * to_f(zd[i]));
+  }
+}
+
+// dabar_t = sum_j da_tj, dbbar_t = sum_j db_tj ; dZg / dZu = dzg / dzu scattered to the expert block
+template <typename T>
+__global__ void __launch_bounds__(ENT)
+combine_bwd_kernel(const T* __restrict__ da_sorted, const T* __restrict__ db_sorted, const T* __restrict__ dzg_sorted,
+                   const T* __restrict__ dzu_sorted, const int* __restrict__ inv, const int* __restrict__ expert_idx,
+                   T* __restrict__ dabar, T* __restrict__ dbbar, T* __restrict__ dZg, T* __restrict__ dZu, int f, int N,
+                   int r, int k) {
+  const int t = blockIdx.x;
+  __shared__ int pos[MIXLORA_MAX_TOP_K], ex[MIXLORA_MAX_TOP_K];
+  if (threadIdx.x < k) {
+    pos[threadIdx.x] = inv[(size_t)t * k + threadIdx.x];
+    ex[threadIdx.x] = expert_idx[(size_t)t * k + threadIdx.x];
+  }
+  __syncthreads();
+  for (int c = threadIdx.x; c < f; c += ENT) {
+    float sa = 0.f, sb = 0.f;
+    for (int j = 0; j < k; ++j) {
+      sa += to_f(da_sorted[(size_t)pos[j] * f + c]);
+      sb += to_f(db_sorted[(size_t)pos[j] * f + c]);
+    }
+    dabar[(size_t)t * f + c] = from_f<T>(sa);
+    dbbar[(size_t)t * f + c] = from_f<T>(sb);
+  }
+  const int nr = N * r;
+  for (int q = threadIdx.x; q < nr; q += ENT) {
+    const int e = q / r, rr = q % r;
+    T vg = from_f<T>(0.f), vu = from_f<T>(0.f);
+    for (int j = 0; j < k; ++j)
+      if (ex[j] == e) {
+        vg = dzg_sorted[(size_t)pos[j] * r + rr];
+        vu = dzu_sorted[(size_t)pos[j] * r + rr];
+      }
+    dZg[(size_t)t * nr + q] = vg;
+    dZu[(size_t)t * nr + q] = vu;
+  }
+}
+
+// Router backward, one thread per token: gate re-normalisation, auxiliary-loss term
+// (F_i is piecewise constant, so only P_i carries gradient), softmax.
+template <typename T>
+__global__ void router_bwd_kernel(const float* __restrict__ probs, const float* __restrict__ gates,
+                                  const int* __restrict__ expert_idx, const float* __restrict__ dgate,
+                                  const float* __restrict__ F, float* __restrict__ dlogits, T* __restrict__ dl_act,
+                                  int tokens, int N, int NP, int k, int renorm, float aux_scale) {
+  const int t = blockIdx.x * blockDim.x + threadIdx.x;
+  if (t >= tokens) return;
+  float dp[MIXLORA_MAX_EXPERTS];
+#pragma unroll
+  for (int e = 0; e < MIXLORA_MAX_EXPERTS; ++e) dp[e] = (e < N) ? aux_scale * F[e] : 0.f;
+  float q = 0.f, inner = 0.f;
+  for (int j = 0; j < k; ++j) {
+    const int e = expert_idx[(size_t)t * k + j];
+    q += probs[(size_t)t * N + e];
+    inner = fmaf(gates[(size_t)t * k + j], dgate[(size_t)t * k + j], inner);
+  }
+  for (int j = 0; j < k; ++j) {
+    const int e = expert_idx[(size_t)t * k + j];
+    const float dg = dgate[(size_t)t * k + j];
+    const float v = renorm ? (dg - inner) / q : dg;
+#pragma unroll
+    for (int ee = 0; ee < MIXLORA_MAX_EXPERTS; ++ee)
+      if (ee == e) dp[ee] += v;
+  }
+  float dot = 0.f;
+#pragma unroll
+  for (int e = 0; e < MIXLORA_MAX_EXPERTS; ++e)
+    if (e < N) dot = fmaf(probs[(size_t)t * N + e], dp[e], dot);
+#pragma unroll
+  for (int e = 0; e < MIXLORA_MAX_EXPERTS; ++e) {
+    if (e < NP) {
+      float v = (e < N) ? probs[(size_t)t * N + e] * (dp[e] - dot) : 0.f;
+      if (e < N) dlogits[(size_t)t * N + e] = v;
+      if (dl_act) dl_act[(size_t)t * NP + e] = from_f<T>(v);
+    }
+  }
+}
+
+// out[e] = sum_t dl[t, e], one block per expert, fixed order.
+__global__ void __launch_bounds__(256)
+colsum_kernel(const float* __restrict__ dl, float* __restrict__ out, int tokens, int N, int accumulate) {
+  __shared__ float sp[256];
+  const int e = blockIdx.x;
+  float s = 0.f;
+  for (int t = threadIdx.x; t < tokens; t += 256) s += dl[(size_t)t * N + e];
+  sp[threadIdx.x] = s;
+  __syncthreads();
+  for (int o = 128; o > 0; o >>= 1) {
+    if (threadIdx.x < o) sp[threadIdx.x] += sp[threadIdx.x + o];
+    __syncthreads();
+  }
+  if (threadIdx.x == 0) out[e] = accumulate ? out[e] + sp[0] : sp[0];
+}
+
+// router weight in the activation type, rows padded to NP with zeros
+template <typename T>
+__global__ void wr_act_kernel(const float* __restrict__ w_router, T* __restrict__ wr_act, int N, int NP, int d) {
+  const long long n = (long long)NP * d;
+  for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < n; i += (long long)gridDim.x * blockDim.x) {
+    int e = (int)(i / d);
+    wr_act[i] = from_f<T>(e < N ? w_router[i] : 0.f);
+  }
+}
+
+inline int grid_for(long long n, int block) {
+  long long g = (n + block - 1) / block;
+  return (int)(g < 1 ? 1 : (g > 148 * 16 ? 148 * 16 : g));
+}
+
+template <typename T>
+cudaError_t bd_cat_t(const Ctx& c) {
+  const long long n = (long long)c.s.d_model * c.s.n_experts * c.s.rank;
+  bd_cat_kernel<T><<<grid_for(n, 256), 256, 0, c.st>>>(reinterpret_cast<const T*>(c.p.b_down), c.at<T>(c.L.bd_cat),
+                                                      c.s.d_model, c.s.n_experts, c.s.rank, c.scale);
+  return cudaGetLastError();
+}
+
+template <typename T>
+cudaError_t lora_b_swiglu_t(const Ctx& c) {
+  const int slots = c.s.tokens * c.s.top_k;
+  const int blocks = (slots + SL - 1) / SL;
+  const size_t smem = 2 * SL * c.s.rank * sizeof(float);
+  lora_b_swiglu_kernel<T><<<blocks, ENT, smem, c.st>>>(
+      c.at<T>(c.L.G), c.at<T>(c.L.U), c.at<T>(c.L.zga), c.at<T>(c.L.zua), reinterpret_cast<const T*>(c.p.b_gate),
+      reinterpret_cast<const T*>(c.p.b_up), c.at<int>(c.L.pos_token), c.at<int>(c.L.pos_expert), c.at<T>(c.L.h_sorted),
+      slots, c.s.d_ff, c.s.n_experts, c.s.rank, c.scale);
+  return cudaGetLastError();
+}
+
+template <typename T>
+cudaError_t combine_h_t(const Ctx& c) {
+  combine_h_kernel<T><<<c.s.tokens, ENT, 0, c.st>>>(c.at<T>(c.L.h_sorted), c.at<T>(c.L.zd), c.at<float>(c.L.gates),
+                                                   c.at<int>(c.L.inv), c.at<int>(c.L.expert_idx), c.at<T>(c.L.hbar),
+                                                   c.at<T>(c.L.Zs), c.s.d_ff, c.s.n_experts, c.s.rank, c.s.top_k);
+  return cudaGetLastError();
+}
+
+template <typename T>
+cudaError_t swiglu_bwd_t(const Ctx& c) {
+  const int slots = c.s.tokens * c.s.top_k;
+  const int blocks = (slots + SL - 1) / SL;
+  const size_t smem = 3 * SL * c.s.rank * sizeof(float);
+  swiglu_bwd_kernel<T><<<blocks, ENT, smem, c.st>>>(
+      c.at<T>(c.L.G), c.at<T>(c.L.U), c.at<T>(c.L.D), c.at<T>(c.L.zga), c.at<T>(c.L.zua), c.at<T>(c.L.spd),
+      reinterpret_cast<const T*>(c.p.b_gate), reinterpret_cast<const T*>(c.p.b_up),
+      reinterpret_cast<const T*>(c.p.a_down), c.at<float>(c.L.gates), c.at<int>(c.L.perm), c.at<int>(c.L.pos_token),
+      c.at<int>(c.L.pos_expert), c.at<T>(c.L.h_sorted), c.at<T>(c.L.da_sorted), c.at<T>(c.L.db_sorted),
+      c.at<T>(c.L.zg_sorted), c.at<T>(c.L.zu_sorted), c.at<float>(c.L.dgate), slots, c.s.d_ff, c.s.n_experts, c.s.rank,
+      c.scale);
+  return cudaGetLastError();
+}
+
+template <typename T>
+cudaError_t slot_prep_bwd_t(const Ctx& c) {
+  const int slots = c.s.tokens * c.s.top_k;
+  slot_prep_bwd_kernel<T><<<grid_for((long long)slots * c.s.rank, 256), 256, 0, c.st>>>(
+      c.at<T>(c.L.spd), c.at<T>(c.L.zd), c.at<float>(c.L.gates), c.at<int>(c.L.perm), c.at<int>(c.L.pos_token),
+      c.at<int>(c.L.pos_expert), c.at<T>(c.L.dzd_sorted), c.at<T>(c.L.gzd_sorted), slots, c.s.n_experts, c.s.rank);
+  return cudaGetLastError();
+}
+
+template <typename T>
+cudaError_t combine_bwd_t(const Ctx& c) {
+  combine_bwd_kernel<T><<<c.s.tokens, ENT, 0, c.st>>>(
+      c.at<T>(c.L.da_sorted), c.at<T>(c.L.db_sorted), c.at<T>(c.L.dzg_sorted), c.at<T>(c.L.dzu_sorted),
+      c.at<int>(c.L.inv), c.at<int>(c.L.expert_idx), c.at<T>(c.L.dabar), c.at<T>(c.L.dbbar), c.at<T>(c.L.dZg),
+      c.at<T>(c.L.dZu), c.s.d_ff, c.s.n_experts, c.s.rank, c.s.top_k);
+  return cudaGetLastError();
+}
+
+template <typename T>
+cudaError_t router_bwd_t(const Ctx& c, float aux_coef, float* d_bias, int accumulate, int want_dx) {
+  const int T_ = c.s.tokens, N = c.s.n_experts, NP = round_up8(N);
+  const float aux_scale = (T_ > 0) ? aux_coef * (float)N / (float)T_ : 0.f;
+  router_bwd_kernel<T><<<(T_ + 127) / 128, 128, 0, c.st>>>(
+      c.at<float>(c.L.probs), c.at<float>(c.L.gates), c.at<int>(c.L.expert_idx), c.at<float>(c.L.dgate),
+      c.at<float>(c.L.stat_F), c.at<float>(c.L.dlogits), want_dx ? c.at<T>(c.L.dl_act) : nullptr, T_, N, NP, c.s.top_k,
+      c.s.renormalize, aux_scale);
+  if (d_bias) colsum_kernel<<<N, 256, 0, c.st>>>(c.at<float>(c.L.dlogits), d_bias, T_, N, accumulate);
+  if (want_dx)
+    wr_act_kernel<T><<<grid_for((long long)NP * c.s.d_model, 256), 256, 0, c.st>>>(c.p.w_router, c.at<T>(c.L.wr_act), N,
+                                                                                 NP, c.s.d_model);
+  return cudaGetLastError();
+}
+
+}  // namespace
+
+cudaError_t launch_bd_cat(const Ctx& c) { return c.bf16 ? bd_cat_t<bf16>(c) : bd_cat_t<float>(c); }
+cudaError_t launch_lora_b_swiglu(const Ctx& c) { return c.bf16 ? lora_b_swiglu_t<bf16>(c) : lora_b_swiglu_t<float>(c); }
+cudaError_t launch_combine_h(const Ctx& c) { return c.bf16 ? combine_h_t<bf16>(c) : combine_h_t<float>(c); }
+cudaError_t launch_swiglu_bwd(const Ctx& c) { return c.bf16 ? swiglu_bwd_t<bf16>(c) : swiglu_bwd_t<float>(c); }
+cudaError_t launch_slot_prep_bwd(const Ctx& c) { return c.bf16 ? slot_prep_bwd_t<bf16>(c) : slot_prep_bwd_t<float>(c); }
+cudaError_t launch_combine_bwd(const Ctx& c) { return c.bf16 ? combine_bwd_t<bf16>(c) : combine_bwd_t<float>(c); }
+cudaError_t launch_router_bwd(const Ctx& c, float aux_coef, float* d_bias, int accumulate, int want_dx) {
+  return c.bf16 ? router_bwd_t<bf16>(c, aux_coef, d_bias, accumulate, want_dx)
+                : router_bwd_t<float>(c, aux_coef, d_bias, accumulate, want_dx);
+}
+
+}  // namespace mixlora
