@@ -1,0 +1,407 @@
+// C ABI of the MixLoRA FFN library: argument checks, workspace layout, and the sequence of
+// kernel launches of the forward and backward passes.
+#include <stdio.h>
+#include <string.h>
+
+#include "common.cuh"
+
+namespace mixlora {
+
+WsLayout ws_layout(const mixlora_shape_t& s) {
+  WsLayout L;
+  memset(&L, 0, sizeof(L));
+  const size_t T = (size_t)s.tokens, d = (size_t)s.d_model, f = (size_t)s.d_ff, N = (size_t)s.n_experts,
+               k = (size_t)s.top_k, r = (size_t)s.rank;
+  const size_t E = act_size(s);
+  const size_t nblk = (size_t)route_blocks(s.tokens);
+  const size_t mt = (size_t)max_seg_tiles(s.tokens, s.top_k, s.n_experts);
+  const size_t NP = (size_t)round_up8(s.n_experts);
+  size_t off = 0;
+  auto take = [&](size_t bytes) {
+    size_t o = off;
+    off = align_up(off + (bytes ? bytes : 1), 256);
+    return o;
+  };
+  L.status = take(64 * 4);
+  L.probs = take(T * N * 4);
+  L.expert_idx = take(T * k * 4);
+  L.gates = take(T * k * 4);
+  L.low_margin = take(T);
+  L.perm = take(T * k * 4);
+  L.inv = take(T * k * 4);
+  L.pos_token = take(T * k * 4);
+  L.pos_expert = take(T * k * 4);
+  L.seg_off = take((N + 1) * 4);
+  L.blk_counts = take(nblk * N * 4);
+  L.blk_off = take(nblk * N * 4);
+  L.stat_F = take(N * 4);
+  L.stat_P = take(N * 4);
+  L.tile_info = take((mt * 4 + 4) * 4);
+  L.G = take(T * f * E);
+  L.U = take(T * f * E);
+  L.zga = take(T * N * r * E);
+  L.zua = take(T * N * r * E);
+  L.zd = take(T * k * r * E);
+  L.Zs = take(T * N * r * E);
+  L.bd_cat = take(d * N * r * E);
+  L.h_sorted = take(T * k * f * E);
+  L.hbar = take(T * f * E);
+  L.total_fwd = off;
+  L.D = take(T * f * E);
+  L.spd = take(T * N * r * E);
+  L.da_sorted = take(T * k * f * E);
+  L.db_sorted = take(T * k * f * E);
+  L.dabar = take(T * f * E);
+  L.dbbar = take(T * f * E);
+  L.zg_sorted = take(T * k * r * E);
+  L.zu_sorted = take(T * k * r * E);
+  L.dzg_sorted = take(T * k * r * E);
+  L.dzu_sorted = take(T * k * r * E);
+  L.dzd_sorted = take(T * k * r * E);
+  L.gzd_sorted = take(T * k * r * E);
+  L.dZg = take(T * N * r * E);
+  L.dZu = take(T * N * r * E);
+  L.dgate = take(T * k * 4);
+  L.dlogits = take(T * N * 4);
+  L.dl_act = take(T * NP * E);
+  L.wr_act = take(NP * d * E);
+  L.total_bwd = off;
+  return L;
+}
+
+namespace {
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+mixlora_status_t check_shape(const mixlora_shape_t* s) {
+  if (!s || s->struct_size != sizeof(mixlora_shape_t)) return MIXLORA_ERR_INVALID_ARG;
+  if (s->tokens < 0 || s->d_model <= 0 || s->d_ff <= 0 || s->n_experts <= 0 || s->top_k <= 0 || s->rank <= 0)
+    return MIXLORA_ERR_INVALID_ARG;
+  if (s->top_k > s->n_experts) return MIXLORA_ERR_INVALID_ARG;
+  if (s->dtype != MIXLORA_DTYPE_BF16 && s->dtype != MIXLORA_DTYPE_FP32) return MIXLORA_ERR_INVALID_ARG;
+  if (!(s->lora_alpha == s->lora_alpha)) return MIXLORA_ERR_INVALID_ARG;
+  if (s->aux_f_mode != 0 && s->aux_f_mode != 1) return MIXLORA_ERR_INVALID_ARG;
+  if (s->renormalize != 0 && s->renormalize != 1) return MIXLORA_ERR_INVALID_ARG;
+  if (s->d_model % 8 || s->d_ff % 8) return MIXLORA_ERR_UNSUPPORTED;
+  if (s->n_experts > MIXLORA_MAX_EXPERTS || s->top_k > MIXLORA_MAX_TOP_K || s->rank > MIXLORA_MAX_RANK)
+    return MIXLORA_ERR_UNSUPPORTED;
+  if (s->dtype == MIXLORA_DTYPE_BF16 && s->rank % 8) return MIXLORA_ERR_UNSUPPORTED;
+  if (s->dtype == MIXLORA_DTYPE_FP32 && s->rank % 4) return MIXLORA_ERR_UNSUPPORTED;
+  if ((long long)s->tokens * s->top_k > 4000000LL) return MIXLORA_ERR_UNSUPPORTED;
+  return MIXLORA_OK;
+}
+
+mixlora_status_t check_params(const mixlora_params_t* p) {
+  if (!p) return MIXLORA_ERR_INVALID_ARG;
+  const void* req[] = {p->x, p->w_gate, p->w_up, p->w_down, p->w_router, p->a_gate, p->b_gate,
+                       p->a_up, p->b_up, p->a_down, p->b_down};
+  for (const void* q : req)
+    if (!q || !aligned16(q)) return MIXLORA_ERR_INVALID_ARG;
+  if (p->router_bias && (reinterpret_cast<uintptr_t>(p->router_bias) & 3u)) return MIXLORA_ERR_INVALID_ARG;
+  return MIXLORA_OK;
+}
+
+#define MIXLORA_CUDA(expr)                              \
+  do {                                                  \
+    cudaError_t e__ = (expr);                           \
+    if (e__ != cudaSuccess) return MIXLORA_ERR_CUDA;    \
+  } while (0)
+
+Ctx make_ctx(const mixlora_shape_t* s, const mixlora_params_t* p, void* ws, void* stream) {
+  Ctx c;
+  c.s = *s;
+  if (p) c.p = *p; else memset(&c.p, 0, sizeof(c.p));
+  c.L = ws_layout(*s);
+  c.ws = reinterpret_cast<char*>(ws);
+  c.st = reinterpret_cast<cudaStream_t>(stream);
+  c.bf16 = (s->dtype == MIXLORA_DTYPE_BF16);
+  c.scale = s->lora_alpha / (float)s->rank;
+  return c;
+}
+
+SGemm sgemm_base(const Ctx& c, void* C, long long c_sm, long long c_sn, int c_bf16, int M, int N) {
+  SGemm g;
+  memset(&g, 0, sizeof(g));
+  g.C = C; g.c_sm = c_sm; g.c_sn = c_sn; g.c_sg = 0; g.c_is_bf16 = c_bf16;
+  g.M = M; g.N = N; g.groups = 1; g.group_mode = 0; g.alpha = 1.f; g.accumulate = 0; g.nseg = 0;
+  g.seg_off = c.at<int>(c.L.seg_off);
+  return g;
+}
+
+void add_seg(SGemm& g, const SOperand& A, const SOperand& B, int K) {
+  g.A[g.nseg] = A; g.B[g.nseg] = B; g.K[g.nseg] = K; ++g.nseg;
+}
+
+// Dense product on the tensor-core kernel when it takes the shape, else on the SIMT kernel.
+cudaError_t dense_product(const Ctx& c, int M, const TcOut* outs, int nout) {
+  if (c.bf16 && tc_gemm_supported(M, outs, nout)) return launch_tc_gemm(M, outs, nout, c.at<int>(c.L.status), c.st);
+  for (int o = 0; o < nout; ++o) {
+    const TcOut& t = outs[o];
+    SGemm g = sgemm_base(c, t.C, t.ldc, 1, c.bf16, M, t.N);
+    for (int i = 0; i < t.nseg; ++i) {
+      const TcSeg& sg = t.seg[i];
+      SOperand A = soperand(sg.A, sg.lda, 1, c.bf16);
+      SOperand B = sg.b_kn ? soperand(sg.B, 1, sg.ldb, c.bf16) : soperand(sg.B, sg.ldb, 1, c.bf16);
+      add_seg(g, A, B, sg.K);
+    }
+    cudaError_t e = launch_simt_gemm(g, c.st);
+    if (e != cudaSuccess) return e;
+  }
+  return cudaSuccess;
+}
+
+TcOut tc_out(void* C, long long ldc, int N) {
+  TcOut o;
+  memset(&o, 0, sizeof(o));
+  o.C = C; o.ldc = ldc; o.N = N; o.nseg = 0;
+  return o;
+}
+void tc_add(TcOut& o, const void* A, long long lda, int K, const void* B, long long ldb, int b_kn) {
+  TcSeg& s = o.seg[o.nseg++];
+  s.A = A; s.lda = lda; s.K = K; s.B = B; s.ldb = ldb; s.b_kn = b_kn;
+}
+
+}  // namespace
+}  // namespace mixlora
+
+using namespace mixlora;
+
+extern "C" {
+
+void mixlora_limits(mixlora_limits_t* out) {
+  if (!out) return;
+  out->max_experts = MIXLORA_MAX_EXPERTS;
+  out->max_top_k = MIXLORA_MAX_TOP_K;
+  out->max_rank = MIXLORA_MAX_RANK;
+}
+
+const char* mixlora_status_string(mixlora_status_t st) {
+  switch (st) {
+    case MIXLORA_OK: return "ok";
+    case MIXLORA_ERR_INVALID_ARG: return "invalid argument";
+    case MIXLORA_ERR_UNSUPPORTED: return "size outside the supported limits";
+    case MIXLORA_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
+    case MIXLORA_ERR_CUDA: return "CUDA call failed";
+    case MIXLORA_ERR_DEVICE_TIMEOUT: return "a bounded wait inside a kernel ran out";
+  }
+  return "unknown status";
+}
+
+size_t mixlora_workspace_bytes(const mixlora_shape_t* shape, int for_backward) {
+  if (check_shape(shape) != MIXLORA_OK) return 0;
+  WsLayout L = ws_layout(*shape);
+  return for_backward ? L.total_bwd : L.total_fwd;
+}
+
+mixlora_status_t mixlora_ffn_forward(const mixlora_shape_t* shape, const mixlora_params_t* params, void* y,
+                                     void* workspace, size_t workspace_bytes, void* stream) {
+  mixlora_status_t st = check_shape(shape);
+  if (st != MIXLORA_OK) return st;
+  st = check_params(params);
+  if (st != MIXLORA_OK) return st;
+  if (!y || !aligned16(y)) return MIXLORA_ERR_INVALID_ARG;
+  Ctx c = make_ctx(shape, params, workspace, stream);
+  if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255u) || workspace_bytes < c.L.total_fwd)
+    return MIXLORA_ERR_WORKSPACE;
+  const int T = shape->tokens, d = shape->d_model, f = shape->d_ff, N = shape->n_experts, r = shape->rank,
+            k = shape->top_k;
+  const int Nr = N * r;
+  MIXLORA_CUDA(cudaMemsetAsync(c.ws + c.L.status, 0, 256, c.st));
+  if (T == 0) return MIXLORA_OK;
+
+  // router (Eq. 7) and dispatch
+  MIXLORA_CUDA(launch_router(c));
+  MIXLORA_CUDA(launch_dispatch(c));
+
+  // shared gate / up projections and LoRA-A of every expert, one pass over x
+  {
+    TcOut outs[4];
+    outs[0] = tc_out(c.ws + c.L.G, f, f);     tc_add(outs[0], params->x, d, d, params->w_gate, d, 0);
+    outs[1] = tc_out(c.ws + c.L.U, f, f);     tc_add(outs[1], params->x, d, d, params->w_up, d, 0);
+    outs[2] = tc_out(c.ws + c.L.zga, Nr, Nr); tc_add(outs[2], params->x, d, d, params->a_gate, d, 0);
+    outs[3] = tc_out(c.ws + c.L.zua, Nr, Nr); tc_add(outs[3], params->x, d, d, params->a_up, d, 0);
+    MIXLORA_CUDA(dense_product(c, T, outs, 4));
+  }
+  // per-slot LoRA-B expansion + SwiGLU
+  MIXLORA_CUDA(launch_lora_b_swiglu(c));
+  // zd = A_d[e] h per slot (rows grouped by expert)
+  {
+    SGemm g = sgemm_base(c, c.ws + c.L.zd, r, 1, c.bf16, T * k, r);
+    g.group_mode = 1; g.groups = N;
+    add_seg(g, soperand(c.ws + c.L.h_sorted, f, 1, c.bf16), soperand(params->a_down, f, 1, c.bf16, (long long)r * f), f);
+    MIXLORA_CUDA(launch_simt_gemm(g, c.st));
+  }
+  MIXLORA_CUDA(launch_combine_h(c));
+  MIXLORA_CUDA(launch_bd_cat(c));
+  // y = [hbar | Zs] [W_d | s B_d]^T : the frozen down projection acts once on the gate-weighted sum of a
+  // token's slots (W_d is linear and shared), its LoRA rides along as extra reduction columns
+  {
+    TcOut out = tc_out(y, d, d);
+    tc_add(out, c.ws + c.L.hbar, f, f, params->w_down, f, 0);
+    tc_add(out, c.ws + c.L.Zs, Nr, Nr, c.ws + c.L.bd_cat, Nr, 0);
+    MIXLORA_CUDA(dense_product(c, T, &out, 1));
+  }
+  return MIXLORA_OK;
+}
+
+mixlora_status_t mixlora_aux_loss(const mixlora_shape_t* shape, const void* workspace, float coef, float* loss,
+                                  float* F, float* P, void* stream) {
+  mixlora_status_t st = check_shape(shape);
+  if (st != MIXLORA_OK) return st;
+  if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255u)) return MIXLORA_ERR_WORKSPACE;
+  if (!loss) return MIXLORA_ERR_INVALID_ARG;
+  Ctx c = make_ctx(shape, nullptr, const_cast<void*>(workspace), stream);
+  if (shape->tokens == 0) {
+    MIXLORA_CUDA(cudaMemsetAsync(loss, 0, sizeof(float), c.st));
+    if (F) MIXLORA_CUDA(cudaMemsetAsync(F, 0, sizeof(float) * shape->n_experts, c.st));
+    if (P) MIXLORA_CUDA(cudaMemsetAsync(P, 0, sizeof(float) * shape->n_experts, c.st));
+    return MIXLORA_OK;
+  }
+  MIXLORA_CUDA(launch_aux_loss(c, coef, loss, F, P));
+  return MIXLORA_OK;
+}
+
+mixlora_status_t mixlora_ffn_backward(const mixlora_shape_t* shape, const mixlora_params_t* params, const void* dy,
+                                      float aux_coef, void* workspace, size_t workspace_bytes,
+                                      const mixlora_grads_t* grads, void* stream) {
+  mixlora_status_t st = check_shape(shape);
+  if (st != MIXLORA_OK) return st;
+  st = check_params(params);
+  if (st != MIXLORA_OK) return st;
+  if (!dy || !aligned16(dy) || !grads) return MIXLORA_ERR_INVALID_ARG;
+  {
+    const void* outs[] = {grads->d_a_gate, grads->d_b_gate, grads->d_a_up, grads->d_b_up, grads->d_a_down,
+                          grads->d_b_down, grads->d_w_router, grads->d_x};
+    for (const void* q : outs)
+      if (q && !aligned16(q)) return MIXLORA_ERR_INVALID_ARG;
+    if (grads->accumulate != 0 && grads->accumulate != 1) return MIXLORA_ERR_INVALID_ARG;
+  }
+  Ctx c = make_ctx(shape, params, workspace, stream);
+  if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255u) || workspace_bytes < c.L.total_bwd)
+    return MIXLORA_ERR_WORKSPACE;
+  const int T = shape->tokens, d = shape->d_model, f = shape->d_ff, N = shape->n_experts, r = shape->rank,
+            k = shape->top_k;
+  const int Nr = N * r, NP = round_up8(N);
+  const int acc = grads->accumulate;
+  const int want_dx = grads->d_x != nullptr;
+  if (T == 0) {
+    if (!acc) {
+      struct { float* p; size_t n; } z[] = {
+          {grads->d_a_gate, (size_t)N * r * d}, {grads->d_b_gate, (size_t)N * f * r}, {grads->d_a_up, (size_t)N * r * d},
+          {grads->d_b_up, (size_t)N * f * r},   {grads->d_a_down, (size_t)N * r * f}, {grads->d_b_down, (size_t)N * d * r},
+          {grads->d_w_router, (size_t)N * d},   {grads->d_router_bias, (size_t)N}};
+      for (auto& q : z)
+        if (q.p) MIXLORA_CUDA(cudaMemsetAsync(q.p, 0, q.n * sizeof(float), c.st));
+    }
+    return MIXLORA_OK;
+  }
+  const int b = c.bf16;
+
+  MIXLORA_CUDA(launch_bd_cat(c));
+  // D = dy W_d (shared by a token's slots) and s B_d^T dy for every expert
+  {
+    TcOut outs[2];
+    outs[0] = tc_out(c.ws + c.L.D, f, f);      tc_add(outs[0], dy, d, d, params->w_down, f, 1);
+    outs[1] = tc_out(c.ws + c.L.spd, Nr, Nr);  tc_add(outs[1], dy, d, d, c.ws + c.L.bd_cat, Nr, 1);
+    MIXLORA_CUDA(dense_product(c, T, outs, 2));
+  }
+  MIXLORA_CUDA(launch_swiglu_bwd(c));
+  MIXLORA_CUDA(launch_slot_prep_bwd(c));
+  // dzg = s da B_g[e], dzu = s db B_u[e] (rows grouped by expert)
+  for (int which = 0; which < 2; ++which) {
+    SGemm g = sgemm_base(c, c.ws + (which ? c.L.dzu_sorted : c.L.dzg_sorted), r, 1, b, T * k, r);
+    g.group_mode = 1; g.groups = N; g.alpha = c.scale;
+    add_seg(g, soperand(c.ws + (which ? c.L.db_sorted : c.L.da_sorted), f, 1, b),
+            soperand(which ? params->b_up : params->b_gate, 1, r, b, (long long)f * r), f);
+    MIXLORA_CUDA(launch_simt_gemm(g, c.st));
+  }
+  // LoRA weight gradients: sums over the slots of each expert's segment
+  const int* pos_token = c.at<int>(c.L.pos_token);
+  auto wgrad = [&](float* out, int M, int Nn, long long c_sm, long long c_sn, long long c_sg, const SOperand& A,
+                   const SOperand& B, float alpha) -> cudaError_t {
+    if (!out) return cudaSuccess;
+    SGemm g = sgemm_base(c, out, c_sm, c_sn, 0, M, Nn);
+    g.c_sg = c_sg; g.group_mode = 2; g.groups = N; g.alpha = alpha; g.accumulate = acc;
+    add_seg(g, A, B, 0);
+    return launch_simt_gemm(g, c.st);
+  };
+  // dB_g[e][f'][rr] = s sum da[pos][f'] zg[pos][rr]
+  MIXLORA_CUDA(wgrad(grads->d_b_gate, f, r, r, 1, (long long)f * r, soperand(c.ws + c.L.da_sorted, 1, f, b),
+                     soperand(c.ws + c.L.zg_sorted, 1, r, b), c.scale));
+  MIXLORA_CUDA(wgrad(grads->d_b_up, f, r, r, 1, (long long)f * r, soperand(c.ws + c.L.db_sorted, 1, f, b),
+                     soperand(c.ws + c.L.zu_sorted, 1, r, b), c.scale));
+  // dA_g[e][rr][c] = sum dzg[pos][rr] x[token(pos)][c]
+  MIXLORA_CUDA(wgrad(grads->d_a_gate, r, d, d, 1, (long long)r * d, soperand(c.ws + c.L.dzg_sorted, 1, r, b),
+                     soperand(params->x, 1, d, b, 0, nullptr, pos_token), 1.f));
+  MIXLORA_CUDA(wgrad(grads->d_a_up, r, d, d, 1, (long long)r * d, soperand(c.ws + c.L.dzu_sorted, 1, r, b),
+                     soperand(params->x, 1, d, b, 0, nullptr, pos_token), 1.f));
+  // dA_d[e][rr][f'] = sum dzd[pos][rr] h[pos][f']
+  MIXLORA_CUDA(wgrad(grads->d_a_down, r, f, f, 1, (long long)r * f, soperand(c.ws + c.L.dzd_sorted, 1, r, b),
+                     soperand(c.ws + c.L.h_sorted, 1, f, b), 1.f));
+  // dB_d[e][c][rr] = s sum dy[token(pos)][c] (g zd)[pos][rr]
+  MIXLORA_CUDA(wgrad(grads->d_b_down, d, r, r, 1, (long long)d * r, soperand(dy, 1, d, b, 0, nullptr, pos_token),
+                     soperand(c.ws + c.L.gzd_sorted, 1, r, b), c.scale));
+
+  // router: gates -> probabilities -> logits -> W_r
+  MIXLORA_CUDA(launch_router_bwd(c, aux_coef, grads->d_router_bias, acc, want_dx));
+  if (grads->d_w_router) {
+    SGemm g = sgemm_base(c, grads->d_w_router, d, 1, 0, N, d);
+    g.accumulate = acc;
+    add_seg(g, soperand(c.ws + c.L.dlogits, 1, N, 0), soperand(params->x, 1, d, b), T);
+    MIXLORA_CUDA(launch_simt_gemm(g, c.st));
+  }
+  if (want_dx) {
+    MIXLORA_CUDA(launch_combine_bwd(c));
+    // dx = [dabar | dbbar | dZg | dZu | dl] [W_g ; W_u ; A_g ; A_u ; W_r]
+    TcOut out = tc_out(grads->d_x, d, d);
+    tc_add(out, c.ws + c.L.dabar, f, f, params->w_gate, d, 1);
+    tc_add(out, c.ws + c.L.dbbar, f, f, params->w_up, d, 1);
+    tc_add(out, c.ws + c.L.dZg, Nr, Nr, params->a_gate, d, 1);
+    tc_add(out, c.ws + c.L.dZu, Nr, Nr, params->a_up, d, 1);
+    tc_add(out, c.ws + c.L.dl_act, NP, NP, c.ws + c.L.wr_act, d, 1);
+    MIXLORA_CUDA(dense_product(c, T, &out, 1));
+  }
+  return MIXLORA_OK;
+}
+
+mixlora_status_t mixlora_routing_view(const mixlora_shape_t* shape, const void* workspace, const int32_t** expert_idx,
+                                      const float** gates, const int32_t** perm, const int32_t** seg_off,
+                                      const uint8_t** low_margin, const float** probs) {
+  mixlora_status_t st = check_shape(shape);
+  if (st != MIXLORA_OK) return st;
+  if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255u)) return MIXLORA_ERR_WORKSPACE;
+  WsLayout L = ws_layout(*shape);
+  const char* ws = reinterpret_cast<const char*>(workspace);
+  if (expert_idx) *expert_idx = reinterpret_cast<const int32_t*>(ws + L.expert_idx);
+  if (gates) *gates = reinterpret_cast<const float*>(ws + L.gates);
+  if (perm) *perm = reinterpret_cast<const int32_t*>(ws + L.perm);
+  if (seg_off) *seg_off = reinterpret_cast<const int32_t*>(ws + L.seg_off);
+  if (low_margin) *low_margin = reinterpret_cast<const uint8_t*>(ws + L.low_margin);
+  if (probs) *probs = reinterpret_cast<const float*>(ws + L.probs);
+  return MIXLORA_OK;
+}
+
+mixlora_status_t mixlora_device_status(const void* workspace, int32_t* code, void* stream) {
+  if (!workspace || !code) return MIXLORA_ERR_INVALID_ARG;
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+  int32_t v = 0;
+  MIXLORA_CUDA(cudaMemcpyAsync(&v, workspace, sizeof(v), cudaMemcpyDeviceToHost, st));
+  MIXLORA_CUDA(cudaStreamSynchronize(st));
+  *code = v;
+  return MIXLORA_OK;
+}
+
+mixlora_status_t mixlora_gemm_bf16(const void* A, const void* B, void* C, int32_t M, int32_t N, int32_t K,
+                                   int32_t b_is_kn, int32_t* status_word, void* stream) {
+  if (!A || !B || !C || !aligned16(A) || !aligned16(B) || !aligned16(C)) return MIXLORA_ERR_INVALID_ARG;
+  if (M < 0 || N <= 0 || K <= 0 || (b_is_kn != 0 && b_is_kn != 1)) return MIXLORA_ERR_INVALID_ARG;
+  if (N % 8 || K % 8) return MIXLORA_ERR_UNSUPPORTED;
+  if (M == 0) return MIXLORA_OK;
+  TcOut out = tc_out(C, N, N);
+  tc_add(out, A, K, K, B, b_is_kn ? N : K, b_is_kn);
+  if (!tc_gemm_supported(M, &out, 1)) return MIXLORA_ERR_UNSUPPORTED;
+  MIXLORA_CUDA(launch_tc_gemm(M, &out, 1, status_word, reinterpret_cast<cudaStream_t>(stream)));
+  return MIXLORA_OK;
+}
+
+}  // extern "C"
