@@ -127,12 +127,12 @@ router_kernel(const T* __restrict__ x, const float* __restrict__ w_router, const
     if (k < N) margin = fminf(margin, last - next);
     if (N > 1) margin = fminf(margin, first - ((k >= 2) ? second : next));
     low_margin[t] = (margin < kMarginFlag) ? 1 : 0;
-    const float gscale = renorm ? 1.f / qsum : 1.f;
+    
 #pragma unroll
     for (int j = 0; j < MIXLORA_MAX_TOP_K; ++j) {
       if (j < k) {
         expert_idx[(size_t)t * k + j] = sel[j];
-        gates[(size_t)t * k + j] = selp[j] * gscale;
+        gates[(size_t)t * k + j] = renorm ? selp[j] / qsum : selp[j];  // k = 1 gives exactly 1
       }
     }
   }
