@@ -1,0 +1,369 @@
+#!/usr/bin/env python
+"""Benchmark of the MixLoRA FFN block (forward + aux loss + backward) on B200.
+
+    python bench.py --gpus N --steps K --warmup W          # the CUDA library
+    python bench.py --impl reference ...                   # the CPU oracle, bounded sample per step
+
+One "step" is one pass of the whole hot path over one synthetic batch of the LLaMA-2-7B
+shaped workload (8192 tokens per GPU, 8 experts, top-2, rank 16): forward, auxiliary loss,
+backward with LoRA, router and input gradients.  Rank 0 prints one JSON line.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np
+
+from paper_2404_15159_b200 import synth
+
+METRIC = "mixlora_ffn_fwd_bwd_tokens_per_s"
+UNIT = "tokens/s"
+AUX_COEF = 0.01
+
+
+def workload_by_name(name: str) -> synth.Workload:
+    table = {"c1": synth.c1, "c2": synth.c2, "c3": synth.c3, "c4": synth.c4}
+    if name in table:
+        return table[name]()
+    if name.startswith("c5:"):                      # c5:N,k,r,T
+        n, k, r, t = (int(v) for v in name[3:].split(","))
+        return synth.c5(n, k, r, t)
+    raise SystemExit(f"unknown workload {name}")
+
+
+# ----------------------------------------------------------------------------------------
+# flop / byte model of the stages (algorithmic, per step)
+# ----------------------------------------------------------------------------------------
+def stage_flops(w: synth.Workload, want_dx: bool) -> dict:
+    T, d, f, N, k, r = w.tokens, w.d_model, w.d_ff, w.n_experts, w.top_k, w.rank
+    U = 2.0 * T * d * f
+    Nr = N * r
+    NP = (N + 7) // 8 * 8
+    fl = {
+        "gemm_gate_up": 2 * U + 2 * 2.0 * T * d * Nr,          # W1, W3 once per token + LoRA-A of every expert
+        "gemm_down": U + 2.0 * T * Nr * d,                     # W2 on the gate-weighted sum + LoRA-B down
+        "gemm_dgrad_down": U + 2.0 * T * d * Nr,               # dy W2 + B_d^T dy
+        "gemm_dx": (2 * U + 2 * 2.0 * T * Nr * d + 2.0 * T * NP * d) if want_dx else 0.0,
+    }
+    return fl
+
+
+def load_peaks() -> dict:
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as fh:
+            p = json.load(fh)
+        return dict(hbm_gbs=p["hbm_gbs"], bf16_tflops=p["bf16_tflops"],
+                    bf16_tflops_sustained=p.get("bf16_tflops_sustained", p["bf16_tflops"]), source="measured")
+    return dict(hbm_gbs=6650.0, bf16_tflops=1590.0, bf16_tflops_sustained=1400.0, source="fallback")
+
+
+# ----------------------------------------------------------------------------------------
+# clocks sampler
+# ----------------------------------------------------------------------------------------
+class ClockSampler:
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index = index
+        self.samples = []
+        self.proc = None
+        self.thread = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
+                                          "-i", str(self.index), "-lms", "100"], stdout=subprocess.PIPE,
+                                         stderr=subprocess.DEVNULL, text=True)
+        except OSError:
+            self.proc = None
+            return
+        self.thread = threading.Thread(target=self._read, daemon=True)
+        self.thread.start()
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.samples.append((time.time(), line.strip()))
+
+    def stop(self, t0: float, t1: float) -> dict:
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=2)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        sm, mx, pw, reasons = [], [], [], set()
+        rows = [s for s in self.samples if t0 <= s[0] <= t1 + 0.1] or self.samples
+        for _, line in rows:
+            parts = [p.strip() for p in line.split(",")]
+            if len(parts) < 7:
+                continue
+            try:
+                sm.append(float(parts[0])); mx.append(float(parts[1])); pw.append(float(parts[2]))
+            except ValueError:
+                continue
+            for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), parts[3:7]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "power_w_max": max(pw) if pw else None, "samples": len(sm), "reasons": sorted(reasons)}
+
+
+# ----------------------------------------------------------------------------------------
+# CPU oracle leg
+# ----------------------------------------------------------------------------------------
+def oracle_sample(w: synth.Workload, tensors: dict, sample_tokens: int, want_dx: bool):
+    """One oracle forward + aux + backward on the first `sample_tokens` tokens.  Returns seconds."""
+    from oracle import mixlora_oracle as orc
+    xs, dys = tensors["x"][:sample_tokens], tensors["dy"][:sample_tokens]
+    params = synth.params_of(tensors)
+    t0 = time.perf_counter()
+    y, saved = orc.ffn_forward(xs, params, w.top_k, w.lora_alpha)
+    orc.aux_loss(saved["route"]["probs"], saved["route"]["expert_idx"], AUX_COEF)
+    orc.ffn_backward(xs, params, dys, saved, aux_coef=AUX_COEF, want_dx=want_dx)
+    return time.perf_counter() - t0
+
+
+def threads_used() -> int:
+    try:
+        from threadpoolctl import threadpool_info
+        n = [p.get("num_threads", 1) for p in threadpool_info() if p.get("user_api") == "blas"]
+        return max(n) if n else (os.cpu_count() or 1)
+    except Exception:
+        return os.cpu_count() or 1
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    w = workload_by_name(args.workload)
+    sample = args.ref_sample
+    tensors = synth.generate(w.with_(tokens=sample))
+    times = []
+    for i in range(args.warmup + args.steps):
+        dt = oracle_sample(w, tensors, sample, True)
+        if i >= args.warmup:
+            times.append(dt)
+    per_step = float(np.mean(times))
+    value = sample / per_step
+    cores = threads_used()
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": per_step * 1e3, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": w.name, "tokens_per_gpu": w.tokens, "d_model": w.d_model, "d_ff": w.d_ff,
+                   "n_experts": w.n_experts, "top_k": w.top_k, "rank": w.rank},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle",
+                         "sample": f"first {sample} tokens of the workload per step, full d_model/d_ff, forward + aux + "
+                                   f"backward with dx, float64 numpy"},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+
+
+# ----------------------------------------------------------------------------------------
+# CUDA leg
+# ----------------------------------------------------------------------------------------
+def run_cuda(args):
+    import torch
+    import torch.distributed as dist
+    from paper_2404_15159_b200 import binding as B
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (the library has no CPU path)")
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+
+    w = workload_by_name(args.workload)
+    want_dx = not args.no_dx
+    bf16 = w.dtype == "bf16"
+    act = torch.bfloat16 if bf16 else torch.float32
+    # every rank holds the same weights and its own batch of tokens (data parallel, weak scaling)
+    tensors = synth.generate(w.with_(seed=w.seed))
+    if rank > 0:
+        rng = np.random.Generator(np.random.Philox(key=w.seed + 1000 + rank))
+        tensors["x"] = synth.round_to_bf16(rng.standard_normal(tensors["x"].shape, dtype=np.float32))
+        tensors["dy"] = synth.round_to_bf16(rng.standard_normal(tensors["dy"].shape, dtype=np.float32))
+    dev = {}
+    for n, v in tensors.items():
+        if v is None:
+            dev[n] = None
+        elif n in ("w_router", "router_bias"):
+            dev[n] = torch.from_numpy(v).cuda()
+        else:
+            dev[n] = torch.from_numpy(v).cuda().to(act)
+    shape = B.make_shape(w.tokens, w.d_model, w.d_ff, w.n_experts, w.top_k, w.rank, w.lora_alpha,
+                         B.MIXLORA_DTYPE_BF16 if bf16 else B.MIXLORA_DTYPE_FP32)
+    params = B.make_params(**{n: dev[n] for n in synth.PARAM_NAMES}, x=dev["x"])
+    ws = B.alloc_workspace(shape, True)
+    y = torch.empty(w.tokens, w.d_model, dtype=act, device="cuda")
+    loss = torch.zeros(1, dtype=torch.float32, device="cuda")
+    gnames = ("d_a_gate", "d_b_gate", "d_a_up", "d_b_up", "d_a_down", "d_b_down", "d_w_router", "d_router_bias")
+    sizes = [int(np.prod(tensors[n[2:]].shape)) if n != "d_router_bias" else w.n_experts for n in gnames]
+    pad = [(s + 63) // 64 * 64 for s in sizes]
+    flat = torch.zeros(sum(pad), dtype=torch.float32, device="cuda")     # one buffer => one all-reduce
+    g, off = {}, 0
+    for n, s, p in zip(gnames, sizes, pad):
+        g[n] = flat[off:off + s]
+        off += p
+    if want_dx:
+        g["d_x"] = torch.empty(w.tokens, w.d_model, dtype=act, device="cuda")
+    grads = B.make_grads(accumulate=0, **g)
+
+    def step():
+        B.mixlora_ffn_forward(shape, params, y, ws)
+        B.mixlora_aux_loss(shape, ws, AUX_COEF, loss)
+        B.mixlora_ffn_backward(shape, params, dev["dy"], AUX_COEF, ws, grads)
+        if world > 1:
+            dist.all_reduce(flat)          # data-parallel sum of the LoRA and router gradients
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def timed(fn, steps, warmup):
+        for _ in range(warmup):
+            fn()
+        barrier()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        t0 = time.time()
+        e0.record()
+        for _ in range(steps):
+            fn()
+        e1.record()
+        barrier()
+        t1 = time.time()
+        ms = torch.tensor([e0.elapsed_time(e1)], dtype=torch.float64, device="cuda")
+        if world > 1:
+            dist.all_reduce(ms, op=dist.ReduceOp.MAX)
+        return float(ms.item()), t0, t1
+
+    B.mixlora_stage_timing(False)
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+    total_ms, t0, t1 = timed(step, args.steps, args.warmup)
+    clocks = sampler.stop(t0, t1) if rank == 0 else None
+    launches = sum(v[1] for v in B.mixlora_stage_timing_read().values())
+    launches_per_step = launches // (args.steps + args.warmup)
+    status = B.mixlora_device_status(ws)
+    ms_per_step = total_ms / args.steps
+    value = world * w.tokens / (ms_per_step * 1e-3)
+
+    # per-stage device time over the same number of steps (events on the launching stream)
+    B.mixlora_stage_timing(True)
+    for _ in range(args.steps):
+        step()
+    torch.cuda.synchronize()
+    stages = B.mixlora_stage_timing_read()
+    B.mixlora_stage_timing(False)
+    stage_ms = {n: v[0] / args.steps for n, v in stages.items()}
+
+    # end to end through the same calls with host buffers: x and dy come from pinned host memory every
+    # step, y and the loss go back
+    hx = torch.from_numpy(tensors["x"]).to(act).pin_memory()
+    hdy = torch.from_numpy(tensors["dy"]).to(act).pin_memory()
+    hy = torch.empty(w.tokens, w.d_model, dtype=act).pin_memory()
+    hloss = torch.empty(1, dtype=torch.float32).pin_memory()
+
+    def step_e2e():
+        dev["x"].copy_(hx, non_blocking=True)
+        dev["dy"].copy_(hdy, non_blocking=True)
+        step()
+        hy.copy_(y, non_blocking=True)
+        hloss.copy_(loss, non_blocking=True)
+        torch.cuda.current_stream().synchronize()
+
+    e2e_ms, _, _ = timed(step_e2e, args.steps, max(1, args.warmup // 2))
+    e2e_value = world * w.tokens / (e2e_ms / args.steps * 1e-3)
+    h2d = hx.numel() * hx.element_size() + hdy.numel() * hdy.element_size()
+    d2h = hy.numel() * hy.element_size() + 4
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    peaks = load_peaks()
+    fl = stage_flops(w, want_dx)
+    gemm_names = [n for n in fl if fl[n] > 0]
+    dom = max(gemm_names, key=lambda n: stage_ms.get(n, 0.0))
+    gemm_ms = sum(stage_ms.get(n, 0.0) for n in gemm_names)
+    gemm_fl = sum(fl[n] for n in gemm_names)
+    peak_tf = peaks["bf16_tflops_sustained"]       # the kernel is timed inside a long step
+    dom_tf = fl[dom] / (stage_ms[dom] * 1e-3) / 1e12 if stage_ms.get(dom) else 0.0
+    roofline = {"bound": "tensor", "kernel": dom, "achieved": dom_tf, "peak": peak_tf, "unit": "TFLOP/s",
+                "frac": dom_tf / peak_tf, "peak_source": peaks["source"] + " (sustained bf16)",
+                "flops_per_launch": fl[dom], "ms_per_launch": stage_ms.get(dom), "traffic": None,
+                "gemm_phases": {"tflops": gemm_fl / (gemm_ms * 1e-3) / 1e12 if gemm_ms else 0.0,
+                                "frac": (gemm_fl / (gemm_ms * 1e-3) / 1e12 / peak_tf) if gemm_ms else 0.0,
+                                "ms": gemm_ms, "share_of_step": gemm_ms / sum(stage_ms.values())}}
+
+    cpu_baseline = None
+    if world == 1 and not args.no_cpu_baseline:
+        sample = args.cpu_sample
+        sec = oracle_sample(w, tensors, sample, want_dx)
+        cpu_baseline = {"value": sample / sec, "unit": UNIT, "cores": threads_used(), "kind": "oracle",
+                        "sample": f"one oracle pass (forward + aux + backward) over the first {sample} tokens of the "
+                                  f"workload at full d_model/d_ff, {sec:.1f} s"}
+
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "bf16" if bf16 else "f32", "data": "synthetic",
+        "config": {"workload": w.name, "tokens_per_gpu": w.tokens, "d_model": w.d_model, "d_ff": w.d_ff,
+                   "n_experts": w.n_experts, "top_k": w.top_k, "rank": w.rank, "lora_alpha": w.lora_alpha,
+                   "backward_dx": want_dx, "aux_coef": AUX_COEF,
+                   "parallelism": f"dp{world} over tokens" + (", NCCL all-reduce of LoRA/router grads" if world > 1 else ""),
+                   "l2": "inputs larger than L2 (weights 270 MB + activations > 126 MB), no flush"},
+        "roofline": roofline, "cpu_baseline": cpu_baseline,
+        "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
+        "gpu_launches": launches_per_step * args.steps, "gpu_launches_per_step": launches_per_step,
+        "stage_ms": {n: round(v, 4) for n, v in stage_ms.items()}, "device_status": status, "clocks": clocks,
+    }
+    print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
+    ap.add_argument("--workload", default="c3")
+    ap.add_argument("--no-dx", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--cpu-sample", type=int, default=512, help="tokens of the oracle's timed sample")
+    ap.add_argument("--ref-sample", type=int, default=256, help="tokens per step of --impl reference")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_cuda(args)
+
+
+if __name__ == "__main__":
+    main()

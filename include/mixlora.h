@@ -149,6 +149,18 @@ mixlora_status_t mixlora_device_status(const void *workspace, int32_t *code /* h
 mixlora_status_t mixlora_gemm_bf16(const void *A, const void *B, void *C, int32_t M, int32_t N, int32_t K,
                                    int32_t b_is_kn, int32_t *status_word, void *stream);
 
+/* Opt-in bookkeeping for measurements (host side, process-wide, not thread-safe).
+ * mixlora_stage_timing(1) clears the counters and makes every later forward / backward /
+ * aux_loss call bracket each stage of the path (router, dispatch, the dense products, the
+ * LoRA stages, ...) with CUDA events on the caller's stream; mixlora_stage_timing(0) clears
+ * and switches the events off (kernel launches are still counted).
+ * mixlora_stage_timing_read waits for the recorded events and fills, for up to max_stages
+ * stages, the stage name (static string), the device milliseconds accumulated since the last
+ * mixlora_stage_timing call and the number of kernels launched.  Returns the number of stages. */
+mixlora_status_t mixlora_stage_timing(int32_t enable);
+int32_t mixlora_stage_timing_read(int32_t max_stages, const char **names /* host */, float *ms /* host */,
+                                  int64_t *launches /* host */);
+
 const char *mixlora_status_string(mixlora_status_t status);
 
 #ifdef __cplusplus

@@ -21,7 +21,7 @@ STATUS_NAMES = {0: "MIXLORA_OK", 1: "MIXLORA_ERR_INVALID_ARG", 2: "MIXLORA_ERR_U
 
 EXPORTS = ("mixlora_limits", "mixlora_workspace_bytes", "mixlora_ffn_forward", "mixlora_aux_loss",
            "mixlora_ffn_backward", "mixlora_routing_view", "mixlora_device_status", "mixlora_gemm_bf16",
-           "mixlora_status_string")
+           "mixlora_status_string", "mixlora_stage_timing", "mixlora_stage_timing_read")
 
 
 class mixlora_shape_t(C.Structure):
@@ -75,6 +75,11 @@ def _load() -> C.CDLL:
     lib.mixlora_gemm_bf16.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.c_int32,
                                       C.c_int32, C.c_void_p, C.c_void_p]
     lib.mixlora_gemm_bf16.restype = C.c_int
+    lib.mixlora_stage_timing.argtypes = [C.c_int32]
+    lib.mixlora_stage_timing.restype = C.c_int
+    lib.mixlora_stage_timing_read.argtypes = [C.c_int32, C.POINTER(C.c_char_p), C.POINTER(C.c_float),
+                                              C.POINTER(C.c_int64)]
+    lib.mixlora_stage_timing_read.restype = C.c_int32
     lib.mixlora_status_string.argtypes = [C.c_int]
     lib.mixlora_status_string.restype = C.c_char_p
     return lib
@@ -190,3 +195,17 @@ def mixlora_device_status(workspace, stream=None) -> int:
 def mixlora_gemm_bf16(A, B, Cout, M, N, K, b_is_kn=False, status_word=None, stream=None) -> None:
     _check(lib.mixlora_gemm_bf16(_ptr(A), _ptr(B), _ptr(Cout), M, N, K, 1 if b_is_kn else 0, _ptr(status_word),
                                  _stream(stream)), "mixlora_gemm_bf16")
+
+
+def mixlora_stage_timing(enable: bool) -> None:
+    _check(lib.mixlora_stage_timing(1 if enable else 0), "mixlora_stage_timing")
+
+
+def mixlora_stage_timing_read() -> dict:
+    """{stage: (milliseconds, kernel launches)} accumulated since the last mixlora_stage_timing call."""
+    n = 32
+    names = (C.c_char_p * n)()
+    ms = (C.c_float * n)()
+    launches = (C.c_int64 * n)()
+    cnt = lib.mixlora_stage_timing_read(n, names, ms, launches)
+    return {names[i].decode(): (float(ms[i]), int(launches[i])) for i in range(min(cnt, n))}

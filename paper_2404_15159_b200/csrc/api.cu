@@ -3,6 +3,8 @@
 #include <stdio.h>
 #include <string.h>
 
+#include <vector>
+
 #include "common.cuh"
 
 namespace mixlora {
@@ -70,6 +72,40 @@ WsLayout ws_layout(const mixlora_shape_t& s) {
 }
 
 namespace {
+
+// ---- opt-in per-stage device timing and launch counting (host-side bookkeeping only) ----
+enum Stage {
+  ST_ROUTER, ST_DISPATCH, ST_GEMM_GATE_UP, ST_LORA_B_SWIGLU, ST_LORA_A_DOWN, ST_COMBINE_H, ST_GEMM_DOWN,
+  ST_GEMM_DGRAD_DOWN, ST_SWIGLU_BWD, ST_LORA_DZ, ST_LORA_WGRAD, ST_ROUTER_BWD, ST_COMBINE_BWD, ST_GEMM_DX, ST_COUNT
+};
+const char* const kStageNames[ST_COUNT] = {
+    "router", "dispatch", "gemm_gate_up", "lora_b_swiglu", "lora_a_down", "combine_h", "gemm_down",
+    "gemm_dgrad_down", "swiglu_bwd", "lora_dz", "lora_wgrad", "router_bwd", "combine_bwd", "gemm_dx"};
+
+struct StageRec { int stage; cudaEvent_t a, b; };
+struct Profiler {
+  bool on = false;
+  std::vector<StageRec> recs;
+  long long launches[ST_COUNT] = {0};
+};
+Profiler g_prof;
+
+struct StageScope {
+  int stage; cudaStream_t st; cudaEvent_t a = nullptr, b = nullptr; bool on;
+  StageScope(int stage_, cudaStream_t st_, int launches) : stage(stage_), st(st_), on(g_prof.on) {
+    g_prof.launches[stage] += launches;
+    if (on) {
+      if (cudaEventCreate(&a) != cudaSuccess || cudaEventCreate(&b) != cudaSuccess) { on = false; return; }
+      cudaEventRecord(a, st);
+    }
+  }
+  ~StageScope() {
+    if (on) {
+      cudaEventRecord(b, st);
+      g_prof.recs.push_back({stage, a, b});
+    }
+  }
+};
 
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
@@ -150,6 +186,10 @@ cudaError_t dense_product(const Ctx& c, int M, const TcOut* outs, int nout) {
   return cudaSuccess;
 }
 
+int dense_launches(const Ctx& c, int M, const TcOut* outs, int nout) {
+  return (c.bf16 && tc_gemm_supported(M, outs, nout)) ? 1 : nout;
+}
+
 TcOut tc_out(void* C, long long ldc, int N) {
   TcOut o;
   memset(&o, 0, sizeof(o));
@@ -210,8 +250,8 @@ mixlora_status_t mixlora_ffn_forward(const mixlora_shape_t* shape, const mixlora
   if (T == 0) return MIXLORA_OK;
 
   // router (Eq. 7) and dispatch
-  MIXLORA_CUDA(launch_router(c));
-  MIXLORA_CUDA(launch_dispatch(c));
+  { StageScope ss(ST_ROUTER, c.st, 2); MIXLORA_CUDA(launch_router(c)); }
+  { StageScope ss(ST_DISPATCH, c.st, 3); MIXLORA_CUDA(launch_dispatch(c)); }
 
   // shared gate / up projections and LoRA-A of every expert, one pass over x
   {
@@ -220,25 +260,27 @@ mixlora_status_t mixlora_ffn_forward(const mixlora_shape_t* shape, const mixlora
     outs[1] = tc_out(c.ws + c.L.U, f, f);     tc_add(outs[1], params->x, d, d, params->w_up, d, 0);
     outs[2] = tc_out(c.ws + c.L.zga, Nr, Nr); tc_add(outs[2], params->x, d, d, params->a_gate, d, 0);
     outs[3] = tc_out(c.ws + c.L.zua, Nr, Nr); tc_add(outs[3], params->x, d, d, params->a_up, d, 0);
+    StageScope ss(ST_GEMM_GATE_UP, c.st, dense_launches(c, T, outs, 4));
     MIXLORA_CUDA(dense_product(c, T, outs, 4));
   }
   // per-slot LoRA-B expansion + SwiGLU
-  MIXLORA_CUDA(launch_lora_b_swiglu(c));
+  { StageScope ss(ST_LORA_B_SWIGLU, c.st, 1); MIXLORA_CUDA(launch_lora_b_swiglu(c)); }
   // zd = A_d[e] h per slot (rows grouped by expert)
   {
+    StageScope ss(ST_LORA_A_DOWN, c.st, 1);
     SGemm g = sgemm_base(c, c.ws + c.L.zd, r, 1, c.bf16, T * k, r);
     g.group_mode = 1; g.groups = N;
     add_seg(g, soperand(c.ws + c.L.h_sorted, f, 1, c.bf16), soperand(params->a_down, f, 1, c.bf16, (long long)r * f), f);
     MIXLORA_CUDA(launch_simt_gemm(g, c.st));
   }
-  MIXLORA_CUDA(launch_combine_h(c));
-  MIXLORA_CUDA(launch_bd_cat(c));
+  { StageScope ss(ST_COMBINE_H, c.st, 2); MIXLORA_CUDA(launch_combine_h(c)); MIXLORA_CUDA(launch_bd_cat(c)); }
   // y = [hbar | Zs] [W_d | s B_d]^T : the frozen down projection acts once on the gate-weighted sum of a
   // token's slots (W_d is linear and shared), its LoRA rides along as extra reduction columns
   {
     TcOut out = tc_out(y, d, d);
     tc_add(out, c.ws + c.L.hbar, f, f, params->w_down, f, 0);
     tc_add(out, c.ws + c.L.Zs, Nr, Nr, c.ws + c.L.bd_cat, Nr, 0);
+    StageScope ss(ST_GEMM_DOWN, c.st, dense_launches(c, T, &out, 1));
     MIXLORA_CUDA(dense_product(c, T, &out, 1));
   }
   return MIXLORA_OK;
@@ -257,7 +299,7 @@ mixlora_status_t mixlora_aux_loss(const mixlora_shape_t* shape, const void* work
     if (P) MIXLORA_CUDA(cudaMemsetAsync(P, 0, sizeof(float) * shape->n_experts, c.st));
     return MIXLORA_OK;
   }
-  MIXLORA_CUDA(launch_aux_loss(c, coef, loss, F, P));
+  { StageScope ss(ST_ROUTER, c.st, 1); MIXLORA_CUDA(launch_aux_loss(c, coef, loss, F, P)); }
   return MIXLORA_OK;
 }
 
@@ -297,18 +339,19 @@ mixlora_status_t mixlora_ffn_backward(const mixlora_shape_t* shape, const mixlor
   }
   const int b = c.bf16;
 
-  MIXLORA_CUDA(launch_bd_cat(c));
   // D = dy W_d (shared by a token's slots) and s B_d^T dy for every expert
   {
     TcOut outs[2];
     outs[0] = tc_out(c.ws + c.L.D, f, f);      tc_add(outs[0], dy, d, d, params->w_down, f, 1);
     outs[1] = tc_out(c.ws + c.L.spd, Nr, Nr);  tc_add(outs[1], dy, d, d, c.ws + c.L.bd_cat, Nr, 1);
+    StageScope ss(ST_GEMM_DGRAD_DOWN, c.st, 1 + dense_launches(c, T, outs, 2));
+    MIXLORA_CUDA(launch_bd_cat(c));
     MIXLORA_CUDA(dense_product(c, T, outs, 2));
   }
-  MIXLORA_CUDA(launch_swiglu_bwd(c));
-  MIXLORA_CUDA(launch_slot_prep_bwd(c));
+  { StageScope ss(ST_SWIGLU_BWD, c.st, 2); MIXLORA_CUDA(launch_swiglu_bwd(c)); MIXLORA_CUDA(launch_slot_prep_bwd(c)); }
   // dzg = s da B_g[e], dzu = s db B_u[e] (rows grouped by expert)
   for (int which = 0; which < 2; ++which) {
+    StageScope ss(ST_LORA_DZ, c.st, 1);
     SGemm g = sgemm_base(c, c.ws + (which ? c.L.dzu_sorted : c.L.dzg_sorted), r, 1, b, T * k, r);
     g.group_mode = 1; g.groups = N; g.alpha = c.scale;
     add_seg(g, soperand(c.ws + (which ? c.L.db_sorted : c.L.da_sorted), f, 1, b),
@@ -320,6 +363,7 @@ mixlora_status_t mixlora_ffn_backward(const mixlora_shape_t* shape, const mixlor
   auto wgrad = [&](float* out, int M, int Nn, long long c_sm, long long c_sn, long long c_sg, const SOperand& A,
                    const SOperand& B, float alpha) -> cudaError_t {
     if (!out) return cudaSuccess;
+    StageScope ss(ST_LORA_WGRAD, c.st, 1);
     SGemm g = sgemm_base(c, out, c_sm, c_sn, 0, M, Nn);
     g.c_sg = c_sg; g.group_mode = 2; g.groups = N; g.alpha = alpha; g.accumulate = acc;
     add_seg(g, A, B, 0);
@@ -343,15 +387,19 @@ mixlora_status_t mixlora_ffn_backward(const mixlora_shape_t* shape, const mixlor
                      soperand(c.ws + c.L.gzd_sorted, 1, r, b), c.scale));
 
   // router: gates -> probabilities -> logits -> W_r
-  MIXLORA_CUDA(launch_router_bwd(c, aux_coef, grads->d_router_bias, acc, want_dx));
+  {
+    StageScope ss(ST_ROUTER_BWD, c.st, 1 + (grads->d_router_bias ? 1 : 0) + (want_dx ? 1 : 0));
+    MIXLORA_CUDA(launch_router_bwd(c, aux_coef, grads->d_router_bias, acc, want_dx));
+  }
   if (grads->d_w_router) {
+    StageScope ss(ST_ROUTER_BWD, c.st, 1);
     SGemm g = sgemm_base(c, grads->d_w_router, d, 1, 0, N, d);
     g.accumulate = acc;
     add_seg(g, soperand(c.ws + c.L.dlogits, 1, N, 0), soperand(params->x, 1, d, b), T);
     MIXLORA_CUDA(launch_simt_gemm(g, c.st));
   }
   if (want_dx) {
-    MIXLORA_CUDA(launch_combine_bwd(c));
+    { StageScope ss(ST_COMBINE_BWD, c.st, 1); MIXLORA_CUDA(launch_combine_bwd(c)); }
     // dx = [dabar | dbbar | dZg | dZu | dl] [W_g ; W_u ; A_g ; A_u ; W_r]
     TcOut out = tc_out(grads->d_x, d, d);
     tc_add(out, c.ws + c.L.dabar, f, f, params->w_gate, d, 1);
@@ -359,6 +407,7 @@ mixlora_status_t mixlora_ffn_backward(const mixlora_shape_t* shape, const mixlor
     tc_add(out, c.ws + c.L.dZg, Nr, Nr, params->a_gate, d, 1);
     tc_add(out, c.ws + c.L.dZu, Nr, Nr, params->a_up, d, 1);
     tc_add(out, c.ws + c.L.dl_act, NP, NP, c.ws + c.L.wr_act, d, 1);
+    StageScope ss(ST_GEMM_DX, c.st, dense_launches(c, T, &out, 1));
     MIXLORA_CUDA(dense_product(c, T, &out, 1));
   }
   return MIXLORA_OK;
@@ -389,6 +438,29 @@ mixlora_status_t mixlora_device_status(const void* workspace, int32_t* code, voi
   MIXLORA_CUDA(cudaStreamSynchronize(st));
   *code = v;
   return MIXLORA_OK;
+}
+
+mixlora_status_t mixlora_stage_timing(int32_t enable) {
+  for (auto& r : g_prof.recs) { cudaEventDestroy(r.a); cudaEventDestroy(r.b); }
+  g_prof.recs.clear();
+  for (int i = 0; i < ST_COUNT; ++i) g_prof.launches[i] = 0;
+  g_prof.on = enable != 0;
+  return MIXLORA_OK;
+}
+
+int32_t mixlora_stage_timing_read(int32_t max_stages, const char** names, float* ms, int64_t* launches) {
+  float acc[ST_COUNT] = {0};
+  for (auto& r : g_prof.recs) {
+    float t = 0.f;
+    if (cudaEventSynchronize(r.b) == cudaSuccess && cudaEventElapsedTime(&t, r.a, r.b) == cudaSuccess) acc[r.stage] += t;
+  }
+  int n = max_stages < ST_COUNT ? max_stages : ST_COUNT;
+  for (int i = 0; i < n; ++i) {
+    if (names) names[i] = kStageNames[i];
+    if (ms) ms[i] = acc[i];
+    if (launches) launches[i] = g_prof.launches[i];
+  }
+  return ST_COUNT;
 }
 
 mixlora_status_t mixlora_gemm_bf16(const void* A, const void* B, void* C, int32_t M, int32_t N, int32_t K,
