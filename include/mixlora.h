@@ -11,7 +11,8 @@
  *   - Every tensor pointer is a DEVICE pointer unless marked "host".  All tensors are
  *     dense, row-major, 16-byte aligned and owned by the caller, including the workspace.
  *     The library allocates no device memory in these calls and keeps no state between
- *     calls other than what it writes into the caller's workspace.
+ *     calls other than what it writes into the caller's workspace (the opt-in measurement
+ *     bookkeeping of mixlora_stage_timing excepted).
  *   - Weights are stored [out, in] as in Eq. 1 (W in R^{d1 x d2}).
  *   - T tokens, d = d_model, f = d_ff, N experts, k = top_k, r = rank, s = lora_alpha / r.
  *     A slot is one (token, selected expert) pair; slot id = t * k + j, j = 0 for the
