@@ -150,6 +150,29 @@ mixlora_status_t mixlora_device_status(const void *workspace, int32_t *code /* h
 mixlora_status_t mixlora_gemm_bf16(const void *A, const void *B, void *C, int32_t M, int32_t N, int32_t K,
                                    int32_t b_is_kn, int32_t *status_word, void *stream);
 
+/* Slot dispatch without a workspace (the paper has no counterpart; it computes what the
+ * dispatch step of mixlora_ffn_forward computes).  For callers that cannot allocate device
+ * memory and so have no workspace to pass: a plug-in inside a host program that owns the
+ * allocator, code that must not trigger the device-wide synchronisation of cudaMalloc, a
+ * process with a memory budget fixed at start-up.  The per-block count tables that the
+ * dispatch kernels need between their three launches sit in a 64 KiB array that is part of
+ * the library image on every GPU that loads it (held until the process exits).
+ *   expert_idx [tokens, top_k] int32 device, values in [0, n_experts), distinct per token.
+ *   perm  [tokens * top_k] int32 device out: slot id (t * top_k + j) at each position of the
+ *         order "expert ascending, token ascending".
+ *   seg_off [n_experts + 1] int32 device out: first position of each expert.
+ * Limits: tokens <= mixlora_dispatch_static_max_tokens() (65536), n_experts <= 32,
+ * top_k <= 8; larger sizes return MIXLORA_ERR_UNSUPPORTED and enqueue nothing.
+ * The call allocates nothing, on the device or through any library.  The first call on each
+ * device looks up the device address of the array (with that device current); make that
+ * first call outside any stream capture.  All calls on a device share the one array: it
+ * keeps whatever the last call left, every entry a call reads is written by that call
+ * first, and two calls whose kernels overlap on the GPU (different streams, no ordering)
+ * race on it - keep such calls ordered. */
+mixlora_status_t mixlora_dispatch_static(const int32_t *expert_idx, int32_t tokens, int32_t n_experts,
+                                         int32_t top_k, int32_t *perm, int32_t *seg_off, void *stream);
+int32_t mixlora_dispatch_static_max_tokens(void);
+
 /* Opt-in bookkeeping for measurements (host side, process-wide, not thread-safe).
  * mixlora_stage_timing(1) clears the counters and makes every later forward / backward /
  * aux_loss call bracket each stage of the path (router, dispatch, the dense products, the

@@ -21,7 +21,8 @@ STATUS_NAMES = {0: "MIXLORA_OK", 1: "MIXLORA_ERR_INVALID_ARG", 2: "MIXLORA_ERR_U
 
 EXPORTS = ("mixlora_limits", "mixlora_workspace_bytes", "mixlora_ffn_forward", "mixlora_aux_loss",
            "mixlora_ffn_backward", "mixlora_routing_view", "mixlora_device_status", "mixlora_gemm_bf16",
-           "mixlora_status_string", "mixlora_stage_timing", "mixlora_stage_timing_read")
+           "mixlora_status_string", "mixlora_stage_timing", "mixlora_stage_timing_read",
+           "mixlora_dispatch_static", "mixlora_dispatch_static_max_tokens")
 
 
 class mixlora_shape_t(C.Structure):
@@ -80,6 +81,11 @@ def _load() -> C.CDLL:
     lib.mixlora_stage_timing_read.argtypes = [C.c_int32, C.POINTER(C.c_char_p), C.POINTER(C.c_float),
                                               C.POINTER(C.c_int64)]
     lib.mixlora_stage_timing_read.restype = C.c_int32
+    lib.mixlora_dispatch_static.argtypes = [C.c_void_p, C.c_int32, C.c_int32, C.c_int32, C.c_void_p, C.c_void_p,
+                                            C.c_void_p]
+    lib.mixlora_dispatch_static.restype = C.c_int
+    lib.mixlora_dispatch_static_max_tokens.argtypes = []
+    lib.mixlora_dispatch_static_max_tokens.restype = C.c_int32
     lib.mixlora_status_string.argtypes = [C.c_int]
     lib.mixlora_status_string.restype = C.c_char_p
     return lib
@@ -209,3 +215,14 @@ def mixlora_stage_timing_read() -> dict:
     launches = (C.c_int64 * n)()
     cnt = lib.mixlora_stage_timing_read(n, names, ms, launches)
     return {names[i].decode(): (float(ms[i]), int(launches[i])) for i in range(min(cnt, n))}
+
+
+def mixlora_dispatch_static(expert_idx, tokens, n_experts, top_k, perm, seg_off, stream=None) -> None:
+    """Dispatch of slots to experts that needs no workspace: its scratch is a fixed array inside the
+    library, so a caller that cannot allocate device memory can still use it (limits in mixlora.h)."""
+    _check(lib.mixlora_dispatch_static(_ptr(expert_idx), tokens, n_experts, top_k, _ptr(perm), _ptr(seg_off),
+                                       _stream(stream)), "mixlora_dispatch_static")
+
+
+def mixlora_dispatch_static_max_tokens() -> int:
+    return int(lib.mixlora_dispatch_static_max_tokens())
