@@ -1,11 +1,446 @@
-// Tensor-core dense product (placeholder until the tcgen05 kernel lands: reports every shape as
-// not taken, so the callers use the SIMT kernel).
+// Dense bf16 product on the Blackwell tensor cores (tcgen05 + TMEM), operands staged by TMA.
+//
+//   C_o[M, N_o] = sum_seg A_seg[M, K_seg] * op(B_o,seg)          fp32 accumulation, bf16 output
+//
+// One persistent CTA per SM walks 128 x tile_n output tiles (tile_n <= 256).  Warp roles:
+//   warp 0    : TMA producer  (one lane)  global -> 128B-swizzled smem ring, kStages deep
+//   warp 1    : MMA issuer    (one lane)  tcgen05.mma 128 x tile_n x 16 into one of two TMEM accumulators
+//   warps 2-5 : epilogue      tcgen05.ld of the finished accumulator, bf16 convert, global stores,
+//               overlapped with the main loop of the next tile (two accumulators of 256 columns)
+// Reduction segments are walked back to back into the same accumulator (K-concatenation);
+// several outputs (column blocks with their own B and C) share one launch when they share A.
+// Every wait is bounded: when a limit runs out the CTA records MIXLORA_ERR_DEVICE_TIMEOUT in the
+// caller's status word, all roles leave their loops, and TMEM is released before exit.
+#include <cuda.h>
+
+#include <mutex>
+
 #include "common.cuh"
 
 namespace mixlora {
 
-bool tc_gemm_supported(int, const TcOut*, int) { return false; }
+namespace {
 
-cudaError_t launch_tc_gemm(int, const TcOut*, int, int*, cudaStream_t) { return cudaErrorNotSupported; }
+constexpr int BM = 128;          // rows per tile (UMMA M, cta_group::1)
+constexpr int BN_MAX = 256;      // columns per tile (UMMA N)
+constexpr int BK = 64;           // reduction elements per stage = one 128-byte swizzle row of bf16
+constexpr int UMMA_K = 16;
+constexpr int kStages = 4;
+constexpr int kMaxSeg = kMaxKSeg;  // A maps
+constexpr int kMaxOut = 4;
+constexpr int kMaxB = 8;           // B maps (outputs x segments)
+constexpr int kThreads = 192;
+constexpr uint32_t kABytes = BM * BK * 2;        // 16 KiB
+constexpr uint32_t kBBytes = BN_MAX * BK * 2;    // 32 KiB
+constexpr uint32_t kStageBytes = kABytes + kBBytes;
+constexpr uint32_t kSmemBytes = kStages * kStageBytes + 1024 /* alignment slack */ + 256 /* barriers */;
+constexpr uint32_t kTmemCols = 512;
+constexpr uint32_t kWaitLimit = 1u << 22;        // try_wait rounds before a wait gives up
+
+struct alignas(64) TcParams {
+  CUtensorMap a_map[kMaxSeg];
+  CUtensorMap b_map[kMaxB];        // index o * nseg + seg
+  void* C[kMaxOut];
+  long long ldc[kMaxOut];
+  int N[kMaxOut];
+  int tile_n[kMaxOut];
+  int tile_start[kMaxOut + 1];     // first tile index of each output
+  int kblocks[kMaxSeg];
+  int nseg, nout, M, m_tiles, total_tiles;
+  int* status;
+};
+
+// ---- PTX wrappers -------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+// Bounded wait.  Returns false when the limit ran out or another role gave up.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+  for (uint32_t it = 0; it < kWaitLimit; ++it) {
+    if (mbar_try_wait(bar, parity)) return true;
+    if ((it & 63u) == 63u && *abort_flag) return false;
+  }
+  return false;
+}
+
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+      ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1)
+      : "memory");
+}
+__device__ __forceinline__ void prefetch_tmap(const CUtensorMap* map) {
+  asm volatile("prefetch.tensormap [%0];" ::"l"(map) : "memory");
+}
+
+__device__ __forceinline__ void tmem_alloc(uint32_t dst_smem, uint32_t cols) {
+  asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dst_smem), "r"(cols) : "memory");
+}
+__device__ __forceinline__ void tmem_relinquish() {
+  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t cols) {
+  asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(cols) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+__device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
+                                          uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+// Arrives on the mbarrier once every tcgen05.mma issued so far by this thread has completed.
+__device__ __forceinline__ void umma_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&v)[32]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]), "=r"(v[8]),
+        "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]), "=r"(v[16]),
+        "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]), "=r"(v[24]),
+        "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
+      : "r"(taddr)
+      : "memory");
+}
+__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+// Shared-memory matrix descriptor of a 128B-swizzled operand tile.
+//   K-major  : rows of 128 bytes (64 bf16 along K); 8-row groups 1024 bytes apart (stride offset).
+//   MN-major : rows of 128 bytes (64 bf16 along N) per k; 8-k groups 1024 bytes apart (stride offset),
+//              64-column blocks `lbo_bytes` apart (leading offset).
+__device__ __forceinline__ uint64_t make_desc(uint32_t saddr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
+  uint64_t d = 0;
+  d |= (uint64_t)((saddr & 0x3FFFFu) >> 4);
+  d |= (uint64_t)((lbo_bytes >> 4) & 0x3FFFu) << 16;
+  d |= (uint64_t)((sbo_bytes >> 4) & 0x3FFFu) << 32;
+  d |= (uint64_t)1 << 46;   // descriptor version of this architecture
+  d |= (uint64_t)2 << 61;   // 128-byte swizzle
+  return d;
+}
+
+// Instruction descriptor: bf16 x bf16 -> fp32, M = 128, N = n, A K-major, B K-major or MN-major.
+__device__ __forceinline__ uint32_t make_idesc(int n, int b_mn_major) {
+  uint32_t d = 0;
+  d |= 1u << 4;                        // accumulator fp32
+  d |= 1u << 7;                        // A bf16
+  d |= 1u << 10;                       // B bf16
+  d |= (uint32_t)(b_mn_major & 1) << 16;
+  d |= (uint32_t)(n >> 3) << 17;
+  d |= (uint32_t)(BM >> 4) << 24;
+  return d;
+}
+
+struct TileCoord { int o, m0, n0; };
+
+__device__ __forceinline__ TileCoord tile_coord(const TcParams& p, int tile) {
+  int o = 0;
+#pragma unroll
+  for (int i = 1; i < kMaxOut; ++i)
+    if (i < p.nout && tile >= p.tile_start[i]) o = i;
+  const int local = tile - p.tile_start[o];
+  TileCoord t;
+  t.o = o;
+  t.m0 = (local % p.m_tiles) * BM;       // rows fastest: neighbouring CTAs share the B tile
+  t.n0 = (local / p.m_tiles) * p.tile_n[o];
+  return t;
+}
+
+template <int B_KN>
+__global__ void __launch_bounds__(kThreads, 1) tc_gemm_kernel(const __grid_constant__ TcParams p) {
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + kStages * kStageBytes);
+  // bars[0..kStages) full, [kStages..2kStages) empty, then tmem_full[2], tmem_empty[2]
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * kStages + 4);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const uint32_t smem_base = smem_u32(smem);
+  const uint32_t bar_base = smem_u32(bars);
+  auto full_bar = [&](int s) { return bar_base + 8u * s; };
+  auto empty_bar = [&](int s) { return bar_base + 8u * (kStages + s); };
+  auto tfull_bar = [&](int b) { return bar_base + 8u * (2 * kStages + b); };
+  auto tempty_bar = [&](int b) { return bar_base + 8u * (2 * kStages + 2 + b); };
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < kStages; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
+    for (int b = 0; b < 2; ++b) { mbar_init(tfull_bar(b), 1); mbar_init(tempty_bar(b), 4); }
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 1) {
+    tmem_alloc(smem_u32(tmem_slot), kTmemCols);
+    tmem_relinquish();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  int total_kb = 0;
+  for (int s = 0; s < p.nseg; ++s) total_kb += p.kblocks[s];
+
+  if (warp == 0) {
+    // ---------------- TMA producer ----------------
+    if (lane == 0) {
+      for (int s = 0; s < p.nseg; ++s) prefetch_tmap(&p.a_map[s]);
+      for (int s = 0; s < p.nseg * p.nout; ++s) prefetch_tmap(&p.b_map[s]);
+      uint32_t it = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; tile < p.total_tiles && ok; tile += gridDim.x) {
+        const TileCoord tc = tile_coord(p, tile);
+        const int tn = p.tile_n[tc.o];
+        const uint32_t tx = kABytes + (uint32_t)tn * BK * 2;
+        for (int sg = 0; sg < p.nseg && ok; ++sg) {
+          const CUtensorMap* am = &p.a_map[sg];
+          const CUtensorMap* bm = &p.b_map[tc.o * p.nseg + sg];
+          for (int kb = 0; kb < p.kblocks[sg]; ++kb, ++it) {
+            const int st = it % kStages;
+            const uint32_t ph = (it / kStages) & 1u;
+            if (!mbar_wait(empty_bar(st), ph ^ 1u, abort_flag)) { ok = false; break; }
+            const uint32_t a_dst = smem_base + st * kStageBytes;
+            const uint32_t b_dst = a_dst + kABytes;
+            mbar_expect_tx(full_bar(st), tx);
+            tma_load_2d(a_dst, am, full_bar(st), kb * BK, tc.m0);
+            if (B_KN == 0) {
+              tma_load_2d(b_dst, bm, full_bar(st), kb * BK, tc.n0);
+            } else {
+              for (int j = 0; j < tn / 64; ++j)
+                tma_load_2d(b_dst + j * (BK * 128), bm, full_bar(st), tc.n0 + j * 64, kb * BK);
+            }
+          }
+        }
+      }
+      if (!ok) {
+        *abort_flag = 1;
+        if (p.status) atomicExch(p.status, (int)MIXLORA_ERR_DEVICE_TIMEOUT);
+      }
+    }
+  } else if (warp == 1) {
+    // ---------------- MMA issuer ----------------
+    if (lane == 0) {
+      uint32_t it = 0, tcount = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; tile < p.total_tiles && ok; tile += gridDim.x, ++tcount) {
+        const TileCoord tc = tile_coord(p, tile);
+        const int tn = p.tile_n[tc.o];
+        const uint32_t idesc = make_idesc(tn, B_KN);
+        const uint32_t buf = tcount & 1u;
+        const uint32_t use = tcount >> 1;                 // how often this accumulator was used before
+        if (!mbar_wait(tempty_bar(buf), (use & 1u) ^ 1u, abort_flag)) { ok = false; break; }
+        tc_fence_after();
+        const uint32_t d_tmem = tmem_base + buf * BN_MAX;
+        for (int kb = 0; kb < total_kb; ++kb, ++it) {
+          const int st = it % kStages;
+          const uint32_t ph = (it / kStages) & 1u;
+          if (!mbar_wait(full_bar(st), ph, abort_flag)) { ok = false; break; }
+          tc_fence_after();
+          const uint32_t a_addr = smem_base + st * kStageBytes;
+          const uint32_t b_addr = a_addr + kABytes;
+#pragma unroll
+          for (int k = 0; k < BK / UMMA_K; ++k) {
+            const uint64_t ad = make_desc(a_addr + k * (UMMA_K * 2), 16, 1024);
+            const uint64_t bd = (B_KN == 0) ? make_desc(b_addr + k * (UMMA_K * 2), 16, 1024)
+                                            : make_desc(b_addr + k * (UMMA_K * 128), BK * 128, 1024);
+            umma_bf16(d_tmem, ad, bd, idesc, (kb | k) != 0);
+          }
+          umma_commit(empty_bar(st));                      // frees the smem stage when the MMAs retire
+        }
+        if (ok) umma_commit(tfull_bar(buf));               // accumulator complete
+      }
+      if (!ok) {
+        *abort_flag = 1;
+        if (p.status) atomicExch(p.status, (int)MIXLORA_ERR_DEVICE_TIMEOUT);
+      }
+    }
+  } else {
+    // ---------------- epilogue: TMEM -> registers -> bf16 -> global ----------------
+    const int q = warp & 3;                                // TMEM lane quarter this warp may read
+    uint32_t tcount = 0;
+    bool ok = true;
+    for (int tile = blockIdx.x; tile < p.total_tiles && ok; tile += gridDim.x, ++tcount) {
+      const TileCoord tc = tile_coord(p, tile);
+      const int tn = p.tile_n[tc.o];
+      const uint32_t buf = tcount & 1u;
+      const uint32_t use = tcount >> 1;
+      // the decision must be the same for the whole warp: the TMEM loads below are warp-collective
+      if (!__all_sync(0xffffffffu, mbar_wait(tfull_bar(buf), use & 1u, abort_flag))) { ok = false; break; }
+      tc_fence_after();
+      const int row = tc.m0 + q * 32 + lane;
+      const int No = p.N[tc.o];
+      bf16* crow = reinterpret_cast<bf16*>(p.C[tc.o]) + (size_t)row * p.ldc[tc.o];
+      const uint32_t t_addr = tmem_base + ((uint32_t)(q * 32) << 16) + buf * BN_MAX;
+      for (int c = 0; c < tn; c += 32) {
+        uint32_t v[32];
+        tmem_ld32(t_addr + c, v);
+        tmem_ld_wait();
+        if (row < p.M) {
+#pragma unroll
+          for (int g8 = 0; g8 < 4; ++g8) {
+            const int col = tc.n0 + c + g8 * 8;
+            if (col < No) {                                // N is a multiple of 8: whole 16-byte groups
+              uint4 o;
+              __nv_bfloat162 h0 = __floats2bfloat162_rn(__uint_as_float(v[g8 * 8 + 0]), __uint_as_float(v[g8 * 8 + 1]));
+              __nv_bfloat162 h1 = __floats2bfloat162_rn(__uint_as_float(v[g8 * 8 + 2]), __uint_as_float(v[g8 * 8 + 3]));
+              __nv_bfloat162 h2 = __floats2bfloat162_rn(__uint_as_float(v[g8 * 8 + 4]), __uint_as_float(v[g8 * 8 + 5]));
+              __nv_bfloat162 h3 = __floats2bfloat162_rn(__uint_as_float(v[g8 * 8 + 6]), __uint_as_float(v[g8 * 8 + 7]));
+              o.x = *reinterpret_cast<uint32_t*>(&h0);
+              o.y = *reinterpret_cast<uint32_t*>(&h1);
+              o.z = *reinterpret_cast<uint32_t*>(&h2);
+              o.w = *reinterpret_cast<uint32_t*>(&h3);
+              *reinterpret_cast<uint4*>(crow + col) = o;
+            }
+          }
+        }
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(tempty_bar(buf));         // 4 arrivals release the accumulator
+    }
+    if (!ok && lane == 0) {
+      *abort_flag = 1;
+      if (p.status) atomicExch(p.status, (int)MIXLORA_ERR_DEVICE_TIMEOUT);
+    }
+  }
+
+  __syncthreads();
+  if (*abort_flag) {
+    // a wait gave up: give copies that may still be in flight time to land before the CTA's smem goes away
+    for (int i = 0; i < 200; ++i) __nanosleep(5000);
+  }
+  tc_fence_after();
+  if (warp == 1) {
+    __syncwarp();
+    tmem_dealloc(tmem_base, kTmemCols);
+  }
+}
+
+// ---- host side ------------------------------------------------------------------------------
+typedef CUresult (*EncodeFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                             const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                             CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeFn get_encode() {
+  static EncodeFn fn = nullptr;
+  static std::once_flag once;
+  std::call_once(once, [] {
+    void* f = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &f, cudaEnableDefault, &q) == cudaSuccess &&
+        q == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeFn>(f);
+  });
+  return fn;
+}
+
+// 2-D bf16 tensor [rows, cols] row-major with leading dimension ld (elements); box = [box_rows, box_cols].
+bool encode_2d(CUtensorMap* map, const void* ptr, long long rows, long long cols, long long ld, int box_rows,
+               int box_cols) {
+  EncodeFn fn = get_encode();
+  if (!fn) return false;
+  cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+  cuuint64_t strides[1] = {(cuuint64_t)ld * 2};
+  cuuint32_t box[2] = {(cuuint32_t)box_cols, (cuuint32_t)box_rows};
+  cuuint32_t estr[2] = {1, 1};
+  CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), dims, strides, box, estr,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS;
+}
+
+int round_up(int v, int a) { return (v + a - 1) / a * a; }
+
+}  // namespace
+
+bool tc_gemm_supported(int M, const TcOut* outs, int nout) {
+  if (M <= 0 || nout <= 0 || nout > kMaxOut) return false;
+  const int nseg = outs[0].nseg;
+  if (nseg <= 0 || nseg > kMaxSeg || nseg * nout > kMaxB) return false;
+  if (!get_encode()) return false;
+  for (int o = 0; o < nout; ++o) {
+    const TcOut& t = outs[o];
+    if (t.nseg != nseg || t.N <= 0 || t.N % 8 || t.ldc % 8 || (reinterpret_cast<uintptr_t>(t.C) & 15u)) return false;
+    for (int s = 0; s < nseg; ++s) {
+      const TcSeg& g = t.seg[s];
+      if (g.K <= 0 || g.K % 8 || g.lda % 8 || g.ldb % 8) return false;
+      if ((reinterpret_cast<uintptr_t>(g.A) & 15u) || (reinterpret_cast<uintptr_t>(g.B) & 15u)) return false;
+      if (g.b_kn != outs[0].seg[0].b_kn) return false;
+      if (g.A != outs[0].seg[s].A || g.lda != outs[0].seg[s].lda || g.K != outs[0].seg[s].K) return false;
+    }
+  }
+  return true;
+}
+
+cudaError_t launch_tc_gemm(int M, const TcOut* outs, int nout, int* status_word, cudaStream_t st) {
+  TcParams p;
+  memset(&p, 0, sizeof(p));
+  const int nseg = outs[0].nseg;
+  const int b_kn = outs[0].seg[0].b_kn;
+  p.nseg = nseg; p.nout = nout; p.M = M; p.m_tiles = (M + BM - 1) / BM; p.status = status_word;
+  for (int s = 0; s < nseg; ++s) {
+    const TcSeg& g = outs[0].seg[s];
+    p.kblocks[s] = (g.K + BK - 1) / BK;
+    if (!encode_2d(&p.a_map[s], g.A, M, g.K, g.lda, BM, BK)) return cudaErrorInvalidValue;
+  }
+  int tiles = 0;
+  for (int o = 0; o < nout; ++o) {
+    const TcOut& t = outs[o];
+    const int tn = b_kn ? (t.N >= BN_MAX ? BN_MAX : round_up(t.N, 64)) : (t.N >= BN_MAX ? BN_MAX : round_up(t.N, 16));
+    p.C[o] = t.C; p.ldc[o] = t.ldc; p.N[o] = t.N; p.tile_n[o] = tn;
+    p.tile_start[o] = tiles;
+    tiles += p.m_tiles * ((t.N + tn - 1) / tn);
+    for (int s = 0; s < nseg; ++s) {
+      const TcSeg& g = t.seg[s];
+      bool ok = b_kn ? encode_2d(&p.b_map[o * nseg + s], g.B, g.K, t.N, g.ldb, BK, 64)
+                     : encode_2d(&p.b_map[o * nseg + s], g.B, t.N, g.K, g.ldb, tn, BK);
+      if (!ok) return cudaErrorInvalidValue;
+    }
+  }
+  p.tile_start[nout] = tiles;
+  for (int o = nout + 1; o <= kMaxOut; ++o) p.tile_start[o] = tiles;
+  p.total_tiles = tiles;
+
+  int dev = 0, sms = 148;
+  cudaGetDevice(&dev);
+  cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  {
+    // per function and per device; cheap enough to repeat on every launch
+    cudaError_t e = b_kn ? cudaFuncSetAttribute(tc_gemm_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes)
+                         : cudaFuncSetAttribute(tc_gemm_kernel<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+    if (e != cudaSuccess) return e;
+  }
+  const int grid = tiles < sms ? tiles : sms;
+  if (b_kn) tc_gemm_kernel<1><<<grid, kThreads, kSmemBytes, st>>>(p);
+  else tc_gemm_kernel<0><<<grid, kThreads, kSmemBytes, st>>>(p);
+  return cudaGetLastError();
+}
 
 }  // namespace mixlora
