@@ -43,7 +43,7 @@ WsLayout ws_layout(const mixlora_shape_t& s) {
   L.U = take(T * f * E);
   L.zga = take(T * N * r * E);
   L.zua = take(T * N * r * E);
-  L.zd = take(T * k * r * E);
+  L.zd_all = take(T * k * N * r * E);
   L.Zs = take(T * N * r * E);
   L.bd_cat = take(d * N * r * E);
   L.h_sorted = take(T * k * f * E);
@@ -55,12 +55,13 @@ WsLayout ws_layout(const mixlora_shape_t& s) {
   L.db_sorted = take(T * k * f * E);
   L.dabar = take(T * f * E);
   L.dbbar = take(T * f * E);
-  L.zg_sorted = take(T * k * r * E);
-  L.zu_sorted = take(T * k * r * E);
-  L.dzg_sorted = take(T * k * r * E);
-  L.dzu_sorted = take(T * k * r * E);
-  L.dzd_sorted = take(T * k * r * E);
-  L.gzd_sorted = take(T * k * r * E);
+  L.bg_cat = take(f * N * r * E);
+  L.bu_cat = take(f * N * r * E);
+  L.Zg_pos = take(T * k * N * r * E);
+  L.Zu_pos = take(T * k * N * r * E);
+  L.dZd_pos = take(T * k * N * r * E);
+  L.dzg_all = take(T * k * N * r * E);
+  L.dzu_all = take(T * k * N * r * E);
   L.dZg = take(T * N * r * E);
   L.dZu = take(T * N * r * E);
   L.dgate = take(T * k * 4);
@@ -170,13 +171,15 @@ void add_seg(SGemm& g, const SOperand& A, const SOperand& B, int K) {
 
 // Dense product on the tensor-core kernel when it takes the shape, else on the SIMT kernel.
 cudaError_t dense_product(const Ctx& c, int M, const TcOut* outs, int nout) {
+  if (nout == 0 || M <= 0) return cudaSuccess;
   if (c.bf16 && tc_gemm_supported(M, outs, nout)) return launch_tc_gemm(M, outs, nout, c.at<int>(c.L.status), c.st);
   for (int o = 0; o < nout; ++o) {
     const TcOut& t = outs[o];
-    SGemm g = sgemm_base(c, t.C, t.ldc, 1, c.bf16, M, t.N);
+    SGemm g = t.mode == 0 ? sgemm_base(c, t.C, t.ldc, 1, c.bf16, M, t.N) : sgemm_base(c, t.C, t.s_m, t.s_n, 0, M, t.N);
+    if (t.mode == 1) { g.c_nb = t.nb; g.c_sblk = t.s_blk; g.alpha = t.alpha; g.accumulate = t.accumulate; }
     for (int i = 0; i < t.nseg; ++i) {
       const TcSeg& sg = t.seg[i];
-      SOperand A = soperand(sg.A, sg.lda, 1, c.bf16);
+      SOperand A = sg.a_mn ? soperand(sg.A, 1, sg.lda, c.bf16) : soperand(sg.A, sg.lda, 1, c.bf16);
       SOperand B = sg.b_kn ? soperand(sg.B, 1, sg.ldb, c.bf16) : soperand(sg.B, sg.ldb, 1, c.bf16);
       add_seg(g, A, B, sg.K);
     }
@@ -187,18 +190,29 @@ cudaError_t dense_product(const Ctx& c, int M, const TcOut* outs, int nout) {
 }
 
 int dense_launches(const Ctx& c, int M, const TcOut* outs, int nout) {
+  if (nout == 0 || M <= 0) return 0;
   return (c.bf16 && tc_gemm_supported(M, outs, nout)) ? 1 : nout;
 }
 
+// activation-type output [M, N] row-major
 TcOut tc_out(void* C, long long ldc, int N) {
   TcOut o;
   memset(&o, 0, sizeof(o));
-  o.C = C; o.ldc = ldc; o.N = N; o.nseg = 0;
+  o.C = C; o.ldc = ldc; o.N = N; o.mode = 0; o.alpha = 1.f; o.nseg = 0;
   return o;
 }
-void tc_add(TcOut& o, const void* A, long long lda, int K, const void* B, long long ldb, int b_kn) {
+// fp32 output at C + (n / nb) * s_blk + (n % nb) * s_n + m * s_m
+TcOut tc_out_f32(float* C, int N, long long s_m, long long s_n, int nb, long long s_blk, float alpha, int accumulate) {
+  TcOut o;
+  memset(&o, 0, sizeof(o));
+  o.C = C; o.N = N; o.mode = 1; o.s_m = s_m; o.s_n = s_n; o.nb = nb; o.s_blk = s_blk; o.alpha = alpha;
+  o.accumulate = accumulate; o.nseg = 0;
+  return o;
+}
+void tc_add(TcOut& o, const void* A, long long lda, int K, const void* B, long long ldb, int b_kn, int a_mn = 0,
+            int b_cols = 0) {
   TcSeg& s = o.seg[o.nseg++];
-  s.A = A; s.lda = lda; s.K = K; s.B = B; s.ldb = ldb; s.b_kn = b_kn;
+  s.A = A; s.lda = lda; s.a_mn = a_mn; s.K = K; s.B = B; s.ldb = ldb; s.b_kn = b_kn; s.b_cols = b_cols;
 }
 
 }  // namespace
@@ -265,13 +279,12 @@ mixlora_status_t mixlora_ffn_forward(const mixlora_shape_t* shape, const mixlora
   }
   // per-slot LoRA-B expansion + SwiGLU
   { StageScope ss(ST_LORA_B_SWIGLU, c.st, 1); MIXLORA_CUDA(launch_lora_b_swiglu(c)); }
-  // zd = A_d[e] h per slot (rows grouped by expert)
+  // zd = A_d h per slot, against every expert's A_d (the slot's own block is picked up by the combine)
   {
-    StageScope ss(ST_LORA_A_DOWN, c.st, 1);
-    SGemm g = sgemm_base(c, c.ws + c.L.zd, r, 1, c.bf16, T * k, r);
-    g.group_mode = 1; g.groups = N;
-    add_seg(g, soperand(c.ws + c.L.h_sorted, f, 1, c.bf16), soperand(params->a_down, f, 1, c.bf16, (long long)r * f), f);
-    MIXLORA_CUDA(launch_simt_gemm(g, c.st));
+    TcOut out = tc_out(c.ws + c.L.zd_all, Nr, Nr);
+    tc_add(out, c.ws + c.L.h_sorted, f, f, params->a_down, f, 0);
+    StageScope ss(ST_LORA_A_DOWN, c.st, dense_launches(c, T * k, &out, 1));
+    MIXLORA_CUDA(dense_product(c, T * k, &out, 1));
   }
   { StageScope ss(ST_COMBINE_H, c.st, 2); MIXLORA_CUDA(launch_combine_h(c)); MIXLORA_CUDA(launch_bd_cat(c)); }
   // y = [hbar | Zs] [W_d | s B_d]^T : the frozen down projection acts once on the gate-weighted sum of a
@@ -337,69 +350,76 @@ mixlora_status_t mixlora_ffn_backward(const mixlora_shape_t* shape, const mixlor
     }
     return MIXLORA_OK;
   }
-  const int b = c.bf16;
-
   // D = dy W_d (shared by a token's slots) and s B_d^T dy for every expert
   {
     TcOut outs[2];
     outs[0] = tc_out(c.ws + c.L.D, f, f);      tc_add(outs[0], dy, d, d, params->w_down, f, 1);
     outs[1] = tc_out(c.ws + c.L.spd, Nr, Nr);  tc_add(outs[1], dy, d, d, c.ws + c.L.bd_cat, Nr, 1);
-    StageScope ss(ST_GEMM_DGRAD_DOWN, c.st, 1 + dense_launches(c, T, outs, 2));
+    StageScope ss(ST_GEMM_DGRAD_DOWN, c.st, 3 + dense_launches(c, T, outs, 2));
     MIXLORA_CUDA(launch_bd_cat(c));
+    MIXLORA_CUDA(launch_bgu_cat(c));
     MIXLORA_CUDA(dense_product(c, T, outs, 2));
   }
   { StageScope ss(ST_SWIGLU_BWD, c.st, 2); MIXLORA_CUDA(launch_swiglu_bwd(c)); MIXLORA_CUDA(launch_slot_prep_bwd(c)); }
-  // dzg = s da B_g[e], dzu = s db B_u[e] (rows grouped by expert)
-  for (int which = 0; which < 2; ++which) {
-    StageScope ss(ST_LORA_DZ, c.st, 1);
-    SGemm g = sgemm_base(c, c.ws + (which ? c.L.dzu_sorted : c.L.dzg_sorted), r, 1, b, T * k, r);
-    g.group_mode = 1; g.groups = N; g.alpha = c.scale;
-    add_seg(g, soperand(c.ws + (which ? c.L.db_sorted : c.L.da_sorted), f, 1, b),
-            soperand(which ? params->b_up : params->b_gate, 1, r, b, (long long)f * r), f);
-    MIXLORA_CUDA(launch_simt_gemm(g, c.st));
+  // dzg = da (s B_g), dzu = db (s B_u), against every expert (the slot's own block is used)
+  {
+    TcOut outs[2];
+    outs[0] = tc_out(c.ws + c.L.dzg_all, Nr, Nr); tc_add(outs[0], c.ws + c.L.da_sorted, f, f, c.ws + c.L.bg_cat, Nr, 1);
+    outs[1] = tc_out(c.ws + c.L.dzu_all, Nr, Nr); tc_add(outs[1], c.ws + c.L.db_sorted, f, f, c.ws + c.L.bu_cat, Nr, 1);
+    StageScope ss(ST_LORA_DZ, c.st, dense_launches(c, T * k, outs, 2));
+    MIXLORA_CUDA(dense_product(c, T * k, outs, 2));
   }
-  // LoRA weight gradients: sums over the slots of each expert's segment
-  const int* pos_token = c.at<int>(c.L.pos_token);
-  auto wgrad = [&](float* out, int M, int Nn, long long c_sm, long long c_sn, long long c_sg, const SOperand& A,
-                   const SOperand& B, float alpha) -> cudaError_t {
-    if (!out) return cudaSuccess;
-    StageScope ss(ST_LORA_WGRAD, c.st, 1);
-    SGemm g = sgemm_base(c, out, c_sm, c_sn, 0, M, Nn);
-    g.c_sg = c_sg; g.group_mode = 2; g.groups = N; g.alpha = alpha; g.accumulate = acc;
-    add_seg(g, A, B, 0);
-    return launch_simt_gemm(g, c.st);
-  };
-  // dB_g[e][f'][rr] = s sum da[pos][f'] zg[pos][rr]
-  MIXLORA_CUDA(wgrad(grads->d_b_gate, f, r, r, 1, (long long)f * r, soperand(c.ws + c.L.da_sorted, 1, f, b),
-                     soperand(c.ws + c.L.zg_sorted, 1, r, b), c.scale));
-  MIXLORA_CUDA(wgrad(grads->d_b_up, f, r, r, 1, (long long)f * r, soperand(c.ws + c.L.db_sorted, 1, f, b),
-                     soperand(c.ws + c.L.zu_sorted, 1, r, b), c.scale));
-  // dA_g[e][rr][c] = sum dzg[pos][rr] x[token(pos)][c]
-  MIXLORA_CUDA(wgrad(grads->d_a_gate, r, d, d, 1, (long long)r * d, soperand(c.ws + c.L.dzg_sorted, 1, r, b),
-                     soperand(params->x, 1, d, b, 0, nullptr, pos_token), 1.f));
-  MIXLORA_CUDA(wgrad(grads->d_a_up, r, d, d, 1, (long long)r * d, soperand(c.ws + c.L.dzu_sorted, 1, r, b),
-                     soperand(params->x, 1, d, b, 0, nullptr, pos_token), 1.f));
-  // dA_d[e][rr][f'] = sum dzd[pos][rr] h[pos][f']
-  MIXLORA_CUDA(wgrad(grads->d_a_down, r, f, f, 1, (long long)r * f, soperand(c.ws + c.L.dzd_sorted, 1, r, b),
-                     soperand(c.ws + c.L.h_sorted, 1, f, b), 1.f));
-  // dB_d[e][c][rr] = s sum dy[token(pos)][c] (g zd)[pos][rr]
-  MIXLORA_CUDA(wgrad(grads->d_b_down, d, r, r, 1, (long long)d * r, soperand(dy, 1, d, b, 0, nullptr, pos_token),
-                     soperand(c.ws + c.L.gzd_sorted, 1, r, b), c.scale));
-
-  // router: gates -> probabilities -> logits -> W_r
+  // router: gates -> probabilities -> logits
   {
     StageScope ss(ST_ROUTER_BWD, c.st, 1 + (grads->d_router_bias ? 1 : 0) + (want_dx ? 1 : 0));
     MIXLORA_CUDA(launch_router_bwd(c, aux_coef, grads->d_router_bias, acc, want_dx));
   }
-  if (grads->d_w_router) {
-    StageScope ss(ST_ROUTER_BWD, c.st, 1);
-    SGemm g = sgemm_base(c, grads->d_w_router, d, 1, 0, N, d);
-    g.accumulate = acc;
-    add_seg(g, soperand(c.ws + c.L.dlogits, 1, N, 0), soperand(params->x, 1, d, b), T);
-    MIXLORA_CUDA(launch_simt_gemm(g, c.st));
+  { StageScope ss(ST_COMBINE_BWD, c.st, 1); MIXLORA_CUDA(launch_combine_bwd(c, want_dx)); }
+  // LoRA and router weight gradients.  Reduction over the sorted slots (f-sized matrices) ...
+  {
+    TcOut outs[3];
+    int n = 0;
+    if (grads->d_b_gate) {   // dB_g[e][f'][rr] = s sum_pos da[pos][f'] zg[pos][rr]
+      outs[n] = tc_out_f32(grads->d_b_gate, Nr, r, 1, r, (long long)f * r, c.scale, acc);
+      tc_add(outs[n++], c.ws + c.L.da_sorted, f, T * k, c.ws + c.L.Zg_pos, Nr, 1, 1);
+    }
+    if (grads->d_b_up) {
+      outs[n] = tc_out_f32(grads->d_b_up, Nr, r, 1, r, (long long)f * r, c.scale, acc);
+      tc_add(outs[n++], c.ws + c.L.db_sorted, f, T * k, c.ws + c.L.Zu_pos, Nr, 1, 1);
+    }
+    if (grads->d_a_down) {   // dA_d[e][rr][f'] = sum_pos (g s pd)[pos][rr] h[pos][f']
+      outs[n] = tc_out_f32(grads->d_a_down, Nr, 1, f, 0, 0, 1.f, acc);
+      tc_add(outs[n++], c.ws + c.L.h_sorted, f, T * k, c.ws + c.L.dZd_pos, Nr, 1, 1);
+    }
+    StageScope ss(ST_LORA_WGRAD, c.st, dense_launches(c, f, outs, n));
+    MIXLORA_CUDA(dense_product(c, f, outs, n));
+  }
+  // ... and over the tokens (d-sized matrices and the router weight)
+  {
+    TcOut outs[4];
+    int n = 0;
+    if (grads->d_a_gate) {   // dA_g[e][rr][c] = sum_t dzg[t][e*r+rr] x[t][c]
+      outs[n] = tc_out_f32(grads->d_a_gate, Nr, 1, d, 0, 0, 1.f, acc);
+      tc_add(outs[n++], params->x, d, T, c.ws + c.L.dZg, Nr, 1, 1);
+    }
+    if (grads->d_a_up) {
+      outs[n] = tc_out_f32(grads->d_a_up, Nr, 1, d, 0, 0, 1.f, acc);
+      tc_add(outs[n++], params->x, d, T, c.ws + c.L.dZu, Nr, 1, 1);
+    }
+    if (grads->d_b_down) {   // dB_d[e][c][rr] = s sum_t dy[t][c] (g zd)[t][e*r+rr]
+      outs[n] = tc_out_f32(grads->d_b_down, Nr, r, 1, r, (long long)d * r, c.scale, acc);
+      tc_add(outs[n++], dy, d, T, c.ws + c.L.Zs, Nr, 1, 1);
+    }
+    StageScope ss(ST_LORA_WGRAD, c.st, dense_launches(c, d, outs, n));
+    MIXLORA_CUDA(dense_product(c, d, outs, n));
+  }
+  if (grads->d_w_router) {     // dW_r[i][c] = sum_t dl[t][i] x[t][c]
+    TcOut out = tc_out_f32(grads->d_w_router, N, 1, d, 0, 0, 1.f, acc);
+    tc_add(out, params->x, d, T, c.ws + c.L.dl_act, NP, 1, 1, NP);
+    StageScope ss(ST_ROUTER_BWD, c.st, dense_launches(c, d, &out, 1));
+    MIXLORA_CUDA(dense_product(c, d, &out, 1));
   }
   if (want_dx) {
-    { StageScope ss(ST_COMBINE_BWD, c.st, 1); MIXLORA_CUDA(launch_combine_bwd(c)); }
     // dx = [dabar | dbbar | dZg | dZu | dl] [W_g ; W_u ; A_g ; A_u ; W_r]
     TcOut out = tc_out(grads->d_x, d, d);
     tc_add(out, c.ws + c.L.dabar, f, f, params->w_gate, d, 1);

@@ -36,7 +36,7 @@ struct WsLayout {
                       //                    the int after the table holds the tile count
   size_t G, U;        // act [T, f]        shared W1 / W3 projections (Section 3.3 (I))
   size_t zga, zua;    // act [T, N*r]      A_g x and A_u x for every expert
-  size_t zd;          // act [T*k, r]      A_d h per sorted slot
+  size_t zd_all;      // act [T*k, N*r]    A_d h of every expert per sorted slot (the slot's own block is used)
   size_t Zs;          // act [T, N*r]      gate * zd scattered to the slot's expert block
   size_t bd_cat;      // act [d, N*r]      s * B_d laid out [c][e*r + rr]
   size_t h_sorted;    // act [T*k, f]
@@ -46,8 +46,10 @@ struct WsLayout {
   size_t spd;         // act [T, N*r]      s * B_d^T dy for every expert
   size_t da_sorted, db_sorted;  // act [T*k, f]
   size_t dabar, dbbar;          // act [T, f]
-  size_t zg_sorted, zu_sorted;  // act [T*k, r]
-  size_t dzg_sorted, dzu_sorted, dzd_sorted, gzd_sorted;  // act [T*k, r]
+  size_t bg_cat, bu_cat;        // act [f, N*r]    s * B_g, s * B_u laid out [f'][e*r + rr]
+  size_t Zg_pos, Zu_pos;        // act [T*k, N*r]  zg / zu of the slot in its expert block, zero elsewhere
+  size_t dZd_pos;               // act [T*k, N*r]  g * s * pd of the slot in its expert block, zero elsewhere
+  size_t dzg_all, dzu_all;      // act [T*k, N*r]  da (s B_g) and db (s B_u) against every expert
   size_t dZg, dZu;    // act [T, N*r]      dzg / dzu scattered dense
   size_t dgate;       // f32 [T*k]         by slot id
   size_t dlogits;     // f32 [T, N]
@@ -93,6 +95,8 @@ struct SGemm {
   int nseg;
   void* C;
   long long c_sm, c_sn, c_sg;
+  int c_nb;             // > 0: column n sits at (n / c_nb) * c_sblk + (n % c_nb) * c_sn
+  long long c_sblk;
   int c_is_bf16;
   int M, N;            // for group_mode 1, M is the upper bound of rows over all groups
   const int* seg_off;  // device
@@ -129,23 +133,30 @@ cudaError_t launch_router(const Ctx& c);              // probs, expert_idx, gate
 cudaError_t launch_dispatch(const Ctx& c);            // perm, inv, pos_token, pos_expert, seg_off, tile_info
 cudaError_t launch_aux_loss(const Ctx& c, float coef, float* loss, float* F, float* P);
 cudaError_t launch_bd_cat(const Ctx& c);
+cudaError_t launch_bgu_cat(const Ctx& c);              // bg_cat, bu_cat
 cudaError_t launch_lora_b_swiglu(const Ctx& c);       // h_sorted from G, U, zga, zua, B_g, B_u
 cudaError_t launch_combine_h(const Ctx& c);           // hbar, Zs
-cudaError_t launch_swiglu_bwd(const Ctx& c);          // h_sorted, da_sorted, db_sorted, dgate, z*_sorted
-cudaError_t launch_slot_prep_bwd(const Ctx& c);       // dzd_sorted, gzd_sorted
-cudaError_t launch_combine_bwd(const Ctx& c);         // dabar, dbbar, dZg, dZu
+cudaError_t launch_swiglu_bwd(const Ctx& c);          // h_sorted, da_sorted, db_sorted, dgate, Zg_pos, Zu_pos
+cudaError_t launch_slot_prep_bwd(const Ctx& c);       // dZd_pos
+cudaError_t launch_combine_bwd(const Ctx& c, int want_dx);  // dZg, dZu and, for dx, dabar, dbbar
 cudaError_t launch_router_bwd(const Ctx& c, float aux_coef, float* d_bias, int accumulate, int want_dx);
 
-// Tensor-core dense product (tc_gemm.cu).  K-concatenated segments; every operand bf16.
-//   C_o[M, N_o] = sum_seg A_seg[M, K_seg] * op(B_o,seg)
-// B is [N, K_seg] row-major (b_kn = 0) or [K_seg, N] row-major (b_kn = 1).  Several outputs
-// (column blocks with their own B and C) may share one launch when they share A.
+// Dense product (tensor-core kernel in tc_gemm.cu, SIMT kernel otherwise), fp32 accumulation:
+//   C_o[M, N_o] = sum_seg op(A_o,seg) * op(B_o,seg)
+// A is [M, K] row-major (a_mn = 0) or [K, M] row-major (a_mn = 1); B is [N, K] row-major
+// (b_kn = 0) or [K, N] row-major (b_kn = 1).  Reduction segments are concatenated; several
+// outputs share one launch.  The tensor-core kernel wants bf16 operands.
+// Output mode 0: activation type, row-major with pitch ldc.  Mode 1: fp32 at
+//   C + (n / nb) * s_blk + (n % nb) * s_n + m * s_m   (nb = 0: C + n * s_n + m * s_m),
+// value alpha * acc, added to the old value when accumulate is set.
 struct TcSeg {
-  const void* A; long long lda; int K;
+  const void* A; long long lda; int a_mn; int K;
   const void* B; long long ldb; int b_kn;
+  int b_cols;   // columns (b_kn = 1) or rows (b_kn = 0) that exist in B when fewer than N_o rounded up; 0 = N_o
 };
 struct TcOut {
   void* C; long long ldc; int N;
+  int mode; long long s_m, s_n, s_blk; int nb; float alpha; int accumulate;
   TcSeg seg[kMaxKSeg]; int nseg;
 };
 bool tc_gemm_supported(int M, const TcOut* outs, int nout);

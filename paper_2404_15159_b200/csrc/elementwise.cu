@@ -18,7 +18,7 @@ __device__ __forceinline__ float sigmoidf_(float v) { return 1.f / (1.f + expf(-
 constexpr int SL = 8;      // sorted slots per block in the per-slot kernels
 constexpr int ENT = 256;   // threads per block
 
-// bd_cat[c][e*r + rr] = s * B_d[e][c][rr]
+// cat[c][e*r + rr] = s * B[e][c][rr]   (B is [N, rows, r]; used for B_d with rows = d and B_g, B_u with rows = f)
 template <typename T>
 __global__ void bd_cat_kernel(const T* __restrict__ b_down, T* __restrict__ bd_cat, int d, int N, int r, float s) {
   const long long n = (long long)d * N * r;
@@ -120,7 +120,7 @@ combine_h_kernel(const T* __restrict__ h_sorted, const T* __restrict__ zd, const
     const int e = q / r, rr = q % r;
     float v = 0.f;
     for (int j = 0; j < k; ++j)
-      if (ex[j] == e) v = g[j] * to_f(zd[(size_t)pos[j] * r + rr]);
+      if (ex[j] == e) v = g[j] * to_f(zd[(size_t)pos[j] * nr + q]);
     Zs[(size_t)t * nr + q] = from_f<T>(v);
   }
 }
@@ -135,7 +135,7 @@ swiglu_bwd_kernel(const T* __restrict__ G, const T* __restrict__ U, const T* __r
                   const T* __restrict__ b_gate, const T* __restrict__ b_up, const T* __restrict__ a_down,
                   const float* __restrict__ gates, const int* __restrict__ perm, const int* __restrict__ pos_token,
                   const int* __restrict__ pos_expert, T* __restrict__ h_sorted, T* __restrict__ da_sorted,
-                  T* __restrict__ db_sorted, T* __restrict__ zg_sorted, T* __restrict__ zu_sorted,
+                  T* __restrict__ db_sorted, T* __restrict__ Zg_pos, T* __restrict__ Zu_pos,
                   float* __restrict__ dgate, int slots, int f, int N, int r, float s) {
   extern __shared__ float sm[];
   float* zg = sm;                 // [SL][r] scaled by s
@@ -159,14 +159,19 @@ swiglu_bwd_kernel(const T* __restrict__ G, const T* __restrict__ U, const T* __r
     float vg = 0.f, vu = 0.f, vp = 0.f;
     if (sl < ns) {
       size_t o = (size_t)tok[sl] * N * r + (size_t)ex[sl] * r + rr;
-      T zgv = zga[o], zuv = zua[o];
-      vg = s * to_f(zgv);
-      vu = s * to_f(zuv);
+      vg = s * to_f(zga[o]);
+      vu = s * to_f(zua[o]);
       vp = to_f(spd[o]);
-      zg_sorted[(size_t)(base + sl) * r + rr] = zgv;
-      zu_sorted[(size_t)(base + sl) * r + rr] = zuv;
     }
     zg[i] = vg; zu[i] = vu; pd[i] = vp;
+  }
+  // the slot's zg / zu in its expert block of a row that is zero elsewhere (operand of the B_g / B_u gradients)
+  for (int i = threadIdx.x; i < ns * N * r; i += ENT) {
+    const int sl = i / (N * r), q = i % (N * r);
+    const bool own = (q / r) == ex[sl];
+    const size_t src = (size_t)tok[sl] * N * r + q;
+    Zg_pos[(size_t)(base + sl) * N * r + q] = own ? zga[src] : from_f<T>(0.f);
+    Zu_pos[(size_t)(base + sl) * N * r + q] = own ? zua[src] : from_f<T>(0.f);
   }
   __syncthreads();
   float dg_acc[SL];
@@ -231,19 +236,19 @@ swiglu_bwd_kernel(const T* __restrict__ G, const T* __restrict__ U, const T* __r
   }
 }
 
-// dzd_sorted = g * (s pd) at the slot's expert ; gzd_sorted = g * zd
+// dZd_pos[pos][q] = g * (s pd)[token, q] inside the slot's expert block, zero elsewhere
 template <typename T>
-__global__ void slot_prep_bwd_kernel(const T* __restrict__ spd, const T* __restrict__ zd, const float* __restrict__ gates,
+__global__ void slot_prep_bwd_kernel(const T* __restrict__ spd, const float* __restrict__ gates,
                                      const int* __restrict__ perm, const int* __restrict__ pos_token,
-                                     const int* __restrict__ pos_expert, T* __restrict__ dzd_sorted,
-                                     T* __restrict__ gzd_sorted, int slots, int N, int r) {
-  const long long n = (long long)slots * r;
+                                     const int* __restrict__ pos_expert, T* __restrict__ dZd_pos, int slots, int N,
+                                     int r) {
+  const long long nr = (long long)N * r;
+  const long long n = (long long)slots * nr;
   for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < n; i += (long long)gridDim.x * blockDim.x) {
-    const int pos = (int)(i / r), rr = (int)(i % r);
-    const float g = gates[perm[pos]];
-    const size_t o = (size_t)pos_token[pos] * N * r + (size_t)pos_expert[pos] * r + rr;
-    dzd_sorted[i] = from_f<T>(g * to_f(spd[o]));
-    gzd_sorted[i] = from_f<T>(g * to_f(zd[i]));
+    const int pos = (int)(i / nr), q = (int)(i % nr);
+    float v = 0.f;
+    if (q / r == pos_expert[pos]) v = gates[perm[pos]] * to_f(spd[(size_t)pos_token[pos] * nr + q]);
+    dZd_pos[i] = from_f<T>(v);
   }
 }
 
@@ -253,7 +258,7 @@ __global__ void __launch_bounds__(ENT)
 combine_bwd_kernel(const T* __restrict__ da_sorted, const T* __restrict__ db_sorted, const T* __restrict__ dzg_sorted,
                    const T* __restrict__ dzu_sorted, const int* __restrict__ inv, const int* __restrict__ expert_idx,
                    T* __restrict__ dabar, T* __restrict__ dbbar, T* __restrict__ dZg, T* __restrict__ dZu, int f, int N,
-                   int r, int k) {
+                   int r, int k, int want_dx) {
   const int t = blockIdx.x;
   __shared__ int pos[MIXLORA_MAX_TOP_K], ex[MIXLORA_MAX_TOP_K];
   if (threadIdx.x < k) {
@@ -261,7 +266,7 @@ combine_bwd_kernel(const T* __restrict__ da_sorted, const T* __restrict__ db_sor
     ex[threadIdx.x] = expert_idx[(size_t)t * k + threadIdx.x];
   }
   __syncthreads();
-  for (int c = threadIdx.x; c < f; c += ENT) {
+  for (int c = threadIdx.x; want_dx && c < f; c += ENT) {
     float sa = 0.f, sb = 0.f;
     for (int j = 0; j < k; ++j) {
       sa += to_f(da_sorted[(size_t)pos[j] * f + c]);
@@ -276,8 +281,8 @@ combine_bwd_kernel(const T* __restrict__ da_sorted, const T* __restrict__ db_sor
     T vg = from_f<T>(0.f), vu = from_f<T>(0.f);
     for (int j = 0; j < k; ++j)
       if (ex[j] == e) {
-        vg = dzg_sorted[(size_t)pos[j] * r + rr];
-        vu = dzu_sorted[(size_t)pos[j] * r + rr];
+        vg = dzg_sorted[(size_t)pos[j] * nr + q];
+        vu = dzu_sorted[(size_t)pos[j] * nr + q];
       }
     dZg[(size_t)t * nr + q] = vg;
     dZu[(size_t)t * nr + q] = vu;
@@ -364,6 +369,16 @@ cudaError_t bd_cat_t(const Ctx& c) {
 }
 
 template <typename T>
+cudaError_t bgu_cat_t(const Ctx& c) {
+  const long long n = (long long)c.s.d_ff * c.s.n_experts * c.s.rank;
+  bd_cat_kernel<T><<<grid_for(n, 256), 256, 0, c.st>>>(reinterpret_cast<const T*>(c.p.b_gate), c.at<T>(c.L.bg_cat),
+                                                      c.s.d_ff, c.s.n_experts, c.s.rank, c.scale);
+  bd_cat_kernel<T><<<grid_for(n, 256), 256, 0, c.st>>>(reinterpret_cast<const T*>(c.p.b_up), c.at<T>(c.L.bu_cat),
+                                                      c.s.d_ff, c.s.n_experts, c.s.rank, c.scale);
+  return cudaGetLastError();
+}
+
+template <typename T>
 cudaError_t lora_b_swiglu_t(const Ctx& c) {
   const int slots = c.s.tokens * c.s.top_k;
   const int blocks = (slots + SL - 1) / SL;
@@ -377,7 +392,7 @@ cudaError_t lora_b_swiglu_t(const Ctx& c) {
 
 template <typename T>
 cudaError_t combine_h_t(const Ctx& c) {
-  combine_h_kernel<T><<<c.s.tokens, ENT, 0, c.st>>>(c.at<T>(c.L.h_sorted), c.at<T>(c.L.zd), c.at<float>(c.L.gates),
+  combine_h_kernel<T><<<c.s.tokens, ENT, 0, c.st>>>(c.at<T>(c.L.h_sorted), c.at<T>(c.L.zd_all), c.at<float>(c.L.gates),
                                                    c.at<int>(c.L.inv), c.at<int>(c.L.expert_idx), c.at<T>(c.L.hbar),
                                                    c.at<T>(c.L.Zs), c.s.d_ff, c.s.n_experts, c.s.rank, c.s.top_k);
   return cudaGetLastError();
@@ -393,7 +408,7 @@ cudaError_t swiglu_bwd_t(const Ctx& c) {
       reinterpret_cast<const T*>(c.p.b_gate), reinterpret_cast<const T*>(c.p.b_up),
       reinterpret_cast<const T*>(c.p.a_down), c.at<float>(c.L.gates), c.at<int>(c.L.perm), c.at<int>(c.L.pos_token),
       c.at<int>(c.L.pos_expert), c.at<T>(c.L.h_sorted), c.at<T>(c.L.da_sorted), c.at<T>(c.L.db_sorted),
-      c.at<T>(c.L.zg_sorted), c.at<T>(c.L.zu_sorted), c.at<float>(c.L.dgate), slots, c.s.d_ff, c.s.n_experts, c.s.rank,
+      c.at<T>(c.L.Zg_pos), c.at<T>(c.L.Zu_pos), c.at<float>(c.L.dgate), slots, c.s.d_ff, c.s.n_experts, c.s.rank,
       c.scale);
   return cudaGetLastError();
 }
@@ -401,18 +416,18 @@ cudaError_t swiglu_bwd_t(const Ctx& c) {
 template <typename T>
 cudaError_t slot_prep_bwd_t(const Ctx& c) {
   const int slots = c.s.tokens * c.s.top_k;
-  slot_prep_bwd_kernel<T><<<grid_for((long long)slots * c.s.rank, 256), 256, 0, c.st>>>(
-      c.at<T>(c.L.spd), c.at<T>(c.L.zd), c.at<float>(c.L.gates), c.at<int>(c.L.perm), c.at<int>(c.L.pos_token),
-      c.at<int>(c.L.pos_expert), c.at<T>(c.L.dzd_sorted), c.at<T>(c.L.gzd_sorted), slots, c.s.n_experts, c.s.rank);
+  slot_prep_bwd_kernel<T><<<grid_for((long long)slots * c.s.rank * c.s.n_experts, 256), 256, 0, c.st>>>(
+      c.at<T>(c.L.spd), c.at<float>(c.L.gates), c.at<int>(c.L.perm), c.at<int>(c.L.pos_token),
+      c.at<int>(c.L.pos_expert), c.at<T>(c.L.dZd_pos), slots, c.s.n_experts, c.s.rank);
   return cudaGetLastError();
 }
 
 template <typename T>
-cudaError_t combine_bwd_t(const Ctx& c) {
+cudaError_t combine_bwd_t(const Ctx& c, int want_dx) {
   combine_bwd_kernel<T><<<c.s.tokens, ENT, 0, c.st>>>(
-      c.at<T>(c.L.da_sorted), c.at<T>(c.L.db_sorted), c.at<T>(c.L.dzg_sorted), c.at<T>(c.L.dzu_sorted),
+      c.at<T>(c.L.da_sorted), c.at<T>(c.L.db_sorted), c.at<T>(c.L.dzg_all), c.at<T>(c.L.dzu_all),
       c.at<int>(c.L.inv), c.at<int>(c.L.expert_idx), c.at<T>(c.L.dabar), c.at<T>(c.L.dbbar), c.at<T>(c.L.dZg),
-      c.at<T>(c.L.dZu), c.s.d_ff, c.s.n_experts, c.s.rank, c.s.top_k);
+      c.at<T>(c.L.dZu), c.s.d_ff, c.s.n_experts, c.s.rank, c.s.top_k, want_dx);
   return cudaGetLastError();
 }
 
@@ -422,7 +437,7 @@ cudaError_t router_bwd_t(const Ctx& c, float aux_coef, float* d_bias, int accumu
   const float aux_scale = (T_ > 0) ? aux_coef * (float)N / (float)T_ : 0.f;
   router_bwd_kernel<T><<<(T_ + 127) / 128, 128, 0, c.st>>>(
       c.at<float>(c.L.probs), c.at<float>(c.L.gates), c.at<int>(c.L.expert_idx), c.at<float>(c.L.dgate),
-      c.at<float>(c.L.stat_F), c.at<float>(c.L.dlogits), want_dx ? c.at<T>(c.L.dl_act) : nullptr, T_, N, NP, c.s.top_k,
+      c.at<float>(c.L.stat_F), c.at<float>(c.L.dlogits), c.at<T>(c.L.dl_act), T_, N, NP, c.s.top_k,
       c.s.renormalize, aux_scale);
   if (d_bias) colsum_kernel<<<N, 256, 0, c.st>>>(c.at<float>(c.L.dlogits), d_bias, T_, N, accumulate);
   if (want_dx)
@@ -438,7 +453,10 @@ cudaError_t launch_lora_b_swiglu(const Ctx& c) { return c.bf16 ? lora_b_swiglu_t
 cudaError_t launch_combine_h(const Ctx& c) { return c.bf16 ? combine_h_t<bf16>(c) : combine_h_t<float>(c); }
 cudaError_t launch_swiglu_bwd(const Ctx& c) { return c.bf16 ? swiglu_bwd_t<bf16>(c) : swiglu_bwd_t<float>(c); }
 cudaError_t launch_slot_prep_bwd(const Ctx& c) { return c.bf16 ? slot_prep_bwd_t<bf16>(c) : slot_prep_bwd_t<float>(c); }
-cudaError_t launch_combine_bwd(const Ctx& c) { return c.bf16 ? combine_bwd_t<bf16>(c) : combine_bwd_t<float>(c); }
+cudaError_t launch_combine_bwd(const Ctx& c, int want_dx) {
+  return c.bf16 ? combine_bwd_t<bf16>(c, want_dx) : combine_bwd_t<float>(c, want_dx);
+}
+cudaError_t launch_bgu_cat(const Ctx& c) { return c.bf16 ? bgu_cat_t<bf16>(c) : bgu_cat_t<float>(c); }
 cudaError_t launch_router_bwd(const Ctx& c, float aux_coef, float* d_bias, int accumulate, int want_dx) {
   return c.bf16 ? router_bwd_t<bf16>(c, aux_coef, d_bias, accumulate, want_dx)
                 : router_bwd_t<float>(c, aux_coef, d_bias, accumulate, want_dx);

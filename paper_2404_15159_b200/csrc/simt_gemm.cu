@@ -89,7 +89,9 @@ __global__ void __launch_bounds__(NT) simt_gemm_kernel(const SGemm g) {
     for (int j = 0; j < 4; ++j) {
       int n = n0 + tx * 4 + j;
       if (n >= g.N) continue;
-      long long idx = cbase + (long long)m * g.c_sm + (long long)n * g.c_sn;
+      long long idx = cbase + (long long)m * g.c_sm +
+                      (g.c_nb > 0 ? (long long)(n / g.c_nb) * g.c_sblk + (long long)(n % g.c_nb) * g.c_sn
+                                  : (long long)n * g.c_sn);
       float v = g.alpha * acc[i][j];
       if (g.c_is_bf16) {
         bf16* C = reinterpret_cast<bf16*>(g.C);

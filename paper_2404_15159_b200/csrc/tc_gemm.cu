@@ -38,11 +38,14 @@ constexpr uint32_t kTmemCols = 512;
 constexpr uint32_t kWaitLimit = 1u << 22;        // try_wait rounds before a wait gives up
 
 struct alignas(64) TcParams {
-  CUtensorMap a_map[kMaxSeg];
+  CUtensorMap a_map[kMaxB];        // index o * nseg + seg
   CUtensorMap b_map[kMaxB];        // index o * nseg + seg
   void* C[kMaxOut];
-  long long ldc[kMaxOut];
-  int N[kMaxOut];
+  long long ldc[kMaxOut];          // mode 0: row pitch; mode 1: stride of m
+  long long s_n[kMaxOut], s_blk[kMaxOut];
+  float alpha[kMaxOut];
+  int mode[kMaxOut], nb[kMaxOut], accumulate[kMaxOut];
+  int N[kMaxOut];                  // columns stored
   int tile_n[kMaxOut];
   int tile_start[kMaxOut + 1];     // first tile index of each output
   int kblocks[kMaxSeg];
@@ -147,11 +150,12 @@ __device__ __forceinline__ uint64_t make_desc(uint32_t saddr, uint32_t lbo_bytes
 }
 
 // Instruction descriptor: bf16 x bf16 -> fp32, M = 128, N = n, A K-major, B K-major or MN-major.
-__device__ __forceinline__ uint32_t make_idesc(int n, int b_mn_major) {
+__device__ __forceinline__ uint32_t make_idesc(int n, int a_mn_major, int b_mn_major) {
   uint32_t d = 0;
   d |= 1u << 4;                        // accumulator fp32
   d |= 1u << 7;                        // A bf16
   d |= 1u << 10;                       // B bf16
+  d |= (uint32_t)(a_mn_major & 1) << 15;
   d |= (uint32_t)(b_mn_major & 1) << 16;
   d |= (uint32_t)(n >> 3) << 17;
   d |= (uint32_t)(BM >> 4) << 24;
@@ -173,7 +177,7 @@ __device__ __forceinline__ TileCoord tile_coord(const TcParams& p, int tile) {
   return t;
 }
 
-template <int B_KN>
+template <int A_MN, int B_KN>
 __global__ void __launch_bounds__(kThreads, 1) tc_gemm_kernel(const __grid_constant__ TcParams p) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -211,8 +215,7 @@ __global__ void __launch_bounds__(kThreads, 1) tc_gemm_kernel(const __grid_const
   if (warp == 0) {
     // ---------------- TMA producer ----------------
     if (lane == 0) {
-      for (int s = 0; s < p.nseg; ++s) prefetch_tmap(&p.a_map[s]);
-      for (int s = 0; s < p.nseg * p.nout; ++s) prefetch_tmap(&p.b_map[s]);
+      for (int s = 0; s < p.nseg * p.nout; ++s) { prefetch_tmap(&p.a_map[s]); prefetch_tmap(&p.b_map[s]); }
       uint32_t it = 0;
       bool ok = true;
       for (int tile = blockIdx.x; tile < p.total_tiles && ok; tile += gridDim.x) {
@@ -220,7 +223,7 @@ __global__ void __launch_bounds__(kThreads, 1) tc_gemm_kernel(const __grid_const
         const int tn = p.tile_n[tc.o];
         const uint32_t tx = kABytes + (uint32_t)tn * BK * 2;
         for (int sg = 0; sg < p.nseg && ok; ++sg) {
-          const CUtensorMap* am = &p.a_map[sg];
+          const CUtensorMap* am = &p.a_map[tc.o * p.nseg + sg];
           const CUtensorMap* bm = &p.b_map[tc.o * p.nseg + sg];
           for (int kb = 0; kb < p.kblocks[sg]; ++kb, ++it) {
             const int st = it % kStages;
@@ -229,7 +232,12 @@ __global__ void __launch_bounds__(kThreads, 1) tc_gemm_kernel(const __grid_const
             const uint32_t a_dst = smem_base + st * kStageBytes;
             const uint32_t b_dst = a_dst + kABytes;
             mbar_expect_tx(full_bar(st), tx);
-            tma_load_2d(a_dst, am, full_bar(st), kb * BK, tc.m0);
+            if (A_MN == 0) {
+              tma_load_2d(a_dst, am, full_bar(st), kb * BK, tc.m0);
+            } else {
+              tma_load_2d(a_dst, am, full_bar(st), tc.m0, kb * BK);
+              tma_load_2d(a_dst + BK * 128, am, full_bar(st), tc.m0 + 64, kb * BK);
+            }
             if (B_KN == 0) {
               tma_load_2d(b_dst, bm, full_bar(st), kb * BK, tc.n0);
             } else {
@@ -252,7 +260,7 @@ __global__ void __launch_bounds__(kThreads, 1) tc_gemm_kernel(const __grid_const
       for (int tile = blockIdx.x; tile < p.total_tiles && ok; tile += gridDim.x, ++tcount) {
         const TileCoord tc = tile_coord(p, tile);
         const int tn = p.tile_n[tc.o];
-        const uint32_t idesc = make_idesc(tn, B_KN);
+        const uint32_t idesc = make_idesc(tn, A_MN, B_KN);
         const uint32_t buf = tcount & 1u;
         const uint32_t use = tcount >> 1;                 // how often this accumulator was used before
         if (!mbar_wait(tempty_bar(buf), (use & 1u) ^ 1u, abort_flag)) { ok = false; break; }
@@ -267,7 +275,8 @@ __global__ void __launch_bounds__(kThreads, 1) tc_gemm_kernel(const __grid_const
           const uint32_t b_addr = a_addr + kABytes;
 #pragma unroll
           for (int k = 0; k < BK / UMMA_K; ++k) {
-            const uint64_t ad = make_desc(a_addr + k * (UMMA_K * 2), 16, 1024);
+            const uint64_t ad = (A_MN == 0) ? make_desc(a_addr + k * (UMMA_K * 2), 16, 1024)
+                                            : make_desc(a_addr + k * (UMMA_K * 128), BK * 128, 1024);
             const uint64_t bd = (B_KN == 0) ? make_desc(b_addr + k * (UMMA_K * 2), 16, 1024)
                                             : make_desc(b_addr + k * (UMMA_K * 128), BK * 128, 1024);
             umma_bf16(d_tmem, ad, bd, idesc, (kb | k) != 0);
@@ -302,7 +311,24 @@ __global__ void __launch_bounds__(kThreads, 1) tc_gemm_kernel(const __grid_const
         uint32_t v[32];
         tmem_ld32(t_addr + c, v);
         tmem_ld_wait();
-        if (row < p.M) {
+        if (row < p.M && p.mode[tc.o] == 1) {
+          // fp32 output at base + (n / nb) * s_blk + (n % nb) * s_n + m * s_m, scaled, optionally accumulated
+          float* base = reinterpret_cast<float*>(p.C[tc.o]) + (size_t)row * p.ldc[tc.o];
+          const int nb = p.nb[tc.o];
+          const long long sn = p.s_n[tc.o], sb = p.s_blk[tc.o];
+          const float alpha = p.alpha[tc.o];
+          const int accum = p.accumulate[tc.o];
+#pragma unroll 4
+          for (int j = 0; j < 32; ++j) {
+            const int n = tc.n0 + c + j;
+            if (n < No) {
+              float* dst = base + (nb > 0 ? (size_t)(n / nb) * sb + (size_t)(n % nb) * sn : (size_t)n * sn);
+              float val = alpha * __uint_as_float(v[j]);
+              if (accum) val += *dst;
+              *dst = val;
+            }
+          }
+        } else if (row < p.M) {
 #pragma unroll
           for (int g8 = 0; g8 < 4; ++g8) {
             const int col = tc.n0 + c + g8 * 8;
@@ -385,62 +411,75 @@ bool tc_gemm_supported(int M, const TcOut* outs, int nout) {
   const int nseg = outs[0].nseg;
   if (nseg <= 0 || nseg > kMaxSeg || nseg * nout > kMaxB) return false;
   if (!get_encode()) return false;
+  const int a_mn = outs[0].seg[0].a_mn, b_kn = outs[0].seg[0].b_kn;
+  if (a_mn && M % 8) return false;
   for (int o = 0; o < nout; ++o) {
     const TcOut& t = outs[o];
-    if (t.nseg != nseg || t.N <= 0 || t.N % 8 || t.ldc % 8 || (reinterpret_cast<uintptr_t>(t.C) & 15u)) return false;
+    if (t.nseg != nseg || t.N <= 0 || !t.C) return false;
+    if (t.mode == 0) {
+      if (t.N % 8 || t.ldc % 8 || (reinterpret_cast<uintptr_t>(t.C) & 15u)) return false;
+    } else if (t.mode != 1 || (reinterpret_cast<uintptr_t>(t.C) & 3u)) {
+      return false;
+    }
     for (int s = 0; s < nseg; ++s) {
       const TcSeg& g = t.seg[s];
-      if (g.K <= 0 || g.K % 8 || g.lda % 8 || g.ldb % 8) return false;
+      if (g.K <= 0 || g.lda % 8 || g.ldb % 8) return false;   // row pitches are multiples of 16 bytes
       if ((reinterpret_cast<uintptr_t>(g.A) & 15u) || (reinterpret_cast<uintptr_t>(g.B) & 15u)) return false;
-      if (g.b_kn != outs[0].seg[0].b_kn) return false;
-      if (g.A != outs[0].seg[s].A || g.lda != outs[0].seg[s].lda || g.K != outs[0].seg[s].K) return false;
+      if (g.b_kn != b_kn || g.a_mn != a_mn) return false;
+      if (g.K != outs[0].seg[s].K) return false;
     }
   }
   return true;
+}
+
+template <int A_MN, int B_KN>
+cudaError_t launch_variant(const TcParams& p, int grid, cudaStream_t st) {
+  // the attribute is per function and per device; cheap enough to repeat on every launch
+  cudaError_t e = cudaFuncSetAttribute(tc_gemm_kernel<A_MN, B_KN>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+  if (e != cudaSuccess) return e;
+  tc_gemm_kernel<A_MN, B_KN><<<grid, kThreads, kSmemBytes, st>>>(p);
+  return cudaGetLastError();
 }
 
 cudaError_t launch_tc_gemm(int M, const TcOut* outs, int nout, int* status_word, cudaStream_t st) {
   TcParams p;
   memset(&p, 0, sizeof(p));
   const int nseg = outs[0].nseg;
-  const int b_kn = outs[0].seg[0].b_kn;
+  const int a_mn = outs[0].seg[0].a_mn, b_kn = outs[0].seg[0].b_kn;
   p.nseg = nseg; p.nout = nout; p.M = M; p.m_tiles = (M + BM - 1) / BM; p.status = status_word;
-  for (int s = 0; s < nseg; ++s) {
-    const TcSeg& g = outs[0].seg[s];
-    p.kblocks[s] = (g.K + BK - 1) / BK;
-    if (!encode_2d(&p.a_map[s], g.A, M, g.K, g.lda, BM, BK)) return cudaErrorInvalidValue;
-  }
+  for (int s = 0; s < nseg; ++s) p.kblocks[s] = (outs[0].seg[s].K + BK - 1) / BK;
   int tiles = 0;
   for (int o = 0; o < nout; ++o) {
     const TcOut& t = outs[o];
-    const int tn = b_kn ? (t.N >= BN_MAX ? BN_MAX : round_up(t.N, 64)) : (t.N >= BN_MAX ? BN_MAX : round_up(t.N, 16));
-    p.C[o] = t.C; p.ldc[o] = t.ldc; p.N[o] = t.N; p.tile_n[o] = tn;
+    // the operand tile covers whole 16-column (K-major B) or 64-column (N-major B) groups; columns past N read as
+    // zero through the tensor map and are never stored
+    const int cols = t.mode == 0 ? t.N : round_up(t.N, 8);
+    const int tn = b_kn ? (cols >= BN_MAX ? BN_MAX : round_up(cols, 64)) : (cols >= BN_MAX ? BN_MAX : round_up(cols, 16));
+    p.C[o] = t.C; p.N[o] = t.N; p.tile_n[o] = tn;
+    p.mode[o] = t.mode;
+    p.ldc[o] = t.mode == 0 ? t.ldc : t.s_m;
+    p.s_n[o] = t.s_n; p.s_blk[o] = t.s_blk; p.nb[o] = t.nb; p.alpha[o] = t.alpha; p.accumulate[o] = t.accumulate;
     p.tile_start[o] = tiles;
     tiles += p.m_tiles * ((t.N + tn - 1) / tn);
     for (int s = 0; s < nseg; ++s) {
       const TcSeg& g = t.seg[s];
-      bool ok = b_kn ? encode_2d(&p.b_map[o * nseg + s], g.B, g.K, t.N, g.ldb, BK, 64)
-                     : encode_2d(&p.b_map[o * nseg + s], g.B, t.N, g.K, g.ldb, tn, BK);
+      bool ok = a_mn ? encode_2d(&p.a_map[o * nseg + s], g.A, g.K, M, g.lda, BK, 64)
+                     : encode_2d(&p.a_map[o * nseg + s], g.A, M, g.K, g.lda, BM, BK);
+      if (!ok) return cudaErrorInvalidValue;
+      ok = b_kn ? encode_2d(&p.b_map[o * nseg + s], g.B, g.K, g.b_cols > 0 ? g.b_cols : t.N, g.ldb, BK, 64)
+                : encode_2d(&p.b_map[o * nseg + s], g.B, g.b_cols > 0 ? g.b_cols : t.N, g.K, g.ldb, tn, BK);
       if (!ok) return cudaErrorInvalidValue;
     }
   }
-  p.tile_start[nout] = tiles;
-  for (int o = nout + 1; o <= kMaxOut; ++o) p.tile_start[o] = tiles;
+  for (int o = nout; o <= kMaxOut; ++o) p.tile_start[o] = tiles;
   p.total_tiles = tiles;
 
   int dev = 0, sms = 148;
   cudaGetDevice(&dev);
   cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-  {
-    // per function and per device; cheap enough to repeat on every launch
-    cudaError_t e = b_kn ? cudaFuncSetAttribute(tc_gemm_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes)
-                         : cudaFuncSetAttribute(tc_gemm_kernel<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
-    if (e != cudaSuccess) return e;
-  }
   const int grid = tiles < sms ? tiles : sms;
-  if (b_kn) tc_gemm_kernel<1><<<grid, kThreads, kSmemBytes, st>>>(p);
-  else tc_gemm_kernel<0><<<grid, kThreads, kSmemBytes, st>>>(p);
-  return cudaGetLastError();
+  if (a_mn) return b_kn ? launch_variant<1, 1>(p, grid, st) : launch_variant<1, 0>(p, grid, st);
+  return b_kn ? launch_variant<0, 1>(p, grid, st) : launch_variant<0, 0>(p, grid, st);
 }
 
 }  // namespace mixlora
