@@ -11,8 +11,8 @@ ROOT = os.path.dirname(PKG)
 CSRC = os.path.join(PKG, "csrc")
 LIB = os.path.join(PKG, "libmixlora.so")
 OBJ_DIR = os.path.join(PKG, "_build")
-SOURCES = ["api.cu", "router.cu", "simt_gemm.cu", "elementwise.cu", "tc_gemm.cu", "static_dispatch.cu"]
-HEADERS = [os.path.join(CSRC, "common.cuh"), os.path.join(ROOT, "include", "mixlora.h")]
+SOURCES = ["api.cu", "router.cu", "simt_gemm.cu", "elementwise.cu", "tc_gemm.cu", "static_dispatch.cu", "fused_swiglu.cu"]
+HEADERS = [os.path.join(CSRC, "common.cuh"), os.path.join(CSRC, "tc_ptx.cuh"), os.path.join(ROOT, "include", "mixlora.h")]
 
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",

@@ -46,6 +46,10 @@ WsLayout ws_layout(const mixlora_shape_t& s) {
   L.zd_all = take(T * k * N * r * E);
   L.Zs = take(T * N * r * E);
   L.bd_cat = take(d * N * r * E);
+  L.bg_cat = take(f * N * r * E);
+  L.bu_cat = take(f * N * r * E);
+  L.Zg_pos = take(T * k * N * r * E);
+  L.Zu_pos = take(T * k * N * r * E);
   L.h_sorted = take(T * k * f * E);
   L.hbar = take(T * f * E);
   L.total_fwd = off;
@@ -55,11 +59,9 @@ WsLayout ws_layout(const mixlora_shape_t& s) {
   L.db_sorted = take(T * k * f * E);
   L.dabar = take(T * f * E);
   L.dbbar = take(T * f * E);
-  L.bg_cat = take(f * N * r * E);
-  L.bu_cat = take(f * N * r * E);
-  L.Zg_pos = take(T * k * N * r * E);
-  L.Zu_pos = take(T * k * N * r * E);
+  L.P_pos = take(T * k * N * r * E);
   L.dZd_pos = take(T * k * N * r * E);
+  L.dgate_part = take((size_t)fused_swiglu_bwd_col_tiles(s.d_ff) * T * k * 4);
   L.dzg_all = take(T * k * N * r * E);
   L.dzu_all = take(T * k * N * r * E);
   L.dZg = take(T * N * r * E);
@@ -278,7 +280,13 @@ mixlora_status_t mixlora_ffn_forward(const mixlora_shape_t* shape, const mixlora
     MIXLORA_CUDA(dense_product(c, T, outs, 4));
   }
   // per-slot LoRA-B expansion + SwiGLU
-  { StageScope ss(ST_LORA_B_SWIGLU, c.st, 1); MIXLORA_CUDA(launch_lora_b_swiglu(c)); }
+  {
+    StageScope ss(ST_LORA_B_SWIGLU, c.st, 4);
+    MIXLORA_CUDA(launch_bgu_cat(c));
+    MIXLORA_CUDA(launch_zpos(c));
+    if (fused_swiglu_supported(c)) MIXLORA_CUDA(launch_fused_swiglu_fwd(c));
+    else MIXLORA_CUDA(launch_lora_b_swiglu(c));
+  }
   // zd = A_d h per slot, against every expert's A_d (the slot's own block is picked up by the combine)
   {
     TcOut out = tc_out(c.ws + c.L.zd_all, Nr, Nr);
@@ -355,12 +363,20 @@ mixlora_status_t mixlora_ffn_backward(const mixlora_shape_t* shape, const mixlor
     TcOut outs[2];
     outs[0] = tc_out(c.ws + c.L.D, f, f);      tc_add(outs[0], dy, d, d, params->w_down, f, 1);
     outs[1] = tc_out(c.ws + c.L.spd, Nr, Nr);  tc_add(outs[1], dy, d, d, c.ws + c.L.bd_cat, Nr, 1);
-    StageScope ss(ST_GEMM_DGRAD_DOWN, c.st, 3 + dense_launches(c, T, outs, 2));
+    StageScope ss(ST_GEMM_DGRAD_DOWN, c.st, 1 + dense_launches(c, T, outs, 2));
     MIXLORA_CUDA(launch_bd_cat(c));
-    MIXLORA_CUDA(launch_bgu_cat(c));
     MIXLORA_CUDA(dense_product(c, T, outs, 2));
   }
-  { StageScope ss(ST_SWIGLU_BWD, c.st, 2); MIXLORA_CUDA(launch_swiglu_bwd(c)); MIXLORA_CUDA(launch_slot_prep_bwd(c)); }
+  {
+    StageScope ss(ST_SWIGLU_BWD, c.st, 3);
+    MIXLORA_CUDA(launch_slot_prep_bwd(c));
+    if (fused_swiglu_supported(c)) {
+      MIXLORA_CUDA(launch_fused_swiglu_bwd(c));
+      MIXLORA_CUDA(launch_dgate_reduce(c, fused_swiglu_bwd_col_tiles(f)));
+    } else {
+      MIXLORA_CUDA(launch_swiglu_bwd(c));
+    }
+  }
   // dzg = da (s B_g), dzu = db (s B_u), against every expert (the slot's own block is used)
   {
     TcOut outs[2];

@@ -39,6 +39,8 @@ struct WsLayout {
   size_t zd_all;      // act [T*k, N*r]    A_d h of every expert per sorted slot (the slot's own block is used)
   size_t Zs;          // act [T, N*r]      gate * zd scattered to the slot's expert block
   size_t bd_cat;      // act [d, N*r]      s * B_d laid out [c][e*r + rr]
+  size_t bg_cat, bu_cat;  // act [f, N*r]  s * B_g, s * B_u laid out [f'][e*r + rr]
+  size_t Zg_pos, Zu_pos;  // act [T*k, N*r]  zg / zu of the slot in its expert block, zero elsewhere
   size_t h_sorted;    // act [T*k, f]
   size_t hbar;        // act [T, f]        sum_j g_j h_j
   size_t total_fwd;
@@ -46,9 +48,9 @@ struct WsLayout {
   size_t spd;         // act [T, N*r]      s * B_d^T dy for every expert
   size_t da_sorted, db_sorted;  // act [T*k, f]
   size_t dabar, dbbar;          // act [T, f]
-  size_t bg_cat, bu_cat;        // act [f, N*r]    s * B_g, s * B_u laid out [f'][e*r + rr]
-  size_t Zg_pos, Zu_pos;        // act [T*k, N*r]  zg / zu of the slot in its expert block, zero elsewhere
-  size_t dZd_pos;               // act [T*k, N*r]  g * s * pd of the slot in its expert block, zero elsewhere
+  size_t P_pos;                 // act [T*k, N*r]  s * pd of the slot in its expert block, zero elsewhere
+  size_t dZd_pos;               // act [T*k, N*r]  gate * P_pos
+  size_t dgate_part;            // f32 [ceil(f/64), T*k]  per column tile partial <Dt, h> of the fused backward
   size_t dzg_all, dzu_all;      // act [T*k, N*r]  da (s B_g) and db (s B_u) against every expert
   size_t dZg, dZu;    // act [T, N*r]      dzg / dzu scattered dense
   size_t dgate;       // f32 [T*k]         by slot id
@@ -134,10 +136,16 @@ cudaError_t launch_dispatch(const Ctx& c);            // perm, inv, pos_token, p
 cudaError_t launch_aux_loss(const Ctx& c, float coef, float* loss, float* F, float* P);
 cudaError_t launch_bd_cat(const Ctx& c);
 cudaError_t launch_bgu_cat(const Ctx& c);              // bg_cat, bu_cat
+cudaError_t launch_zpos(const Ctx& c);                 // Zg_pos, Zu_pos
+cudaError_t launch_dgate_reduce(const Ctx& c, int col_tiles);   // dgate from dgate_part
+bool fused_swiglu_supported(const Ctx& c);
+int fused_swiglu_bwd_col_tiles(int f);
+cudaError_t launch_fused_swiglu_fwd(const Ctx& c);     // tensor-core version of lora_b_swiglu
+cudaError_t launch_fused_swiglu_bwd(const Ctx& c);     // tensor-core version of swiglu_bwd (writes dgate_part)
 cudaError_t launch_lora_b_swiglu(const Ctx& c);       // h_sorted from G, U, zga, zua, B_g, B_u
 cudaError_t launch_combine_h(const Ctx& c);           // hbar, Zs
 cudaError_t launch_swiglu_bwd(const Ctx& c);          // h_sorted, da_sorted, db_sorted, dgate, Zg_pos, Zu_pos
-cudaError_t launch_slot_prep_bwd(const Ctx& c);       // dZd_pos
+cudaError_t launch_slot_prep_bwd(const Ctx& c);       // P_pos, dZd_pos
 cudaError_t launch_combine_bwd(const Ctx& c, int want_dx);  // dZg, dZu and, for dx, dabar, dbbar
 cudaError_t launch_router_bwd(const Ctx& c, float aux_coef, float* d_bias, int accumulate, int want_dx);
 

@@ -135,8 +135,7 @@ swiglu_bwd_kernel(const T* __restrict__ G, const T* __restrict__ U, const T* __r
                   const T* __restrict__ b_gate, const T* __restrict__ b_up, const T* __restrict__ a_down,
                   const float* __restrict__ gates, const int* __restrict__ perm, const int* __restrict__ pos_token,
                   const int* __restrict__ pos_expert, T* __restrict__ h_sorted, T* __restrict__ da_sorted,
-                  T* __restrict__ db_sorted, T* __restrict__ Zg_pos, T* __restrict__ Zu_pos,
-                  float* __restrict__ dgate, int slots, int f, int N, int r, float s) {
+                  T* __restrict__ db_sorted, float* __restrict__ dgate, int slots, int f, int N, int r, float s) {
   extern __shared__ float sm[];
   float* zg = sm;                 // [SL][r] scaled by s
   float* zu = sm + SL * r;        // [SL][r] scaled by s
@@ -164,14 +163,6 @@ swiglu_bwd_kernel(const T* __restrict__ G, const T* __restrict__ U, const T* __r
       vp = to_f(spd[o]);
     }
     zg[i] = vg; zu[i] = vu; pd[i] = vp;
-  }
-  // the slot's zg / zu in its expert block of a row that is zero elsewhere (operand of the B_g / B_u gradients)
-  for (int i = threadIdx.x; i < ns * N * r; i += ENT) {
-    const int sl = i / (N * r), q = i % (N * r);
-    const bool own = (q / r) == ex[sl];
-    const size_t src = (size_t)tok[sl] * N * r + q;
-    Zg_pos[(size_t)(base + sl) * N * r + q] = own ? zga[src] : from_f<T>(0.f);
-    Zu_pos[(size_t)(base + sl) * N * r + q] = own ? zua[src] : from_f<T>(0.f);
   }
   __syncthreads();
   float dg_acc[SL];
@@ -240,16 +231,47 @@ swiglu_bwd_kernel(const T* __restrict__ G, const T* __restrict__ U, const T* __r
 template <typename T>
 __global__ void slot_prep_bwd_kernel(const T* __restrict__ spd, const float* __restrict__ gates,
                                      const int* __restrict__ perm, const int* __restrict__ pos_token,
-                                     const int* __restrict__ pos_expert, T* __restrict__ dZd_pos, int slots, int N,
-                                     int r) {
+                                     const int* __restrict__ pos_expert, T* __restrict__ P_pos,
+                                     T* __restrict__ dZd_pos, int slots, int N, int r) {
   const long long nr = (long long)N * r;
   const long long n = (long long)slots * nr;
   for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < n; i += (long long)gridDim.x * blockDim.x) {
     const int pos = (int)(i / nr), q = (int)(i % nr);
+    T pv = from_f<T>(0.f);
     float v = 0.f;
-    if (q / r == pos_expert[pos]) v = gates[perm[pos]] * to_f(spd[(size_t)pos_token[pos] * nr + q]);
+    if (q / r == pos_expert[pos]) {
+      pv = spd[(size_t)pos_token[pos] * nr + q];
+      v = gates[perm[pos]] * to_f(pv);
+    }
+    P_pos[i] = pv;
     dZd_pos[i] = from_f<T>(v);
   }
+}
+
+// Zg_pos[pos][q] = zga[token(pos)][q] inside the slot's expert block, zero elsewhere (same for Zu_pos)
+template <typename T>
+__global__ void zpos_kernel(const T* __restrict__ zga, const T* __restrict__ zua, const int* __restrict__ pos_token,
+                            const int* __restrict__ pos_expert, T* __restrict__ Zg_pos, T* __restrict__ Zu_pos,
+                            int slots, int N, int r) {
+  const long long nr = (long long)N * r;
+  const long long n = (long long)slots * nr;
+  for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < n; i += (long long)gridDim.x * blockDim.x) {
+    const int pos = (int)(i / nr), q = (int)(i % nr);
+    const bool own = (q / r) == pos_expert[pos];
+    const size_t src = (size_t)pos_token[pos] * nr + q;
+    Zg_pos[i] = own ? zga[src] : from_f<T>(0.f);
+    Zu_pos[i] = own ? zua[src] : from_f<T>(0.f);
+  }
+}
+
+// dgate[slot] = sum over column tiles of the partial <Dt, h> (fixed order)
+__global__ void dgate_reduce_kernel(const float* __restrict__ part, const int* __restrict__ perm,
+                                    float* __restrict__ dgate, int slots, int col_tiles) {
+  const int pos = blockIdx.x * blockDim.x + threadIdx.x;
+  if (pos >= slots) return;
+  float s = 0.f;
+  for (int ct = 0; ct < col_tiles; ++ct) s += part[(size_t)ct * slots + pos];
+  dgate[perm[pos]] = s;
 }
 
 // dabar_t = sum_j da_tj, dbbar_t = sum_j db_tj ; dZg / dZu = dzg / dzu scattered to the expert block
@@ -379,6 +401,15 @@ cudaError_t bgu_cat_t(const Ctx& c) {
 }
 
 template <typename T>
+cudaError_t zpos_t(const Ctx& c) {
+  const int slots = c.s.tokens * c.s.top_k;
+  zpos_kernel<T><<<grid_for((long long)slots * c.s.rank * c.s.n_experts, 256), 256, 0, c.st>>>(
+      c.at<T>(c.L.zga), c.at<T>(c.L.zua), c.at<int>(c.L.pos_token), c.at<int>(c.L.pos_expert), c.at<T>(c.L.Zg_pos),
+      c.at<T>(c.L.Zu_pos), slots, c.s.n_experts, c.s.rank);
+  return cudaGetLastError();
+}
+
+template <typename T>
 cudaError_t lora_b_swiglu_t(const Ctx& c) {
   const int slots = c.s.tokens * c.s.top_k;
   const int blocks = (slots + SL - 1) / SL;
@@ -408,7 +439,7 @@ cudaError_t swiglu_bwd_t(const Ctx& c) {
       reinterpret_cast<const T*>(c.p.b_gate), reinterpret_cast<const T*>(c.p.b_up),
       reinterpret_cast<const T*>(c.p.a_down), c.at<float>(c.L.gates), c.at<int>(c.L.perm), c.at<int>(c.L.pos_token),
       c.at<int>(c.L.pos_expert), c.at<T>(c.L.h_sorted), c.at<T>(c.L.da_sorted), c.at<T>(c.L.db_sorted),
-      c.at<T>(c.L.Zg_pos), c.at<T>(c.L.Zu_pos), c.at<float>(c.L.dgate), slots, c.s.d_ff, c.s.n_experts, c.s.rank,
+      c.at<float>(c.L.dgate), slots, c.s.d_ff, c.s.n_experts, c.s.rank,
       c.scale);
   return cudaGetLastError();
 }
@@ -418,7 +449,7 @@ cudaError_t slot_prep_bwd_t(const Ctx& c) {
   const int slots = c.s.tokens * c.s.top_k;
   slot_prep_bwd_kernel<T><<<grid_for((long long)slots * c.s.rank * c.s.n_experts, 256), 256, 0, c.st>>>(
       c.at<T>(c.L.spd), c.at<float>(c.L.gates), c.at<int>(c.L.perm), c.at<int>(c.L.pos_token),
-      c.at<int>(c.L.pos_expert), c.at<T>(c.L.dZd_pos), slots, c.s.n_experts, c.s.rank);
+      c.at<int>(c.L.pos_expert), c.at<T>(c.L.P_pos), c.at<T>(c.L.dZd_pos), slots, c.s.n_experts, c.s.rank);
   return cudaGetLastError();
 }
 
@@ -455,6 +486,13 @@ cudaError_t launch_swiglu_bwd(const Ctx& c) { return c.bf16 ? swiglu_bwd_t<bf16>
 cudaError_t launch_slot_prep_bwd(const Ctx& c) { return c.bf16 ? slot_prep_bwd_t<bf16>(c) : slot_prep_bwd_t<float>(c); }
 cudaError_t launch_combine_bwd(const Ctx& c, int want_dx) {
   return c.bf16 ? combine_bwd_t<bf16>(c, want_dx) : combine_bwd_t<float>(c, want_dx);
+}
+cudaError_t launch_zpos(const Ctx& c) { return c.bf16 ? zpos_t<bf16>(c) : zpos_t<float>(c); }
+cudaError_t launch_dgate_reduce(const Ctx& c, int col_tiles) {
+  const int slots = c.s.tokens * c.s.top_k;
+  dgate_reduce_kernel<<<(slots + 255) / 256, 256, 0, c.st>>>(c.at<float>(c.L.dgate_part), c.at<int>(c.L.perm),
+                                                            c.at<float>(c.L.dgate), slots, col_tiles);
+  return cudaGetLastError();
 }
 cudaError_t launch_bgu_cat(const Ctx& c) { return c.bf16 ? bgu_cat_t<bf16>(c) : bgu_cat_t<float>(c); }
 cudaError_t launch_router_bwd(const Ctx& c, float aux_coef, float* d_bias, int accumulate, int want_dx) {
