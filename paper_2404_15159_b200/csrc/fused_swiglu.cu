@@ -21,7 +21,8 @@ using namespace tc;
 constexpr int BK = 64;
 constexpr int UMMA_K = 16;
 constexpr int kStages = 4;
-constexpr int kThreads = 192;
+constexpr int kEpiSplit = 2;                       // epilogue warps per TMEM lane quarter, each takes COLS / kEpiSplit columns
+constexpr int kThreads = 64 + 128 * kEpiSplit;
 constexpr uint32_t kABytes = BM * BK * 2;
 constexpr uint32_t kTmemCols = 512;
 constexpr uint32_t kBufStride = 256;
@@ -78,7 +79,7 @@ __global__ void __launch_bounds__(kThreads, 1) fused_swiglu_kernel(const __grid_
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < kStages; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
-    for (int b = 0; b < 2; ++b) { mbar_init(tfull_bar(b), 1); mbar_init(tempty_bar(b), 4); }
+    for (int b = 0; b < 2; ++b) { mbar_init(tfull_bar(b), 1); mbar_init(tempty_bar(b), 4 * kEpiSplit); }
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -158,12 +159,14 @@ __global__ void __launch_bounds__(kThreads, 1) fused_swiglu_kernel(const __grid_
       }
     }
   } else {
-    const int q = warp & 3;
+    constexpr int WCOLS = COLS / kEpiSplit;            // columns this warp handles
+    const int q = warp & 3;                            // TMEM lane quarter this warp may read
+    const int part = (warp - 2) >> 2;                  // which column share of the tile
     uint32_t wcount = 0;
     bool ok = true;
     for (int w = blockIdx.x; w < p.total && ok; w += gridDim.x, ++wcount) {
       const int ct = w % p.col_tiles;
-      const int row0 = (w / p.col_tiles) * BM, col0 = ct * COLS;
+      const int row0 = (w / p.col_tiles) * BM, col0 = ct * COLS + part * WCOLS;
       const uint32_t buf = wcount & 1u, use = wcount >> 1;
       const int pos = row0 + q * 32 + lane;
       const bool valid = pos < p.slots;
@@ -171,14 +174,24 @@ __global__ void __launch_bounds__(kThreads, 1) fused_swiglu_kernel(const __grid_
       const int tok = valid ? p.pos_token[pos] : 0;
       float gate = 0.f;
       if (BWD && valid) gate = p.gates[p.perm[pos]];
-      if (!__all_sync(0xffffffffu, mbar_wait(tfull_bar(buf), use & 1u, abort_flag))) { ok = false; break; }
-      tc_fence_after();
-      const uint32_t t_addr = tmem_base + ((uint32_t)(q * 32) << 16) + buf * kBufStride;
       const size_t src = (size_t)tok * p.f + col0;
       const size_t dst = (size_t)pos * p.f + col0;
+      // the token's G, U (and D) values of this column tile do not depend on the accumulator: fetch the whole
+      // row segment now, so that the gathers are in flight while the MMAs finish
+      uint4 gq[WCOLS / 8], uq[WCOLS / 8], dq[BWD ? WCOLS / 8 : 1];
+#pragma unroll
+      for (int i = 0; i < WCOLS / 8; ++i) {
+        const bool in = valid && (col0 + i * 8 < p.f);
+        gq[i] = in ? __ldg(reinterpret_cast<const uint4*>(p.G + src + i * 8)) : make_uint4(0, 0, 0, 0);
+        uq[i] = in ? __ldg(reinterpret_cast<const uint4*>(p.U + src + i * 8)) : make_uint4(0, 0, 0, 0);
+        if (BWD) dq[i] = in ? __ldg(reinterpret_cast<const uint4*>(p.D + src + i * 8)) : make_uint4(0, 0, 0, 0);
+      }
+      if (!__all_sync(0xffffffffu, mbar_wait(tfull_bar(buf), use & 1u, abort_flag))) { ok = false; break; }
+      tc_fence_after();
+      const uint32_t t_addr = tmem_base + ((uint32_t)(q * 32) << 16) + buf * kBufStride + part * WCOLS;
       float dg = 0.f;
-#pragma unroll 1
-      for (int c = 0; c < COLS; c += 16) {
+#pragma unroll
+      for (int c = 0; c < WCOLS; c += 16) {
         uint32_t va[16], vb[16], vd[16];
         tmem_ld16(t_addr + c, va);
         tmem_ld16(t_addr + COLS + c, vb);
@@ -190,24 +203,24 @@ __global__ void __launch_bounds__(kThreads, 1) fused_swiglu_kernel(const __grid_
             const int col = col0 + c + g8 * 8;
             if (col < p.f) {
               float gv[8], uv[8], hv[8];
-              unpack8(*reinterpret_cast<const uint4*>(p.G + src + c + g8 * 8), gv);
-              unpack8(*reinterpret_cast<const uint4*>(p.U + src + c + g8 * 8), uv);
+              unpack8(gq[c / 8 + g8], gv);
+              unpack8(uq[c / 8 + g8], uv);
               if (!BWD) {
 #pragma unroll
                 for (int i = 0; i < 8; ++i) {
                   const float a = gv[i] + __uint_as_float(va[g8 * 8 + i]);
                   const float b = uv[i] + __uint_as_float(vb[g8 * 8 + i]);
-                  hv[i] = a / (1.f + __expf(-a)) * b;
+                  hv[i] = __fdividef(a, 1.f + __expf(-a)) * b;
                 }
                 *reinterpret_cast<uint4*>(p.h + dst + c + g8 * 8) = pack8(hv);
               } else {
                 float dv[8], dav[8], dbv[8];
-                unpack8(*reinterpret_cast<const uint4*>(p.D + src + c + g8 * 8), dv);
+                unpack8(dq[c / 8 + g8], dv);
 #pragma unroll
                 for (int i = 0; i < 8; ++i) {
                   const float a = gv[i] + __uint_as_float(va[g8 * 8 + i]);
                   const float b = uv[i] + __uint_as_float(vb[g8 * 8 + i]);
-                  const float sg = 1.f / (1.f + __expf(-a));
+                  const float sg = __fdividef(1.f, 1.f + __expf(-a));
                   const float sa = a * sg;
                   const float hh = sa * b;
                   const float Dt = dv[i] + __uint_as_float(vd[g8 * 8 + i]);
@@ -228,7 +241,7 @@ __global__ void __launch_bounds__(kThreads, 1) fused_swiglu_kernel(const __grid_
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(tempty_bar(buf));
-      if (BWD && valid) p.dgate_part[(size_t)ct * p.slots + pos] = dg;
+      if (BWD && valid) p.dgate_part[(size_t)(ct * kEpiSplit + part) * p.slots + pos] = dg;
     }
     if (!ok && lane == 0) {
       *abort_flag = 1;
@@ -284,7 +297,7 @@ cudaError_t launch_t(const Ctx& c) {
 }  // namespace
 
 bool fused_swiglu_supported(const Ctx& c) { return c.bf16 && c.s.tokens > 0; }
-int fused_swiglu_bwd_col_tiles(int f) { return (f + 63) / 64; }
+int fused_swiglu_bwd_col_tiles(int f) { return (f + 63) / 64 * kEpiSplit; }
 cudaError_t launch_fused_swiglu_fwd(const Ctx& c) { return launch_t<0>(c); }
 cudaError_t launch_fused_swiglu_bwd(const Ctx& c) { return launch_t<1>(c); }
 
