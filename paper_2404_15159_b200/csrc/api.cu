@@ -294,7 +294,7 @@ mixlora_status_t mixlora_ffn_forward(const mixlora_shape_t* shape, const mixlora
     StageScope ss(ST_LORA_A_DOWN, c.st, dense_launches(c, T * k, &out, 1));
     MIXLORA_CUDA(dense_product(c, T * k, &out, 1));
   }
-  { StageScope ss(ST_COMBINE_H, c.st, 2); MIXLORA_CUDA(launch_combine_h(c)); MIXLORA_CUDA(launch_bd_cat(c)); }
+  { StageScope ss(ST_COMBINE_H, c.st, c.bf16 ? 3 : 2); MIXLORA_CUDA(launch_combine_h(c)); MIXLORA_CUDA(launch_bd_cat(c)); }
   // y = [hbar | Zs] [W_d | s B_d]^T : the frozen down projection acts once on the gate-weighted sum of a
   // token's slots (W_d is linear and shared), its LoRA rides along as extra reduction columns
   {
@@ -390,7 +390,7 @@ mixlora_status_t mixlora_ffn_backward(const mixlora_shape_t* shape, const mixlor
     StageScope ss(ST_ROUTER_BWD, c.st, 1 + (grads->d_router_bias ? 1 : 0) + (want_dx ? 1 : 0));
     MIXLORA_CUDA(launch_router_bwd(c, aux_coef, grads->d_router_bias, acc, want_dx));
   }
-  { StageScope ss(ST_COMBINE_BWD, c.st, 1); MIXLORA_CUDA(launch_combine_bwd(c, want_dx)); }
+  { StageScope ss(ST_COMBINE_BWD, c.st, (c.bf16 && want_dx) ? 2 : 1); MIXLORA_CUDA(launch_combine_bwd(c, want_dx)); }
   // LoRA and router weight gradients.  Reduction over the sorted slots (f-sized matrices) ...
   {
     TcOut outs[3];

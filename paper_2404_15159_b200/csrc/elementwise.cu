@@ -100,7 +100,7 @@ template <typename T>
 __global__ void __launch_bounds__(ENT)
 combine_h_kernel(const T* __restrict__ h_sorted, const T* __restrict__ zd, const float* __restrict__ gates,
                  const int* __restrict__ inv, const int* __restrict__ expert_idx, T* __restrict__ hbar,
-                 T* __restrict__ Zs, int f, int N, int r, int k) {
+                 T* __restrict__ Zs, int f, int N, int r, int k, int do_wide) {
   const int t = blockIdx.x;
   __shared__ int pos[MIXLORA_MAX_TOP_K], ex[MIXLORA_MAX_TOP_K];
   __shared__ float g[MIXLORA_MAX_TOP_K];
@@ -110,18 +110,85 @@ combine_h_kernel(const T* __restrict__ h_sorted, const T* __restrict__ zd, const
     g[threadIdx.x] = gates[(size_t)t * k + threadIdx.x];
   }
   __syncthreads();
-  for (int c = threadIdx.x; c < f; c += ENT) {
+  for (int c = threadIdx.x; do_wide && c < f; c += ENT) {
     float acc = 0.f;
     for (int j = 0; j < k; ++j) acc = fmaf(g[j], to_f(h_sorted[(size_t)pos[j] * f + c]), acc);
     hbar[(size_t)t * f + c] = from_f<T>(acc);
   }
   const int nr = N * r;
-  for (int q = threadIdx.x; q < nr; q += ENT) {
+  for (int q = threadIdx.x; q < nr; q += blockDim.x) {
     const int e = q / r, rr = q % r;
     float v = 0.f;
     for (int j = 0; j < k; ++j)
       if (ex[j] == e) v = g[j] * to_f(zd[(size_t)pos[j] * nr + q]);
     Zs[(size_t)t * nr + q] = from_f<T>(v);
+  }
+}
+
+// bf16 version of the f-wide part of combine_h, 8 values per thread per step
+__global__ void __launch_bounds__(ENT)
+combine_h_vec_kernel(const bf16* __restrict__ h_sorted, const float* __restrict__ gates, const int* __restrict__ inv,
+                     bf16* __restrict__ hbar, int f, int k) {
+  const int t = blockIdx.x;
+  __shared__ int pos[MIXLORA_MAX_TOP_K];
+  __shared__ float g[MIXLORA_MAX_TOP_K];
+  if (threadIdx.x < k) {
+    pos[threadIdx.x] = inv[(size_t)t * k + threadIdx.x];
+    g[threadIdx.x] = gates[(size_t)t * k + threadIdx.x];
+  }
+  __syncthreads();
+  for (int c = threadIdx.x * 8; c < f; c += ENT * 8) {
+    float acc[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+    for (int j = 0; j < k; ++j) {
+      const uint4 raw = __ldg(reinterpret_cast<const uint4*>(h_sorted + (size_t)pos[j] * f + c));
+      const __nv_bfloat162* pr = reinterpret_cast<const __nv_bfloat162*>(&raw);
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        const float2 v = __bfloat1622float2(pr[i]);
+        acc[2 * i] = fmaf(g[j], v.x, acc[2 * i]);
+        acc[2 * i + 1] = fmaf(g[j], v.y, acc[2 * i + 1]);
+      }
+    }
+    uint4 o;
+    __nv_bfloat162* po = reinterpret_cast<__nv_bfloat162*>(&o);
+#pragma unroll
+    for (int i = 0; i < 4; ++i) po[i] = __floats2bfloat162_rn(acc[2 * i], acc[2 * i + 1]);
+    *reinterpret_cast<uint4*>(hbar + (size_t)t * f + c) = o;
+  }
+}
+
+// bf16 version of the f-wide part of combine_bwd
+__global__ void __launch_bounds__(ENT)
+combine_bwd_vec_kernel(const bf16* __restrict__ da_sorted, const bf16* __restrict__ db_sorted,
+                       const int* __restrict__ inv, bf16* __restrict__ dabar, bf16* __restrict__ dbbar, int f, int k) {
+  const int t = blockIdx.x;
+  __shared__ int pos[MIXLORA_MAX_TOP_K];
+  if (threadIdx.x < k) pos[threadIdx.x] = inv[(size_t)t * k + threadIdx.x];
+  __syncthreads();
+  for (int c = threadIdx.x * 8; c < f; c += ENT * 8) {
+    float sa[8] = {0, 0, 0, 0, 0, 0, 0, 0}, sb[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+    for (int j = 0; j < k; ++j) {
+      const uint4 ra = __ldg(reinterpret_cast<const uint4*>(da_sorted + (size_t)pos[j] * f + c));
+      const uint4 rb = __ldg(reinterpret_cast<const uint4*>(db_sorted + (size_t)pos[j] * f + c));
+      const __nv_bfloat162* pa = reinterpret_cast<const __nv_bfloat162*>(&ra);
+      const __nv_bfloat162* pb = reinterpret_cast<const __nv_bfloat162*>(&rb);
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        const float2 va = __bfloat1622float2(pa[i]), vb = __bfloat1622float2(pb[i]);
+        sa[2 * i] += va.x; sa[2 * i + 1] += va.y;
+        sb[2 * i] += vb.x; sb[2 * i + 1] += vb.y;
+      }
+    }
+    uint4 oa, ob;
+    __nv_bfloat162* qa = reinterpret_cast<__nv_bfloat162*>(&oa);
+    __nv_bfloat162* qb = reinterpret_cast<__nv_bfloat162*>(&ob);
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      qa[i] = __floats2bfloat162_rn(sa[2 * i], sa[2 * i + 1]);
+      qb[i] = __floats2bfloat162_rn(sb[2 * i], sb[2 * i + 1]);
+    }
+    *reinterpret_cast<uint4*>(dabar + (size_t)t * f + c) = oa;
+    *reinterpret_cast<uint4*>(dbbar + (size_t)t * f + c) = ob;
   }
 }
 
@@ -298,7 +365,7 @@ combine_bwd_kernel(const T* __restrict__ da_sorted, const T* __restrict__ db_sor
     dbbar[(size_t)t * f + c] = from_f<T>(sb);
   }
   const int nr = N * r;
-  for (int q = threadIdx.x; q < nr; q += ENT) {
+  for (int q = threadIdx.x; q < nr; q += blockDim.x) {
     const int e = q / r, rr = q % r;
     T vg = from_f<T>(0.f), vu = from_f<T>(0.f);
     for (int j = 0; j < k; ++j)
@@ -423,9 +490,11 @@ cudaError_t lora_b_swiglu_t(const Ctx& c) {
 
 template <typename T>
 cudaError_t combine_h_t(const Ctx& c) {
-  combine_h_kernel<T><<<c.s.tokens, ENT, 0, c.st>>>(c.at<T>(c.L.h_sorted), c.at<T>(c.L.zd_all), c.at<float>(c.L.gates),
-                                                   c.at<int>(c.L.inv), c.at<int>(c.L.expert_idx), c.at<T>(c.L.hbar),
-                                                   c.at<T>(c.L.Zs), c.s.d_ff, c.s.n_experts, c.s.rank, c.s.top_k);
+  // with bf16 activations the f-wide sum runs in its own vectorised kernel; this one then only scatters Zs
+  constexpr bool vec = sizeof(T) == 2;
+  combine_h_kernel<T><<<c.s.tokens, vec ? 128 : ENT, 0, c.st>>>(
+      c.at<T>(c.L.h_sorted), c.at<T>(c.L.zd_all), c.at<float>(c.L.gates), c.at<int>(c.L.inv), c.at<int>(c.L.expert_idx),
+      c.at<T>(c.L.hbar), c.at<T>(c.L.Zs), c.s.d_ff, c.s.n_experts, c.s.rank, c.s.top_k, vec ? 0 : 1);
   return cudaGetLastError();
 }
 
@@ -455,10 +524,11 @@ cudaError_t slot_prep_bwd_t(const Ctx& c) {
 
 template <typename T>
 cudaError_t combine_bwd_t(const Ctx& c, int want_dx) {
-  combine_bwd_kernel<T><<<c.s.tokens, ENT, 0, c.st>>>(
+  constexpr bool vec = sizeof(T) == 2;
+  combine_bwd_kernel<T><<<c.s.tokens, vec ? 128 : ENT, 0, c.st>>>(
       c.at<T>(c.L.da_sorted), c.at<T>(c.L.db_sorted), c.at<T>(c.L.dzg_all), c.at<T>(c.L.dzu_all),
       c.at<int>(c.L.inv), c.at<int>(c.L.expert_idx), c.at<T>(c.L.dabar), c.at<T>(c.L.dbbar), c.at<T>(c.L.dZg),
-      c.at<T>(c.L.dZu), c.s.d_ff, c.s.n_experts, c.s.rank, c.s.top_k, want_dx);
+      c.at<T>(c.L.dZu), c.s.d_ff, c.s.n_experts, c.s.rank, c.s.top_k, vec ? 0 : want_dx);
   return cudaGetLastError();
 }
 
@@ -481,11 +551,21 @@ cudaError_t router_bwd_t(const Ctx& c, float aux_coef, float* d_bias, int accumu
 
 cudaError_t launch_bd_cat(const Ctx& c) { return c.bf16 ? bd_cat_t<bf16>(c) : bd_cat_t<float>(c); }
 cudaError_t launch_lora_b_swiglu(const Ctx& c) { return c.bf16 ? lora_b_swiglu_t<bf16>(c) : lora_b_swiglu_t<float>(c); }
-cudaError_t launch_combine_h(const Ctx& c) { return c.bf16 ? combine_h_t<bf16>(c) : combine_h_t<float>(c); }
+cudaError_t launch_combine_h(const Ctx& c) {
+  if (!c.bf16) return combine_h_t<float>(c);
+  combine_h_vec_kernel<<<c.s.tokens, ENT, 0, c.st>>>(c.at<bf16>(c.L.h_sorted), c.at<float>(c.L.gates), c.at<int>(c.L.inv),
+                                                    c.at<bf16>(c.L.hbar), c.s.d_ff, c.s.top_k);
+  return combine_h_t<bf16>(c);
+}
 cudaError_t launch_swiglu_bwd(const Ctx& c) { return c.bf16 ? swiglu_bwd_t<bf16>(c) : swiglu_bwd_t<float>(c); }
 cudaError_t launch_slot_prep_bwd(const Ctx& c) { return c.bf16 ? slot_prep_bwd_t<bf16>(c) : slot_prep_bwd_t<float>(c); }
 cudaError_t launch_combine_bwd(const Ctx& c, int want_dx) {
-  return c.bf16 ? combine_bwd_t<bf16>(c, want_dx) : combine_bwd_t<float>(c, want_dx);
+  if (!c.bf16) return combine_bwd_t<float>(c, want_dx);
+  if (want_dx)
+    combine_bwd_vec_kernel<<<c.s.tokens, ENT, 0, c.st>>>(c.at<bf16>(c.L.da_sorted), c.at<bf16>(c.L.db_sorted),
+                                                        c.at<int>(c.L.inv), c.at<bf16>(c.L.dabar),
+                                                        c.at<bf16>(c.L.dbbar), c.s.d_ff, c.s.top_k);
+  return combine_bwd_t<bf16>(c, want_dx);
 }
 cudaError_t launch_zpos(const Ctx& c) { return c.bf16 ? zpos_t<bf16>(c) : zpos_t<float>(c); }
 cudaError_t launch_dgate_reduce(const Ctx& c, int col_tiles) {

@@ -21,8 +21,9 @@ using namespace tc;
 constexpr int BK = 64;
 constexpr int UMMA_K = 16;
 constexpr int kStages = 4;
-constexpr int kEpiSplit = 2;                       // epilogue warps per TMEM lane quarter, each takes COLS / kEpiSplit columns
-constexpr int kThreads = 64 + 128 * kEpiSplit;
+// epilogue warps per TMEM lane quarter (each takes COLS / split columns of a tile)
+constexpr int epi_split(int bwd) { return bwd ? 2 : 4; }
+constexpr int threads_of(int bwd) { return 64 + 128 * epi_split(bwd); }
 constexpr uint32_t kABytes = BM * BK * 2;
 constexpr uint32_t kTmemCols = 512;
 constexpr uint32_t kBufStride = 256;
@@ -57,8 +58,9 @@ __device__ __forceinline__ uint4 pack8(const float* v) {
 }
 
 template <int BWD>
-__global__ void __launch_bounds__(kThreads, 1) fused_swiglu_kernel(const __grid_constant__ FsParams p) {
+__global__ void __launch_bounds__(threads_of(BWD), 1) fused_swiglu_kernel(const __grid_constant__ FsParams p) {
   constexpr int COLS = BWD ? 64 : 128;
+  constexpr int kEpiSplit = epi_split(BWD);
   constexpr int NSUB = BWD ? 3 : 2;
   constexpr uint32_t kBBytes = COLS * BK * 2;
   constexpr uint32_t kStageBytes = kABytes + kBBytes;
@@ -290,14 +292,14 @@ cudaError_t launch_t(const Ctx& c) {
   cudaError_t e = cudaFuncSetAttribute(fused_swiglu_kernel<BWD>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem);
   if (e != cudaSuccess) return e;
   const int grid = p.total < sms ? p.total : sms;
-  fused_swiglu_kernel<BWD><<<grid, kThreads, kSmem, c.st>>>(p);
+  fused_swiglu_kernel<BWD><<<grid, threads_of(BWD), kSmem, c.st>>>(p);
   return cudaGetLastError();
 }
 
 }  // namespace
 
 bool fused_swiglu_supported(const Ctx& c) { return c.bf16 && c.s.tokens > 0; }
-int fused_swiglu_bwd_col_tiles(int f) { return (f + 63) / 64 * kEpiSplit; }
+int fused_swiglu_bwd_col_tiles(int f) { return (f + 63) / 64 * epi_split(1); }
 cudaError_t launch_fused_swiglu_fwd(const Ctx& c) { return launch_t<0>(c); }
 cudaError_t launch_fused_swiglu_bwd(const Ctx& c) { return launch_t<1>(c); }
 

@@ -9,22 +9,37 @@ namespace {
 constexpr int kWarpsPerBlock = 8;
 constexpr float kMarginFlag = 1e-4f;
 
-__device__ __forceinline__ float4 ld4(const float* p) { return *reinterpret_cast<const float4*>(p); }
-__device__ __forceinline__ float4 ld4(const bf16* p) {
-  uint2 raw = *reinterpret_cast<const uint2*>(p);
-  __nv_bfloat162 lo = *reinterpret_cast<__nv_bfloat162*>(&raw.x);
-  __nv_bfloat162 hi = *reinterpret_cast<__nv_bfloat162*>(&raw.y);
-  float2 a = __bfloat1622float2(lo), b = __bfloat1622float2(hi);
-  return make_float4(a.x, a.y, b.x, b.y);
+// VEC consecutive features of one row as floats (16-byte load)
+template <int VEC> struct FeatVec { float v[VEC]; };
+__device__ __forceinline__ FeatVec<4> ld_feat(const float* p) {
+  const float4 r = *reinterpret_cast<const float4*>(p);
+  FeatVec<4> o; o.v[0] = r.x; o.v[1] = r.y; o.v[2] = r.z; o.v[3] = r.w;
+  return o;
 }
+__device__ __forceinline__ FeatVec<8> ld_feat(const bf16* p) {
+  const uint4 raw = *reinterpret_cast<const uint4*>(p);
+  const __nv_bfloat162* h = reinterpret_cast<const __nv_bfloat162*>(&raw);
+  FeatVec<8> o;
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const float2 f = __bfloat1622float2(h[i]);
+    o.v[2 * i] = f.x; o.v[2 * i + 1] = f.y;
+  }
+  return o;
+}
+template <typename T> struct VecOf;
+template <> struct VecOf<float> { static constexpr int value = 4; };
+template <> struct VecOf<bf16> { static constexpr int value = 8; };
 
 // One warp handles TOK tokens at a time and NE (>= N) logits per token, TOK * NE = 32
-// accumulators per lane.  Each lane covers 4 consecutive features per 128-feature step.
+// accumulators per lane.  Each lane covers VEC consecutive features (one 16-byte load of x)
+// per step of 32 * VEC features.
 template <typename T, int NE, int TOK>
 __global__ void __launch_bounds__(kWarpsPerBlock * 32)
 router_kernel(const T* __restrict__ x, const float* __restrict__ w_router, const float* __restrict__ bias,
               float* __restrict__ probs, int* __restrict__ expert_idx, float* __restrict__ gates,
               uint8_t* __restrict__ low_margin, int tokens, int d, int N, int k, int renorm) {
+  constexpr int VEC = VecOf<T>::value;
   const int lane = threadIdx.x & 31;
   const int warp = (blockIdx.x * kWarpsPerBlock) + (threadIdx.x >> 5);
   const int t0 = warp * TOK;
@@ -36,24 +51,26 @@ router_kernel(const T* __restrict__ x, const float* __restrict__ w_router, const
 #pragma unroll
     for (int e = 0; e < NE; ++e) acc[a][e] = 0.f;
 
-  for (int c = lane * 4; c < d; c += 128) {
-    float4 xv[TOK];
+  for (int c = lane * VEC; c < d; c += 32 * VEC) {
+    FeatVec<VEC> xv[TOK];
 #pragma unroll
     for (int a = 0; a < TOK; ++a) {
-      int t = t0 + a;
-      xv[a] = (t < tokens) ? ld4(x + (size_t)t * d + c) : make_float4(0.f, 0.f, 0.f, 0.f);
+      const int t = min(t0 + a, tokens - 1);       // rows past the end repeat the last token; never written
+      xv[a] = ld_feat(x + (size_t)t * d + c);
     }
 #pragma unroll
     for (int e = 0; e < NE; ++e) {
       if (e < N) {
-        float4 w = ld4(w_router + (size_t)e * d + c);
+        float w[VEC];
 #pragma unroll
-        for (int a = 0; a < TOK; ++a) {
-          acc[a][e] = fmaf(xv[a].x, w.x, acc[a][e]);
-          acc[a][e] = fmaf(xv[a].y, w.y, acc[a][e]);
-          acc[a][e] = fmaf(xv[a].z, w.z, acc[a][e]);
-          acc[a][e] = fmaf(xv[a].w, w.w, acc[a][e]);
+        for (int i = 0; i < VEC; i += 4) {
+          const float4 r = __ldg(reinterpret_cast<const float4*>(w_router + (size_t)e * d + c + i));
+          w[i] = r.x; w[i + 1] = r.y; w[i + 2] = r.z; w[i + 3] = r.w;
         }
+#pragma unroll
+        for (int a = 0; a < TOK; ++a)
+#pragma unroll
+          for (int i = 0; i < VEC; ++i) acc[a][e] = fmaf(xv[a].v[i], w[i], acc[a][e]);
       }
     }
   }
