@@ -218,14 +218,10 @@ def run_cuda(args):
     ws = B.alloc_workspace(shape, True)
     y = torch.empty(w.tokens, w.d_model, dtype=act, device="cuda")
     loss = torch.zeros(1, dtype=torch.float32, device="cuda")
-    gnames = ("d_a_gate", "d_b_gate", "d_a_up", "d_b_up", "d_a_down", "d_b_down", "d_w_router", "d_router_bias")
-    sizes = [int(np.prod(tensors[n[2:]].shape)) if n != "d_router_bias" else w.n_experts for n in gnames]
-    pad = [(s + 63) // 64 * 64 for s in sizes]
-    flat = torch.zeros(sum(pad), dtype=torch.float32, device="cuda")     # one buffer => one all-reduce
-    g, off = {}, 0
-    for n, s, p in zip(gnames, sizes, pad):
-        g[n] = flat[off:off + s]
-        off += p
+    from paper_2404_15159_b200 import dp
+    offsets, total = dp.flat_grad_layout(w.d_model, w.d_ff, w.n_experts, w.rank)
+    flat = torch.zeros(total, dtype=torch.float32, device="cuda")        # one buffer => one all-reduce
+    g = {n: flat[off:off + size] for n, (off, size) in offsets.items()}
     if want_dx:
         g["d_x"] = torch.empty(w.tokens, w.d_model, dtype=act, device="cuda")
     grads = B.make_grads(accumulate=0, **g)
