@@ -50,6 +50,13 @@ WsLayout ws_layout(const mixlora_shape_t& s) {
   L.bu_cat = take(f * N * r * E);
   L.Zg_pos = take(T * k * N * r * E);
   L.Zu_pos = take(T * k * N * r * E);
+  {
+    const size_t rp = r < 16 ? 16 : r;
+    L.zg_s = take(T * k * rp * E);
+    L.zu_s = take(T * k * rp * E);
+    L.bgp = take(N * f * 16 * E);
+    L.bup = take(N * f * 16 * E);
+  }
   L.h_sorted = take(T * k * f * E);
   L.hbar = take(T * f * E);
   L.total_fwd = off;
@@ -60,8 +67,12 @@ WsLayout ws_layout(const mixlora_shape_t& s) {
   L.dabar = take(T * f * E);
   L.dbbar = take(T * f * E);
   L.P_pos = take(T * k * N * r * E);
+  L.p_s = take(T * k * (r < 16 ? 16 : r) * E);
   L.dZd_pos = take(T * k * N * r * E);
-  L.dgate_part = take((size_t)fused_swiglu_bwd_col_tiles(s.d_ff) * T * k * 4);
+  {
+    const int a = fused_swiglu_bwd_col_tiles(s.d_ff), b = grouped_swiglu_bwd_col_tiles(s.d_ff);
+    L.dgate_part = take((size_t)(a > b ? a : b) * T * k * 4);
+  }
   L.dzg_all = take(T * k * N * r * E);
   L.dzu_all = take(T * k * N * r * E);
   L.dZg = take(T * N * r * E);
@@ -281,11 +292,17 @@ mixlora_status_t mixlora_ffn_forward(const mixlora_shape_t* shape, const mixlora
   }
   // per-slot LoRA-B expansion + SwiGLU
   {
-    StageScope ss(ST_LORA_B_SWIGLU, c.st, 4);
+    StageScope ss(ST_LORA_B_SWIGLU, c.st, 5);
     MIXLORA_CUDA(launch_bgu_cat(c));
     MIXLORA_CUDA(launch_zpos(c));
-    if (fused_swiglu_supported(c)) MIXLORA_CUDA(launch_fused_swiglu_fwd(c));
-    else MIXLORA_CUDA(launch_lora_b_swiglu(c));
+    if (grouped_swiglu_supported(c)) {
+      MIXLORA_CUDA(launch_zcompact(c));
+      MIXLORA_CUDA(launch_grouped_swiglu_fwd(c));
+    } else if (fused_swiglu_supported(c)) {
+      MIXLORA_CUDA(launch_fused_swiglu_fwd(c));
+    } else {
+      MIXLORA_CUDA(launch_lora_b_swiglu(c));
+    }
   }
   // zd = A_d h per slot, against every expert's A_d (the slot's own block is picked up by the combine)
   {
@@ -370,7 +387,10 @@ mixlora_status_t mixlora_ffn_backward(const mixlora_shape_t* shape, const mixlor
   {
     StageScope ss(ST_SWIGLU_BWD, c.st, 3);
     MIXLORA_CUDA(launch_slot_prep_bwd(c));
-    if (fused_swiglu_supported(c)) {
+    if (grouped_swiglu_supported(c)) {
+      MIXLORA_CUDA(launch_grouped_swiglu_bwd(c));
+      MIXLORA_CUDA(launch_dgate_reduce(c, grouped_swiglu_bwd_col_tiles(f)));
+    } else if (fused_swiglu_supported(c)) {
       MIXLORA_CUDA(launch_fused_swiglu_bwd(c));
       MIXLORA_CUDA(launch_dgate_reduce(c, fused_swiglu_bwd_col_tiles(f)));
     } else {

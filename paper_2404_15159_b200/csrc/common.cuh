@@ -41,6 +41,8 @@ struct WsLayout {
   size_t bd_cat;      // act [d, N*r]      s * B_d laid out [c][e*r + rr]
   size_t bg_cat, bu_cat;  // act [f, N*r]  s * B_g, s * B_u laid out [f'][e*r + rr]
   size_t Zg_pos, Zu_pos;  // act [T*k, N*r]  zg / zu of the slot in its expert block, zero elsewhere
+  size_t zg_s, zu_s;  // act [T*k, max(r,16)]  s * zg, s * zu of the slot's own expert, zero padded
+  size_t bgp, bup;    // act [N*f, 16]     B_g, B_u zero padded to 16 columns (used when r < 16)
   size_t h_sorted;    // act [T*k, f]
   size_t hbar;        // act [T, f]        sum_j g_j h_j
   size_t total_fwd;
@@ -49,6 +51,7 @@ struct WsLayout {
   size_t da_sorted, db_sorted;  // act [T*k, f]
   size_t dabar, dbbar;          // act [T, f]
   size_t P_pos;                 // act [T*k, N*r]  s * pd of the slot in its expert block, zero elsewhere
+  size_t p_s;                   // act [T*k, max(r,16)]  s * pd of the slot's own expert, zero padded
   size_t dZd_pos;               // act [T*k, N*r]  gate * P_pos
   size_t dgate_part;            // f32 [ceil(f/64), T*k]  per column tile partial <Dt, h> of the fused backward
   size_t dzg_all, dzu_all;      // act [T*k, N*r]  da (s B_g) and db (s B_u) against every expert
@@ -138,6 +141,11 @@ cudaError_t launch_bd_cat(const Ctx& c);
 cudaError_t launch_bgu_cat(const Ctx& c);              // bg_cat, bu_cat
 cudaError_t launch_zpos(const Ctx& c);                 // Zg_pos, Zu_pos
 cudaError_t launch_dgate_reduce(const Ctx& c, int col_tiles);   // dgate from dgate_part
+cudaError_t launch_zcompact(const Ctx& c);             // zg_s, zu_s (and bgp, bup when r < 16)
+bool grouped_swiglu_supported(const Ctx& c);
+int grouped_swiglu_bwd_col_tiles(int f);
+cudaError_t launch_grouped_swiglu_fwd(const Ctx& c);   // per-expert tiles, K = r (grouped_swiglu.cu)
+cudaError_t launch_grouped_swiglu_bwd(const Ctx& c);
 bool fused_swiglu_supported(const Ctx& c);
 int fused_swiglu_bwd_col_tiles(int f);
 cudaError_t launch_fused_swiglu_fwd(const Ctx& c);     // tensor-core version of lora_b_swiglu

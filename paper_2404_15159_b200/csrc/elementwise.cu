@@ -299,7 +299,7 @@ template <typename T>
 __global__ void slot_prep_bwd_kernel(const T* __restrict__ spd, const float* __restrict__ gates,
                                      const int* __restrict__ perm, const int* __restrict__ pos_token,
                                      const int* __restrict__ pos_expert, T* __restrict__ P_pos,
-                                     T* __restrict__ dZd_pos, int slots, int N, int r) {
+                                     T* __restrict__ dZd_pos, T* __restrict__ p_s, int slots, int N, int r, int rp) {
   const long long nr = (long long)N * r;
   const long long n = (long long)slots * nr;
   for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < n; i += (long long)gridDim.x * blockDim.x) {
@@ -312,6 +312,12 @@ __global__ void slot_prep_bwd_kernel(const T* __restrict__ spd, const float* __r
     }
     P_pos[i] = pv;
     dZd_pos[i] = from_f<T>(v);
+  }
+  // compact copy: the slot's own r values, zero padded to rp
+  const long long n2 = (long long)slots * rp;
+  for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < n2; i += (long long)gridDim.x * blockDim.x) {
+    const int pos = (int)(i / rp), cidx = (int)(i % rp);
+    p_s[i] = cidx < r ? spd[((size_t)pos_token[pos] * N + pos_expert[pos]) * r + cidx] : from_f<T>(0.f);
   }
 }
 
@@ -328,6 +334,36 @@ __global__ void zpos_kernel(const T* __restrict__ zga, const T* __restrict__ zua
     const size_t src = (size_t)pos_token[pos] * nr + q;
     Zg_pos[i] = own ? zga[src] : from_f<T>(0.f);
     Zu_pos[i] = own ? zua[src] : from_f<T>(0.f);
+  }
+}
+
+// zg_s[pos][c] = s * zga[token][e*r + c] for c < r, zero up to the padded width rp (same for zu_s)
+template <typename T>
+__global__ void zcompact_kernel(const T* __restrict__ zga, const T* __restrict__ zua, const int* __restrict__ pos_token,
+                                const int* __restrict__ pos_expert, T* __restrict__ zg_s, T* __restrict__ zu_s,
+                                int slots, int N, int r, int rp, float s) {
+  const long long n = (long long)slots * rp;
+  for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < n; i += (long long)gridDim.x * blockDim.x) {
+    const int pos = (int)(i / rp), cidx = (int)(i % rp);
+    float vg = 0.f, vu = 0.f;
+    if (cidx < r) {
+      const size_t src = ((size_t)pos_token[pos] * N + pos_expert[pos]) * r + cidx;
+      vg = s * to_f(zga[src]);
+      vu = s * to_f(zua[src]);
+    }
+    zg_s[i] = from_f<T>(vg);
+    zu_s[i] = from_f<T>(vu);
+  }
+}
+
+// out[row][c] = in[row][c] for c < r, zero up to 16 columns (rows = N * f)
+template <typename T>
+__global__ void pad16_kernel(const T* __restrict__ in, T* __restrict__ out, long long rows, int r) {
+  const long long n = rows * 16;
+  for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < n; i += (long long)gridDim.x * blockDim.x) {
+    const long long row = i / 16;
+    const int cidx = (int)(i % 16);
+    out[i] = cidx < r ? in[row * r + cidx] : from_f<T>(0.f);
   }
 }
 
@@ -477,6 +513,22 @@ cudaError_t zpos_t(const Ctx& c) {
 }
 
 template <typename T>
+cudaError_t zcompact_t(const Ctx& c) {
+  const int slots = c.s.tokens * c.s.top_k, r = c.s.rank, rp = r < 16 ? 16 : r;
+  zcompact_kernel<T><<<grid_for((long long)slots * rp, 256), 256, 0, c.st>>>(
+      c.at<T>(c.L.zga), c.at<T>(c.L.zua), c.at<int>(c.L.pos_token), c.at<int>(c.L.pos_expert), c.at<T>(c.L.zg_s),
+      c.at<T>(c.L.zu_s), slots, c.s.n_experts, r, rp, c.scale);
+  if (r < 16) {
+    const long long rows = (long long)c.s.n_experts * c.s.d_ff;
+    pad16_kernel<T><<<grid_for(rows * 16, 256), 256, 0, c.st>>>(reinterpret_cast<const T*>(c.p.b_gate),
+                                                               c.at<T>(c.L.bgp), rows, r);
+    pad16_kernel<T><<<grid_for(rows * 16, 256), 256, 0, c.st>>>(reinterpret_cast<const T*>(c.p.b_up), c.at<T>(c.L.bup),
+                                                               rows, r);
+  }
+  return cudaGetLastError();
+}
+
+template <typename T>
 cudaError_t lora_b_swiglu_t(const Ctx& c) {
   const int slots = c.s.tokens * c.s.top_k;
   const int blocks = (slots + SL - 1) / SL;
@@ -518,7 +570,8 @@ cudaError_t slot_prep_bwd_t(const Ctx& c) {
   const int slots = c.s.tokens * c.s.top_k;
   slot_prep_bwd_kernel<T><<<grid_for((long long)slots * c.s.rank * c.s.n_experts, 256), 256, 0, c.st>>>(
       c.at<T>(c.L.spd), c.at<float>(c.L.gates), c.at<int>(c.L.perm), c.at<int>(c.L.pos_token),
-      c.at<int>(c.L.pos_expert), c.at<T>(c.L.P_pos), c.at<T>(c.L.dZd_pos), slots, c.s.n_experts, c.s.rank);
+      c.at<int>(c.L.pos_expert), c.at<T>(c.L.P_pos), c.at<T>(c.L.dZd_pos), c.at<T>(c.L.p_s), slots, c.s.n_experts,
+      c.s.rank, c.s.rank < 16 ? 16 : c.s.rank);
   return cudaGetLastError();
 }
 
@@ -567,6 +620,7 @@ cudaError_t launch_combine_bwd(const Ctx& c, int want_dx) {
                                                         c.at<bf16>(c.L.dbbar), c.s.d_ff, c.s.top_k);
   return combine_bwd_t<bf16>(c, want_dx);
 }
+cudaError_t launch_zcompact(const Ctx& c) { return c.bf16 ? zcompact_t<bf16>(c) : zcompact_t<float>(c); }
 cudaError_t launch_zpos(const Ctx& c) { return c.bf16 ? zpos_t<bf16>(c) : zpos_t<float>(c); }
 cudaError_t launch_dgate_reduce(const Ctx& c, int col_tiles) {
   const int slots = c.s.tokens * c.s.top_k;

@@ -280,7 +280,7 @@ EncodeFn get_encode() {
 
 // 2-D bf16 tensor [rows, cols] row-major with leading dimension ld (elements); box = [box_rows, box_cols].
 bool encode_2d(CUtensorMap* map, const void* ptr, long long rows, long long cols, long long ld, int box_rows,
-               int box_cols) {
+               int box_cols, int swizzle_bytes = 128) {
   EncodeFn fn = get_encode();
   if (!fn) return false;
   cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
@@ -288,7 +288,10 @@ bool encode_2d(CUtensorMap* map, const void* ptr, long long rows, long long cols
   cuuint32_t box[2] = {(cuuint32_t)box_cols, (cuuint32_t)box_rows};
   cuuint32_t estr[2] = {1, 1};
   CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), dims, strides, box, estr,
-                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE,
+                  swizzle_bytes == 128 ? CU_TENSOR_MAP_SWIZZLE_128B
+                                       : (swizzle_bytes == 64 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_32B),
+                  CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   return r == CUDA_SUCCESS;
 }
@@ -298,8 +301,8 @@ int round_up(int v, int a) { return (v + a - 1) / a * a; }
 }  // namespace
 
 bool tc_encode_2d(CUtensorMap* map, const void* ptr, long long rows, long long cols, long long ld, int box_rows,
-                  int box_cols) {
-  return encode_2d(map, ptr, rows, cols, ld, box_rows, box_cols);
+                  int box_cols, int swizzle_bytes) {
+  return encode_2d(map, ptr, rows, cols, ld, box_rows, box_cols, swizzle_bytes);
 }
 
 bool tc_gemm_supported(int M, const TcOut* outs, int nout) {

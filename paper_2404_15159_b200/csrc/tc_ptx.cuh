@@ -105,14 +105,43 @@ __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.
 //   K-major  : rows of 128 bytes (64 bf16 along K); 8-row groups 1024 bytes apart (stride offset).
 //   MN-major : rows of 128 bytes (64 bf16 along N) per k; 8-k groups 1024 bytes apart (stride offset),
 //              64-column blocks `lbo_bytes` apart (leading offset).
-__device__ __forceinline__ uint64_t make_desc(uint32_t saddr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
+__device__ __forceinline__ uint64_t make_desc_mode(uint32_t saddr, uint32_t lbo_bytes, uint32_t sbo_bytes,
+                                                  uint32_t layout_type) {
   uint64_t d = 0;
   d |= (uint64_t)((saddr & 0x3FFFFu) >> 4);
   d |= (uint64_t)((lbo_bytes >> 4) & 0x3FFFu) << 16;
   d |= (uint64_t)((sbo_bytes >> 4) & 0x3FFFu) << 32;
   d |= (uint64_t)1 << 46;   // descriptor version of this architecture
-  d |= (uint64_t)2 << 61;   // 128-byte swizzle
+  d |= (uint64_t)layout_type << 61;
   return d;
+}
+__device__ __forceinline__ uint64_t make_desc(uint32_t saddr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
+  return make_desc_mode(saddr, lbo_bytes, sbo_bytes, 2);   // 128-byte swizzle
+}
+// K-major operand tile whose rows are `row_bytes` (32, 64 or 128) long and swizzled with the span of one row:
+// 8-row groups are 8 * row_bytes apart.  Layout-type codes: 128 B -> 2, 64 B -> 4, 32 B -> 6.
+__device__ __forceinline__ uint64_t make_desc_kmajor_rows(uint32_t saddr, uint32_t row_bytes) {
+  const uint32_t lt = row_bytes == 128 ? 2u : (row_bytes == 64 ? 4u : 6u);
+  return make_desc_mode(saddr, 16, 8 * row_bytes, lt);
+}
+
+// TMA tile store smem -> global (bulk async group of the issuing thread)
+__device__ __forceinline__ void tma_store_2d(const CUtensorMap* map, uint32_t src, int c0, int c1) {
+  asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];"
+               ::"l"(map), "r"(src), "r"(c0), "r"(c1)
+               : "memory");
+}
+__device__ __forceinline__ void tma_store_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+// waits until the smem sources of all but the newest `N` store groups of this thread have been read
+template <int N> __device__ __forceinline__ void tma_store_wait_read() {
+  asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory");
+}
+template <int N> __device__ __forceinline__ void tma_store_wait_all() {
+  asm volatile("cp.async.bulk.wait_group %0;" ::"n"(N) : "memory");
+}
+__device__ __forceinline__ void fence_proxy_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+__device__ __forceinline__ void named_barrier(int id, int threads) {
+  asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(threads) : "memory");
 }
 
 // Instruction descriptor: bf16 x bf16 -> fp32, M = 128, N = n, A K-major, B K-major or MN-major.
@@ -134,6 +163,6 @@ __device__ __forceinline__ uint32_t make_idesc(int n, int a_mn_major, int b_mn_m
 // Host: tensor map of a 2-D bf16 tensor [rows, cols], row-major with leading dimension ld (elements),
 // 128-byte swizzle, box = [box_rows, box_cols]; out-of-range elements read as zero.  False on failure.
 bool tc_encode_2d(CUtensorMap* map, const void* ptr, long long rows, long long cols, long long ld, int box_rows,
-                  int box_cols);
+                  int box_cols, int swizzle_bytes = 128);
 
 }  // namespace mixlora
