@@ -446,14 +446,12 @@ mixlora_status_t mixlora_ffn_backward(const mixlora_shape_t* shape, const mixlor
       outs[n] = tc_out_f32(grads->d_b_down, Nr, r, 1, r, (long long)d * r, c.scale, acc);
       tc_add(outs[n++], dy, d, T, c.ws + c.L.Zs, Nr, 1, 1);
     }
+    if (grads->d_w_router) {   // dW_r[i][c] = sum_t dl[t][i] x[t][c]
+      outs[n] = tc_out_f32(grads->d_w_router, N, 1, d, 0, 0, 1.f, acc);
+      tc_add(outs[n++], params->x, d, T, c.ws + c.L.dl_act, NP, 1, 1, NP);
+    }
     StageScope ss(ST_LORA_WGRAD, c.st, dense_launches(c, d, outs, n));
     MIXLORA_CUDA(dense_product(c, d, outs, n));
-  }
-  if (grads->d_w_router) {     // dW_r[i][c] = sum_t dl[t][i] x[t][c]
-    TcOut out = tc_out_f32(grads->d_w_router, N, 1, d, 0, 0, 1.f, acc);
-    tc_add(out, params->x, d, T, c.ws + c.L.dl_act, NP, 1, 1, NP);
-    StageScope ss(ST_ROUTER_BWD, c.st, dense_launches(c, d, &out, 1));
-    MIXLORA_CUDA(dense_product(c, d, &out, 1));
   }
   if (want_dx) {
     // dx = [dabar | dbbar | dZg | dZu | dl] [W_g ; W_u ; A_g ; A_u ; W_r]

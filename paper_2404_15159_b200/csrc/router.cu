@@ -6,7 +6,7 @@ namespace mixlora {
 
 namespace {
 
-constexpr int kWarpsPerBlock = 8;
+constexpr int kWarpsPerBlock = 4;
 constexpr float kMarginFlag = 1e-4f;
 
 // VEC consecutive features of one row as floats (16-byte load)
@@ -156,15 +156,15 @@ router_kernel(const T* __restrict__ x, const float* __restrict__ w_router, const
 }
 
 // F_i and P_i of Eq. 9, one block per expert, fixed summation order (deterministic).
-__global__ void __launch_bounds__(256)
+__global__ void __launch_bounds__(1024)
 router_stats_kernel(const float* __restrict__ probs, const int* __restrict__ expert_idx, float* __restrict__ F,
                     float* __restrict__ P, int tokens, int N, int k, int f_mode) {
-  __shared__ float sp[256];
-  __shared__ int sc[256];
+  __shared__ float sp[1024];
+  __shared__ int sc[1024];
   const int e = blockIdx.x;
   float ps = 0.f;
   int cnt = 0;
-  for (int t = threadIdx.x; t < tokens; t += 256) {
+  for (int t = threadIdx.x; t < tokens; t += 1024) {
     ps += probs[(size_t)t * N + e];
     if (f_mode == 0) {
       cnt += (expert_idx[(size_t)t * k] == e);
@@ -175,7 +175,7 @@ router_stats_kernel(const float* __restrict__ probs, const int* __restrict__ exp
   sp[threadIdx.x] = ps;
   sc[threadIdx.x] = cnt;
   __syncthreads();
-  for (int o = 128; o > 0; o >>= 1) {
+  for (int o = 512; o > 0; o >>= 1) {
     if (threadIdx.x < o) {
       sp[threadIdx.x] += sp[threadIdx.x + o];
       sc[threadIdx.x] += sc[threadIdx.x + o];
@@ -320,7 +320,7 @@ cudaError_t launch_router_t(const Ctx& c) {
         x, c.p.w_router, c.p.router_bias, probs, idx, gates, flags, s.tokens, s.d_model, s.n_experts, s.top_k, \
         s.renormalize);                                                                                        \
   }
-  if (s.n_experts <= 8) MIXLORA_ROUTER_LAUNCH(8, 4)
+  if (s.n_experts <= 8) MIXLORA_ROUTER_LAUNCH(8, 2)
   else if (s.n_experts <= 16) MIXLORA_ROUTER_LAUNCH(16, 2)
   else MIXLORA_ROUTER_LAUNCH(32, 1)
 #undef MIXLORA_ROUTER_LAUNCH
@@ -332,7 +332,7 @@ cudaError_t launch_router_t(const Ctx& c) {
 cudaError_t launch_router(const Ctx& c) {
   cudaError_t e = c.bf16 ? launch_router_t<bf16>(c) : launch_router_t<float>(c);
   if (e != cudaSuccess) return e;
-  router_stats_kernel<<<c.s.n_experts, 256, 0, c.st>>>(c.at<float>(c.L.probs), c.at<int>(c.L.expert_idx),
+  router_stats_kernel<<<c.s.n_experts, 1024, 0, c.st>>>(c.at<float>(c.L.probs), c.at<int>(c.L.expert_idx),
                                                        c.at<float>(c.L.stat_F), c.at<float>(c.L.stat_P), c.s.tokens,
                                                        c.s.n_experts, c.s.top_k, c.s.aux_f_mode);
   return cudaGetLastError();
