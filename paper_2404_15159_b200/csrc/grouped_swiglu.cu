@@ -38,7 +38,7 @@ struct alignas(64) GsParams {
   const int* pos_token; const int* perm; const float* gates; const int* tile_info;
   bf16* h; bf16* da; bf16* db;
   float* dgate_part;       // [col_tiles * kSplit, slots]
-  int max_tiles, slots, f, r, row_bytes, kblocks, ksteps, krows, col_tiles, nstages;
+  int max_tiles, slots, f, r, row_bytes, kblocks, ksteps, krows, col_tiles, nstages, out_sets;
   uint32_t stage_bytes, a_bytes;
   int* status;
 };
@@ -59,6 +59,13 @@ __device__ __forceinline__ uint4 pack8(const float* v) {
   r.x = *reinterpret_cast<uint32_t*>(&h0); r.y = *reinterpret_cast<uint32_t*>(&h1);
   r.z = *reinterpret_cast<uint32_t*>(&h2); r.w = *reinterpret_cast<uint32_t*>(&h3);
   return r;
+}
+// sigmoid(a) = 0.5 tanh(a / 2) + 0.5 with the hardware tanh approximation (one special-function op;
+// its error is below the bf16 rounding of every value stored from here)
+__device__ __forceinline__ float fast_sigmoid(float a) {
+  float t;
+  asm("tanh.approx.f32 %0, %1;" : "=f"(t) : "f"(0.5f * a));
+  return fmaf(t, 0.5f, 0.5f);
 }
 __device__ __forceinline__ void tmem_ld8(uint32_t taddr, uint32_t (&v)[8]) {
   asm volatile("tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
@@ -83,7 +90,7 @@ __global__ void __launch_bounds__(kThreads, 1) grouped_swiglu_kernel(const __gri
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   uint8_t* gather_smem = smem;                                    // two sets
   uint8_t* out_smem = gather_smem + 2 * kSetBytes;
-  uint8_t* stage_smem = out_smem + kOutBytes;
+  uint8_t* stage_smem = out_smem + p.out_sets * kOutBytes;          // one or two output tiles
   uint64_t* bars = reinterpret_cast<uint64_t*>(stage_smem + p.nstages * p.stage_bytes);
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * kMaxStages + 4);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
@@ -195,22 +202,32 @@ __global__ void __launch_bounds__(kThreads, 1) grouped_swiglu_kernel(const __gri
     const uint32_t gs_base = smem_u32(gather_smem);
     const uint32_t out_base = smem_u32(out_smem);
 
-    // cooperative gather of item w into `set`: thread -> (block, row, 16-byte chunk), 4 rows x 128 B per warp instruction
+    // Cooperative gather of item w into `set`.  Thread -> rows g_r0 and g_r0 + 64 of every 64-column block and the
+    // 16-byte chunk g_cb of those rows, so a warp instruction reads 4 rows x 128 contiguous bytes.  Everything
+    // that does not depend on the item is computed once here.
+    const int g_r0 = et >> 3, g_cb = et & 7;
+    const uint32_t g_dst0 = gs_base + g_r0 * 128 + ((g_cb ^ (g_r0 & 7)) << 4);
     auto gather = [&](int w, int set) {
       const int tile = w / p.col_tiles, col0 = (w % p.col_tiles) * COLS;
       const int p0 = p.tile_info[tile * 4 + 1], rows = p.tile_info[tile * 4 + 2];
+      const bool in0 = g_r0 < rows, in1 = g_r0 + 64 < rows;
+      const size_t row0 = (size_t)(in0 ? p.pos_token[p0 + g_r0] : 0) * p.f + col0 + g_cb * 8;
+      const size_t row1 = (size_t)(in1 ? p.pos_token[p0 + g_r0 + 64] : 0) * p.f + col0 + g_cb * 8;
+      const uint32_t dst_set = g_dst0 + set * kSetBytes;
 #pragma unroll
-      for (int i = 0; i < (NMAT * CB * 1024) / NET; ++i) {
-        const int idx = et + i * NET;
-        const int blk = idx >> 10, within = idx & 1023;
-        const int m = blk / CB, j = blk % CB;
-        const int rr = within >> 3, cb = within & 7;
-        const int col = col0 + j * 64 + cb * 8;
-        const bool in = rr < rows && col < p.f;
+      for (int m = 0; m < NMAT; ++m) {
         const bf16* base = m == 0 ? p.G : (m == 1 ? p.U : p.D);
-        const bf16* src = in ? base + (size_t)p.pos_token[p0 + rr] * p.f + col : base;
-        const uint32_t dst = gs_base + set * kSetBytes + blk * kBlockBytes + rr * 128 + ((cb ^ (rr & 7)) << 4);
-        asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(in ? 16 : 0) : "memory");
+#pragma unroll
+        for (int j = 0; j < CB; ++j) {
+          const bool cin = col0 + j * 64 + g_cb * 8 < p.f;
+          const uint32_t dst = dst_set + (m * CB + j) * kBlockBytes;
+          const bool a0 = in0 && cin, a1 = in1 && cin;
+          const bf16* s0 = a0 ? base + row0 + j * 64 : base;
+          const bf16* s1 = a1 ? base + row1 + j * 64 : base;
+          asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(s0), "r"(a0 ? 16 : 0) : "memory");
+          asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst + 64 * 128), "l"(s1), "r"(a1 ? 16 : 0)
+                       : "memory");
+        }
       }
       asm volatile("cp.async.commit_group;" ::: "memory");
     };
@@ -232,7 +249,10 @@ __global__ void __launch_bounds__(kThreads, 1) grouped_swiglu_kernel(const __gri
       if (w + (int)gridDim.x < total) gather(w + gridDim.x, set ^ 1);
       else asm volatile("cp.async.commit_group;" ::: "memory");
       asm volatile("cp.async.wait_group 1;" ::: "memory");
-      if (et == 0) tma_store_wait_read<0>();           // the previous item's stores have read the output tile
+      const int oidx = p.out_sets == 2 ? set : 0;      // output tile of this item
+      if (et == 0) {                                   // earlier stores have finished reading that tile
+        if (p.out_sets == 2) tma_store_wait_read<1>(); else tma_store_wait_read<0>();
+      }
       named_barrier(1, NET);                           // this item's gathers are visible; the output tile is free
 
       const bool got = __all_sync(0xffffffffu, mbar_wait(tfull_bar(buf), use & 1u, abort_flag));
@@ -240,59 +260,65 @@ __global__ void __launch_bounds__(kThreads, 1) grouped_swiglu_kernel(const __gri
         tc_fence_after();
         const uint32_t t_addr = tmem_base + ((uint32_t)(q * 32) << 16) + buf * kBufStride + part * WCOLS;
         const uint8_t* gset = gather_smem + set * kSetBytes;
+        uint8_t* oset = out_smem + oidx * kOutBytes;
+        // this thread's columns are chunks c8 = part * NCH + ch of the tile; all lie in one 64-column block
+        const int jblk = (part * NCH) >> 3, cb0 = (part * NCH) & 7, rx = row & 7;
+        const uint32_t row_off = jblk * kBlockBytes + row * 128;
         float dg = 0.f;
 #pragma unroll
-        for (int ch = 0; ch < NCH; ++ch) {
-          uint32_t va[8], vb[8], vd[8];
-          tmem_ld8(t_addr + ch * 8, va);
-          tmem_ld8(t_addr + COLS + ch * 8, vb);
-          if (BWD) tmem_ld8(t_addr + 2 * COLS + ch * 8, vd);
+        for (int c16 = 0; c16 < WCOLS; c16 += 16) {
+          uint32_t va[16], vb[16], vd[BWD ? 16 : 1];
+          tmem_ld16(t_addr + c16, va);
+          tmem_ld16(t_addr + COLS + c16, vb);
+          if (BWD) tmem_ld16(t_addr + 2 * COLS + c16, reinterpret_cast<uint32_t(&)[16]>(vd));
           tmem_ld_wait();
-          const int c8 = part * NCH + ch;              // 8-column chunk inside the tile
-          const int j = c8 >> 3, cb = c8 & 7;
-          const uint32_t off = j * kBlockBytes + row * 128 + ((cb ^ (row & 7)) << 4);
-          float gv[8], uv[8], hv[8];
-          unpack8(*reinterpret_cast<const uint4*>(gset + 0 * CB * kBlockBytes + off), gv);
-          unpack8(*reinterpret_cast<const uint4*>(gset + 1 * CB * kBlockBytes + off), uv);
-          const int col = col0 + c8 * 8;
-          const size_t gdst = (size_t)pos * p.f + col;
-          const bool direct = !full_tile && valid && col < p.f;
-          if (!BWD) {
 #pragma unroll
-            for (int i = 0; i < 8; ++i) {
-              const float a = gv[i] + __uint_as_float(va[i]);
-              const float b = uv[i] + __uint_as_float(vb[i]);
-              hv[i] = __fdividef(a, 1.f + __expf(-a)) * b;
-            }
-            const uint4 ho = pack8(hv);
-            if (full_tile) *reinterpret_cast<uint4*>(out_smem + off) = ho;
-            else if (direct) *reinterpret_cast<uint4*>(p.h + gdst) = ho;
-          } else {
-            float dv[8], dav[8], dbv[8];
-            unpack8(*reinterpret_cast<const uint4*>(gset + 2 * CB * kBlockBytes + off), dv);
+          for (int hh8 = 0; hh8 < 2; ++hh8) {
+            const int ch = c16 / 8 + hh8;
+            const uint32_t off = row_off + (((cb0 + ch) ^ rx) << 4);
+            float gv[8], uv[8], hv[8];
+            unpack8(*reinterpret_cast<const uint4*>(gset + 0 * CB * kBlockBytes + off), gv);
+            unpack8(*reinterpret_cast<const uint4*>(gset + 1 * CB * kBlockBytes + off), uv);
+            const int col = col0 + (part * NCH + ch) * 8;
+            const size_t gdst = (size_t)pos * p.f + col;
+            const bool direct = !full_tile && valid && col < p.f;
+            if (!BWD) {
 #pragma unroll
-            for (int i = 0; i < 8; ++i) {
-              const float a = gv[i] + __uint_as_float(va[i]);
-              const float b = uv[i] + __uint_as_float(vb[i]);
-              const float sg = __fdividef(1.f, 1.f + __expf(-a));
-              const float sa = a * sg;
-              const float hh = sa * b;
-              const float Dt = dv[i] + __uint_as_float(vd[i]);
-              dg = fmaf(Dt, hh, dg);
-              const float dh = gate * Dt;
-              hv[i] = hh;
-              dav[i] = dh * b * sg * (1.f + a * (1.f - sg));
-              dbv[i] = dh * sa;
-            }
-            const uint4 ho = pack8(hv), ao = pack8(dav), bo = pack8(dbv);
-            if (full_tile) {
-              *reinterpret_cast<uint4*>(out_smem + 0 * CB * kBlockBytes + off) = ho;
-              *reinterpret_cast<uint4*>(out_smem + 1 * CB * kBlockBytes + off) = ao;
-              *reinterpret_cast<uint4*>(out_smem + 2 * CB * kBlockBytes + off) = bo;
-            } else if (direct) {
-              *reinterpret_cast<uint4*>(p.h + gdst) = ho;
-              *reinterpret_cast<uint4*>(p.da + gdst) = ao;
-              *reinterpret_cast<uint4*>(p.db + gdst) = bo;
+              for (int i = 0; i < 8; ++i) {
+                const float a = gv[i] + __uint_as_float(va[hh8 * 8 + i]);
+                const float b = uv[i] + __uint_as_float(vb[hh8 * 8 + i]);
+                hv[i] = a * fast_sigmoid(a) * b;
+              }
+              const uint4 ho = pack8(hv);
+              if (full_tile) *reinterpret_cast<uint4*>(oset + off) = ho;
+              else if (direct) *reinterpret_cast<uint4*>(p.h + gdst) = ho;
+            } else {
+              float dv[8], dav[8], dbv[8];
+              unpack8(*reinterpret_cast<const uint4*>(gset + 2 * CB * kBlockBytes + off), dv);
+#pragma unroll
+              for (int i = 0; i < 8; ++i) {
+                const float a = gv[i] + __uint_as_float(va[hh8 * 8 + i]);
+                const float b = uv[i] + __uint_as_float(vb[hh8 * 8 + i]);
+                const float sg = fast_sigmoid(a);
+                const float sa = a * sg;
+                const float hh = sa * b;
+                const float Dt = dv[i] + __uint_as_float(vd[BWD ? hh8 * 8 + i : 0]);
+                dg = fmaf(Dt, hh, dg);
+                const float dh = gate * Dt;
+                hv[i] = hh;
+                dav[i] = dh * b * sg * (1.f + a * (1.f - sg));
+                dbv[i] = dh * sa;
+              }
+              const uint4 ho = pack8(hv), ao = pack8(dav), bo = pack8(dbv);
+              if (full_tile) {
+                *reinterpret_cast<uint4*>(oset + 0 * CB * kBlockBytes + off) = ho;
+                *reinterpret_cast<uint4*>(oset + 1 * CB * kBlockBytes + off) = ao;
+                *reinterpret_cast<uint4*>(oset + 2 * CB * kBlockBytes + off) = bo;
+              } else if (direct) {
+                *reinterpret_cast<uint4*>(p.h + gdst) = ho;
+                *reinterpret_cast<uint4*>(p.da + gdst) = ao;
+                *reinterpret_cast<uint4*>(p.db + gdst) = bo;
+              }
             }
           }
         }
@@ -312,9 +338,9 @@ __global__ void __launch_bounds__(kThreads, 1) grouped_swiglu_kernel(const __gri
         for (int m = 0; m < NOUT; ++m)
 #pragma unroll
           for (int j = 0; j < CB; ++j)
-            tma_store_2d(&p.o_map[m], out_base + (m * CB + j) * kBlockBytes, col0 + j * 64, p0);
-        tma_store_commit();
+            tma_store_2d(&p.o_map[m], out_base + oidx * kOutBytes + (m * CB + j) * kBlockBytes, col0 + j * 64, p0);
       }
+      if (et == 0) tma_store_commit();                 // one group per item, also when nothing was stored
       if (*epi_stop) break;                            // same value for every epilogue thread after the barrier
     }
     asm volatile("cp.async.wait_all;" ::: "memory");
@@ -348,8 +374,13 @@ cudaError_t launch_t(const Ctx& c) {
   p.a_bytes = 128 * p.row_bytes;
   const uint32_t b_bytes_k = COLS * p.row_bytes, b_bytes_n = CB * p.krows * 128;
   p.stage_bytes = (uint32_t)align_up(p.a_bytes + (b_bytes_k > b_bytes_n ? b_bytes_k : b_bytes_n), 1024);
-  const uint32_t fixed = 2 * NMAT * CB * kBlockBytes + NOUT * CB * kBlockBytes + 1024 + 256;
   const uint32_t budget = 227 * 1024;
+  p.out_sets = 2;
+  uint32_t fixed = 2 * NMAT * CB * kBlockBytes + 2 * NOUT * CB * kBlockBytes + 1024 + 256;
+  if (fixed + 2 * p.stage_bytes > budget) {            // wide operands: fall back to one output tile
+    p.out_sets = 1;
+    fixed -= NOUT * CB * kBlockBytes;
+  }
   int nst = (int)((budget - fixed) / p.stage_bytes);
   if (nst > kMaxStages) nst = kMaxStages;
   if (nst < 2) return cudaErrorInvalidConfiguration;
