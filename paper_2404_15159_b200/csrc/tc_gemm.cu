@@ -13,6 +13,8 @@
 // caller's status word, all roles leave their loops, and TMEM is released before exit.
 #include <cuda.h>
 
+#include <stdlib.h>
+
 #include <mutex>
 
 #include "common.cuh"
@@ -260,6 +262,224 @@ __global__ void __launch_bounds__(kThreads, 1) tc_gemm_kernel(const __grid_const
   }
 }
 
+// ---- CTA-pair variant ------------------------------------------------------------------------
+// Two CTAs of a cluster work on one 256 x tile_n output tile with cta_group::2 MMAs: each CTA stages its own 128 rows
+// of A and HALF of the B tile, so the operand bytes per CTA and k-block drop from 48 KB to 32 KB and the same shared
+// memory holds a 6-stage ring.  Protocol (no TMA multicast anywhere):
+//   - both CTAs allocate TMEM (cta_group::2) and run a producer warp; every load signals the LEADER's full barrier,
+//     on which the leader's producer has posted the byte count of both CTAs;
+//   - the leader's MMA thread issues the MMAs for the pair and multicast-commits onto both CTAs' empty barriers
+//     (stage free) and accumulator-full barriers;
+//   - each CTA's epilogue warps drain that CTA's 128 accumulator rows and arrive on the leader's accumulator-empty
+//     barrier through its cluster address;
+//   - a cluster barrier at the end keeps either CTA's smem and barriers alive until both are done.
+constexpr int kStages2 = 6;
+constexpr uint32_t kBBytes2 = 128 * BK * 2;              // half of a 256-column B tile
+constexpr uint32_t kStageBytes2 = kABytes + kBBytes2;    // 32 KiB
+constexpr uint32_t kSmemBytes2 = kStages2 * kStageBytes2 + 1024 + 256;
+
+__device__ __forceinline__ void store_chunk32(const TcParams& p, int o, int row, int n0c, const uint32_t (&v)[32]) {
+  const int No = p.N[o];
+  if (row >= p.M) return;
+  if (p.mode[o] == 1) {
+    float* base = reinterpret_cast<float*>(p.C[o]) + (size_t)row * p.ldc[o];
+    const int nb = p.nb[o];
+    const long long sn = p.s_n[o], sb = p.s_blk[o];
+    const float alpha = p.alpha[o];
+    const int accum = p.accumulate[o];
+#pragma unroll
+    for (int j = 0; j < 32; ++j) {
+      const int n = n0c + j;
+      if (n < No) {
+        float* dst = base + (nb > 0 ? (size_t)(n / nb) * sb + (size_t)(n % nb) * sn : (size_t)n * sn);
+        float val = alpha * __uint_as_float(v[j]);
+        if (accum) val += *dst;
+        *dst = val;
+      }
+    }
+  } else {
+    bf16* crow = reinterpret_cast<bf16*>(p.C[o]) + (size_t)row * p.ldc[o];
+#pragma unroll
+    for (int g8 = 0; g8 < 4; ++g8) {
+      const int col = n0c + g8 * 8;
+      if (col < No) {
+        uint4 q4;
+        __nv_bfloat162 h0 = __floats2bfloat162_rn(__uint_as_float(v[g8 * 8 + 0]), __uint_as_float(v[g8 * 8 + 1]));
+        __nv_bfloat162 h1 = __floats2bfloat162_rn(__uint_as_float(v[g8 * 8 + 2]), __uint_as_float(v[g8 * 8 + 3]));
+        __nv_bfloat162 h2 = __floats2bfloat162_rn(__uint_as_float(v[g8 * 8 + 4]), __uint_as_float(v[g8 * 8 + 5]));
+        __nv_bfloat162 h3 = __floats2bfloat162_rn(__uint_as_float(v[g8 * 8 + 6]), __uint_as_float(v[g8 * 8 + 7]));
+        q4.x = *reinterpret_cast<uint32_t*>(&h0);
+        q4.y = *reinterpret_cast<uint32_t*>(&h1);
+        q4.z = *reinterpret_cast<uint32_t*>(&h2);
+        q4.w = *reinterpret_cast<uint32_t*>(&h3);
+        *reinterpret_cast<uint4*>(crow + col) = q4;
+      }
+    }
+  }
+}
+
+template <int A_MN, int B_KN>
+__global__ void __launch_bounds__(kThreads, 1) tc_gemm_pair_kernel(const __grid_constant__ TcParams p) {
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + kStages2 * kStageBytes2);
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * kStages2 + 4);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const uint32_t rank = cluster_ctarank();               // 0 = leader of the pair
+  const bool leader = rank == 0;
+  const uint32_t smem_base = smem_u32(smem);
+  const uint32_t bar_base = smem_u32(bars);
+  auto full_bar = [&](int s) { return bar_base + 8u * s; };
+  auto empty_bar = [&](int s) { return bar_base + 8u * (kStages2 + s); };
+  auto tfull_bar = [&](int b) { return bar_base + 8u * (2 * kStages2 + b); };
+  auto tempty_bar = [&](int b) { return bar_base + 8u * (2 * kStages2 + 2 + b); };
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < kStages2; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
+    for (int b = 0; b < 2; ++b) { mbar_init(tfull_bar(b), 1); mbar_init(tempty_bar(b), 8); }   // 4 warps of each CTA
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 1) {
+    tmem_alloc_pair(smem_u32(tmem_slot), kTmemCols);
+    tmem_relinquish_pair();
+  }
+  tc_fence_before();
+  __syncthreads();
+  cluster_sync_all();                                    // the peer's barriers exist before anything signals them
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  int total_kb = 0;
+  for (int s = 0; s < p.nseg; ++s) total_kb += p.kblocks[s];
+  const int pair = blockIdx.x >> 1, npairs = gridDim.x >> 1;
+
+  if (warp == 0) {
+    // ---------------- TMA producer (both CTAs) ----------------
+    if (lane == 0) {
+      for (int s = 0; s < p.nseg * p.nout; ++s) { prefetch_tmap(&p.a_map[s]); prefetch_tmap(&p.b_map[s]); }
+      uint32_t it = 0;
+      bool ok = true;
+      for (int tile = pair; tile < p.total_tiles && ok; tile += npairs) {
+        const TileCoord tc = tile_coord(p, tile);        // m0 counts 256-row tiles here (m_tiles set by the host)
+        const int tn = p.tile_n[tc.o], half = tn >> 1;
+        const int m0 = tc.m0 * 2 + (int)rank * BM;
+        const int n0 = tc.n0 + (int)rank * half;
+        const uint32_t tx_pair = 2u * (kABytes + (uint32_t)half * BK * 2);
+        for (int sg = 0; sg < p.nseg && ok; ++sg) {
+          const CUtensorMap* am = &p.a_map[tc.o * p.nseg + sg];
+          const CUtensorMap* bm = &p.b_map[tc.o * p.nseg + sg];
+          for (int kb = 0; kb < p.kblocks[sg]; ++kb, ++it) {
+            const int st = it % kStages2;
+            const uint32_t ph = (it / kStages2) & 1u;
+            if (!mbar_wait(empty_bar(st), ph ^ 1u, abort_flag)) { ok = false; break; }
+            const uint32_t a_dst = smem_base + st * kStageBytes2;
+            const uint32_t b_dst = a_dst + kABytes;
+            const uint32_t lbar = map_to_cta(full_bar(st), 0);
+            if (leader) mbar_expect_tx(full_bar(st), tx_pair);
+            if (A_MN == 0) {
+              tma_load_2d_pair(a_dst, am, lbar, kb * BK, m0);
+            } else {
+              tma_load_2d_pair(a_dst, am, lbar, m0, kb * BK);
+              tma_load_2d_pair(a_dst + BK * 128, am, lbar, m0 + 64, kb * BK);
+            }
+            if (B_KN == 0) {
+              tma_load_2d_pair(b_dst, bm, lbar, kb * BK, n0);
+            } else {
+              for (int j = 0; j < half / 64; ++j)
+                tma_load_2d_pair(b_dst + j * (BK * 128), bm, lbar, n0 + j * 64, kb * BK);
+            }
+          }
+        }
+      }
+      if (!ok) {
+        *abort_flag = 1;
+        if (p.status) atomicExch(p.status, (int)MIXLORA_ERR_DEVICE_TIMEOUT);
+      }
+    }
+  } else if (warp == 1) {
+    // ---------------- MMA issuer (leader CTA only) ----------------
+    if (lane == 0 && leader) {
+      uint32_t it = 0, tcount = 0;
+      bool ok = true;
+      for (int tile = pair; tile < p.total_tiles && ok; tile += npairs, ++tcount) {
+        const TileCoord tc = tile_coord(p, tile);
+        const int tn = p.tile_n[tc.o];
+        const uint32_t idesc = make_idesc_m(2 * BM, tn, A_MN, B_KN);
+        const uint32_t buf = tcount & 1u;
+        const uint32_t use = tcount >> 1;
+        if (!mbar_wait(tempty_bar(buf), (use & 1u) ^ 1u, abort_flag)) { ok = false; break; }
+        tc_fence_after();
+        const uint32_t d_tmem = tmem_base + buf * BN_MAX;
+        for (int kb = 0; kb < total_kb; ++kb, ++it) {
+          const int st = it % kStages2;
+          const uint32_t ph = (it / kStages2) & 1u;
+          if (!mbar_wait(full_bar(st), ph, abort_flag)) { ok = false; break; }
+          tc_fence_after();
+          const uint32_t a_addr = smem_base + st * kStageBytes2;
+          const uint32_t b_addr = a_addr + kABytes;
+#pragma unroll
+          for (int k = 0; k < BK / UMMA_K; ++k) {
+            const uint64_t ad = (A_MN == 0) ? make_desc(a_addr + k * (UMMA_K * 2), 16, 1024)
+                                            : make_desc(a_addr + k * (UMMA_K * 128), BK * 128, 1024);
+            const uint64_t bd = (B_KN == 0) ? make_desc(b_addr + k * (UMMA_K * 2), 16, 1024)
+                                            : make_desc(b_addr + k * (UMMA_K * 128), BK * 128, 1024);
+            umma_bf16_pair(d_tmem, ad, bd, idesc, (kb | k) != 0);
+          }
+          umma_commit_pair(empty_bar(st), 3);            // frees the stage in both CTAs
+        }
+        if (ok) umma_commit_pair(tfull_bar(buf), 3);     // accumulator complete, for both CTAs' epilogues
+      }
+      if (!ok) {
+        *abort_flag = 1;
+        if (p.status) atomicExch(p.status, (int)MIXLORA_ERR_DEVICE_TIMEOUT);
+      }
+    }
+  } else {
+    // ---------------- epilogue (both CTAs, own 128 rows) ----------------
+    const int q = warp & 3;
+    uint32_t tcount = 0;
+    bool ok = true;
+    for (int tile = pair; tile < p.total_tiles && ok; tile += npairs, ++tcount) {
+      const TileCoord tc = tile_coord(p, tile);
+      const int tn = p.tile_n[tc.o];
+      const uint32_t buf = tcount & 1u;
+      const uint32_t use = tcount >> 1;
+      if (!__all_sync(0xffffffffu, mbar_wait(tfull_bar(buf), use & 1u, abort_flag))) { ok = false; break; }
+      tc_fence_after();
+      const int row = tc.m0 * 2 + (int)rank * BM + q * 32 + lane;
+      const uint32_t t_addr = tmem_base + ((uint32_t)(q * 32) << 16) + buf * BN_MAX;
+      for (int c = 0; c < tn; c += 32) {
+        uint32_t v[32];
+        tmem_ld32(t_addr + c, v);
+        tmem_ld_wait();
+        store_chunk32(p, tc.o, row, tc.n0 + c, v);
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive_cluster(map_to_cta(tempty_bar(buf), 0));   // 8 arrivals release the accumulator
+    }
+    if (!ok && lane == 0) {
+      *abort_flag = 1;
+      if (p.status) atomicExch(p.status, (int)MIXLORA_ERR_DEVICE_TIMEOUT);
+    }
+  }
+
+  __syncthreads();
+  if (*abort_flag) {
+    for (int i = 0; i < 200; ++i) __nanosleep(5000);     // let copies that may still be in flight land
+  }
+  tc_fence_before();
+  cluster_sync_all();                                    // neither CTA leaves while its peer may still touch it
+  tc_fence_after();
+  if (warp == 1) {
+    __syncwarp();
+    tmem_dealloc_pair(tmem_base, kTmemCols);
+  }
+}
+
 // ---- host side ------------------------------------------------------------------------------
 typedef CUresult (*EncodeFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
                              const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
@@ -340,33 +560,67 @@ cudaError_t launch_variant(const TcParams& p, int grid, cudaStream_t st) {
   return cudaGetLastError();
 }
 
+template <int A_MN, int B_KN>
+cudaError_t launch_pair_variant(const TcParams& p, int grid, cudaStream_t st) {
+  cudaError_t e = cudaFuncSetAttribute(tc_gemm_pair_kernel<A_MN, B_KN>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes2);
+  if (e != cudaSuccess) return e;
+  cudaLaunchConfig_t cfg;
+  memset(&cfg, 0, sizeof(cfg));
+  cfg.gridDim = dim3(grid, 1, 1);
+  cfg.blockDim = dim3(kThreads, 1, 1);
+  cfg.dynamicSmemBytes = kSmemBytes2;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = 2;
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, tc_gemm_pair_kernel<A_MN, B_KN>, p);
+}
+
+// CTA pairs are used whenever the problem has at least 256 rows; MIXLORA_TC_SINGLE=1 in the environment keeps the
+// single-CTA kernel for every shape (a measurement switch, read once)
+bool tc_force_single() {
+  static const bool v = [] {
+    const char* e = getenv("MIXLORA_TC_SINGLE");
+    return e && e[0] == '1';
+  }();
+  return v;
+}
+
 cudaError_t launch_tc_gemm(int M, const TcOut* outs, int nout, int* status_word, cudaStream_t st) {
   TcParams p;
   memset(&p, 0, sizeof(p));
   const int nseg = outs[0].nseg;
   const int a_mn = outs[0].seg[0].a_mn, b_kn = outs[0].seg[0].b_kn;
-  p.nseg = nseg; p.nout = nout; p.M = M; p.m_tiles = (M + BM - 1) / BM; p.status = status_word;
+  const bool pair = !tc_force_single() && M >= 2 * BM;
+  const int tile_m = pair ? 2 * BM : BM;
+  p.nseg = nseg; p.nout = nout; p.M = M; p.m_tiles = (M + tile_m - 1) / tile_m; p.status = status_word;
   for (int s = 0; s < nseg; ++s) p.kblocks[s] = (outs[0].seg[s].K + BK - 1) / BK;
   int tiles = 0;
   for (int o = 0; o < nout; ++o) {
     const TcOut& t = outs[o];
-    // the operand tile covers whole 16-column (K-major B) or 64-column (N-major B) groups; columns past N read as
-    // zero through the tensor map and are never stored
+    // the operand tile covers whole groups of columns (16 for a K-major B, 64 for an N-major B, per CTA); columns
+    // past N read as zero through the tensor map and are never stored
     const int cols = t.mode == 0 ? t.N : round_up(t.N, 8);
-    const int tn = b_kn ? (cols >= BN_MAX ? BN_MAX : round_up(cols, 64)) : (cols >= BN_MAX ? BN_MAX : round_up(cols, 16));
+    const int gran = (b_kn ? 64 : 16) * (pair ? 2 : 1);
+    const int tn = cols >= BN_MAX ? BN_MAX : round_up(cols, gran);
     p.C[o] = t.C; p.N[o] = t.N; p.tile_n[o] = tn;
     p.mode[o] = t.mode;
     p.ldc[o] = t.mode == 0 ? t.ldc : t.s_m;
     p.s_n[o] = t.s_n; p.s_blk[o] = t.s_blk; p.nb[o] = t.nb; p.alpha[o] = t.alpha; p.accumulate[o] = t.accumulate;
     p.tile_start[o] = tiles;
     tiles += p.m_tiles * ((t.N + tn - 1) / tn);
+    const int b_rows = pair ? tn / 2 : tn;               // rows of a K-major B tile held by one CTA
     for (int s = 0; s < nseg; ++s) {
       const TcSeg& g = t.seg[s];
       bool ok = a_mn ? encode_2d(&p.a_map[o * nseg + s], g.A, g.K, M, g.lda, BK, 64)
                      : encode_2d(&p.a_map[o * nseg + s], g.A, M, g.K, g.lda, BM, BK);
       if (!ok) return cudaErrorInvalidValue;
       ok = b_kn ? encode_2d(&p.b_map[o * nseg + s], g.B, g.K, g.b_cols > 0 ? g.b_cols : t.N, g.ldb, BK, 64)
-                : encode_2d(&p.b_map[o * nseg + s], g.B, g.b_cols > 0 ? g.b_cols : t.N, g.K, g.ldb, tn, BK);
+                : encode_2d(&p.b_map[o * nseg + s], g.B, g.b_cols > 0 ? g.b_cols : t.N, g.K, g.ldb, b_rows, BK);
       if (!ok) return cudaErrorInvalidValue;
     }
   }
@@ -376,6 +630,11 @@ cudaError_t launch_tc_gemm(int M, const TcOut* outs, int nout, int* status_word,
   int dev = 0, sms = 148;
   cudaGetDevice(&dev);
   cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  if (pair) {
+    const int pairs = tiles < sms / 2 ? tiles : sms / 2;
+    if (a_mn) return b_kn ? launch_pair_variant<1, 1>(p, 2 * pairs, st) : launch_pair_variant<1, 0>(p, 2 * pairs, st);
+    return b_kn ? launch_pair_variant<0, 1>(p, 2 * pairs, st) : launch_pair_variant<0, 0>(p, 2 * pairs, st);
+  }
   const int grid = tiles < sms ? tiles : sms;
   if (a_mn) return b_kn ? launch_variant<1, 1>(p, grid, st) : launch_variant<1, 0>(p, grid, st);
   return b_kn ? launch_variant<0, 1>(p, grid, st) : launch_variant<0, 0>(p, grid, st);
