@@ -362,7 +362,7 @@ def run_cuda(args):
         "router": T_ * d_ * E + N_ * d_ * 4 + T_ * N_ * 4 * 2,
         "lora_b_swiglu": (T_ * f_ * 2 + T_ * k_ * f_) * E,                      # G, U once per token + h per slot
         "combine_h": (T_ * k_ * f_ + T_ * f_) * E,
-        "swiglu_bwd": (T_ * f_ * 3 + T_ * k_ * f_ * 3) * E,                     # G, U, D once + h, da, db per slot
+        "swiglu_bwd": (T_ * f_ * 3 + T_ * k_ * f_ * 2) * E,                     # G, U, D once + da, db per slot
         "combine_bwd": (2 * T_ * k_ * f_ + 2 * T_ * f_) * E if want_dx else 0,
     }
     hbm = {n: {"gbs": round(bts / (stage_ms[n] * 1e-3) / 1e9, 1), "frac": round(bts / (stage_ms[n] * 1e-3) / 1e9 / peaks["hbm_gbs"], 3),

@@ -37,7 +37,7 @@ struct alignas(64) GsParams {
   const bf16* G; const bf16* U; const bf16* D;
   const int* pos_token; const int* perm; const float* gates; const int* tile_info;
   bf16* h; bf16* da; bf16* db;
-  float* dgate_part;       // [col_tiles * kSplit, slots]
+  float* dgate_part;       // [col_tiles, slots]
   int max_tiles, slots, f, r, row_bytes, kblocks, ksteps, krows, col_tiles, nstages, out_sets;
   uint32_t stage_bytes, a_bytes;
   int* status;
@@ -67,20 +67,14 @@ __device__ __forceinline__ float fast_sigmoid(float a) {
   asm("tanh.approx.f32 %0, %1;" : "=f"(t) : "f"(0.5f * a));
   return fmaf(t, 0.5f, 0.5f);
 }
-__device__ __forceinline__ void tmem_ld8(uint32_t taddr, uint32_t (&v)[8]) {
-  asm volatile("tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
-               : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7])
-               : "r"(taddr)
-               : "memory");
-}
-
 template <int BWD>
 __global__ void __launch_bounds__(kThreads, 1) grouped_swiglu_kernel(const __grid_constant__ GsParams p) {
   constexpr int COLS = BWD ? 64 : 128;
   constexpr int CB = COLS / 64;                        // 64-column blocks per tile
   constexpr int NSUB = BWD ? 3 : 2;                    // MMAs per item
   constexpr int NMAT = BWD ? 3 : 2;                    // gathered matrices G, U (, D)
-  constexpr int NOUT = BWD ? 3 : 1;                    // stored matrices h (, da, db)
+  constexpr int NOUT = BWD ? 2 : 1;                    // stored matrices: h forward; da, db backward (the forward's h
+                                                       // is still in the workspace and serves the A_d gradient)
   constexpr uint32_t kSetBytes = NMAT * CB * kBlockBytes;
   constexpr uint32_t kOutBytes = NOUT * CB * kBlockBytes;
   constexpr int WCOLS = COLS / kSplit;                 // columns per epilogue thread
@@ -91,7 +85,8 @@ __global__ void __launch_bounds__(kThreads, 1) grouped_swiglu_kernel(const __gri
   uint8_t* gather_smem = smem;                                    // two sets
   uint8_t* out_smem = gather_smem + 2 * kSetBytes;
   uint8_t* stage_smem = out_smem + p.out_sets * kOutBytes;          // one or two output tiles
-  uint64_t* bars = reinterpret_cast<uint64_t*>(stage_smem + p.nstages * p.stage_bytes);
+  float* dg_smem = reinterpret_cast<float*>(stage_smem + p.nstages * p.stage_bytes);   // [kSplit][128]
+  uint64_t* bars = reinterpret_cast<uint64_t*>(dg_smem + (BWD ? kSplit * BM : 0));
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * kMaxStages + 4);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
   volatile int* epi_stop = reinterpret_cast<volatile int*>(tmem_slot + 2);
@@ -305,17 +300,14 @@ __global__ void __launch_bounds__(kThreads, 1) grouped_swiglu_kernel(const __gri
                 const float Dt = dv[i] + __uint_as_float(vd[BWD ? hh8 * 8 + i : 0]);
                 dg = fmaf(Dt, hh, dg);
                 const float dh = gate * Dt;
-                hv[i] = hh;
                 dav[i] = dh * b * sg * (1.f + a * (1.f - sg));
                 dbv[i] = dh * sa;
               }
-              const uint4 ho = pack8(hv), ao = pack8(dav), bo = pack8(dbv);
+              const uint4 ao = pack8(dav), bo = pack8(dbv);
               if (full_tile) {
-                *reinterpret_cast<uint4*>(oset + 0 * CB * kBlockBytes + off) = ho;
-                *reinterpret_cast<uint4*>(oset + 1 * CB * kBlockBytes + off) = ao;
-                *reinterpret_cast<uint4*>(oset + 2 * CB * kBlockBytes + off) = bo;
+                *reinterpret_cast<uint4*>(oset + 0 * CB * kBlockBytes + off) = ao;
+                *reinterpret_cast<uint4*>(oset + 1 * CB * kBlockBytes + off) = bo;
               } else if (direct) {
-                *reinterpret_cast<uint4*>(p.h + gdst) = ho;
                 *reinterpret_cast<uint4*>(p.da + gdst) = ao;
                 *reinterpret_cast<uint4*>(p.db + gdst) = bo;
               }
@@ -325,7 +317,7 @@ __global__ void __launch_bounds__(kThreads, 1) grouped_swiglu_kernel(const __gri
         tc_fence_before();
         __syncwarp();
         if (lane == 0) mbar_arrive(tempty_bar(buf));
-        if (BWD && valid) p.dgate_part[(size_t)(ct * kSplit + part) * p.slots + pos] = dg;
+        if (BWD) dg_smem[part * BM + row] = dg;
       } else if (lane == 0) {
         *abort_flag = 1;
         if (p.status) atomicExch(p.status, (int)MIXLORA_ERR_DEVICE_TIMEOUT);
@@ -341,6 +333,12 @@ __global__ void __launch_bounds__(kThreads, 1) grouped_swiglu_kernel(const __gri
             tma_store_2d(&p.o_map[m], out_base + oidx * kOutBytes + (m * CB + j) * kBlockBytes, col0 + j * 64, p0);
       }
       if (et == 0) tma_store_commit();                 // one group per item, also when nothing was stored
+      if (BWD && got && part == 0 && valid) {          // the row's partial <Dt, h> over this column tile, fixed order
+        float sdg = 0.f;
+#pragma unroll
+        for (int pp = 0; pp < kSplit; ++pp) sdg += dg_smem[pp * BM + row];
+        p.dgate_part[(size_t)ct * p.slots + pos] = sdg;
+      }
       if (*epi_stop) break;                            // same value for every epilogue thread after the barrier
     }
     asm volatile("cp.async.wait_all;" ::: "memory");
@@ -362,7 +360,7 @@ template <int BWD>
 cudaError_t launch_t(const Ctx& c) {
   constexpr int COLS = BWD ? 64 : 128;
   constexpr int CB = COLS / 64;
-  constexpr int NMAT = BWD ? 3 : 2, NOUT = BWD ? 3 : 1;
+  constexpr int NMAT = BWD ? 3 : 2, NOUT = BWD ? 2 : 1;
   const int slots = c.s.tokens * c.s.top_k, f = c.s.d_ff, r = c.s.rank, N = c.s.n_experts;
   const int rp = r < 16 ? 16 : r;
   GsParams p;
@@ -376,7 +374,7 @@ cudaError_t launch_t(const Ctx& c) {
   p.stage_bytes = (uint32_t)align_up(p.a_bytes + (b_bytes_k > b_bytes_n ? b_bytes_k : b_bytes_n), 1024);
   const uint32_t budget = 227 * 1024;
   p.out_sets = 2;
-  uint32_t fixed = 2 * NMAT * CB * kBlockBytes + 2 * NOUT * CB * kBlockBytes + 1024 + 256;
+  uint32_t fixed = 2 * NMAT * CB * kBlockBytes + 2 * NOUT * CB * kBlockBytes + (BWD ? kSplit * BM * 4 : 0) + 1024 + 256;
   if (fixed + 2 * p.stage_bytes > budget) {            // wide operands: fall back to one output tile
     p.out_sets = 1;
     fixed -= NOUT * CB * kBlockBytes;
@@ -398,8 +396,8 @@ cudaError_t launch_t(const Ctx& c) {
   if (BWD)
     ok = ok && tc_encode_2d(&p.a_map[2], c.ws + c.L.p_s, slots, rp, rp, BM, kbc, p.row_bytes) &&
          tc_encode_2d(&p.b_map[2], c.p.a_down, (long long)N * r, f, f, p.krows, 64, 128) &&
-         tc_encode_2d(&p.o_map[1], c.ws + c.L.da_sorted, slots, f, f, BM, 64, 128) &&
-         tc_encode_2d(&p.o_map[2], c.ws + c.L.db_sorted, slots, f, f, BM, 64, 128);
+         tc_encode_2d(&p.o_map[0], c.ws + c.L.da_sorted, slots, f, f, BM, 64, 128) &&
+         tc_encode_2d(&p.o_map[1], c.ws + c.L.db_sorted, slots, f, f, BM, 64, 128);
   if (!ok) return cudaErrorInvalidValue;
   p.G = c.at<bf16>(c.L.G); p.U = c.at<bf16>(c.L.U); p.D = c.at<bf16>(c.L.D);
   p.pos_token = c.at<int>(c.L.pos_token); p.perm = c.at<int>(c.L.perm); p.gates = c.at<float>(c.L.gates);
@@ -427,7 +425,7 @@ bool grouped_swiglu_supported(const Ctx& c) {
   const int r = c.s.rank;
   return c.bf16 && c.s.tokens > 0 && (r == 8 || r == 16 || r == 32 || r == 64 || r == 128);
 }
-int grouped_swiglu_bwd_col_tiles(int f) { return (f + 63) / 64 * kSplit; }
+int grouped_swiglu_bwd_col_tiles(int f) { return (f + 63) / 64; }
 cudaError_t launch_grouped_swiglu_fwd(const Ctx& c) { return launch_t<0>(c); }
 cudaError_t launch_grouped_swiglu_bwd(const Ctx& c) { return launch_t<1>(c); }
 
