@@ -59,6 +59,8 @@ WsLayout ws_layout(const mixlora_shape_t& s) {
   }
   L.h_sorted = take(T * k * f * E);
   L.hbar = take(T * f * E);
+  L.work_count = take(8 * 4);
+  L.work_rows1 = take((size_t)rows_worklist_max(s.tokens * s.top_k, s.n_experts, 1) * 32);
   L.total_fwd = off;
   L.D = take(T * f * E);
   L.spd = take(T * N * r * E);
@@ -81,6 +83,8 @@ WsLayout ws_layout(const mixlora_shape_t& s) {
   L.dlogits = take(T * N * 4);
   L.dl_act = take(T * NP * E);
   L.wr_act = take(NP * d * E);
+  L.work_rows2 = take((size_t)rows_worklist_max(s.tokens * s.top_k, s.n_experts, 2) * 32);
+  L.work_red = take((size_t)reduce_worklist_max(s.d_ff, s.n_experts, 3) * 32);
   L.total_bwd = off;
   return L;
 }
@@ -183,9 +187,10 @@ void add_seg(SGemm& g, const SOperand& A, const SOperand& B, int K) {
 }
 
 // Dense product on the tensor-core kernel when it takes the shape, else on the SIMT kernel.
-cudaError_t dense_product(const Ctx& c, int M, const TcOut* outs, int nout) {
+cudaError_t dense_product(const Ctx& c, int M, const TcOut* outs, int nout, const TcWork* wl = nullptr) {
   if (nout == 0 || M <= 0) return cudaSuccess;
-  if (c.bf16 && tc_gemm_supported(M, outs, nout)) return launch_tc_gemm(M, outs, nout, c.at<int>(c.L.status), c.st);
+  if (c.bf16 && tc_gemm_supported(M, outs, nout))
+    return launch_tc_gemm(M, outs, nout, c.at<int>(c.L.status), c.st, wl);   // the SIMT kernel below computes every block
   for (int o = 0; o < nout; ++o) {
     const TcOut& t = outs[o];
     SGemm g = t.mode == 0 ? sgemm_base(c, t.C, t.ldc, 1, c.bf16, M, t.N) : sgemm_base(c, t.C, t.s_m, t.s_n, 0, M, t.N);
@@ -308,8 +313,12 @@ mixlora_status_t mixlora_ffn_forward(const mixlora_shape_t* shape, const mixlora
   {
     TcOut out = tc_out(c.ws + c.L.zd_all, Nr, Nr);
     tc_add(out, c.ws + c.L.h_sorted, f, f, params->a_down, f, 0);
-    StageScope ss(ST_LORA_A_DOWN, c.st, dense_launches(c, T * k, &out, 1));
-    MIXLORA_CUDA(dense_product(c, T * k, &out, 1));
+    StageScope ss(ST_LORA_A_DOWN, c.st, 1 + dense_launches(c, T * k, &out, 1));
+    // only the block of a slot's own expert is needed: schedule (row tile, expert) pairs that exist
+    TcWork wl = {c.at<int>(c.L.work_rows1), c.at<int>(c.L.work_count) + 0, rows_worklist_max(T * k, N, 1), r};
+    MIXLORA_CUDA(launch_rows_worklist(c, tc_gemm_tile_rows(T * k), 1, (f + 63) / 64, c.at<int>(c.L.work_rows1),
+                                      c.at<int>(c.L.work_count) + 0));
+    MIXLORA_CUDA(dense_product(c, T * k, &out, 1, &wl));
   }
   { StageScope ss(ST_COMBINE_H, c.st, c.bf16 ? 3 : 2); MIXLORA_CUDA(launch_combine_h(c)); MIXLORA_CUDA(launch_bd_cat(c)); }
   // y = [hbar | Zs] [W_d | s B_d]^T : the frozen down projection acts once on the gate-weighted sum of a
@@ -402,8 +411,11 @@ mixlora_status_t mixlora_ffn_backward(const mixlora_shape_t* shape, const mixlor
     TcOut outs[2];
     outs[0] = tc_out(c.ws + c.L.dzg_all, Nr, Nr); tc_add(outs[0], c.ws + c.L.da_sorted, f, f, c.ws + c.L.bg_cat, Nr, 1);
     outs[1] = tc_out(c.ws + c.L.dzu_all, Nr, Nr); tc_add(outs[1], c.ws + c.L.db_sorted, f, f, c.ws + c.L.bu_cat, Nr, 1);
-    StageScope ss(ST_LORA_DZ, c.st, dense_launches(c, T * k, outs, 2));
-    MIXLORA_CUDA(dense_product(c, T * k, outs, 2));
+    StageScope ss(ST_LORA_DZ, c.st, 1 + dense_launches(c, T * k, outs, 2));
+    TcWork wl = {c.at<int>(c.L.work_rows2), c.at<int>(c.L.work_count) + 1, rows_worklist_max(T * k, N, 2), r};
+    MIXLORA_CUDA(launch_rows_worklist(c, tc_gemm_tile_rows(T * k), 2, (f + 63) / 64, c.at<int>(c.L.work_rows2),
+                                      c.at<int>(c.L.work_count) + 1));
+    MIXLORA_CUDA(dense_product(c, T * k, outs, 2, &wl));
   }
   // router: gates -> probabilities -> logits
   {
@@ -427,8 +439,14 @@ mixlora_status_t mixlora_ffn_backward(const mixlora_shape_t* shape, const mixlor
       outs[n] = tc_out_f32(grads->d_a_down, Nr, 1, f, 0, 0, 1.f, acc);
       tc_add(outs[n++], c.ws + c.L.h_sorted, f, T * k, c.ws + c.L.dZd_pos, Nr, 1, 1);
     }
-    StageScope ss(ST_LORA_WGRAD, c.st, dense_launches(c, f, outs, n));
-    MIXLORA_CUDA(dense_product(c, f, outs, n));
+    StageScope ss(ST_LORA_WGRAD, c.st, 1 + dense_launches(c, f, outs, n));
+    if (n > 0) {
+      // each expert's block is a sum over that expert's segment of sorted slots only
+      TcWork wl = {c.at<int>(c.L.work_red), c.at<int>(c.L.work_count) + 2, reduce_worklist_max(f, N, n), r};
+      MIXLORA_CUDA(launch_reduce_worklist(c, f, tc_gemm_tile_rows(f), n, c.at<int>(c.L.work_red),
+                                          c.at<int>(c.L.work_count) + 2));
+      MIXLORA_CUDA(dense_product(c, f, outs, n, &wl));
+    }
   }
   // ... and over the tokens (d-sized matrices and the router weight)
   {

@@ -45,6 +45,8 @@ struct WsLayout {
   size_t bgp, bup;    // act [N*f, 16]     B_g, B_u zero padded to 16 columns (used when r < 16)
   size_t h_sorted;    // act [T*k, f]
   size_t hbar;        // act [T, f]        sum_j g_j h_j
+  size_t work_count;  // i32 [8]  item counts of the work lists below
+  size_t work_rows1;  // i32 [.., 8]  rows list with one output (A_d h)
   size_t total_fwd;
   size_t D;           // act [T, f]        dy W_d
   size_t spd;         // act [T, N*r]      s * B_d^T dy for every expert
@@ -60,6 +62,8 @@ struct WsLayout {
   size_t dlogits;     // f32 [T, N]
   size_t dl_act;      // act [T, NP]       dlogits in the activation type, NP = N rounded up to 8
   size_t wr_act;      // act [NP, d]       router weight in the activation type
+  size_t work_rows2;  // i32 [.., 8]  rows list with two outputs (da sB_g, db sB_u)
+  size_t work_red;    // i32 [.., 8]  reduce list of the f-sized weight gradients
   size_t total_bwd;
 };
 
@@ -175,7 +179,27 @@ struct TcOut {
   int mode; long long s_m, s_n, s_blk; int nb; float alpha; int accumulate;
   TcSeg seg[kMaxKSeg]; int nseg;
 };
+// Optional block-sparse schedule built on the device from the segment offsets (router.cu): only the listed
+// (row tile, column block) items are computed, each with its own range of 64-deep reduction blocks and its own
+// window of stored columns.  Items are 8 ints {output, m0, n0, kb_begin, kb_end, n_lo, n_hi, 0}.
+struct TcWork {
+  const int* items;   // device
+  const int* count;   // device, number of items
+  int max_items;      // bound used to size the launch
+  int block_cols;     // columns of one block (the LoRA rank)
+};
 bool tc_gemm_supported(int M, const TcOut* outs, int nout);
-cudaError_t launch_tc_gemm(int M, const TcOut* outs, int nout, int* status_word, cudaStream_t st);
+int tc_gemm_tile_rows(int M);   // rows of the tiles the tensor-core kernel will use for a problem with M rows
+cudaError_t launch_tc_gemm(int M, const TcOut* outs, int nout, int* status_word, cudaStream_t st,
+                           const TcWork* wl = nullptr);
+// Work lists over the sorted slots (need seg_off of the dispatch step):
+//   rows list : for every tile of `tile_rows` sorted slots and every expert with slots in it, `nout` items that
+//               compute that expert's block of r columns for the tile's rows (all k-blocks);
+//   reduce list: for every output, expert and tile of `tile_rows` output rows, one item whose reduction runs over
+//               the k-blocks that touch the expert's segment of sorted slots.
+cudaError_t launch_rows_worklist(const Ctx& c, int tile_rows, int nout, int kblocks, int* items, int* count);
+cudaError_t launch_reduce_worklist(const Ctx& c, int out_rows, int tile_rows, int nout, int* items, int* count);
+static inline int rows_worklist_max(int slots, int N, int nout) { return ((slots + kSegTile - 1) / kSegTile + N) * nout; }
+static inline int reduce_worklist_max(int out_rows, int N, int nout) { return ((out_rows + kSegTile - 1) / kSegTile) * N * nout; }
 
 }  // namespace mixlora

@@ -304,6 +304,40 @@ dispatch_scatter_kernel(const int* __restrict__ expert_idx, const int* __restric
   }
 }
 
+// ---- work lists for the block-sparse dense products ------------------------------------------
+__global__ void rows_worklist_kernel(const int* __restrict__ seg_off, int N, int slots, int tile_rows, int r, int nout,
+                                     int kblocks, int max_items, int* __restrict__ items, int* __restrict__ count) {
+  const int m_tiles = (slots + tile_rows - 1) / tile_rows;
+  const int idx = blockIdx.x * blockDim.x + threadIdx.x;
+  if (idx >= m_tiles * N) return;
+  const int mt = idx / N, e = idx % N;
+  const int lo = mt * tile_rows, hi = min(lo + tile_rows, slots);
+  const int sb = seg_off[e], se = seg_off[e + 1];
+  if (se <= sb || se <= lo || sb >= hi) return;            // expert e has no slot in this tile
+  const int at = atomicAdd(count, nout);                   // the order of items does not affect any result
+  if (at + nout > max_items) return;
+  for (int o = 0; o < nout; ++o) {
+    int* it = items + (size_t)(at + o) * 8;
+    it[0] = o; it[1] = lo; it[2] = e * r; it[3] = 0; it[4] = kblocks; it[5] = e * r; it[6] = e * r + r; it[7] = 0;
+  }
+}
+
+__global__ void reduce_worklist_kernel(const int* __restrict__ seg_off, int N, int out_rows, int tile_rows, int r,
+                                       int nout, int* __restrict__ items, int* __restrict__ count) {
+  const int m_tiles = (out_rows + tile_rows - 1) / tile_rows;
+  const int total = nout * N * m_tiles;
+  const int idx = blockIdx.x * blockDim.x + threadIdx.x;
+  if (idx == 0) *count = total;
+  if (idx >= total) return;
+  // tile index fastest, then expert, then output: neighbouring CTAs work on the same expert's operand rows
+  const int mt = idx % m_tiles, e = (idx / m_tiles) % N, o = idx / (m_tiles * N);
+  const int sb = seg_off[e], se = seg_off[e + 1];
+  int* it = items + (size_t)idx * 8;
+  it[0] = o; it[1] = mt * tile_rows; it[2] = e * r;
+  it[3] = sb / 64; it[4] = se > sb ? (se + 63) / 64 : sb / 64;   // k-blocks that touch the segment (none if empty)
+  it[5] = e * r; it[6] = e * r + r; it[7] = 0;
+}
+
 template <typename T>
 cudaError_t launch_router_t(const Ctx& c) {
   const mixlora_shape_t& s = c.s;
@@ -351,6 +385,25 @@ cudaError_t launch_dispatch(const Ctx& c) {
                                                                 c.at<int>(c.L.inv), c.at<int>(c.L.pos_token),
                                                                 c.at<int>(c.L.pos_expert), s.tokens, s.n_experts,
                                                                 s.top_k);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_rows_worklist(const Ctx& c, int tile_rows, int nout, int kblocks, int* items, int* count) {
+  const int slots = c.s.tokens * c.s.top_k, N = c.s.n_experts;
+  const int m_tiles = (slots + tile_rows - 1) / tile_rows;
+  cudaError_t e = cudaMemsetAsync(count, 0, sizeof(int), c.st);
+  if (e != cudaSuccess) return e;
+  const int n = m_tiles * N;
+  rows_worklist_kernel<<<(n + 255) / 256, 256, 0, c.st>>>(c.at<int>(c.L.seg_off), N, slots, tile_rows, c.s.rank, nout,
+                                                         kblocks, rows_worklist_max(slots, N, nout), items, count);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_reduce_worklist(const Ctx& c, int out_rows, int tile_rows, int nout, int* items, int* count) {
+  const int N = c.s.n_experts;
+  const int n = nout * N * ((out_rows + tile_rows - 1) / tile_rows);
+  reduce_worklist_kernel<<<(n + 255) / 256, 256, 0, c.st>>>(c.at<int>(c.L.seg_off), N, out_rows, tile_rows, c.s.rank,
+                                                           nout, items, count);
   return cudaGetLastError();
 }
 

@@ -51,23 +51,82 @@ struct alignas(64) TcParams {
   int tile_n[kMaxOut];
   int tile_start[kMaxOut + 1];     // first tile index of each output
   int kblocks[kMaxSeg];
-  int nseg, nout, M, m_tiles, total_tiles;
+  int nseg, nout, M, m_tiles, total_tiles, tile_m;
+  // Optional device-built work list (block-sparse schedule over the sorted slots): item = 8 ints
+  // {output, m0, n0, first k-block, end k-block, first stored column, end stored column, 0}; *work_count items.
+  const int* work;
+  const int* work_count;
   int* status;
 };
 
-struct TileCoord { int o, m0, n0; };
+struct TileCoord { int o, m0, n0, kb0, kb1, n_lo, n_hi; };
+
+__device__ __forceinline__ int tile_total(const TcParams& p) {
+  if (!p.work) return p.total_tiles;
+  const int n = *p.work_count;
+  return n < p.total_tiles ? n : p.total_tiles;
+}
 
 __device__ __forceinline__ TileCoord tile_coord(const TcParams& p, int tile) {
+  TileCoord t;
+  if (p.work) {
+    const int4 a = *reinterpret_cast<const int4*>(p.work + (size_t)tile * 8);
+    const int4 b = *reinterpret_cast<const int4*>(p.work + (size_t)tile * 8 + 4);
+    t.o = a.x; t.m0 = a.y; t.n0 = a.z; t.kb0 = a.w; t.kb1 = b.x; t.n_lo = b.y; t.n_hi = b.z;
+    return t;
+  }
   int o = 0;
 #pragma unroll
   for (int i = 1; i < kMaxOut; ++i)
     if (i < p.nout && tile >= p.tile_start[i]) o = i;
   const int local = tile - p.tile_start[o];
-  TileCoord t;
   t.o = o;
-  t.m0 = (local % p.m_tiles) * BM;       // rows fastest: neighbouring CTAs share the B tile
+  t.m0 = (local % p.m_tiles) * p.tile_m;  // rows fastest: neighbouring CTAs share the B tile
   t.n0 = (local / p.m_tiles) * p.tile_n[o];
+  t.kb0 = 0; t.kb1 = -1;                  // all k-blocks of every segment
+  t.n_lo = 0; t.n_hi = p.N[o];
   return t;
+}
+
+// Stores 32 accumulator columns [n0c, n0c + 32) of one row; only columns inside [n_lo, n_hi) are written.
+__device__ __forceinline__ void store_chunk32(const TcParams& p, int o, int row, int n0c, int n_lo, int n_hi,
+                                              const uint32_t (&v)[32]) {
+  if (row >= p.M) return;
+  if (p.mode[o] == 1) {
+    float* base = reinterpret_cast<float*>(p.C[o]) + (size_t)row * p.ldc[o];
+    const int nb = p.nb[o];
+    const long long sn = p.s_n[o], sb = p.s_blk[o];
+    const float alpha = p.alpha[o];
+    const int accum = p.accumulate[o];
+#pragma unroll
+    for (int j = 0; j < 32; ++j) {
+      const int n = n0c + j;
+      if (n >= n_lo && n < n_hi) {
+        float* dst = base + (nb > 0 ? (size_t)(n / nb) * sb + (size_t)(n % nb) * sn : (size_t)n * sn);
+        float val = alpha * __uint_as_float(v[j]);
+        if (accum) val += *dst;
+        *dst = val;
+      }
+    }
+  } else {
+    bf16* crow = reinterpret_cast<bf16*>(p.C[o]) + (size_t)row * p.ldc[o];
+#pragma unroll
+    for (int g8 = 0; g8 < 4; ++g8) {
+      const int col = n0c + g8 * 8;
+      if (col >= n_lo && col < n_hi) {
+        uint4 q4;
+        __nv_bfloat162 h0 = __floats2bfloat162_rn(__uint_as_float(v[g8 * 8 + 0]), __uint_as_float(v[g8 * 8 + 1]));
+        __nv_bfloat162 h1 = __floats2bfloat162_rn(__uint_as_float(v[g8 * 8 + 2]), __uint_as_float(v[g8 * 8 + 3]));
+        __nv_bfloat162 h2 = __floats2bfloat162_rn(__uint_as_float(v[g8 * 8 + 4]), __uint_as_float(v[g8 * 8 + 5]));
+        __nv_bfloat162 h3 = __floats2bfloat162_rn(__uint_as_float(v[g8 * 8 + 6]), __uint_as_float(v[g8 * 8 + 7]));
+        q4.x = *reinterpret_cast<uint32_t*>(&h0);
+        q4.y = *reinterpret_cast<uint32_t*>(&h1);
+        q4.z = *reinterpret_cast<uint32_t*>(&h2);
+        q4.w = *reinterpret_cast<uint32_t*>(&h3);
+        *reinterpret_cast<uint4*>(crow + col) = q4;
+      }
+    }
+  }
 }
 
 template <int A_MN, int B_KN>
@@ -104,6 +163,7 @@ __global__ void __launch_bounds__(kThreads, 1) tc_gemm_kernel(const __grid_const
 
   int total_kb = 0;
   for (int s = 0; s < p.nseg; ++s) total_kb += p.kblocks[s];
+  const int total = tile_total(p);
 
   if (warp == 0) {
     // ---------------- TMA producer ----------------
@@ -111,14 +171,15 @@ __global__ void __launch_bounds__(kThreads, 1) tc_gemm_kernel(const __grid_const
       for (int s = 0; s < p.nseg * p.nout; ++s) { prefetch_tmap(&p.a_map[s]); prefetch_tmap(&p.b_map[s]); }
       uint32_t it = 0;
       bool ok = true;
-      for (int tile = blockIdx.x; tile < p.total_tiles && ok; tile += gridDim.x) {
+      for (int tile = blockIdx.x; tile < total && ok; tile += gridDim.x) {
         const TileCoord tc = tile_coord(p, tile);
         const int tn = p.tile_n[tc.o];
         const uint32_t tx = kABytes + (uint32_t)tn * BK * 2;
         for (int sg = 0; sg < p.nseg && ok; ++sg) {
           const CUtensorMap* am = &p.a_map[tc.o * p.nseg + sg];
           const CUtensorMap* bm = &p.b_map[tc.o * p.nseg + sg];
-          for (int kb = 0; kb < p.kblocks[sg]; ++kb, ++it) {
+          const int kb_begin = tc.kb1 < 0 ? 0 : tc.kb0, kb_end = tc.kb1 < 0 ? p.kblocks[sg] : tc.kb1;
+          for (int kb = kb_begin; kb < kb_end; ++kb, ++it) {
             const int st = it % kStages;
             const uint32_t ph = (it / kStages) & 1u;
             if (!mbar_wait(empty_bar(st), ph ^ 1u, abort_flag)) { ok = false; break; }
@@ -150,16 +211,17 @@ __global__ void __launch_bounds__(kThreads, 1) tc_gemm_kernel(const __grid_const
     if (lane == 0) {
       uint32_t it = 0, tcount = 0;
       bool ok = true;
-      for (int tile = blockIdx.x; tile < p.total_tiles && ok; tile += gridDim.x, ++tcount) {
+      for (int tile = blockIdx.x; tile < total && ok; tile += gridDim.x, ++tcount) {
         const TileCoord tc = tile_coord(p, tile);
         const int tn = p.tile_n[tc.o];
+        const int nkb = tc.kb1 < 0 ? total_kb : tc.kb1 - tc.kb0;
         const uint32_t idesc = make_idesc(tn, A_MN, B_KN);
         const uint32_t buf = tcount & 1u;
         const uint32_t use = tcount >> 1;                 // how often this accumulator was used before
         if (!mbar_wait(tempty_bar(buf), (use & 1u) ^ 1u, abort_flag)) { ok = false; break; }
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + buf * BN_MAX;
-        for (int kb = 0; kb < total_kb; ++kb, ++it) {
+        for (int kb = 0; kb < nkb; ++kb, ++it) {
           const int st = it % kStages;
           const uint32_t ph = (it / kStages) & 1u;
           if (!mbar_wait(full_bar(st), ph, abort_flag)) { ok = false; break; }
@@ -188,57 +250,27 @@ __global__ void __launch_bounds__(kThreads, 1) tc_gemm_kernel(const __grid_const
     const int q = warp & 3;                                // TMEM lane quarter this warp may read
     uint32_t tcount = 0;
     bool ok = true;
-    for (int tile = blockIdx.x; tile < p.total_tiles && ok; tile += gridDim.x, ++tcount) {
+    for (int tile = blockIdx.x; tile < total && ok; tile += gridDim.x, ++tcount) {
       const TileCoord tc = tile_coord(p, tile);
       const int tn = p.tile_n[tc.o];
+      const bool empty = tc.kb1 >= 0 && tc.kb1 <= tc.kb0;   // no k-block: the result is zero, TMEM holds nothing for it
       const uint32_t buf = tcount & 1u;
       const uint32_t use = tcount >> 1;
       // the decision must be the same for the whole warp: the TMEM loads below are warp-collective
       if (!__all_sync(0xffffffffu, mbar_wait(tfull_bar(buf), use & 1u, abort_flag))) { ok = false; break; }
       tc_fence_after();
       const int row = tc.m0 + q * 32 + lane;
-      const int No = p.N[tc.o];
-      bf16* crow = reinterpret_cast<bf16*>(p.C[tc.o]) + (size_t)row * p.ldc[tc.o];
       const uint32_t t_addr = tmem_base + ((uint32_t)(q * 32) << 16) + buf * BN_MAX;
       for (int c = 0; c < tn; c += 32) {
         uint32_t v[32];
-        tmem_ld32(t_addr + c, v);
-        tmem_ld_wait();
-        if (row < p.M && p.mode[tc.o] == 1) {
-          // fp32 output at base + (n / nb) * s_blk + (n % nb) * s_n + m * s_m, scaled, optionally accumulated
-          float* base = reinterpret_cast<float*>(p.C[tc.o]) + (size_t)row * p.ldc[tc.o];
-          const int nb = p.nb[tc.o];
-          const long long sn = p.s_n[tc.o], sb = p.s_blk[tc.o];
-          const float alpha = p.alpha[tc.o];
-          const int accum = p.accumulate[tc.o];
-#pragma unroll 4
-          for (int j = 0; j < 32; ++j) {
-            const int n = tc.n0 + c + j;
-            if (n < No) {
-              float* dst = base + (nb > 0 ? (size_t)(n / nb) * sb + (size_t)(n % nb) * sn : (size_t)n * sn);
-              float val = alpha * __uint_as_float(v[j]);
-              if (accum) val += *dst;
-              *dst = val;
-            }
-          }
-        } else if (row < p.M) {
+        if (empty) {
 #pragma unroll
-          for (int g8 = 0; g8 < 4; ++g8) {
-            const int col = tc.n0 + c + g8 * 8;
-            if (col < No) {                                // N is a multiple of 8: whole 16-byte groups
-              uint4 o;
-              __nv_bfloat162 h0 = __floats2bfloat162_rn(__uint_as_float(v[g8 * 8 + 0]), __uint_as_float(v[g8 * 8 + 1]));
-              __nv_bfloat162 h1 = __floats2bfloat162_rn(__uint_as_float(v[g8 * 8 + 2]), __uint_as_float(v[g8 * 8 + 3]));
-              __nv_bfloat162 h2 = __floats2bfloat162_rn(__uint_as_float(v[g8 * 8 + 4]), __uint_as_float(v[g8 * 8 + 5]));
-              __nv_bfloat162 h3 = __floats2bfloat162_rn(__uint_as_float(v[g8 * 8 + 6]), __uint_as_float(v[g8 * 8 + 7]));
-              o.x = *reinterpret_cast<uint32_t*>(&h0);
-              o.y = *reinterpret_cast<uint32_t*>(&h1);
-              o.z = *reinterpret_cast<uint32_t*>(&h2);
-              o.w = *reinterpret_cast<uint32_t*>(&h3);
-              *reinterpret_cast<uint4*>(crow + col) = o;
-            }
-          }
+          for (int j = 0; j < 32; ++j) v[j] = 0u;
+        } else {
+          tmem_ld32(t_addr + c, v);
+          tmem_ld_wait();
         }
+        store_chunk32(p, tc.o, row, tc.n0 + c, tc.n_lo, tc.n_hi, v);
       }
       tc_fence_before();
       __syncwarp();
@@ -278,46 +310,6 @@ constexpr uint32_t kBBytes2 = 128 * BK * 2;              // half of a 256-column
 constexpr uint32_t kStageBytes2 = kABytes + kBBytes2;    // 32 KiB
 constexpr uint32_t kSmemBytes2 = kStages2 * kStageBytes2 + 1024 + 256;
 
-__device__ __forceinline__ void store_chunk32(const TcParams& p, int o, int row, int n0c, const uint32_t (&v)[32]) {
-  const int No = p.N[o];
-  if (row >= p.M) return;
-  if (p.mode[o] == 1) {
-    float* base = reinterpret_cast<float*>(p.C[o]) + (size_t)row * p.ldc[o];
-    const int nb = p.nb[o];
-    const long long sn = p.s_n[o], sb = p.s_blk[o];
-    const float alpha = p.alpha[o];
-    const int accum = p.accumulate[o];
-#pragma unroll
-    for (int j = 0; j < 32; ++j) {
-      const int n = n0c + j;
-      if (n < No) {
-        float* dst = base + (nb > 0 ? (size_t)(n / nb) * sb + (size_t)(n % nb) * sn : (size_t)n * sn);
-        float val = alpha * __uint_as_float(v[j]);
-        if (accum) val += *dst;
-        *dst = val;
-      }
-    }
-  } else {
-    bf16* crow = reinterpret_cast<bf16*>(p.C[o]) + (size_t)row * p.ldc[o];
-#pragma unroll
-    for (int g8 = 0; g8 < 4; ++g8) {
-      const int col = n0c + g8 * 8;
-      if (col < No) {
-        uint4 q4;
-        __nv_bfloat162 h0 = __floats2bfloat162_rn(__uint_as_float(v[g8 * 8 + 0]), __uint_as_float(v[g8 * 8 + 1]));
-        __nv_bfloat162 h1 = __floats2bfloat162_rn(__uint_as_float(v[g8 * 8 + 2]), __uint_as_float(v[g8 * 8 + 3]));
-        __nv_bfloat162 h2 = __floats2bfloat162_rn(__uint_as_float(v[g8 * 8 + 4]), __uint_as_float(v[g8 * 8 + 5]));
-        __nv_bfloat162 h3 = __floats2bfloat162_rn(__uint_as_float(v[g8 * 8 + 6]), __uint_as_float(v[g8 * 8 + 7]));
-        q4.x = *reinterpret_cast<uint32_t*>(&h0);
-        q4.y = *reinterpret_cast<uint32_t*>(&h1);
-        q4.z = *reinterpret_cast<uint32_t*>(&h2);
-        q4.w = *reinterpret_cast<uint32_t*>(&h3);
-        *reinterpret_cast<uint4*>(crow + col) = q4;
-      }
-    }
-  }
-}
-
 template <int A_MN, int B_KN>
 __global__ void __launch_bounds__(kThreads, 1) tc_gemm_pair_kernel(const __grid_constant__ TcParams p) {
   extern __shared__ uint8_t smem_raw[];
@@ -354,6 +346,7 @@ __global__ void __launch_bounds__(kThreads, 1) tc_gemm_pair_kernel(const __grid_
 
   int total_kb = 0;
   for (int s = 0; s < p.nseg; ++s) total_kb += p.kblocks[s];
+  const int total = tile_total(p);
   const int pair = blockIdx.x >> 1, npairs = gridDim.x >> 1;
 
   if (warp == 0) {
@@ -362,16 +355,17 @@ __global__ void __launch_bounds__(kThreads, 1) tc_gemm_pair_kernel(const __grid_
       for (int s = 0; s < p.nseg * p.nout; ++s) { prefetch_tmap(&p.a_map[s]); prefetch_tmap(&p.b_map[s]); }
       uint32_t it = 0;
       bool ok = true;
-      for (int tile = pair; tile < p.total_tiles && ok; tile += npairs) {
-        const TileCoord tc = tile_coord(p, tile);        // m0 counts 256-row tiles here (m_tiles set by the host)
+      for (int tile = pair; tile < total && ok; tile += npairs) {
+        const TileCoord tc = tile_coord(p, tile);
         const int tn = p.tile_n[tc.o], half = tn >> 1;
-        const int m0 = tc.m0 * 2 + (int)rank * BM;
+        const int m0 = tc.m0 + (int)rank * BM;
         const int n0 = tc.n0 + (int)rank * half;
         const uint32_t tx_pair = 2u * (kABytes + (uint32_t)half * BK * 2);
         for (int sg = 0; sg < p.nseg && ok; ++sg) {
           const CUtensorMap* am = &p.a_map[tc.o * p.nseg + sg];
           const CUtensorMap* bm = &p.b_map[tc.o * p.nseg + sg];
-          for (int kb = 0; kb < p.kblocks[sg]; ++kb, ++it) {
+          const int kb_begin = tc.kb1 < 0 ? 0 : tc.kb0, kb_end = tc.kb1 < 0 ? p.kblocks[sg] : tc.kb1;
+          for (int kb = kb_begin; kb < kb_end; ++kb, ++it) {
             const int st = it % kStages2;
             const uint32_t ph = (it / kStages2) & 1u;
             if (!mbar_wait(empty_bar(st), ph ^ 1u, abort_flag)) { ok = false; break; }
@@ -404,16 +398,17 @@ __global__ void __launch_bounds__(kThreads, 1) tc_gemm_pair_kernel(const __grid_
     if (lane == 0 && leader) {
       uint32_t it = 0, tcount = 0;
       bool ok = true;
-      for (int tile = pair; tile < p.total_tiles && ok; tile += npairs, ++tcount) {
+      for (int tile = pair; tile < total && ok; tile += npairs, ++tcount) {
         const TileCoord tc = tile_coord(p, tile);
         const int tn = p.tile_n[tc.o];
+        const int nkb = tc.kb1 < 0 ? total_kb : tc.kb1 - tc.kb0;
         const uint32_t idesc = make_idesc_m(2 * BM, tn, A_MN, B_KN);
         const uint32_t buf = tcount & 1u;
         const uint32_t use = tcount >> 1;
         if (!mbar_wait(tempty_bar(buf), (use & 1u) ^ 1u, abort_flag)) { ok = false; break; }
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + buf * BN_MAX;
-        for (int kb = 0; kb < total_kb; ++kb, ++it) {
+        for (int kb = 0; kb < nkb; ++kb, ++it) {
           const int st = it % kStages2;
           const uint32_t ph = (it / kStages2) & 1u;
           if (!mbar_wait(full_bar(st), ph, abort_flag)) { ok = false; break; }
@@ -442,20 +437,26 @@ __global__ void __launch_bounds__(kThreads, 1) tc_gemm_pair_kernel(const __grid_
     const int q = warp & 3;
     uint32_t tcount = 0;
     bool ok = true;
-    for (int tile = pair; tile < p.total_tiles && ok; tile += npairs, ++tcount) {
+    for (int tile = pair; tile < total && ok; tile += npairs, ++tcount) {
       const TileCoord tc = tile_coord(p, tile);
       const int tn = p.tile_n[tc.o];
+      const bool empty = tc.kb1 >= 0 && tc.kb1 <= tc.kb0;
       const uint32_t buf = tcount & 1u;
       const uint32_t use = tcount >> 1;
       if (!__all_sync(0xffffffffu, mbar_wait(tfull_bar(buf), use & 1u, abort_flag))) { ok = false; break; }
       tc_fence_after();
-      const int row = tc.m0 * 2 + (int)rank * BM + q * 32 + lane;
+      const int row = tc.m0 + (int)rank * BM + q * 32 + lane;
       const uint32_t t_addr = tmem_base + ((uint32_t)(q * 32) << 16) + buf * BN_MAX;
       for (int c = 0; c < tn; c += 32) {
         uint32_t v[32];
-        tmem_ld32(t_addr + c, v);
-        tmem_ld_wait();
-        store_chunk32(p, tc.o, row, tc.n0 + c, v);
+        if (empty) {
+#pragma unroll
+          for (int j = 0; j < 32; ++j) v[j] = 0u;
+        } else {
+          tmem_ld32(t_addr + c, v);
+          tmem_ld_wait();
+        }
+        store_chunk32(p, tc.o, row, tc.n0 + c, tc.n_lo, tc.n_hi, v);
       }
       tc_fence_before();
       __syncwarp();
@@ -590,7 +591,9 @@ bool tc_force_single() {
   return v;
 }
 
-cudaError_t launch_tc_gemm(int M, const TcOut* outs, int nout, int* status_word, cudaStream_t st) {
+int tc_gemm_tile_rows(int M) { return (!tc_force_single() && M >= 2 * BM) ? 2 * BM : BM; }
+
+cudaError_t launch_tc_gemm(int M, const TcOut* outs, int nout, int* status_word, cudaStream_t st, const TcWork* wl) {
   TcParams p;
   memset(&p, 0, sizeof(p));
   const int nseg = outs[0].nseg;
@@ -598,6 +601,11 @@ cudaError_t launch_tc_gemm(int M, const TcOut* outs, int nout, int* status_word,
   const bool pair = !tc_force_single() && M >= 2 * BM;
   const int tile_m = pair ? 2 * BM : BM;
   p.nseg = nseg; p.nout = nout; p.M = M; p.m_tiles = (M + tile_m - 1) / tile_m; p.status = status_word;
+  p.tile_m = tile_m;
+  if (wl) {
+    if (nseg != 1) return cudaErrorInvalidValue;   // a work list carries one k-range per item
+    p.work = wl->items; p.work_count = wl->count;
+  }
   for (int s = 0; s < nseg; ++s) p.kblocks[s] = (outs[0].seg[s].K + BK - 1) / BK;
   int tiles = 0;
   for (int o = 0; o < nout; ++o) {
@@ -606,7 +614,10 @@ cudaError_t launch_tc_gemm(int M, const TcOut* outs, int nout, int* status_word,
     // past N read as zero through the tensor map and are never stored
     const int cols = t.mode == 0 ? t.N : round_up(t.N, 8);
     const int gran = (b_kn ? 64 : 16) * (pair ? 2 : 1);
-    const int tn = cols >= BN_MAX ? BN_MAX : round_up(cols, gran);
+    // with a work list every item covers one block of `block_cols` columns, rounded up to the tile granularity
+    const int want = wl ? wl->block_cols : cols;
+    const int tn = want >= BN_MAX ? BN_MAX : round_up(want, gran);
+    if (wl && wl->block_cols > BN_MAX) return cudaErrorInvalidValue;
     p.C[o] = t.C; p.N[o] = t.N; p.tile_n[o] = tn;
     p.mode[o] = t.mode;
     p.ldc[o] = t.mode == 0 ? t.ldc : t.s_m;
@@ -625,7 +636,8 @@ cudaError_t launch_tc_gemm(int M, const TcOut* outs, int nout, int* status_word,
     }
   }
   for (int o = nout; o <= kMaxOut; ++o) p.tile_start[o] = tiles;
-  p.total_tiles = tiles;
+  p.total_tiles = wl ? wl->max_items : tiles;
+  tiles = p.total_tiles;
 
   int dev = 0, sms = 148;
   cudaGetDevice(&dev);
