@@ -49,6 +49,7 @@ typedef enum {
 
 #define MIXLORA_MAX_EXPERTS 32   /* N <= 32                                              */
 #define MIXLORA_MAX_TOP_K 8      /* k <= min(N, 8)                                       */
+#define MIXLORA_MAX_MODELS 16    /* adapters per multi-model call                         */
 #define MIXLORA_MAX_RANK 128     /* r <= 128; r % 8 == 0 in bf16 mode, r % 4 == 0 in fp32 */
 
 /* Problem shape.  Plain data; set struct_size = sizeof(mixlora_shape_t). */
@@ -126,6 +127,25 @@ mixlora_status_t mixlora_ffn_backward(const mixlora_shape_t *shape /* host */,
                                       const mixlora_params_t *params /* host struct of device ptrs */,
                                       const void *dy, float aux_coef, void *workspace, size_t workspace_bytes,
                                       const mixlora_grads_t *grads /* host struct of device ptrs */, void *stream);
+
+/* Multi-model forward and backward (Section 3.3 (II), the task loop of Algorithm 1): n_models MixLoRA adapters,
+ * each with its own tokens, router, experts, rank and workspace, share ONE frozen FFN (same w_gate, w_up, w_down
+ * pointers, same d_model, d_ff and dtype; anything else returns MIXLORA_ERR_INVALID_ARG).  The frozen weights are
+ * held once, and the adapters' tokens pass through W1 / W3 (forward) and W2 (backward) two adapters per launch;
+ * every other step runs per adapter exactly as in the single-model calls, so each adapter's results equal those of
+ * mixlora_ffn_forward / mixlora_ffn_backward on it alone, bit for bit.  All arrays are HOST arrays of n_models
+ * entries (of structs / device pointers / sizes); workspaces and outputs must be distinct per adapter.
+ * mixlora_aux_loss and mixlora_routing_view are called per adapter on its own workspace. */
+mixlora_status_t mixlora_multi_ffn_forward(int32_t n_models, const mixlora_shape_t *shapes /* host [n] */,
+                                           const mixlora_params_t *params /* host [n] */, void *const *y /* host [n] */,
+                                           void *const *workspaces /* host [n] */,
+                                           const size_t *workspace_bytes /* host [n] */, void *stream);
+mixlora_status_t mixlora_multi_ffn_backward(int32_t n_models, const mixlora_shape_t *shapes /* host [n] */,
+                                            const mixlora_params_t *params /* host [n] */,
+                                            const void *const *dy /* host [n] */, const float *aux_coef /* host [n] */,
+                                            void *const *workspaces /* host [n] */,
+                                            const size_t *workspace_bytes /* host [n] */,
+                                            const mixlora_grads_t *grads /* host [n] */, void *stream);
 
 /* Device pointers into the workspace, for inspection after a forward call:
  * expert_idx [T, k] (descending logit), gates [T, k], perm [T*k] (slot id at each position

@@ -22,7 +22,8 @@ STATUS_NAMES = {0: "MIXLORA_OK", 1: "MIXLORA_ERR_INVALID_ARG", 2: "MIXLORA_ERR_U
 EXPORTS = ("mixlora_limits", "mixlora_workspace_bytes", "mixlora_ffn_forward", "mixlora_aux_loss",
            "mixlora_ffn_backward", "mixlora_routing_view", "mixlora_device_status", "mixlora_gemm_bf16",
            "mixlora_status_string", "mixlora_stage_timing", "mixlora_stage_timing_read",
-           "mixlora_dispatch_static", "mixlora_dispatch_static_max_tokens")
+           "mixlora_dispatch_static", "mixlora_dispatch_static_max_tokens",
+           "mixlora_multi_ffn_forward", "mixlora_multi_ffn_backward")
 
 
 class mixlora_shape_t(C.Structure):
@@ -86,6 +87,14 @@ def _load() -> C.CDLL:
     lib.mixlora_dispatch_static.restype = C.c_int
     lib.mixlora_dispatch_static_max_tokens.argtypes = []
     lib.mixlora_dispatch_static_max_tokens.restype = C.c_int32
+    lib.mixlora_multi_ffn_forward.argtypes = [C.c_int32, C.POINTER(mixlora_shape_t), C.POINTER(mixlora_params_t),
+                                              C.POINTER(C.c_void_p), C.POINTER(C.c_void_p), C.POINTER(C.c_size_t),
+                                              C.c_void_p]
+    lib.mixlora_multi_ffn_forward.restype = C.c_int
+    lib.mixlora_multi_ffn_backward.argtypes = [C.c_int32, C.POINTER(mixlora_shape_t), C.POINTER(mixlora_params_t),
+                                               C.POINTER(C.c_void_p), C.POINTER(C.c_float), C.POINTER(C.c_void_p),
+                                               C.POINTER(C.c_size_t), C.POINTER(mixlora_grads_t), C.c_void_p]
+    lib.mixlora_multi_ffn_backward.restype = C.c_int
     lib.mixlora_status_string.argtypes = [C.c_int]
     lib.mixlora_status_string.restype = C.c_char_p
     return lib
@@ -226,3 +235,25 @@ def mixlora_dispatch_static(expert_idx, tokens, n_experts, top_k, perm, seg_off,
 
 def mixlora_dispatch_static_max_tokens() -> int:
     return int(lib.mixlora_dispatch_static_max_tokens())
+
+
+def _ptr_array(tensors):
+    return (C.c_void_p * len(tensors))(*[_ptr(t) for t in tensors])
+
+
+def mixlora_multi_ffn_forward(shapes, params, ys, workspaces, stream=None) -> None:
+    """Forward of several adapters that share one frozen FFN (lists of equal length, one entry per adapter)."""
+    n = len(shapes)
+    _check(lib.mixlora_multi_ffn_forward(n, (mixlora_shape_t * n)(*shapes), (mixlora_params_t * n)(*params),
+                                         _ptr_array(ys), _ptr_array(workspaces),
+                                         (C.c_size_t * n)(*[w.numel() for w in workspaces]), _stream(stream)),
+           "mixlora_multi_ffn_forward")
+
+
+def mixlora_multi_ffn_backward(shapes, params, dys, aux_coefs, workspaces, grads, stream=None) -> None:
+    n = len(shapes)
+    _check(lib.mixlora_multi_ffn_backward(n, (mixlora_shape_t * n)(*shapes), (mixlora_params_t * n)(*params),
+                                          _ptr_array(dys), (C.c_float * n)(*[float(a) for a in aux_coefs]),
+                                          _ptr_array(workspaces), (C.c_size_t * n)(*[w.numel() for w in workspaces]),
+                                          (mixlora_grads_t * n)(*grads), _stream(stream)),
+           "mixlora_multi_ffn_backward")

@@ -193,7 +193,8 @@ cudaError_t dense_product(const Ctx& c, int M, const TcOut* outs, int nout, cons
     return launch_tc_gemm(M, outs, nout, c.at<int>(c.L.status), c.st, wl);   // the SIMT kernel below computes every block
   for (int o = 0; o < nout; ++o) {
     const TcOut& t = outs[o];
-    SGemm g = t.mode == 0 ? sgemm_base(c, t.C, t.ldc, 1, c.bf16, M, t.N) : sgemm_base(c, t.C, t.s_m, t.s_n, 0, M, t.N);
+    const int Mo = t.M > 0 ? t.M : M;
+    SGemm g = t.mode == 0 ? sgemm_base(c, t.C, t.ldc, 1, c.bf16, Mo, t.N) : sgemm_base(c, t.C, t.s_m, t.s_n, 0, Mo, t.N);
     if (t.mode == 1) { g.c_nb = t.nb; g.c_sblk = t.s_blk; g.alpha = t.alpha; g.accumulate = t.accumulate; }
     for (int i = 0; i < t.nseg; ++i) {
       const TcSeg& sg = t.seg[i];
@@ -265,36 +266,77 @@ size_t mixlora_workspace_bytes(const mixlora_shape_t* shape, int for_backward) {
   return for_backward ? L.total_bwd : L.total_fwd;
 }
 
-mixlora_status_t mixlora_ffn_forward(const mixlora_shape_t* shape, const mixlora_params_t* params, void* y,
-                                     void* workspace, size_t workspace_bytes, void* stream) {
+// ---- forward, in three steps so that several adapters can share the frozen-projection launch ----
+static mixlora_status_t fwd_check(const mixlora_shape_t* shape, const mixlora_params_t* params, void* y,
+                                  void* workspace, size_t workspace_bytes, void* stream, Ctx* out) {
   mixlora_status_t st = check_shape(shape);
   if (st != MIXLORA_OK) return st;
   st = check_params(params);
   if (st != MIXLORA_OK) return st;
   if (!y || !aligned16(y)) return MIXLORA_ERR_INVALID_ARG;
-  Ctx c = make_ctx(shape, params, workspace, stream);
-  if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255u) || workspace_bytes < c.L.total_fwd)
+  *out = make_ctx(shape, params, workspace, stream);
+  if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255u) || workspace_bytes < out->L.total_fwd)
     return MIXLORA_ERR_WORKSPACE;
-  const int T = shape->tokens, d = shape->d_model, f = shape->d_ff, N = shape->n_experts, r = shape->rank,
-            k = shape->top_k;
-  const int Nr = N * r;
-  MIXLORA_CUDA(cudaMemsetAsync(c.ws + c.L.status, 0, 256, c.st));
-  if (T == 0) return MIXLORA_OK;
+  return MIXLORA_OK;
+}
 
-  // router (Eq. 7) and dispatch
+// router (Eq. 7) and dispatch
+static mixlora_status_t fwd_route(const Ctx& c) {
+  MIXLORA_CUDA(cudaMemsetAsync(c.ws + c.L.status, 0, 256, c.st));
+  if (c.s.tokens == 0) return MIXLORA_OK;
   { StageScope ss(ST_ROUTER, c.st, 2); MIXLORA_CUDA(launch_router(c)); }
   { StageScope ss(ST_DISPATCH, c.st, 3); MIXLORA_CUDA(launch_dispatch(c)); }
+  return MIXLORA_OK;
+}
 
-  // shared gate / up projections and LoRA-A of every expert, one pass over x
-  {
-    TcOut outs[4];
-    outs[0] = tc_out(c.ws + c.L.G, f, f);     tc_add(outs[0], params->x, d, d, params->w_gate, d, 0);
-    outs[1] = tc_out(c.ws + c.L.U, f, f);     tc_add(outs[1], params->x, d, d, params->w_up, d, 0);
-    outs[2] = tc_out(c.ws + c.L.zga, Nr, Nr); tc_add(outs[2], params->x, d, d, params->a_gate, d, 0);
-    outs[3] = tc_out(c.ws + c.L.zua, Nr, Nr); tc_add(outs[3], params->x, d, d, params->a_up, d, 0);
+// Shared gate / up projections, once per token (Section 3.3 (I)), for one adapter (then the LoRA-A columns of every
+// expert ride along in the same pass over x) or for two adapters that share W1, W3 (Section 3.3 (II): their tokens
+// go through the frozen weights in one launch; each adapter's LoRA-A product follows on its own).
+static mixlora_status_t fwd_shared_projections(const Ctx* cs, int n) {
+  TcOut outs[4];
+  int no = 0, Tmax = 0;
+  for (int i = 0; i < n; ++i) {
+    const Ctx& c = cs[i];
+    const int T = c.s.tokens, d = c.s.d_model, f = c.s.d_ff;
+    if (T == 0) continue;
+    Tmax = T > Tmax ? T : Tmax;
+    outs[no] = tc_out(c.ws + c.L.G, f, f); outs[no].M = T; tc_add(outs[no++], c.p.x, d, d, c.p.w_gate, d, 0);
+    outs[no] = tc_out(c.ws + c.L.U, f, f); outs[no].M = T; tc_add(outs[no++], c.p.x, d, d, c.p.w_up, d, 0);
+  }
+  if (no == 0) return MIXLORA_OK;
+  const Ctx& c0 = cs[0].s.tokens ? cs[0] : cs[n - 1];
+  if (n == 1) {
+    const Ctx& c = cs[0];
+    const int T = c.s.tokens, d = c.s.d_model, Nr = c.s.n_experts * c.s.rank;
+    outs[2] = tc_out(c.ws + c.L.zga, Nr, Nr); tc_add(outs[2], c.p.x, d, d, c.p.a_gate, d, 0);
+    outs[3] = tc_out(c.ws + c.L.zua, Nr, Nr); tc_add(outs[3], c.p.x, d, d, c.p.a_up, d, 0);
     StageScope ss(ST_GEMM_GATE_UP, c.st, dense_launches(c, T, outs, 4));
     MIXLORA_CUDA(dense_product(c, T, outs, 4));
+    return MIXLORA_OK;
   }
+  {
+    StageScope ss(ST_GEMM_GATE_UP, c0.st, dense_launches(c0, Tmax, outs, no));
+    MIXLORA_CUDA(dense_product(c0, Tmax, outs, no));
+  }
+  for (int i = 0; i < n; ++i) {
+    const Ctx& c = cs[i];
+    const int T = c.s.tokens, d = c.s.d_model, Nr = c.s.n_experts * c.s.rank;
+    if (T == 0) continue;
+    TcOut z[2];
+    z[0] = tc_out(c.ws + c.L.zga, Nr, Nr); tc_add(z[0], c.p.x, d, d, c.p.a_gate, d, 0);
+    z[1] = tc_out(c.ws + c.L.zua, Nr, Nr); tc_add(z[1], c.p.x, d, d, c.p.a_up, d, 0);
+    StageScope ss(ST_GEMM_GATE_UP, c.st, dense_launches(c, T, z, 2));
+    MIXLORA_CUDA(dense_product(c, T, z, 2));
+  }
+  return MIXLORA_OK;
+}
+
+// everything after the shared projections: per-expert deltas, SwiGLU, down projection, combine
+static mixlora_status_t fwd_experts(const Ctx& c, void* y) {
+  const mixlora_params_t* params = &c.p;
+  const int T = c.s.tokens, d = c.s.d_model, f = c.s.d_ff, N = c.s.n_experts, r = c.s.rank, k = c.s.top_k;
+  const int Nr = N * r;
+  if (T == 0) return MIXLORA_OK;
   // per-slot LoRA-B expansion + SwiGLU
   {
     StageScope ss(ST_LORA_B_SWIGLU, c.st, 5);
@@ -333,6 +375,44 @@ mixlora_status_t mixlora_ffn_forward(const mixlora_shape_t* shape, const mixlora
   return MIXLORA_OK;
 }
 
+mixlora_status_t mixlora_ffn_forward(const mixlora_shape_t* shape, const mixlora_params_t* params, void* y,
+                                     void* workspace, size_t workspace_bytes, void* stream) {
+  Ctx c;
+  mixlora_status_t st = fwd_check(shape, params, y, workspace, workspace_bytes, stream, &c);
+  if (st != MIXLORA_OK) return st;
+  if ((st = fwd_route(c)) != MIXLORA_OK) return st;
+  if ((st = fwd_shared_projections(&c, 1)) != MIXLORA_OK) return st;
+  return fwd_experts(c, y);
+}
+
+static bool same_frozen_ffn(const Ctx& a, const Ctx& b) {
+  return a.s.d_model == b.s.d_model && a.s.d_ff == b.s.d_ff && a.s.dtype == b.s.dtype && a.p.w_gate == b.p.w_gate &&
+         a.p.w_up == b.p.w_up && a.p.w_down == b.p.w_down;
+}
+
+mixlora_status_t mixlora_multi_ffn_forward(int32_t n_models, const mixlora_shape_t* shapes,
+                                           const mixlora_params_t* params, void* const* y, void* const* workspaces,
+                                           const size_t* workspace_bytes, void* stream) {
+  if (n_models < 1 || n_models > MIXLORA_MAX_MODELS || !shapes || !params || !y || !workspaces || !workspace_bytes)
+    return MIXLORA_ERR_INVALID_ARG;
+  Ctx cs[MIXLORA_MAX_MODELS];
+  for (int m = 0; m < n_models; ++m) {
+    mixlora_status_t st = fwd_check(&shapes[m], &params[m], y[m], workspaces[m], workspace_bytes[m], stream, &cs[m]);
+    if (st != MIXLORA_OK) return st;
+    if (!same_frozen_ffn(cs[0], cs[m])) return MIXLORA_ERR_INVALID_ARG;   // the adapters must share one frozen FFN
+    for (int o = 0; o < m; ++o)
+      if (workspaces[o] == workspaces[m] || y[o] == y[m]) return MIXLORA_ERR_INVALID_ARG;
+  }
+  mixlora_status_t st;
+  for (int m = 0; m < n_models; ++m)
+    if ((st = fwd_route(cs[m])) != MIXLORA_OK) return st;
+  for (int m = 0; m < n_models; m += 2)
+    if ((st = fwd_shared_projections(&cs[m], n_models - m >= 2 ? 2 : 1)) != MIXLORA_OK) return st;
+  for (int m = 0; m < n_models; ++m)
+    if ((st = fwd_experts(cs[m], y[m])) != MIXLORA_OK) return st;
+  return MIXLORA_OK;
+}
+
 mixlora_status_t mixlora_aux_loss(const mixlora_shape_t* shape, const void* workspace, float coef, float* loss,
                                   float* F, float* P, void* stream) {
   mixlora_status_t st = check_shape(shape);
@@ -350,9 +430,10 @@ mixlora_status_t mixlora_aux_loss(const mixlora_shape_t* shape, const void* work
   return MIXLORA_OK;
 }
 
-mixlora_status_t mixlora_ffn_backward(const mixlora_shape_t* shape, const mixlora_params_t* params, const void* dy,
-                                      float aux_coef, void* workspace, size_t workspace_bytes,
-                                      const mixlora_grads_t* grads, void* stream) {
+// ---- backward, split the same way: checks, the shared dy W_d launch, the rest ----
+static mixlora_status_t bwd_check(const mixlora_shape_t* shape, const mixlora_params_t* params, const void* dy,
+                                  void* workspace, size_t workspace_bytes, const mixlora_grads_t* grads, void* stream,
+                                  Ctx* out) {
   mixlora_status_t st = check_shape(shape);
   if (st != MIXLORA_OK) return st;
   st = check_params(params);
@@ -365,34 +446,76 @@ mixlora_status_t mixlora_ffn_backward(const mixlora_shape_t* shape, const mixlor
       if (q && !aligned16(q)) return MIXLORA_ERR_INVALID_ARG;
     if (grads->accumulate != 0 && grads->accumulate != 1) return MIXLORA_ERR_INVALID_ARG;
   }
-  Ctx c = make_ctx(shape, params, workspace, stream);
-  if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255u) || workspace_bytes < c.L.total_bwd)
+  *out = make_ctx(shape, params, workspace, stream);
+  if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255u) || workspace_bytes < out->L.total_bwd)
     return MIXLORA_ERR_WORKSPACE;
-  const int T = shape->tokens, d = shape->d_model, f = shape->d_ff, N = shape->n_experts, r = shape->rank,
-            k = shape->top_k;
-  const int Nr = N * r, NP = round_up8(N);
-  const int acc = grads->accumulate;
-  const int want_dx = grads->d_x != nullptr;
-  if (T == 0) {
-    if (!acc) {
-      struct { float* p; size_t n; } z[] = {
-          {grads->d_a_gate, (size_t)N * r * d}, {grads->d_b_gate, (size_t)N * f * r}, {grads->d_a_up, (size_t)N * r * d},
-          {grads->d_b_up, (size_t)N * f * r},   {grads->d_a_down, (size_t)N * r * f}, {grads->d_b_down, (size_t)N * d * r},
-          {grads->d_w_router, (size_t)N * d},   {grads->d_router_bias, (size_t)N}};
-      for (auto& q : z)
-        if (q.p) MIXLORA_CUDA(cudaMemsetAsync(q.p, 0, q.n * sizeof(float), c.st));
-    }
-    return MIXLORA_OK;
-  }
-  // D = dy W_d (shared by a token's slots) and s B_d^T dy for every expert
-  {
+  return MIXLORA_OK;
+}
+
+// D = dy W_d (shared by a token's slots) and s B_d^T dy for every expert; two adapters that share W_d send their
+// dy through it in one launch
+static mixlora_status_t bwd_shared_dgrad(const Ctx* cs, const void* const* dys, int n) {
+  if (n == 1) {
+    const Ctx& c = cs[0];
+    const int T = c.s.tokens, d = c.s.d_model, f = c.s.d_ff, Nr = c.s.n_experts * c.s.rank;
+    if (T == 0) return MIXLORA_OK;
     TcOut outs[2];
-    outs[0] = tc_out(c.ws + c.L.D, f, f);      tc_add(outs[0], dy, d, d, params->w_down, f, 1);
-    outs[1] = tc_out(c.ws + c.L.spd, Nr, Nr);  tc_add(outs[1], dy, d, d, c.ws + c.L.bd_cat, Nr, 1);
+    outs[0] = tc_out(c.ws + c.L.D, f, f);      tc_add(outs[0], dys[0], d, d, c.p.w_down, f, 1);
+    outs[1] = tc_out(c.ws + c.L.spd, Nr, Nr);  tc_add(outs[1], dys[0], d, d, c.ws + c.L.bd_cat, Nr, 1);
     StageScope ss(ST_GEMM_DGRAD_DOWN, c.st, 1 + dense_launches(c, T, outs, 2));
     MIXLORA_CUDA(launch_bd_cat(c));
     MIXLORA_CUDA(dense_product(c, T, outs, 2));
+    return MIXLORA_OK;
   }
+  TcOut outs[2];
+  int no = 0, Tmax = 0, last = 0;
+  for (int i = 0; i < n; ++i) {
+    const Ctx& c = cs[i];
+    const int T = c.s.tokens, d = c.s.d_model, f = c.s.d_ff;
+    if (T == 0) continue;
+    Tmax = T > Tmax ? T : Tmax;
+    last = i;
+    outs[no] = tc_out(c.ws + c.L.D, f, f); outs[no].M = T; tc_add(outs[no++], dys[i], d, d, c.p.w_down, f, 1);
+  }
+  if (no == 0) return MIXLORA_OK;
+  {
+    const Ctx& c0 = cs[last];
+    StageScope ss(ST_GEMM_DGRAD_DOWN, c0.st, dense_launches(c0, Tmax, outs, no));
+    MIXLORA_CUDA(dense_product(c0, Tmax, outs, no));
+  }
+  for (int i = 0; i < n; ++i) {
+    const Ctx& c = cs[i];
+    const int T = c.s.tokens, d = c.s.d_model, Nr = c.s.n_experts * c.s.rank;
+    if (T == 0) continue;
+    TcOut z = tc_out(c.ws + c.L.spd, Nr, Nr);
+    tc_add(z, dys[i], d, d, c.ws + c.L.bd_cat, Nr, 1);
+    StageScope ss(ST_GEMM_DGRAD_DOWN, c.st, 1 + dense_launches(c, T, &z, 1));
+    MIXLORA_CUDA(launch_bd_cat(c));
+    MIXLORA_CUDA(dense_product(c, T, &z, 1));
+  }
+  return MIXLORA_OK;
+}
+
+static mixlora_status_t bwd_zero_tokens(const Ctx& c, const mixlora_grads_t* grads) {
+  const int d = c.s.d_model, f = c.s.d_ff, N = c.s.n_experts, r = c.s.rank;
+  if (!grads->accumulate) {
+    struct { float* p; size_t n; } z[] = {
+        {grads->d_a_gate, (size_t)N * r * d}, {grads->d_b_gate, (size_t)N * f * r}, {grads->d_a_up, (size_t)N * r * d},
+        {grads->d_b_up, (size_t)N * f * r},   {grads->d_a_down, (size_t)N * r * f}, {grads->d_b_down, (size_t)N * d * r},
+        {grads->d_w_router, (size_t)N * d},   {grads->d_router_bias, (size_t)N}};
+    for (auto& q : z)
+      if (q.p) MIXLORA_CUDA(cudaMemsetAsync(q.p, 0, q.n * sizeof(float), c.st));
+  }
+  return MIXLORA_OK;
+}
+
+static mixlora_status_t bwd_experts(const Ctx& c, const void* dy, float aux_coef, const mixlora_grads_t* grads) {
+  const mixlora_params_t* params = &c.p;
+  const int T = c.s.tokens, d = c.s.d_model, f = c.s.d_ff, N = c.s.n_experts, r = c.s.rank, k = c.s.top_k;
+  const int Nr = N * r, NP = round_up8(N);
+  const int acc = grads->accumulate;
+  const int want_dx = grads->d_x != nullptr;
+  if (T == 0) return bwd_zero_tokens(c, grads);
   {
     StageScope ss(ST_SWIGLU_BWD, c.st, 3);
     MIXLORA_CUDA(launch_slot_prep_bwd(c));
@@ -484,6 +607,41 @@ mixlora_status_t mixlora_ffn_backward(const mixlora_shape_t* shape, const mixlor
   }
   return MIXLORA_OK;
 }
+
+mixlora_status_t mixlora_ffn_backward(const mixlora_shape_t* shape, const mixlora_params_t* params, const void* dy,
+                                      float aux_coef, void* workspace, size_t workspace_bytes,
+                                      const mixlora_grads_t* grads, void* stream) {
+  Ctx c;
+  mixlora_status_t st = bwd_check(shape, params, dy, workspace, workspace_bytes, grads, stream, &c);
+  if (st != MIXLORA_OK) return st;
+  if ((st = bwd_shared_dgrad(&c, &dy, 1)) != MIXLORA_OK) return st;
+  return bwd_experts(c, dy, aux_coef, grads);
+}
+
+mixlora_status_t mixlora_multi_ffn_backward(int32_t n_models, const mixlora_shape_t* shapes,
+                                            const mixlora_params_t* params, const void* const* dy,
+                                            const float* aux_coef, void* const* workspaces,
+                                            const size_t* workspace_bytes, const mixlora_grads_t* grads, void* stream) {
+  if (n_models < 1 || n_models > MIXLORA_MAX_MODELS || !shapes || !params || !dy || !aux_coef || !workspaces ||
+      !workspace_bytes || !grads)
+    return MIXLORA_ERR_INVALID_ARG;
+  Ctx cs[MIXLORA_MAX_MODELS];
+  for (int m = 0; m < n_models; ++m) {
+    mixlora_status_t st = bwd_check(&shapes[m], &params[m], dy[m], workspaces[m], workspace_bytes[m], &grads[m], stream,
+                                    &cs[m]);
+    if (st != MIXLORA_OK) return st;
+    if (!same_frozen_ffn(cs[0], cs[m])) return MIXLORA_ERR_INVALID_ARG;
+    for (int o = 0; o < m; ++o)
+      if (workspaces[o] == workspaces[m]) return MIXLORA_ERR_INVALID_ARG;
+  }
+  mixlora_status_t st;
+  for (int m = 0; m < n_models; m += 2)
+    if ((st = bwd_shared_dgrad(&cs[m], &dy[m], n_models - m >= 2 ? 2 : 1)) != MIXLORA_OK) return st;
+  for (int m = 0; m < n_models; ++m)
+    if ((st = bwd_experts(cs[m], dy[m], aux_coef[m], &grads[m])) != MIXLORA_OK) return st;
+  return MIXLORA_OK;
+}
+
 
 mixlora_status_t mixlora_routing_view(const mixlora_shape_t* shape, const void* workspace, const int32_t** expert_idx,
                                       const float** gates, const int32_t** perm, const int32_t** seg_off,

@@ -176,6 +176,7 @@ struct TcSeg {
 };
 struct TcOut {
   void* C; long long ldc; int N;
+  int M;        // rows of this output when it differs from the launch's M (0 = same)
   int mode; long long s_m, s_n, s_blk; int nb; float alpha; int accumulate;
   TcSeg seg[kMaxKSeg]; int nseg;
 };

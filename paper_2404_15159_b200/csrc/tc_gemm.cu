@@ -51,7 +51,9 @@ struct alignas(64) TcParams {
   int tile_n[kMaxOut];
   int tile_start[kMaxOut + 1];     // first tile index of each output
   int kblocks[kMaxSeg];
-  int nseg, nout, M, m_tiles, total_tiles, tile_m;
+  int Mo[kMaxOut];                 // rows of each output (outputs of one launch may differ in rows)
+  int m_tiles_o[kMaxOut];
+  int nseg, nout, total_tiles, tile_m;
   // Optional device-built work list (block-sparse schedule over the sorted slots): item = 8 ints
   // {output, m0, n0, first k-block, end k-block, first stored column, end stored column, 0}; *work_count items.
   const int* work;
@@ -81,8 +83,8 @@ __device__ __forceinline__ TileCoord tile_coord(const TcParams& p, int tile) {
     if (i < p.nout && tile >= p.tile_start[i]) o = i;
   const int local = tile - p.tile_start[o];
   t.o = o;
-  t.m0 = (local % p.m_tiles) * p.tile_m;  // rows fastest: neighbouring CTAs share the B tile
-  t.n0 = (local / p.m_tiles) * p.tile_n[o];
+  t.m0 = (local % p.m_tiles_o[o]) * p.tile_m;  // rows fastest: neighbouring CTAs share the B tile
+  t.n0 = (local / p.m_tiles_o[o]) * p.tile_n[o];
   t.kb0 = 0; t.kb1 = -1;                  // all k-blocks of every segment
   t.n_lo = 0; t.n_hi = p.N[o];
   return t;
@@ -91,7 +93,7 @@ __device__ __forceinline__ TileCoord tile_coord(const TcParams& p, int tile) {
 // Stores 32 accumulator columns [n0c, n0c + 32) of one row; only columns inside [n_lo, n_hi) are written.
 __device__ __forceinline__ void store_chunk32(const TcParams& p, int o, int row, int n0c, int n_lo, int n_hi,
                                               const uint32_t (&v)[32]) {
-  if (row >= p.M) return;
+  if (row >= p.Mo[o]) return;
   if (p.mode[o] == 1) {
     float* base = reinterpret_cast<float*>(p.C[o]) + (size_t)row * p.ldc[o];
     const int nb = p.nb[o];
@@ -600,7 +602,7 @@ cudaError_t launch_tc_gemm(int M, const TcOut* outs, int nout, int* status_word,
   const int a_mn = outs[0].seg[0].a_mn, b_kn = outs[0].seg[0].b_kn;
   const bool pair = !tc_force_single() && M >= 2 * BM;
   const int tile_m = pair ? 2 * BM : BM;
-  p.nseg = nseg; p.nout = nout; p.M = M; p.m_tiles = (M + tile_m - 1) / tile_m; p.status = status_word;
+  p.nseg = nseg; p.nout = nout; p.status = status_word;
   p.tile_m = tile_m;
   if (wl) {
     if (nseg != 1) return cudaErrorInvalidValue;   // a work list carries one k-range per item
@@ -618,17 +620,19 @@ cudaError_t launch_tc_gemm(int M, const TcOut* outs, int nout, int* status_word,
     const int want = wl ? wl->block_cols : cols;
     const int tn = want >= BN_MAX ? BN_MAX : round_up(want, gran);
     if (wl && wl->block_cols > BN_MAX) return cudaErrorInvalidValue;
+    const int Mrows = t.M > 0 ? t.M : M;
+    p.Mo[o] = Mrows; p.m_tiles_o[o] = (Mrows + tile_m - 1) / tile_m;
     p.C[o] = t.C; p.N[o] = t.N; p.tile_n[o] = tn;
     p.mode[o] = t.mode;
     p.ldc[o] = t.mode == 0 ? t.ldc : t.s_m;
     p.s_n[o] = t.s_n; p.s_blk[o] = t.s_blk; p.nb[o] = t.nb; p.alpha[o] = t.alpha; p.accumulate[o] = t.accumulate;
     p.tile_start[o] = tiles;
-    tiles += p.m_tiles * ((t.N + tn - 1) / tn);
+    tiles += p.m_tiles_o[o] * ((t.N + tn - 1) / tn);
     const int b_rows = pair ? tn / 2 : tn;               // rows of a K-major B tile held by one CTA
     for (int s = 0; s < nseg; ++s) {
       const TcSeg& g = t.seg[s];
-      bool ok = a_mn ? encode_2d(&p.a_map[o * nseg + s], g.A, g.K, M, g.lda, BK, 64)
-                     : encode_2d(&p.a_map[o * nseg + s], g.A, M, g.K, g.lda, BM, BK);
+      bool ok = a_mn ? encode_2d(&p.a_map[o * nseg + s], g.A, g.K, Mrows, g.lda, BK, 64)
+                     : encode_2d(&p.a_map[o * nseg + s], g.A, Mrows, g.K, g.lda, BM, BK);
       if (!ok) return cudaErrorInvalidValue;
       ok = b_kn ? encode_2d(&p.b_map[o * nseg + s], g.B, g.K, g.b_cols > 0 ? g.b_cols : t.N, g.ldb, BK, 64)
                 : encode_2d(&p.b_map[o * nseg + s], g.B, g.b_cols > 0 ? g.b_cols : t.N, g.K, g.ldb, b_rows, BK);
