@@ -233,6 +233,38 @@ def run_cuda(args):
         if world > 1:
             dist.all_reduce(flat)          # data-parallel sum of the LoRA and router gradients
 
+    M = max(1, args.models)
+    if M > 1:
+        # Multi-model variant (Section 3.3 (II)): the batch is split over M adapters that share the frozen FFN and
+        # go through one multi-model call; each adapter has its own workspace, outputs and gradient buffers (the
+        # LoRA / router tensors are re-used between adapters here, which does not change the work).
+        Tm = w.tokens // M
+        m_shapes, m_params, m_ys, m_ws, m_dys, m_grads, m_keep = [], [], [], [], [], [], []
+        for m in range(M):
+            sl = slice(m * Tm, (m + 1) * Tm)
+            sh = B.make_shape(Tm, w.d_model, w.d_ff, w.n_experts, w.top_k, w.rank, w.lora_alpha,
+                              B.MIXLORA_DTYPE_BF16 if bf16 else B.MIXLORA_DTYPE_FP32)
+            m_shapes.append(sh)
+            m_params.append(B.make_params(**{n: dev[n] for n in synth.PARAM_NAMES}, x=dev["x"][sl]))
+            m_ys.append(y[sl])
+            m_ws.append(B.alloc_workspace(sh, True))
+            m_dys.append(dev["dy"][sl])
+            fl = torch.zeros(total, dtype=torch.float32, device="cuda")
+            gm = {n: fl[off:off + size] for n, (off, size) in offsets.items()}
+            if want_dx:
+                gm["d_x"] = g["d_x"][sl]
+            m_keep.append((fl, gm))
+            m_grads.append(B.make_grads(accumulate=0, **gm))
+
+        def step():                        # noqa: F811
+            B.mixlora_multi_ffn_forward(m_shapes, m_params, m_ys, m_ws)
+            for m in range(M):
+                B.mixlora_aux_loss(m_shapes[m], m_ws[m], AUX_COEF, loss)
+            B.mixlora_multi_ffn_backward(m_shapes, m_params, m_dys, [AUX_COEF] * M, m_ws, m_grads)
+            if world > 1:
+                for fl, _ in m_keep:
+                    dist.all_reduce(fl)
+
     def barrier():
         if world > 1:
             dist.barrier()
@@ -263,7 +295,7 @@ def run_cuda(args):
     clocks = sampler.stop(t0, t1) if rank == 0 else None
     launches = sum(v[1] for v in B.mixlora_stage_timing_read().values())
     launches_per_step = launches // (args.steps + args.warmup)
-    status = B.mixlora_device_status(ws)
+    status = B.mixlora_device_status(ws) if M == 1 else max(B.mixlora_device_status(x_) for x_ in m_ws)
     ms_per_step = total_ms / args.steps
     value = world * w.tokens / (ms_per_step * 1e-3)
 
@@ -387,7 +419,7 @@ def run_cuda(args):
         "dtype": "bf16" if bf16 else "f32", "data": "synthetic",
         "config": {"workload": w.name, "tokens_per_gpu": w.tokens, "d_model": w.d_model, "d_ff": w.d_ff,
                    "n_experts": w.n_experts, "top_k": w.top_k, "rank": w.rank, "lora_alpha": w.lora_alpha,
-                   "backward_dx": want_dx, "aux_coef": AUX_COEF,
+                   "backward_dx": want_dx, "aux_coef": AUX_COEF, "adapters": M,
                    "parallelism": f"dp{world} over tokens" + (", NCCL all-reduce of LoRA/router grads" if world > 1 else ""),
                    "l2": "inputs larger than L2 (weights 270 MB + activations > 126 MB), no flush"},
         "roofline": roofline, "cpu_baseline": cpu_baseline,
@@ -410,6 +442,9 @@ def main():
     ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
     ap.add_argument("--workload", default="c3")
     ap.add_argument("--no-dx", action="store_true")
+    ap.add_argument("--models", type=int, default=1,
+                    help="split the batch over this many adapters sharing the frozen FFN (multi-model calls); the "
+                         "end-to-end leg still runs the single-model calls")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--cpu-sample", type=int, default=512, help="tokens of the oracle's timed sample")
     ap.add_argument("--ref-sample", type=int, default=256, help="tokens per step of --impl reference")
