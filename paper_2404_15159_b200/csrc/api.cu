@@ -208,6 +208,11 @@ cudaError_t dense_product(const Ctx& c, int M, const TcOut* outs, int nout, cons
   return cudaSuccess;
 }
 
+// The LoRA-side products against every expert's block are scheduled block-sparsely (device-built work lists) once
+// the N r columns span more than one 128-column tile; up to one tile the dense form does no extra loads and has
+// fewer, longer work items, which measured faster.
+bool block_sparse(const Ctx& c) { return c.s.n_experts * c.s.rank > 128; }
+
 int dense_launches(const Ctx& c, int M, const TcOut* outs, int nout) {
   if (nout == 0 || M <= 0) return 0;
   return (c.bf16 && tc_gemm_supported(M, outs, nout)) ? 1 : nout;
@@ -355,12 +360,13 @@ static mixlora_status_t fwd_experts(const Ctx& c, void* y) {
   {
     TcOut out = tc_out(c.ws + c.L.zd_all, Nr, Nr);
     tc_add(out, c.ws + c.L.h_sorted, f, f, params->a_down, f, 0);
-    StageScope ss(ST_LORA_A_DOWN, c.st, 1 + dense_launches(c, T * k, &out, 1));
+    StageScope ss(ST_LORA_A_DOWN, c.st, (block_sparse(c) ? 1 : 0) + dense_launches(c, T * k, &out, 1));
     // only the block of a slot's own expert is needed: schedule (row tile, expert) pairs that exist
     TcWork wl = {c.at<int>(c.L.work_rows1), c.at<int>(c.L.work_count) + 0, rows_worklist_max(T * k, N, 1), r};
-    MIXLORA_CUDA(launch_rows_worklist(c, tc_gemm_tile_rows(T * k), 1, (f + 63) / 64, c.at<int>(c.L.work_rows1),
-                                      c.at<int>(c.L.work_count) + 0));
-    MIXLORA_CUDA(dense_product(c, T * k, &out, 1, &wl));
+    if (block_sparse(c))
+      MIXLORA_CUDA(launch_rows_worklist(c, tc_gemm_tile_rows(T * k), 1, (f + 63) / 64, c.at<int>(c.L.work_rows1),
+                                        c.at<int>(c.L.work_count) + 0));
+    MIXLORA_CUDA(dense_product(c, T * k, &out, 1, block_sparse(c) ? &wl : nullptr));
   }
   { StageScope ss(ST_COMBINE_H, c.st, c.bf16 ? 3 : 2); MIXLORA_CUDA(launch_combine_h(c)); MIXLORA_CUDA(launch_bd_cat(c)); }
   // y = [hbar | Zs] [W_d | s B_d]^T : the frozen down projection acts once on the gate-weighted sum of a
@@ -534,11 +540,12 @@ static mixlora_status_t bwd_experts(const Ctx& c, const void* dy, float aux_coef
     TcOut outs[2];
     outs[0] = tc_out(c.ws + c.L.dzg_all, Nr, Nr); tc_add(outs[0], c.ws + c.L.da_sorted, f, f, c.ws + c.L.bg_cat, Nr, 1);
     outs[1] = tc_out(c.ws + c.L.dzu_all, Nr, Nr); tc_add(outs[1], c.ws + c.L.db_sorted, f, f, c.ws + c.L.bu_cat, Nr, 1);
-    StageScope ss(ST_LORA_DZ, c.st, 1 + dense_launches(c, T * k, outs, 2));
+    StageScope ss(ST_LORA_DZ, c.st, (block_sparse(c) ? 1 : 0) + dense_launches(c, T * k, outs, 2));
     TcWork wl = {c.at<int>(c.L.work_rows2), c.at<int>(c.L.work_count) + 1, rows_worklist_max(T * k, N, 2), r};
-    MIXLORA_CUDA(launch_rows_worklist(c, tc_gemm_tile_rows(T * k), 2, (f + 63) / 64, c.at<int>(c.L.work_rows2),
-                                      c.at<int>(c.L.work_count) + 1));
-    MIXLORA_CUDA(dense_product(c, T * k, outs, 2, &wl));
+    if (block_sparse(c))
+      MIXLORA_CUDA(launch_rows_worklist(c, tc_gemm_tile_rows(T * k), 2, (f + 63) / 64, c.at<int>(c.L.work_rows2),
+                                        c.at<int>(c.L.work_count) + 1));
+    MIXLORA_CUDA(dense_product(c, T * k, outs, 2, block_sparse(c) ? &wl : nullptr));
   }
   // router: gates -> probabilities -> logits
   {
@@ -562,13 +569,14 @@ static mixlora_status_t bwd_experts(const Ctx& c, const void* dy, float aux_coef
       outs[n] = tc_out_f32(grads->d_a_down, Nr, 1, f, 0, 0, 1.f, acc);
       tc_add(outs[n++], c.ws + c.L.h_sorted, f, T * k, c.ws + c.L.dZd_pos, Nr, 1, 1);
     }
-    StageScope ss(ST_LORA_WGRAD, c.st, 1 + dense_launches(c, f, outs, n));
+    StageScope ss(ST_LORA_WGRAD, c.st, (block_sparse(c) ? 1 : 0) + dense_launches(c, f, outs, n));
     if (n > 0) {
       // each expert's block is a sum over that expert's segment of sorted slots only
       TcWork wl = {c.at<int>(c.L.work_red), c.at<int>(c.L.work_count) + 2, reduce_worklist_max(f, N, n), r};
-      MIXLORA_CUDA(launch_reduce_worklist(c, f, tc_gemm_tile_rows(f), n, c.at<int>(c.L.work_red),
-                                          c.at<int>(c.L.work_count) + 2));
-      MIXLORA_CUDA(dense_product(c, f, outs, n, &wl));
+      if (block_sparse(c))
+        MIXLORA_CUDA(launch_reduce_worklist(c, f, tc_gemm_tile_rows(f), n, c.at<int>(c.L.work_red),
+                                            c.at<int>(c.L.work_count) + 2));
+      MIXLORA_CUDA(dense_product(c, f, outs, n, block_sparse(c) ? &wl : nullptr));
     }
   }
   // ... and over the tokens (d-sized matrices and the router weight)
