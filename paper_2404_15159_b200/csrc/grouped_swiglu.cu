@@ -6,13 +6,19 @@
 //   producer warp : TMA loads of the rank-r operands: the tile's rows of zg / zu (/ s pd) and the COLS rows of
 //                   B_g[e] / B_u[e] (/ the r rows of A_d[e]); a few KB per item
 //   MMA warp      : da = zg B_g[e]^T, db = zu B_u[e]^T (, dd = (s pd) A_d[e]) as tcgen05.mma with K = r into TMEM
-//   16 epilogue warps:
-//     - gather the shared projections G, U (and D = dy W_d) of the tile's tokens with cp.async, four rows of 128
-//       contiguous bytes per warp instruction, one item ahead, into 128B-swizzled smem tiles
-//     - a = G + da, b = U + db, h = SiLU(a) b            (backward: Dt = D + dd, dgate, d a, d b as well)
-//     - results go to swizzled smem tiles and leave with TMA tile stores (full tiles) or predicated stores
-//       (the last, shorter tile of a segment, whose remaining rows belong to the next expert)
-// All waits are bounded as in the dense product; the epilogue warps leave their loop together.
+//   gather warps  : fetch the shared projections G, U (and D = dy W_d) of the tile's tokens with cp.async, four
+//                   rows of 128 contiguous bytes per warp instruction, into a ring of 128B-swizzled smem tiles,
+//                   up to three items ahead of the epilogue; they also look up the item's slot range and gates
+//   16 epilogue warps: a = G + da, b = U + db, h = SiLU(a) b (backward: Dt = D + dd, dgate, d a, d b as well) in
+//                   packed fp32 pairs, into one of two swizzled output tiles; one CTA-wide barrier per item
+//   store warp    : after that barrier, sends full tiles out by TMA, waits until the copy has read the tile and
+//                   hands it back; the last, shorter tile of a segment (whose remaining rows belong to the next
+//                   expert) is copied out by the epilogue threads with predicated stores instead
+// The TMA stores of these 128-byte-wide boxes drain at about 15 cycles per row and SM, which paces the kernel; both
+// other ways out (coalesced stores from the smem tile, 32-byte stores straight from the registers) measured slower.
+// All waits are bounded as in the dense product.
+#include <algorithm>
+
 #include "common.cuh"
 #include "tc_ptx.cuh"
 
@@ -24,48 +30,83 @@ using namespace tc;
 
 constexpr int kSplit = 4;                 // epilogue warps per TMEM lane quarter
 constexpr int NET = 128 * kSplit;         // epilogue threads
-constexpr int kThreads = 64 + NET;
+constexpr int kStoreWarp = 2;             // issues the TMA stores of the results
+constexpr int kGatherWarps = 4;           // warps that fetch the G / U / D rows
+constexpr int NGT = 32 * kGatherWarps;
+constexpr int kFirstGatherWarp = 3;
+constexpr int kFirstEpiWarp = kFirstGatherWarp + kGatherWarps;
+constexpr int kThreads = 32 * kFirstEpiWarp + NET;
+constexpr int kRowsPerPass = NGT / 8;     // rows one pass of the gather threads covers
+constexpr int kPasses = 128 / kRowsPerPass;
 constexpr uint32_t kTmemCols = 512;
 constexpr uint32_t kBufStride = 256;
 constexpr int kMaxStages = 4;
+constexpr int kMaxSets = 4;               // gathered tiles in flight per CTA
+constexpr int kHdrFloats = 128 + 4;       // per set: gates of the 128 rows, first slot, row count, column tile
 constexpr uint32_t kBlockBytes = 128 * 128;   // one 64-column block of a 128-row tile
 
 struct alignas(64) GsParams {
   CUtensorMap a_map[3];    // zg_s, zu_s, p_s : [slots, RP]
   CUtensorMap b_map[3];    // B_g, B_u as [N f, RP] ; A_d as [N r, f]
-  CUtensorMap o_map[3];    // h, da, db : [slots, f]
+  CUtensorMap o_map[2];    // h (forward) ; da, db (backward) : [slots, f]
   const bf16* G; const bf16* U; const bf16* D;
   const int* pos_token; const int* perm; const float* gates; const int* tile_info;
   bf16* h; bf16* da; bf16* db;
   float* dgate_part;       // [col_tiles, slots]
-  int max_tiles, slots, f, r, row_bytes, kblocks, ksteps, krows, col_tiles, nstages, out_sets;
+  int max_tiles, slots, f, r, row_bytes, kblocks, ksteps, krows, col_tiles, col_group, nstages, nsets, out_sets;
   uint32_t stage_bytes, a_bytes;
   int* status;
 };
 
-__device__ __forceinline__ void unpack8(const uint4& raw, float* o) {
-  const __nv_bfloat162* p = reinterpret_cast<const __nv_bfloat162*>(&raw);
-#pragma unroll
-  for (int i = 0; i < 4; ++i) {
-    float2 v = __bfloat1622float2(p[i]);
-    o[2 * i] = v.x;
-    o[2 * i + 1] = v.y;
-  }
-}
-__device__ __forceinline__ uint4 pack8(const float* v) {
-  uint4 r;
-  __nv_bfloat162 h0 = __floats2bfloat162_rn(v[0], v[1]), h1 = __floats2bfloat162_rn(v[2], v[3]);
-  __nv_bfloat162 h2 = __floats2bfloat162_rn(v[4], v[5]), h3 = __floats2bfloat162_rn(v[6], v[7]);
-  r.x = *reinterpret_cast<uint32_t*>(&h0); r.y = *reinterpret_cast<uint32_t*>(&h1);
-  r.z = *reinterpret_cast<uint32_t*>(&h2); r.w = *reinterpret_cast<uint32_t*>(&h3);
+// Packed fp32 pairs: one add / mul / fma instruction works on both halves of a 64-bit register pair, which halves
+// the issue slots of the element-wise math (the kernel is bound by instruction issue, not by a pipe).
+__device__ __forceinline__ uint64_t pk2(float lo, float hi) {
+  uint64_t r;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
   return r;
 }
-// sigmoid(a) = 0.5 tanh(a / 2) + 0.5 with the hardware tanh approximation (one special-function op;
+__device__ __forceinline__ uint64_t pk2u(uint32_t lo, uint32_t hi) {
+  uint64_t r;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "r"(lo), "r"(hi));
+  return r;
+}
+__device__ __forceinline__ void upk2(uint64_t v, float& lo, float& hi) {
+  asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ uint64_t add2(uint64_t a, uint64_t b) {
+  uint64_t r;
+  asm("add.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+  return r;
+}
+__device__ __forceinline__ uint64_t mul2(uint64_t a, uint64_t b) {
+  uint64_t r;
+  asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+  return r;
+}
+__device__ __forceinline__ uint64_t fma2(uint64_t a, uint64_t b, uint64_t c) {
+  uint64_t r;
+  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(r) : "l"(a), "l"(b), "l"(c));
+  return r;
+}
+constexpr uint64_t kHalf2 = 0x3f0000003f000000ull;      // (0.5f, 0.5f)
+constexpr uint64_t kOne2 = 0x3f8000003f800000ull;       // (1.0f, 1.0f)
+constexpr uint64_t kMinusOne2 = 0xbf800000bf800000ull;  // (-1.0f, -1.0f)
+// two bf16 in one word -> two fp32 (exact)
+__device__ __forceinline__ uint64_t bf2_to_f2(uint32_t v) { return pk2u(v << 16, v & 0xffff0000u); }
+__device__ __forceinline__ uint32_t f2_to_bf2(uint64_t v) {
+  float lo, hi;
+  upk2(v, lo, hi);
+  __nv_bfloat162 h = __floats2bfloat162_rn(lo, hi);
+  return *reinterpret_cast<uint32_t*>(&h);
+}
+// sigmoid(a) = 0.5 tanh(a / 2) + 0.5 with the hardware tanh approximation (one special-function op per value;
 // its error is below the bf16 rounding of every value stored from here)
-__device__ __forceinline__ float fast_sigmoid(float a) {
-  float t;
-  asm("tanh.approx.f32 %0, %1;" : "=f"(t) : "f"(0.5f * a));
-  return fmaf(t, 0.5f, 0.5f);
+__device__ __forceinline__ uint64_t sigmoid2(uint64_t a) {
+  float lo, hi, tl, th;
+  upk2(mul2(a, kHalf2), lo, hi);
+  asm("tanh.approx.f32 %0, %1;" : "=f"(tl) : "f"(lo));
+  asm("tanh.approx.f32 %0, %1;" : "=f"(th) : "f"(hi));
+  return fma2(pk2(tl, th), kHalf2, kHalf2);
 }
 template <int BWD>
 __global__ void __launch_bounds__(kThreads, 1) grouped_swiglu_kernel(const __grid_constant__ GsParams p) {
@@ -78,17 +119,18 @@ __global__ void __launch_bounds__(kThreads, 1) grouped_swiglu_kernel(const __gri
   constexpr uint32_t kSetBytes = NMAT * CB * kBlockBytes;
   constexpr uint32_t kOutBytes = NOUT * CB * kBlockBytes;
   constexpr int WCOLS = COLS / kSplit;                 // columns per epilogue thread
-  constexpr int NCH = WCOLS / 8;
 
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-  uint8_t* gather_smem = smem;                                    // two sets
-  uint8_t* out_smem = gather_smem + 2 * kSetBytes;
-  uint8_t* stage_smem = out_smem + p.out_sets * kOutBytes;          // one or two output tiles
-  float* dg_smem = reinterpret_cast<float*>(stage_smem + p.nstages * p.stage_bytes);   // [kSplit][128]
-  uint64_t* bars = reinterpret_cast<uint64_t*>(dg_smem + (BWD ? kSplit * BM : 0));
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * kMaxStages + 4);
+  uint8_t* gather_smem = smem;                                    // nsets sets
+  uint8_t* out_smem = gather_smem + p.nsets * kSetBytes;           // one or two output tiles
+  uint8_t* stage_smem = out_smem + p.out_sets * kOutBytes;
+  float* dg_smem = reinterpret_cast<float*>(stage_smem + p.nstages * p.stage_bytes);   // [2][kSplit][128]
+  float* hdr_smem = dg_smem + (BWD ? 2 * kSplit * BM : 0);                              // [nsets][kHdrFloats]
+  uint64_t* bars = reinterpret_cast<uint64_t*>(hdr_smem + p.nsets * kHdrFloats);
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * kMaxStages + 6 + 2 * kMaxSets);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+  int* out_hdr = reinterpret_cast<int*>(tmem_slot + 4);   // [2][4]: first slot, rows, column tile of the item in each output tile's turn
   volatile int* epi_stop = reinterpret_cast<volatile int*>(tmem_slot + 2);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -98,10 +140,18 @@ __global__ void __launch_bounds__(kThreads, 1) grouped_swiglu_kernel(const __gri
   auto empty_bar = [&](int s) { return bar_base + 8u * (kMaxStages + s); };
   auto tfull_bar = [&](int b) { return bar_base + 8u * (2 * kMaxStages + b); };
   auto tempty_bar = [&](int b) { return bar_base + 8u * (2 * kMaxStages + 2 + b); };
+  auto gfull_bar = [&](int b) { return bar_base + 8u * (2 * kMaxStages + 4 + b); };
+  auto gempty_bar = [&](int b) { return bar_base + 8u * (2 * kMaxStages + 4 + kMaxSets + b); };
+  auto ofree_bar = [&](int b) { return bar_base + 8u * (2 * kMaxStages + 4 + 2 * kMaxSets + b); };
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < kMaxStages; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
-    for (int b = 0; b < 2; ++b) { mbar_init(tfull_bar(b), 1); mbar_init(tempty_bar(b), 4 * kSplit); }
+    for (int b = 0; b < 2; ++b) {
+      mbar_init(tfull_bar(b), 1); mbar_init(tempty_bar(b), 4 * kSplit); mbar_init(ofree_bar(b), 1);
+    }
+    // a set is full when every gather thread's copies have landed (one asynchronous arrival each) and its header
+    // is written (one plain arrival each); it is empty again when every epilogue warp has read it
+    for (int b = 0; b < kMaxSets; ++b) { mbar_init(gfull_bar(b), 2 * NGT); mbar_init(gempty_bar(b), 4 * kSplit); }
     *abort_flag = 0;
     *epi_stop = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -117,6 +167,16 @@ __global__ void __launch_bounds__(kThreads, 1) grouped_swiglu_kernel(const __gri
   const int ntiles = min(p.tile_info[p.max_tiles * 4], p.max_tiles);
   const int total = ntiles * p.col_tiles;
   const int kb_cols = p.row_bytes / 2;                 // K elements per k-block (16, 32 or 64)
+  // Item order: groups of col_group column tiles, inside a group every segment tile in turn.  The slots of a token
+  // (they sit in different experts' segments) are then worked on while the token's piece of G / U / D is still in
+  // L2, so DRAM sees each piece once; inside a group the CTAs still sweep col_group tiles of the same rows together.
+  const int per_group = ntiles * p.col_group;
+  auto item_at = [&](int w, int& tile, int& ct) {
+    const int g = w / per_group, rem = w - g * per_group;
+    const int gw = min(p.col_group, p.col_tiles - g * p.col_group);   // the last group may be narrower
+    tile = rem / gw;
+    ct = g * p.col_group + rem % gw;
+  };
 
   if (warp == 0) {
     // ---------------- producer: rank-r operands ----------------
@@ -125,7 +185,9 @@ __global__ void __launch_bounds__(kThreads, 1) grouped_swiglu_kernel(const __gri
       uint32_t it = 0;
       bool ok = true;
       for (int w = blockIdx.x; w < total && ok; w += gridDim.x) {
-        const int tile = w / p.col_tiles, col0 = (w % p.col_tiles) * COLS;
+        int tile, ct;
+        item_at(w, tile, ct);
+        const int col0 = ct * COLS;
         const int e = p.tile_info[tile * 4 + 0], p0 = p.tile_info[tile * 4 + 1];
         for (int sub = 0; sub < NSUB && ok; ++sub) {
           for (int kb = 0; kb < p.kblocks; ++kb, ++it) {
@@ -188,78 +250,156 @@ __global__ void __launch_bounds__(kThreads, 1) grouped_swiglu_kernel(const __gri
         if (p.status) atomicExch(p.status, (int)MIXLORA_ERR_DEVICE_TIMEOUT);
       }
     }
+  } else if (warp == kStoreWarp) {
+    // ---------------- store warp ----------------
+    if (lane == 0) {
+      for (int m = 0; m < NOUT; ++m) prefetch_tmap(&p.o_map[m]);
+    }
+    const uint32_t out_base = smem_u32(out_smem);
+    int prev_o = -1;
+    uint32_t n = 0;
+    for (int w = blockIdx.x; w < total; w += gridDim.x, ++n) {
+      named_barrier(1, NET + 32);                      // the item's results are complete in its output tile
+      if (*epi_stop) break;
+      if (lane == 0) {
+        // every epilogue thread is past the previous item (also past copying a short tile out), and that item's
+        // TMA stores have read its tile (waited for below): the tile may be written again
+        if (prev_o >= 0) mbar_arrive(ofree_bar(prev_o));
+        const int o = p.out_sets == 2 ? (int)(n & 1u) : 0;
+        const int* hdr = reinterpret_cast<const int*>(out_hdr + 4 * (n & 1u));
+        const int p0 = hdr[0], rows = hdr[1], col0 = hdr[2] * COLS;
+        if (rows == BM) {
+#pragma unroll
+          for (int m = 0; m < NOUT; ++m)
+#pragma unroll
+            for (int j = 0; j < CB; ++j)
+              tma_store_2d(&p.o_map[m], out_base + o * kOutBytes + (m * CB + j) * kBlockBytes, col0 + j * 64, p0);
+        }
+        tma_store_commit();
+        tma_store_wait_read<0>();
+        prev_o = o;
+      }
+      if (p.out_sets == 1) {
+        // a single output tile is handed back at once: after the copy has read it or, for a short tile, after
+        // the epilogue threads have copied it out (they meet the store warp once more)
+        const int rows = out_hdr[4 * (n & 1u) + 1];
+        if (rows < BM) named_barrier(2, NET + 32);
+        if (lane == 0) mbar_arrive(ofree_bar(0));
+        prev_o = -1;
+      }
+      __syncwarp();
+    }
+    if (lane == 0) tma_store_wait_all<0>();
+  } else if (warp < kFirstEpiWarp) {
+    // ---------------- gather warps: rows of G, U (, D) of the item's tokens ----------------
+    // Thread -> 16-byte chunk g_cb of rows g_r0, g_r0 + kRowsPerPass, ... of every 64-column block, so a warp
+    // instruction reads 4 rows x 128 contiguous bytes.  The copies of one item signal gfull[set] when they have
+    // landed; the warps run ahead of the epilogue by the depth of the ring and never block on the data.
+    const int gt = threadIdx.x - 32 * kFirstGatherWarp;
+    const int g_r0 = gt >> 3, g_cb = gt & 7;
+    const uint32_t g_dst0 = smem_u32(gather_smem) + g_r0 * 128 + ((g_cb ^ (g_r0 & 7)) << 4);
+    int set = 0;
+    uint32_t set_use = 0;                              // times the ring has wrapped
+    bool ok = true;
+    for (int w = blockIdx.x; w < total; w += gridDim.x) {
+      // everything the item needs from global memory besides the rows themselves is fetched before the wait for
+      // a free set, so those dependent loads never delay the copies
+      int tile, ct;
+      item_at(w, tile, ct);
+      const int col0 = ct * COLS;
+      const int p0 = p.tile_info[tile * 4 + 1], rows = p.tile_info[tile * 4 + 2];
+      // rows past the tile's end and columns past f are clamped to valid data: what is computed from them is
+      // never stored (kRowsPerPass is a multiple of 8, so the swizzle term of a thread's rows is constant)
+      size_t roff[kPasses];
+#pragma unroll
+      for (int ps = 0; ps < kPasses; ++ps)
+        roff[ps] = (size_t)p.pos_token[p0 + min(g_r0 + kRowsPerPass * ps, rows - 1)] * p.f;
+      float gate0 = 0.f, gate1 = 0.f;                  // gates of rows gt and (fewer than 128 gather threads) gt + NGT
+      if (BWD) {
+        if (gt < rows) gate0 = p.gates[p.perm[p0 + gt]];
+        if (NGT < 128 && gt + NGT < rows) gate1 = p.gates[p.perm[p0 + gt + NGT]];
+      }
+      if (!mbar_wait(gempty_bar(set), (set_use & 1u) ^ 1u, abort_flag)) { ok = false; break; }
+      float* hdr = hdr_smem + set * kHdrFloats;
+      if (BWD) {
+        hdr[gt] = gate0;
+        if (NGT < 128) hdr[gt + NGT] = gate1;
+      }
+      if (gt == 0) {
+        reinterpret_cast<int*>(hdr)[128] = p0;
+        reinterpret_cast<int*>(hdr)[129] = rows;
+        reinterpret_cast<int*>(hdr)[130] = ct;
+      }
+      const uint32_t dst_set = g_dst0 + set * kSetBytes;
+#pragma unroll
+      for (int j = 0; j < CB; ++j) {
+        const int col = min(col0 + j * 64 + g_cb * 8, p.f - 8);
+        // D is zero-filled past column f: those columns must not add to the row's <Dt, h>
+        const uint32_t d_bytes = col0 + j * 64 + g_cb * 8 < p.f ? 16u : 0u;
+#pragma unroll
+        for (int m = 0; m < NMAT; ++m) {
+          const bf16* base = (m == 0 ? p.G : (m == 1 ? p.U : p.D)) + col;
+          const uint32_t dst = dst_set + (m * CB + j) * kBlockBytes;
+#pragma unroll
+          for (int ps = 0; ps < kPasses; ++ps) {
+            if (m < 2)
+              asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst + ps * kRowsPerPass * 128),
+                           "l"(base + roff[ps])
+                           : "memory");
+            else
+              asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst + ps * kRowsPerPass * 128),
+                           "l"(base + roff[ps]), "r"(d_bytes)
+                           : "memory");
+          }
+        }
+      }
+      asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];" ::"r"(gfull_bar(set)) : "memory");
+      mbar_arrive(gfull_bar(set));                     // publishes the header
+      if (++set == p.nsets) { set = 0; ++set_use; }
+    }
+    asm volatile("cp.async.wait_all;" ::: "memory");
+    if (!ok && lane == 0) {
+      *abort_flag = 1;
+      if (p.status) atomicExch(p.status, (int)MIXLORA_ERR_DEVICE_TIMEOUT);
+    }
   } else {
     // ---------------- epilogue ----------------
     const int q = warp & 3;                            // TMEM lane quarter this warp may read
-    const int part = (warp - 2) >> 2;                  // column share of the tile
-    const int et = threadIdx.x - 64;
+    const int part = (warp - kFirstEpiWarp) >> 2;      // column share of the tile
+    const int et = threadIdx.x - 32 * kFirstEpiWarp;
     const int row = q * 32 + lane;                     // this thread's row of the tile
-    const uint32_t gs_base = smem_u32(gather_smem);
-    const uint32_t out_base = smem_u32(out_smem);
-
-    // Cooperative gather of item w into `set`.  Thread -> rows g_r0 and g_r0 + 64 of every 64-column block and the
-    // 16-byte chunk g_cb of those rows, so a warp instruction reads 4 rows x 128 contiguous bytes.  Everything
-    // that does not depend on the item is computed once here.
-    const int g_r0 = et >> 3, g_cb = et & 7;
-    const uint32_t g_dst0 = gs_base + g_r0 * 128 + ((g_cb ^ (g_r0 & 7)) << 4);
-    auto gather = [&](int w, int set) {
-      const int tile = w / p.col_tiles, col0 = (w % p.col_tiles) * COLS;
-      const int p0 = p.tile_info[tile * 4 + 1], rows = p.tile_info[tile * 4 + 2];
-      const bool in0 = g_r0 < rows, in1 = g_r0 + 64 < rows;
-      const size_t row0 = (size_t)(in0 ? p.pos_token[p0 + g_r0] : 0) * p.f + col0 + g_cb * 8;
-      const size_t row1 = (size_t)(in1 ? p.pos_token[p0 + g_r0 + 64] : 0) * p.f + col0 + g_cb * 8;
-      const uint32_t dst_set = g_dst0 + set * kSetBytes;
-#pragma unroll
-      for (int m = 0; m < NMAT; ++m) {
-        const bf16* base = m == 0 ? p.G : (m == 1 ? p.U : p.D);
-#pragma unroll
-        for (int j = 0; j < CB; ++j) {
-          const bool cin = col0 + j * 64 + g_cb * 8 < p.f;
-          const uint32_t dst = dst_set + (m * CB + j) * kBlockBytes;
-          const bool a0 = in0 && cin, a1 = in1 && cin;
-          const bf16* s0 = a0 ? base + row0 + j * 64 : base;
-          const bf16* s1 = a1 ? base + row1 + j * 64 : base;
-          asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(s0), "r"(a0 ? 16 : 0) : "memory");
-          asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst + 64 * 128), "l"(s1), "r"(a1 ? 16 : 0)
-                       : "memory");
-        }
-      }
-      asm volatile("cp.async.commit_group;" ::: "memory");
-    };
+    // this thread's columns are 16-byte chunks part * (WCOLS / 8) + ch of the tile; all lie in one 64-column block
+    const int jblk = (part * (WCOLS / 8)) >> 3, cb0 = (part * (WCOLS / 8)) & 7, rx = row & 7;
+    const uint32_t row_off = jblk * kBlockBytes + row * 128;
 
     uint32_t wcount = 0;
-    if ((int)blockIdx.x < total) gather(blockIdx.x, 0);
+    int set = 0;
+    uint32_t set_use = 0;
     for (int w = blockIdx.x; w < total; w += gridDim.x, ++wcount) {
-      const int tile = w / p.col_tiles, ct = w % p.col_tiles;
-      const int col0 = ct * COLS;
-      const int p0 = p.tile_info[tile * 4 + 1], rows = p.tile_info[tile * 4 + 2];
       const uint32_t buf = wcount & 1u, use = wcount >> 1;
-      const int set = wcount & 1u;
-      const bool valid = row < rows;
-      const bool full_tile = rows == BM;
-      const int pos = p0 + row;
-      float gate = 0.f;
-      if (BWD && valid) gate = p.gates[p.perm[pos]];
-
-      if (w + (int)gridDim.x < total) gather(w + gridDim.x, set ^ 1);
-      else asm volatile("cp.async.commit_group;" ::: "memory");
-      asm volatile("cp.async.wait_group 1;" ::: "memory");
-      const int oidx = p.out_sets == 2 ? set : 0;      // output tile of this item
-      if (et == 0) {                                   // earlier stores have finished reading that tile
-        if (p.out_sets == 2) tma_store_wait_read<1>(); else tma_store_wait_read<0>();
-      }
-      named_barrier(1, NET);                           // this item's gathers are visible; the output tile is free
-
-      const bool got = __all_sync(0xffffffffu, mbar_wait(tfull_bar(buf), use & 1u, abort_flag));
+      const int oidx = p.out_sets == 2 ? (int)buf : 0;  // output tile of this item
+      const uint32_t o_use = p.out_sets == 2 ? use : wcount;
+      const bool got = __all_sync(0xffffffffu, mbar_wait(gfull_bar(set), set_use & 1u, abort_flag) &&
+                                                   mbar_wait(tfull_bar(buf), use & 1u, abort_flag) &&
+                                                   mbar_wait(ofree_bar(oidx), (o_use & 1u) ^ 1u, abort_flag));
+      int ct = 0, pos = 0, p0 = 0, rows = 0;
       if (got) {
         tc_fence_after();
+        const float* hdr = hdr_smem + set * kHdrFloats;
+        p0 = reinterpret_cast<const int*>(hdr)[128];
+        rows = reinterpret_cast<const int*>(hdr)[129];
+        ct = reinterpret_cast<const int*>(hdr)[130];
+        pos = p0 + row;
+        if (et == 0) {                                 // for the store warp: the set itself is released earlier
+          int* oh = out_hdr + 4 * (wcount & 1u);
+          oh[0] = p0; oh[1] = rows; oh[2] = ct;
+        }
         const uint32_t t_addr = tmem_base + ((uint32_t)(q * 32) << 16) + buf * kBufStride + part * WCOLS;
         const uint8_t* gset = gather_smem + set * kSetBytes;
         uint8_t* oset = out_smem + oidx * kOutBytes;
-        // this thread's columns are chunks c8 = part * NCH + ch of the tile; all lie in one 64-column block
-        const int jblk = (part * NCH) >> 3, cb0 = (part * NCH) & 7, rx = row & 7;
-        const uint32_t row_off = jblk * kBlockBytes + row * 128;
-        float dg = 0.f;
+        uint64_t dg2 = 0;
+        const float gate = BWD ? hdr[row] : 0.f;
+        const uint64_t gate2 = pk2(gate, gate);
 #pragma unroll
         for (int c16 = 0; c16 < WCOLS; c16 += 16) {
           uint32_t va[16], vb[16], vd[BWD ? 16 : 1];
@@ -271,78 +411,84 @@ __global__ void __launch_bounds__(kThreads, 1) grouped_swiglu_kernel(const __gri
           for (int hh8 = 0; hh8 < 2; ++hh8) {
             const int ch = c16 / 8 + hh8;
             const uint32_t off = row_off + (((cb0 + ch) ^ rx) << 4);
-            float gv[8], uv[8], hv[8];
-            unpack8(*reinterpret_cast<const uint4*>(gset + 0 * CB * kBlockBytes + off), gv);
-            unpack8(*reinterpret_cast<const uint4*>(gset + 1 * CB * kBlockBytes + off), uv);
-            const int col = col0 + (part * NCH + ch) * 8;
-            const size_t gdst = (size_t)pos * p.f + col;
-            const bool direct = !full_tile && valid && col < p.f;
+            const uint4 rg = *reinterpret_cast<const uint4*>(gset + 0 * CB * kBlockBytes + off);
+            const uint4 ru = *reinterpret_cast<const uint4*>(gset + 1 * CB * kBlockBytes + off);
+            const uint32_t wg[4] = {rg.x, rg.y, rg.z, rg.w}, wu[4] = {ru.x, ru.y, ru.z, ru.w};
             if (!BWD) {
+              uint32_t ho[4];
 #pragma unroll
-              for (int i = 0; i < 8; ++i) {
-                const float a = gv[i] + __uint_as_float(va[hh8 * 8 + i]);
-                const float b = uv[i] + __uint_as_float(vb[hh8 * 8 + i]);
-                hv[i] = a * fast_sigmoid(a) * b;
+              for (int i = 0; i < 4; ++i) {
+                const int v = hh8 * 8 + 2 * i;
+                const uint64_t a = add2(bf2_to_f2(wg[i]), pk2u(va[v], va[v + 1]));
+                const uint64_t b = add2(bf2_to_f2(wu[i]), pk2u(vb[v], vb[v + 1]));
+                ho[i] = f2_to_bf2(mul2(mul2(a, sigmoid2(a)), b));
               }
-              const uint4 ho = pack8(hv);
-              if (full_tile) *reinterpret_cast<uint4*>(oset + off) = ho;
-              else if (direct) *reinterpret_cast<uint4*>(p.h + gdst) = ho;
+              *reinterpret_cast<uint4*>(oset + off) = make_uint4(ho[0], ho[1], ho[2], ho[3]);
             } else {
-              float dv[8], dav[8], dbv[8];
-              unpack8(*reinterpret_cast<const uint4*>(gset + 2 * CB * kBlockBytes + off), dv);
+              const uint4 rd = *reinterpret_cast<const uint4*>(gset + 2 * CB * kBlockBytes + off);
+              const uint32_t wd[4] = {rd.x, rd.y, rd.z, rd.w};
+              uint32_t ao[4], bo[4];
 #pragma unroll
-              for (int i = 0; i < 8; ++i) {
-                const float a = gv[i] + __uint_as_float(va[hh8 * 8 + i]);
-                const float b = uv[i] + __uint_as_float(vb[hh8 * 8 + i]);
-                const float sg = fast_sigmoid(a);
-                const float sa = a * sg;
-                const float hh = sa * b;
-                const float Dt = dv[i] + __uint_as_float(vd[BWD ? hh8 * 8 + i : 0]);
-                dg = fmaf(Dt, hh, dg);
-                const float dh = gate * Dt;
-                dav[i] = dh * b * sg * (1.f + a * (1.f - sg));
-                dbv[i] = dh * sa;
+              for (int i = 0; i < 4; ++i) {
+                const int v = hh8 * 8 + 2 * i;
+                const uint64_t a = add2(bf2_to_f2(wg[i]), pk2u(va[v], va[v + 1]));
+                const uint64_t b = add2(bf2_to_f2(wu[i]), pk2u(vb[v], vb[v + 1]));
+                const uint64_t Dt = add2(bf2_to_f2(wd[i]), pk2u(vd[BWD ? v : 0], vd[BWD ? v + 1 : 0]));
+                const uint64_t sg = sigmoid2(a);
+                const uint64_t sa = mul2(a, sg);                         // SiLU(a)
+                dg2 = fma2(Dt, mul2(sa, b), dg2);                        // <Dt, h>
+                const uint64_t dh = mul2(gate2, Dt);
+                // SiLU'(a) = sg (1 + a (1 - sg))
+                const uint64_t ds = mul2(sg, fma2(a, fma2(sg, kMinusOne2, kOne2), kOne2));
+                ao[i] = f2_to_bf2(mul2(mul2(dh, b), ds));
+                bo[i] = f2_to_bf2(mul2(dh, sa));
               }
-              const uint4 ao = pack8(dav), bo = pack8(dbv);
-              if (full_tile) {
-                *reinterpret_cast<uint4*>(oset + 0 * CB * kBlockBytes + off) = ao;
-                *reinterpret_cast<uint4*>(oset + 1 * CB * kBlockBytes + off) = bo;
-              } else if (direct) {
-                *reinterpret_cast<uint4*>(p.da + gdst) = ao;
-                *reinterpret_cast<uint4*>(p.db + gdst) = bo;
-              }
+              *reinterpret_cast<uint4*>(oset + 0 * CB * kBlockBytes + off) = make_uint4(ao[0], ao[1], ao[2], ao[3]);
+              *reinterpret_cast<uint4*>(oset + 1 * CB * kBlockBytes + off) = make_uint4(bo[0], bo[1], bo[2], bo[3]);
             }
           }
         }
         tc_fence_before();
         __syncwarp();
-        if (lane == 0) mbar_arrive(tempty_bar(buf));
-        if (BWD) dg_smem[part * BM + row] = dg;
+        if (lane == 0) { mbar_arrive(tempty_bar(buf)); mbar_arrive(gempty_bar(set)); }
+        if (BWD) {
+          float dlo, dhi;
+          upk2(dg2, dlo, dhi);
+          dg_smem[(wcount & 1u) * (kSplit * BM) + part * BM + row] = dlo + dhi;
+        }
       } else if (lane == 0) {
         *abort_flag = 1;
         if (p.status) atomicExch(p.status, (int)MIXLORA_ERR_DEVICE_TIMEOUT);
       }
       fence_proxy_async_smem();                        // the tile written above is read by the TMA unit
-      if (et == 0 && *abort_flag) *epi_stop = 1;
-      named_barrier(1, NET);
-      if (et == 0 && got && full_tile) {
-#pragma unroll
-        for (int m = 0; m < NOUT; ++m)
-#pragma unroll
-          for (int j = 0; j < CB; ++j)
-            tma_store_2d(&p.o_map[m], out_base + oidx * kOutBytes + (m * CB + j) * kBlockBytes, col0 + j * 64, p0);
+      if (!got) *epi_stop = 1;
+      // the one CTA-wide barrier of an item (with the store warp): the results are complete in the output tile
+      named_barrier(1, NET + 32);
+      if (got && rows < BM) {
+        // a segment's last, shorter tile: the rows behind it belong to the next expert, so the valid rows are
+        // copied out of the smem tile one 16-byte chunk per thread and turn
+        const uint8_t* otile = out_smem + oidx * kOutBytes;
+        const int col0 = ct * COLS;
+        for (int idx = et; idx < NOUT * CB * 128 * 8; idx += NET) {
+          const int c = idx & 7, rr = (idx >> 3) & 127, blk = idx >> 10;   // blk = matrix * CB + column block
+          const int col = col0 + (blk % CB) * 64 + c * 8;
+          if (rr < rows && col < p.f) {
+            bf16* dst = (BWD ? (blk / CB == 0 ? p.da : p.db) : p.h) + (size_t)(p0 + rr) * p.f + col;
+            *reinterpret_cast<uint4*>(dst) =
+                *reinterpret_cast<const uint4*>(otile + blk * kBlockBytes + rr * 128 + ((c ^ (rr & 7)) << 4));
+          }
+        }
       }
-      if (et == 0) tma_store_commit();                 // one group per item, also when nothing was stored
-      if (BWD && got && part == 0 && valid) {          // the row's partial <Dt, h> over this column tile, fixed order
+      if (p.out_sets == 1 && got && rows < BM) named_barrier(2, NET + 32);
+      if (BWD && got && part == 0 && row < rows) {     // the row's partial <Dt, h> over this column tile, fixed order
         float sdg = 0.f;
 #pragma unroll
-        for (int pp = 0; pp < kSplit; ++pp) sdg += dg_smem[pp * BM + row];
+        for (int pp = 0; pp < kSplit; ++pp) sdg += dg_smem[(wcount & 1u) * (kSplit * BM) + pp * BM + row];
         p.dgate_part[(size_t)ct * p.slots + pos] = sdg;
       }
-      if (*epi_stop) break;                            // same value for every epilogue thread after the barrier
+      if (*epi_stop) break;                            // same value for every thread after the barrier
+      if (++set == p.nsets) { set = 0; ++set_use; }
     }
-    asm volatile("cp.async.wait_all;" ::: "memory");
-    if (et == 0) tma_store_wait_all<0>();
   }
 
   __syncthreads();
@@ -360,7 +506,7 @@ template <int BWD>
 cudaError_t launch_t(const Ctx& c) {
   constexpr int COLS = BWD ? 64 : 128;
   constexpr int CB = COLS / 64;
-  constexpr int NMAT = BWD ? 3 : 2, NOUT = BWD ? 2 : 1;
+  constexpr int NMAT = BWD ? 3 : 2;
   const int slots = c.s.tokens * c.s.top_k, f = c.s.d_ff, r = c.s.rank, N = c.s.n_experts;
   const int rp = r < 16 ? 16 : r;
   GsParams p;
@@ -373,15 +519,22 @@ cudaError_t launch_t(const Ctx& c) {
   const uint32_t b_bytes_k = COLS * p.row_bytes, b_bytes_n = CB * p.krows * 128;
   p.stage_bytes = (uint32_t)align_up(p.a_bytes + (b_bytes_k > b_bytes_n ? b_bytes_k : b_bytes_n), 1024);
   const uint32_t budget = 227 * 1024;
-  p.out_sets = 2;
-  uint32_t fixed = 2 * NMAT * CB * kBlockBytes + 2 * NOUT * CB * kBlockBytes + (BWD ? kSplit * BM * 4 : 0) + 1024 + 256;
-  if (fixed + 2 * p.stage_bytes > budget) {            // wide operands: fall back to one output tile
-    p.out_sets = 1;
-    fixed -= NOUT * CB * kBlockBytes;
-  }
+  // two output tiles and as many gathered tiles in flight as fit beside two operand stages (one output tile for
+  // wide operands), then as many operand stages as fit
+  constexpr int NOUT = BWD ? 2 : 1;
+  const uint32_t set_bytes = NMAT * CB * kBlockBytes, out_bytes = NOUT * CB * kBlockBytes;
+  const uint32_t base = (BWD ? 2 * kSplit * BM * 4 : 0) + 1024 + 256;
+  auto need = [&](int ns, int os) { return ns * (set_bytes + kHdrFloats * 4) + os * out_bytes + base + 2 * p.stage_bytes; };
+  int nsets = kMaxSets, out_sets = 2;
+  while (nsets > 2 && need(nsets, out_sets) > budget) --nsets;
+  if (need(nsets, out_sets) > budget) out_sets = 1;
+  const uint32_t other = base + nsets * kHdrFloats * 4;
+  const uint32_t fixed = nsets * set_bytes + out_sets * out_bytes + other;
+  if (fixed + 2 * p.stage_bytes > budget) return cudaErrorInvalidConfiguration;
   int nst = (int)((budget - fixed) / p.stage_bytes);
   if (nst > kMaxStages) nst = kMaxStages;
-  if (nst < 2) return cudaErrorInvalidConfiguration;
+  p.nsets = nsets;
+  p.out_sets = out_sets;
   p.nstages = nst;
   const uint32_t smem_bytes = fixed + nst * p.stage_bytes;
 
@@ -407,6 +560,9 @@ cudaError_t launch_t(const Ctx& c) {
   p.max_tiles = max_seg_tiles(c.s.tokens, c.s.top_k, N);
   p.slots = slots; p.f = f; p.r = r;
   p.col_tiles = (f + COLS - 1) / COLS;
+  // columns per group: the group's pieces of the gathered matrices (tokens x columns x NMAT) stay well inside L2
+  const long long group_cols = (32ll << 20) / ((long long)c.s.tokens * 2 * NMAT);
+  p.col_group = (int)std::min<long long>(std::max<long long>(group_cols / COLS, 1), p.col_tiles);
   p.status = c.at<int>(c.L.status);
   int dev = 0, sms = 148;
   cudaGetDevice(&dev);
