@@ -327,3 +327,41 @@ def token_forward(x_t, params, top_k, lora_alpha, renormalize=True, forced_exper
         h = silu(a) * b
         y += gates[j] * (P["w_down"] @ h + s * (P["b_down"][e] @ (P["a_down"][e] @ h)))
     return y, route
+
+
+# --------------------------------------------------------------------------- #
+# the block inside its transformer layer (Eq. 5 / Eq. 6)
+# --------------------------------------------------------------------------- #
+def rmsnorm(z, w_norm, eps):
+    """LN of Eq. 5 for LLaMA-class models: root-mean-square normalisation over the model width with a learned
+    per-channel weight (frozen here), `xn = w_norm * z / sqrt(mean(z^2) + eps)`.  Returns (xn [T, d], inv_rms [T])."""
+    z = np.asarray(z, F64)
+    inv_rms = 1.0 / np.sqrt(np.mean(z * z, axis=1) + eps)
+    return z * inv_rms[:, None] * np.asarray(w_norm, F64)[None, :], inv_rms
+
+
+def layer_forward(z, params, w_norm, eps, top_k, lora_alpha, renormalize=True, forced_expert_idx=None):
+    """Eq. 6: `h = MixLoRA(LN(z)) + z`.  Returns (h [T, d], saved) where saved is that of `ffn_forward` on the
+    normalised input plus `xn` and `inv_rms`."""
+    xn, inv_rms = rmsnorm(z, w_norm, eps)
+    y, saved = ffn_forward(xn, params, top_k, lora_alpha, renormalize=renormalize,
+                           forced_expert_idx=forced_expert_idx)
+    saved = dict(saved)
+    saved["xn"] = xn
+    saved["inv_rms"] = inv_rms
+    return np.asarray(z, F64) + y, saved
+
+
+def layer_backward(z, params, w_norm, dh, saved, aux_coef=0.0, aux_f_mode=0):
+    """Chain rule through Eq. 6.  `dh` = dL/dh.  The LoRA and router gradients are those of `ffn_backward` at the
+    normalised input; `d_x` becomes dL/dz = dh (residual path) + the normalisation's Jacobian applied to dL/dxn:
+    with `xh = z * inv_rms`, `u = dL/dxn * w_norm`:  `inv_rms * (u - xh * mean(u * xh))`."""
+    z = np.asarray(z, F64)
+    dh = np.asarray(dh, F64)
+    g = ffn_backward(saved["xn"], params, dh, saved, aux_coef=aux_coef, aux_f_mode=aux_f_mode, want_dx=True)
+    inv_rms = saved["inv_rms"]
+    xh = z * inv_rms[:, None]
+    u = g["d_x"] * np.asarray(w_norm, F64)[None, :]
+    g = dict(g)
+    g["d_x"] = dh + inv_rms[:, None] * (u - xh * np.mean(u * xh, axis=1, keepdims=True))
+    return g

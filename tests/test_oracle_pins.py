@@ -339,3 +339,79 @@ def test_pins_catch_a_wrong_silu_derivative(monkeypatch):
         arr[i] = old
         worst = max(worst, abs((lp - lm) / (2 * step) - g["d_a_gate"].reshape(-1)[i]))
     assert worst > 1e-4
+
+
+# ---- the block inside its layer (Eq. 5 / Eq. 6) -------------------------------
+def test_rmsnorm_rows_have_unit_mean_square_and_ignore_the_input_scale():
+    rng = np.random.default_rng(3)
+    z = rng.normal(size=(6, 16)) * 3.0
+    xn, inv = orc.rmsnorm(z, np.ones(16), 0.0)
+    np.testing.assert_allclose(np.mean(xn * xn, axis=1), 1.0, rtol=1e-12)
+    np.testing.assert_allclose(inv, 1.0 / np.linalg.norm(z, axis=1) * np.sqrt(16), rtol=1e-12)
+    xn2, _ = orc.rmsnorm(7.5 * z, np.ones(16), 0.0)
+    np.testing.assert_allclose(xn2, xn, rtol=1e-12)
+    # the weight is per channel, and eps enters under the root
+    w = rng.normal(size=16)
+    xn3, _ = orc.rmsnorm(z, w, 0.0)
+    np.testing.assert_allclose(xn3, xn * w[None, :], rtol=1e-12)
+    one = np.full((1, 4), 2.0)
+    np.testing.assert_allclose(orc.rmsnorm(one, np.ones(4), 5.0)[0], 2.0 / 3.0, rtol=1e-12)   # 2 / sqrt(4 + 5)
+
+
+def test_layer_is_the_residual_stream_plus_the_block_on_the_normalised_input():
+    z, p, dh, kw = make_case(T=6, d=8, f=12, N=3, k=2, r=2)
+    w = np.linspace(0.5, 1.5, 8)
+    h, saved = orc.layer_forward(z, p, w, 1e-5, **kw)
+    xn = z / np.sqrt(np.mean(z * z, axis=1, keepdims=True) + 1e-5) * w
+    y, _ = orc.ffn_forward(xn, p, **kw)
+    np.testing.assert_allclose(h, z + y, rtol=1e-12, atol=1e-12)
+    # a block whose down projections are zero leaves the residual stream untouched, and its input gradient is dh
+    p0 = dict(p, w_down=np.zeros_like(p["w_down"]), b_down=np.zeros_like(p["b_down"]))
+    h0, s0 = orc.layer_forward(z, p0, w, 1e-5, **kw)
+    np.testing.assert_array_equal(h0, z)
+    g0 = orc.layer_backward(z, p0, w, dh, s0, aux_coef=0.0)
+    np.testing.assert_allclose(g0["d_x"], dh, rtol=0, atol=1e-14)
+
+
+def layer_loss(z, p, w, eps, dh, kw, coef):
+    h, saved = orc.layer_forward(z, p, w, eps, **kw)
+    la, _, _ = orc.aux_loss(saved["route"]["probs"], saved["route"]["expert_idx"], coef)
+    return float(np.sum(dh * h)) + la
+
+
+@pytest.mark.parametrize("k,N,coef", [(2, 3, 0.6), (1, 4, 0.0)])
+def test_layer_backward_matches_central_differences(k, N, coef):
+    z, p, dh, kw = make_case(T=5, d=8, f=12, N=N, k=k, r=2, alpha=4.0, seed=21 + k, bias=True)
+    z = z * 1.7
+    w = np.random.default_rng(8).normal(size=8) * 0.3 + 1.0
+    eps = 1e-3
+    h, saved = orc.layer_forward(z, p, w, eps, **kw)
+    assert saved["route"]["margin"].min() > 1e-3
+    g = orc.layer_backward(z, p, w, dh, saved, aux_coef=coef)
+    step = 1e-6
+
+    def check(arr, grad, count, name):
+        flat = arr.reshape(-1)
+        for i in np.random.default_rng(2).choice(flat.size, size=min(flat.size, count), replace=False):
+            old = flat[i]
+            flat[i] = old + step
+            lp = layer_loss(z, p, w, eps, dh, kw, coef)
+            flat[i] = old - step
+            lm = layer_loss(z, p, w, eps, dh, kw, coef)
+            flat[i] = old
+            assert grad.reshape(-1)[i] == pytest.approx((lp - lm) / (2 * step), rel=2e-5, abs=2e-7), (name, i)
+
+    check(z, g["d_x"], 40, "z")
+    check(p["a_gate"], g["d_a_gate"], 10, "a_gate")
+    check(p["b_down"], g["d_b_down"], 10, "b_down")
+    check(p["w_router"], g["d_w_router"], 10, "w_router")
+
+
+def test_layer_pins_catch_a_dropped_projection_term_in_the_norm_gradient(monkeypatch):
+    # without the `xh * mean(u * xh)` term the gradient is not orthogonal to z (for eps = 0 the normalised
+    # vector does not change along z, so <dL/dz - dh, z> must vanish)
+    z, p, dh, kw = make_case(T=5, d=8, f=12, N=3, k=2, r=2, seed=4)
+    w = np.ones(8)
+    h, saved = orc.layer_forward(z, p, w, 0.0, **kw)
+    g = orc.layer_backward(z, p, w, dh, saved)
+    np.testing.assert_allclose(np.sum((g["d_x"] - dh) * z, axis=1), 0.0, atol=1e-10)
