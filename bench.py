@@ -265,6 +265,19 @@ def run_cuda(args):
                 for fl, _ in m_keep:
                     dist.all_reduce(fl)
 
+    if args.layer and M == 1 and want_dx:
+        # the block inside its layer (Eq. 5 / Eq. 6): RMS normalisation in front, residual stream behind
+        wn = torch.ones(w.d_model, dtype=act, device="cuda")
+        xn = torch.empty(w.tokens, w.d_model, dtype=act, device="cuda")
+        inv_rms = torch.empty(w.tokens, dtype=torch.float32, device="cuda")
+
+        def step():                        # noqa: F811
+            B.mixlora_layer_forward(shape, params, wn, 1e-5, xn, inv_rms, y, ws)
+            B.mixlora_aux_loss(shape, ws, AUX_COEF, loss)
+            B.mixlora_layer_backward(shape, params, wn, 1e-5, xn, inv_rms, dev["dy"], AUX_COEF, ws, grads)
+            if world > 1:
+                dist.all_reduce(flat)
+
     def barrier():
         if world > 1:
             dist.barrier()
@@ -419,7 +432,7 @@ def run_cuda(args):
         "dtype": "bf16" if bf16 else "f32", "data": "synthetic",
         "config": {"workload": w.name, "tokens_per_gpu": w.tokens, "d_model": w.d_model, "d_ff": w.d_ff,
                    "n_experts": w.n_experts, "top_k": w.top_k, "rank": w.rank, "lora_alpha": w.lora_alpha,
-                   "backward_dx": want_dx, "aux_coef": AUX_COEF, "adapters": M,
+                   "backward_dx": want_dx, "aux_coef": AUX_COEF, "adapters": M, "layer_slice": bool(args.layer and M == 1 and want_dx),
                    "parallelism": f"dp{world} over tokens" + (", NCCL all-reduce of LoRA/router grads" if world > 1 else ""),
                    "l2": "inputs larger than L2 (weights 270 MB + activations > 126 MB), no flush"},
         "roofline": roofline, "cpu_baseline": cpu_baseline,
@@ -442,6 +455,8 @@ def main():
     ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
     ap.add_argument("--workload", default="c3")
     ap.add_argument("--no-dx", action="store_true")
+    ap.add_argument("--layer", action="store_true",
+                    help="time the block inside its layer (RMSNorm in front, residual behind) instead of the block alone")
     ap.add_argument("--models", type=int, default=1,
                     help="split the batch over this many adapters sharing the frozen FFN (multi-model calls); the "
                          "end-to-end leg still runs the single-model calls")

@@ -147,6 +147,26 @@ mixlora_status_t mixlora_multi_ffn_backward(int32_t n_models, const mixlora_shap
                                             const size_t *workspace_bytes /* host [n] */,
                                             const mixlora_grads_t *grads /* host [n] */, void *stream);
 
+/* The block inside its transformer layer (Eq. 5 / Eq. 6): h = MixLoRA(LN(z)) + z, with LN the root-mean-square
+ * normalisation of LLaMA-class models, xn = norm_weight * z / sqrt(mean(z^2) + eps) over the model width.
+ * params->x is z, the residual stream [T, d]; norm_weight is [d]; both, like xn, h, dh and grads->d_x, are device
+ * arrays of shape.dtype.  The forward call writes xn [T, d] and inv_rms [T] (fp32), which the caller owns and must
+ * pass unchanged to the backward call, together with the workspace as the forward call left it.  The residual is
+ * added in the down projection's epilogue; nothing else differs from mixlora_ffn_forward on xn.
+ * The backward call returns the LoRA and router gradients of mixlora_ffn_backward at xn and, in grads->d_x (may be
+ * NULL), dL/dz = dh + J_LN^T dL/dxn; norm_weight is frozen and gets no gradient.  xn, h and d_x must not alias z or
+ * each other; d_model <= 8192 (bf16) or 4096 (fp32), else MIXLORA_ERR_UNSUPPORTED.  mixlora_aux_loss and
+ * mixlora_routing_view work on the workspace as after mixlora_ffn_forward. */
+mixlora_status_t mixlora_layer_forward(const mixlora_shape_t *shape /* host */,
+                                       const mixlora_params_t *params /* host struct of device ptrs */,
+                                       const void *norm_weight, float eps, void *xn, float *inv_rms, void *h,
+                                       void *workspace, size_t workspace_bytes, void *stream);
+mixlora_status_t mixlora_layer_backward(const mixlora_shape_t *shape /* host */,
+                                        const mixlora_params_t *params /* host struct of device ptrs */,
+                                        const void *norm_weight, float eps, const void *xn, const float *inv_rms,
+                                        const void *dh, float aux_coef, void *workspace, size_t workspace_bytes,
+                                        const mixlora_grads_t *grads /* host struct of device ptrs */, void *stream);
+
 /* Device pointers into the workspace, for inspection after a forward call:
  * expert_idx [T, k] (descending logit), gates [T, k], perm [T*k] (slot id at each position
  * of the order "expert ascending, token ascending"), seg_off [N+1] (first position of each

@@ -340,10 +340,15 @@ def rmsnorm(z, w_norm, eps):
     return z * inv_rms[:, None] * np.asarray(w_norm, F64)[None, :], inv_rms
 
 
-def layer_forward(z, params, w_norm, eps, top_k, lora_alpha, renormalize=True, forced_expert_idx=None):
+def layer_forward(z, params, w_norm, eps, top_k, lora_alpha, renormalize=True, forced_expert_idx=None,
+                  xn_round=None):
     """Eq. 6: `h = MixLoRA(LN(z)) + z`.  Returns (h [T, d], saved) where saved is that of `ffn_forward` on the
-    normalised input plus `xn` and `inv_rms`."""
+    normalised input plus `xn` and `inv_rms`.  `xn_round` (optional callable) is the rounding of the storage type
+    in which an implementation keeps the normalised input: the router's discrete choice is then taken on the same
+    values on both sides of a comparison."""
     xn, inv_rms = rmsnorm(z, w_norm, eps)
+    if xn_round is not None:
+        xn = np.asarray(xn_round(xn), F64)
     y, saved = ffn_forward(xn, params, top_k, lora_alpha, renormalize=renormalize,
                            forced_expert_idx=forced_expert_idx)
     saved = dict(saved)

@@ -23,7 +23,8 @@ EXPORTS = ("mixlora_limits", "mixlora_workspace_bytes", "mixlora_ffn_forward", "
            "mixlora_ffn_backward", "mixlora_routing_view", "mixlora_device_status", "mixlora_gemm_bf16",
            "mixlora_status_string", "mixlora_stage_timing", "mixlora_stage_timing_read",
            "mixlora_dispatch_static", "mixlora_dispatch_static_max_tokens",
-           "mixlora_multi_ffn_forward", "mixlora_multi_ffn_backward")
+           "mixlora_multi_ffn_forward", "mixlora_multi_ffn_backward", "mixlora_layer_forward",
+           "mixlora_layer_backward")
 
 
 class mixlora_shape_t(C.Structure):
@@ -95,6 +96,13 @@ def _load() -> C.CDLL:
                                                C.POINTER(C.c_void_p), C.POINTER(C.c_float), C.POINTER(C.c_void_p),
                                                C.POINTER(C.c_size_t), C.POINTER(mixlora_grads_t), C.c_void_p]
     lib.mixlora_multi_ffn_backward.restype = C.c_int
+    lib.mixlora_layer_forward.argtypes = [C.POINTER(mixlora_shape_t), C.POINTER(mixlora_params_t), C.c_void_p, C.c_float,
+                                          C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p]
+    lib.mixlora_layer_forward.restype = C.c_int
+    lib.mixlora_layer_backward.argtypes = [C.POINTER(mixlora_shape_t), C.POINTER(mixlora_params_t), C.c_void_p,
+                                           C.c_float, C.c_void_p, C.c_void_p, C.c_void_p, C.c_float, C.c_void_p,
+                                           C.c_size_t, C.POINTER(mixlora_grads_t), C.c_void_p]
+    lib.mixlora_layer_backward.restype = C.c_int
     lib.mixlora_status_string.argtypes = [C.c_int]
     lib.mixlora_status_string.restype = C.c_char_p
     return lib
@@ -257,3 +265,19 @@ def mixlora_multi_ffn_backward(shapes, params, dys, aux_coefs, workspaces, grads
                                           _ptr_array(workspaces), (C.c_size_t * n)(*[w.numel() for w in workspaces]),
                                           (mixlora_grads_t * n)(*grads), _stream(stream)),
            "mixlora_multi_ffn_backward")
+
+
+def mixlora_layer_forward(shape, params, norm_weight, eps, xn, inv_rms, h, workspace, stream=None) -> None:
+    """h = MixLoRA(RMSNorm(z)) + z with z = params.x; writes xn and inv_rms for the backward call."""
+    _check(lib.mixlora_layer_forward(C.byref(shape), C.byref(params), _ptr(norm_weight), float(eps), _ptr(xn),
+                                     _ptr(inv_rms), _ptr(h), _ptr(workspace),
+                                     workspace.numel() if workspace is not None else 0, _stream(stream)),
+           "mixlora_layer_forward")
+
+
+def mixlora_layer_backward(shape, params, norm_weight, eps, xn, inv_rms, dh, aux_coef, workspace, grads,
+                           stream=None) -> None:
+    _check(lib.mixlora_layer_backward(C.byref(shape), C.byref(params), _ptr(norm_weight), float(eps), _ptr(xn),
+                                      _ptr(inv_rms), _ptr(dh), float(aux_coef), _ptr(workspace),
+                                      workspace.numel() if workspace is not None else 0, C.byref(grads),
+                                      _stream(stream)), "mixlora_layer_backward")

@@ -94,11 +94,11 @@ namespace {
 // ---- opt-in per-stage device timing and launch counting (host-side bookkeeping only) ----
 enum Stage {
   ST_ROUTER, ST_DISPATCH, ST_GEMM_GATE_UP, ST_LORA_B_SWIGLU, ST_LORA_A_DOWN, ST_COMBINE_H, ST_GEMM_DOWN,
-  ST_GEMM_DGRAD_DOWN, ST_SWIGLU_BWD, ST_LORA_DZ, ST_LORA_WGRAD, ST_ROUTER_BWD, ST_COMBINE_BWD, ST_GEMM_DX, ST_COUNT
+  ST_GEMM_DGRAD_DOWN, ST_SWIGLU_BWD, ST_LORA_DZ, ST_LORA_WGRAD, ST_ROUTER_BWD, ST_COMBINE_BWD, ST_GEMM_DX, ST_NORM, ST_COUNT
 };
 const char* const kStageNames[ST_COUNT] = {
     "router", "dispatch", "gemm_gate_up", "lora_b_swiglu", "lora_a_down", "combine_h", "gemm_down",
-    "gemm_dgrad_down", "swiglu_bwd", "lora_dz", "lora_wgrad", "router_bwd", "combine_bwd", "gemm_dx"};
+    "gemm_dgrad_down", "swiglu_bwd", "lora_dz", "lora_wgrad", "router_bwd", "combine_bwd", "gemm_dx", "norm"};
 
 struct StageRec { int stage; cudaEvent_t a, b; };
 struct Profiler {
@@ -204,6 +204,7 @@ cudaError_t dense_product(const Ctx& c, int M, const TcOut* outs, int nout, cons
     }
     cudaError_t e = launch_simt_gemm(g, c.st);
     if (e != cudaSuccess) return e;
+    if (t.mode == 0 && t.R && (e = launch_residual_add(c, t.C, t.ldc, t.R, t.ldr, Mo, t.N)) != cudaSuccess) return e;
   }
   return cudaSuccess;
 }
@@ -337,7 +338,8 @@ static mixlora_status_t fwd_shared_projections(const Ctx* cs, int n) {
 }
 
 // everything after the shared projections: per-expert deltas, SwiGLU, down projection, combine
-static mixlora_status_t fwd_experts(const Ctx& c, void* y) {
+// `residual` (optional, [T, d] of the activation type) is added to y in the down product's epilogue (Eq. 6).
+static mixlora_status_t fwd_experts(const Ctx& c, void* y, const void* residual = nullptr) {
   const mixlora_params_t* params = &c.p;
   const int T = c.s.tokens, d = c.s.d_model, f = c.s.d_ff, N = c.s.n_experts, r = c.s.rank, k = c.s.top_k;
   const int Nr = N * r;
@@ -373,6 +375,7 @@ static mixlora_status_t fwd_experts(const Ctx& c, void* y) {
   // token's slots (W_d is linear and shared), its LoRA rides along as extra reduction columns
   {
     TcOut out = tc_out(y, d, d);
+    out.R = residual; out.ldr = d;
     tc_add(out, c.ws + c.L.hbar, f, f, params->w_down, f, 0);
     tc_add(out, c.ws + c.L.Zs, Nr, Nr, c.ws + c.L.bd_cat, Nr, 0);
     StageScope ss(ST_GEMM_DOWN, c.st, dense_launches(c, T, &out, 1));
@@ -650,6 +653,61 @@ mixlora_status_t mixlora_multi_ffn_backward(int32_t n_models, const mixlora_shap
   return MIXLORA_OK;
 }
 
+
+// ---- the block inside its layer (Eq. 5 / Eq. 6) ----
+static mixlora_status_t layer_check(const mixlora_shape_t* shape, const mixlora_params_t* params, const void* norm_weight,
+                                    float eps, const void* xn, const float* inv_rms) {
+  mixlora_status_t st = check_shape(shape);
+  if (st != MIXLORA_OK) return st;
+  if (!params || !norm_weight || !xn || !inv_rms || !aligned16(norm_weight) || !aligned16(xn) ||
+      (reinterpret_cast<uintptr_t>(inv_rms) & 3u) || !(eps >= 0.f))
+    return MIXLORA_ERR_INVALID_ARG;
+  if (xn == params->x) return MIXLORA_ERR_INVALID_ARG;   // the residual stream is read again after xn is written
+  if (shape->d_model > rmsnorm_max_width(shape->dtype == MIXLORA_DTYPE_BF16)) return MIXLORA_ERR_UNSUPPORTED;
+  return MIXLORA_OK;
+}
+
+mixlora_status_t mixlora_layer_forward(const mixlora_shape_t* shape, const mixlora_params_t* params,
+                                       const void* norm_weight, float eps, void* xn, float* inv_rms, void* h,
+                                       void* workspace, size_t workspace_bytes, void* stream) {
+  mixlora_status_t st = layer_check(shape, params, norm_weight, eps, xn, inv_rms);
+  if (st != MIXLORA_OK) return st;
+  if (h == xn) return MIXLORA_ERR_INVALID_ARG;
+  mixlora_params_t inner = *params;                    // the block itself sees the normalised input
+  inner.x = xn;
+  Ctx c;
+  if ((st = fwd_check(shape, &inner, h, workspace, workspace_bytes, stream, &c)) != MIXLORA_OK) return st;
+  if (!params->x || !aligned16(params->x)) return MIXLORA_ERR_INVALID_ARG;
+  {
+    StageScope ss(ST_NORM, c.st, shape->tokens > 0 ? 1 : 0);
+    MIXLORA_CUDA(launch_rmsnorm_fwd(c, params->x, norm_weight, eps, xn, inv_rms));
+  }
+  if ((st = fwd_route(c)) != MIXLORA_OK) return st;
+  if ((st = fwd_shared_projections(&c, 1)) != MIXLORA_OK) return st;
+  return fwd_experts(c, h, params->x);
+}
+
+mixlora_status_t mixlora_layer_backward(const mixlora_shape_t* shape, const mixlora_params_t* params,
+                                        const void* norm_weight, float eps, const void* xn, const float* inv_rms,
+                                        const void* dh, float aux_coef, void* workspace, size_t workspace_bytes,
+                                        const mixlora_grads_t* grads, void* stream) {
+  mixlora_status_t st = layer_check(shape, params, norm_weight, eps, xn, inv_rms);
+  if (st != MIXLORA_OK) return st;
+  mixlora_params_t inner = *params;
+  inner.x = xn;
+  Ctx c;
+  if ((st = bwd_check(shape, &inner, dh, workspace, workspace_bytes, grads, stream, &c)) != MIXLORA_OK) return st;
+  if (!params->x || !aligned16(params->x)) return MIXLORA_ERR_INVALID_ARG;
+  if (grads->d_x && (grads->d_x == dh || grads->d_x == params->x || grads->d_x == xn)) return MIXLORA_ERR_INVALID_ARG;
+  if ((st = bwd_shared_dgrad(&c, &dh, 1)) != MIXLORA_OK) return st;
+  if ((st = bwd_experts(c, dh, aux_coef, grads)) != MIXLORA_OK) return st;
+  if (grads->d_x) {
+    // d_x holds dL/dxn now; the norm's Jacobian and the residual path turn it into dL/dz in place
+    StageScope ss(ST_NORM, c.st, shape->tokens > 0 ? 1 : 0);
+    MIXLORA_CUDA(launch_rmsnorm_bwd(c, params->x, norm_weight, inv_rms, grads->d_x, dh, grads->d_x));
+  }
+  return MIXLORA_OK;
+}
 
 mixlora_status_t mixlora_routing_view(const mixlora_shape_t* shape, const void* workspace, const int32_t** expert_idx,
                                       const float** gates, const int32_t** perm, const int32_t** seg_off,

@@ -160,6 +160,12 @@ cudaError_t launch_swiglu_bwd(const Ctx& c);          // h_sorted, da_sorted, db
 cudaError_t launch_slot_prep_bwd(const Ctx& c);       // P_pos, dZd_pos
 cudaError_t launch_combine_bwd(const Ctx& c, int want_dx);  // dZg, dZu and, for dx, dabar, dbbar
 cudaError_t launch_router_bwd(const Ctx& c, float aux_coef, float* d_bias, int accumulate, int want_dx);
+// the block inside its layer (Eq. 5 / Eq. 6)
+int rmsnorm_max_width(int bf16_mode);   // widest model the norm kernels take (8192 bf16, 4096 fp32)
+cudaError_t launch_rmsnorm_fwd(const Ctx& c, const void* z, const void* w_norm, float eps, void* xn, float* inv_rms);
+cudaError_t launch_rmsnorm_bwd(const Ctx& c, const void* z, const void* w_norm, const float* inv_rms, const void* dxn,
+                               const void* dh, void* dz);
+cudaError_t launch_residual_add(const Ctx& c, void* C, long long ldc, const void* R, long long ldr, int M, int N);
 
 // Dense product (tensor-core kernel in tc_gemm.cu, SIMT kernel otherwise), fp32 accumulation:
 //   C_o[M, N_o] = sum_seg op(A_o,seg) * op(B_o,seg)
@@ -178,6 +184,7 @@ struct TcOut {
   void* C; long long ldc; int N;
   int M;        // rows of this output when it differs from the launch's M (0 = same)
   int mode; long long s_m, s_n, s_blk; int nb; float alpha; int accumulate;
+  const void* R; long long ldr;   // mode 0 only: optional [M, N] matrix of the output's type added to the product
   TcSeg seg[kMaxKSeg]; int nseg;
 };
 // Optional block-sparse schedule built on the device from the segment offsets (router.cu): only the listed

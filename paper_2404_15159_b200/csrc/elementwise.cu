@@ -600,6 +600,128 @@ cudaError_t router_bwd_t(const Ctx& c, float aux_coef, float* d_bias, int accumu
   return cudaGetLastError();
 }
 
+
+// ---- the block inside its layer (Eq. 5 / Eq. 6): RMS normalisation in front, its Jacobian behind -------------
+// One block per token, 16-byte loads and stores; a thread keeps its chunks of the row in registers between the
+// reduction and the write, so the row is read once.  kNormChunks * kNormThreads 16-byte chunks bound the width.
+constexpr int kNormThreads = 256;
+constexpr int kNormChunks = 4;
+
+template <typename T> struct Vec16 { static constexpr int n = 16 / sizeof(T); };
+template <typename T>
+__device__ __forceinline__ void load16(const T* p, float* o) {
+  const uint4 raw = *reinterpret_cast<const uint4*>(p);
+  const T* e = reinterpret_cast<const T*>(&raw);
+#pragma unroll
+  for (int j = 0; j < Vec16<T>::n; ++j) o[j] = to_f(e[j]);
+}
+template <typename T>
+__device__ __forceinline__ void store16(T* p, const float* v) {
+  uint4 raw;
+  T* e = reinterpret_cast<T*>(&raw);
+#pragma unroll
+  for (int j = 0; j < Vec16<T>::n; ++j) e[j] = from_f<T>(v[j]);
+  *reinterpret_cast<uint4*>(p) = raw;
+}
+
+__device__ __forceinline__ float block_sum(float v, float* red) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  if (lane == 0) red[warp] = v;
+  __syncthreads();
+  float t = 0.f;
+#pragma unroll
+  for (int w = 0; w < kNormThreads / 32; ++w) t += red[w];   // fixed order: the same bits in every thread and run
+  return t;
+}
+
+// xn = w_norm * z * inv_rms (one rounding), inv_rms = 1 / sqrt(mean(z^2) + eps)
+template <typename T>
+__global__ void __launch_bounds__(kNormThreads) rmsnorm_fwd_kernel(const T* __restrict__ z, const T* __restrict__ w_norm,
+                                                                  float eps, T* __restrict__ xn,
+                                                                  float* __restrict__ inv_rms, int d) {
+  constexpr int V = Vec16<T>::n;
+  __shared__ float red[kNormThreads / 32];
+  const size_t row = (size_t)blockIdx.x * d;
+  float v[kNormChunks][V];
+  float ss = 0.f;
+#pragma unroll
+  for (int i = 0; i < kNormChunks; ++i) {
+    const int c = (threadIdx.x + i * kNormThreads) * V;
+    if (c < d) {
+      load16(z + row + c, v[i]);
+#pragma unroll
+      for (int j = 0; j < V; ++j) ss = fmaf(v[i][j], v[i][j], ss);
+    }
+  }
+  const float inv = rsqrtf(block_sum(ss, red) / (float)d + eps);
+  if (threadIdx.x == 0) inv_rms[blockIdx.x] = inv;
+#pragma unroll
+  for (int i = 0; i < kNormChunks; ++i) {
+    const int c = (threadIdx.x + i * kNormThreads) * V;
+    if (c < d) {
+      float w[V];
+      load16(w_norm + c, w);
+#pragma unroll
+      for (int j = 0; j < V; ++j) w[j] = w[j] * v[i][j] * inv;
+      store16(xn + row + c, w);
+    }
+  }
+}
+
+// dz = dh + inv_rms * (u - xh * mean(u * xh)),  u = dxn * w_norm,  xh = z * inv_rms.  dxn and dz may be the same
+// buffer: every element is read before the block writes it.
+template <typename T>
+__global__ void __launch_bounds__(kNormThreads) rmsnorm_bwd_kernel(const T* __restrict__ z, const T* __restrict__ w_norm,
+                                                                  const float* __restrict__ inv_rms, const T* dxn,
+                                                                  const T* __restrict__ dh, T* dz, int d) {
+  constexpr int V = Vec16<T>::n;
+  __shared__ float red[kNormThreads / 32];
+  const size_t row = (size_t)blockIdx.x * d;
+  const float inv = inv_rms[blockIdx.x];
+  float u[kNormChunks][V], xh[kNormChunks][V];
+  float dot = 0.f;
+#pragma unroll
+  for (int i = 0; i < kNormChunks; ++i) {
+    const int c = (threadIdx.x + i * kNormThreads) * V;
+    if (c < d) {
+      float w[V];
+      load16(dxn + row + c, u[i]);
+      load16(w_norm + c, w);
+      load16(z + row + c, xh[i]);
+#pragma unroll
+      for (int j = 0; j < V; ++j) {
+        u[i][j] *= w[j];
+        xh[i][j] *= inv;
+        dot = fmaf(u[i][j], xh[i][j], dot);
+      }
+    }
+  }
+  const float m = block_sum(dot, red) / (float)d;
+#pragma unroll
+  for (int i = 0; i < kNormChunks; ++i) {
+    const int c = (threadIdx.x + i * kNormThreads) * V;
+    if (c < d) {
+      float g[V];
+      load16(dh + row + c, g);
+#pragma unroll
+      for (int j = 0; j < V; ++j) g[j] += inv * (u[i][j] - xh[i][j] * m);
+      store16(dz + row + c, g);
+    }
+  }
+}
+
+// C[m][n] += R[m][n] (fp32 check mode; the tensor-core path adds the residual in its epilogue)
+template <typename T>
+__global__ void residual_add_kernel(T* __restrict__ C, long long ldc, const T* __restrict__ R, long long ldr, int M, int N) {
+  const long long n = (long long)M * N;
+  for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < n; i += (long long)gridDim.x * blockDim.x) {
+    const long long m = i / N, col = i % N;
+    C[m * ldc + col] = from_f<T>(to_f(C[m * ldc + col]) + to_f(R[m * ldr + col]));
+  }
+}
+
 }  // namespace
 
 cudaError_t launch_bd_cat(const Ctx& c) { return c.bf16 ? bd_cat_t<bf16>(c) : bd_cat_t<float>(c); }
@@ -632,6 +754,45 @@ cudaError_t launch_bgu_cat(const Ctx& c) { return c.bf16 ? bgu_cat_t<bf16>(c) : 
 cudaError_t launch_router_bwd(const Ctx& c, float aux_coef, float* d_bias, int accumulate, int want_dx) {
   return c.bf16 ? router_bwd_t<bf16>(c, aux_coef, d_bias, accumulate, want_dx)
                 : router_bwd_t<float>(c, aux_coef, d_bias, accumulate, want_dx);
+}
+
+int rmsnorm_max_width(int bf16_mode) { return kNormThreads * kNormChunks * (bf16_mode ? 8 : 4); }
+cudaError_t launch_rmsnorm_fwd(const Ctx& c, const void* z, const void* w_norm, float eps, void* xn, float* inv_rms) {
+  if (c.s.tokens == 0) return cudaSuccess;
+  if (c.bf16)
+    rmsnorm_fwd_kernel<bf16><<<c.s.tokens, kNormThreads, 0, c.st>>>(
+        reinterpret_cast<const bf16*>(z), reinterpret_cast<const bf16*>(w_norm), eps, reinterpret_cast<bf16*>(xn), inv_rms,
+        c.s.d_model);
+  else
+    rmsnorm_fwd_kernel<float><<<c.s.tokens, kNormThreads, 0, c.st>>>(
+        reinterpret_cast<const float*>(z), reinterpret_cast<const float*>(w_norm), eps, reinterpret_cast<float*>(xn),
+        inv_rms, c.s.d_model);
+  return cudaGetLastError();
+}
+cudaError_t launch_rmsnorm_bwd(const Ctx& c, const void* z, const void* w_norm, const float* inv_rms, const void* dxn,
+                               const void* dh, void* dz) {
+  if (c.s.tokens == 0) return cudaSuccess;
+  if (c.bf16)
+    rmsnorm_bwd_kernel<bf16><<<c.s.tokens, kNormThreads, 0, c.st>>>(
+        reinterpret_cast<const bf16*>(z), reinterpret_cast<const bf16*>(w_norm), inv_rms,
+        reinterpret_cast<const bf16*>(dxn), reinterpret_cast<const bf16*>(dh), reinterpret_cast<bf16*>(dz), c.s.d_model);
+  else
+    rmsnorm_bwd_kernel<float><<<c.s.tokens, kNormThreads, 0, c.st>>>(
+        reinterpret_cast<const float*>(z), reinterpret_cast<const float*>(w_norm), inv_rms,
+        reinterpret_cast<const float*>(dxn), reinterpret_cast<const float*>(dh), reinterpret_cast<float*>(dz),
+        c.s.d_model);
+  return cudaGetLastError();
+}
+cudaError_t launch_residual_add(const Ctx& c, void* C, long long ldc, const void* R, long long ldr, int M, int N) {
+  if (M <= 0 || N <= 0) return cudaSuccess;
+  const int grid = grid_for((long long)M * N, 256);
+  if (c.bf16)
+    residual_add_kernel<bf16><<<grid, 256, 0, c.st>>>(reinterpret_cast<bf16*>(C), ldc, reinterpret_cast<const bf16*>(R),
+                                                      ldr, M, N);
+  else
+    residual_add_kernel<float><<<grid, 256, 0, c.st>>>(reinterpret_cast<float*>(C), ldc,
+                                                       reinterpret_cast<const float*>(R), ldr, M, N);
+  return cudaGetLastError();
 }
 
 }  // namespace mixlora

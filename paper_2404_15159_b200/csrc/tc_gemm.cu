@@ -44,6 +44,8 @@ struct alignas(64) TcParams {
   CUtensorMap b_map[kMaxB];        // index o * nseg + seg
   void* C[kMaxOut];
   long long ldc[kMaxOut];          // mode 0: row pitch; mode 1: stride of m
+  const void* R[kMaxOut];          // mode 0: optional matrix added to the product (a residual stream), or null
+  long long ldr[kMaxOut];
   long long s_n[kMaxOut], s_blk[kMaxOut];
   float alpha[kMaxOut];
   int mode[kMaxOut], nb[kMaxOut], accumulate[kMaxOut];
@@ -112,15 +114,29 @@ __device__ __forceinline__ void store_chunk32(const TcParams& p, int o, int row,
     }
   } else {
     bf16* crow = reinterpret_cast<bf16*>(p.C[o]) + (size_t)row * p.ldc[o];
+    const bf16* rrow = p.R[o] ? reinterpret_cast<const bf16*>(p.R[o]) + (size_t)row * p.ldr[o] : nullptr;
 #pragma unroll
     for (int g8 = 0; g8 < 4; ++g8) {
       const int col = n0c + g8 * 8;
       if (col >= n_lo && col < n_hi) {
         uint4 q4;
-        __nv_bfloat162 h0 = __floats2bfloat162_rn(__uint_as_float(v[g8 * 8 + 0]), __uint_as_float(v[g8 * 8 + 1]));
-        __nv_bfloat162 h1 = __floats2bfloat162_rn(__uint_as_float(v[g8 * 8 + 2]), __uint_as_float(v[g8 * 8 + 3]));
-        __nv_bfloat162 h2 = __floats2bfloat162_rn(__uint_as_float(v[g8 * 8 + 4]), __uint_as_float(v[g8 * 8 + 5]));
-        __nv_bfloat162 h3 = __floats2bfloat162_rn(__uint_as_float(v[g8 * 8 + 6]), __uint_as_float(v[g8 * 8 + 7]));
+        float w[8];
+#pragma unroll
+        for (int j = 0; j < 8; ++j) w[j] = __uint_as_float(v[g8 * 8 + j]);
+        if (rrow) {                                   // fused residual add, in fp32 before the one rounding
+          const uint4 r4 = *reinterpret_cast<const uint4*>(rrow + col);
+          const __nv_bfloat162* rp = reinterpret_cast<const __nv_bfloat162*>(&r4);
+#pragma unroll
+          for (int j = 0; j < 4; ++j) {
+            const float2 rf = __bfloat1622float2(rp[j]);
+            w[2 * j] += rf.x;
+            w[2 * j + 1] += rf.y;
+          }
+        }
+        __nv_bfloat162 h0 = __floats2bfloat162_rn(w[0], w[1]);
+        __nv_bfloat162 h1 = __floats2bfloat162_rn(w[2], w[3]);
+        __nv_bfloat162 h2 = __floats2bfloat162_rn(w[4], w[5]);
+        __nv_bfloat162 h3 = __floats2bfloat162_rn(w[6], w[7]);
         q4.x = *reinterpret_cast<uint32_t*>(&h0);
         q4.y = *reinterpret_cast<uint32_t*>(&h1);
         q4.z = *reinterpret_cast<uint32_t*>(&h2);
@@ -540,6 +556,7 @@ bool tc_gemm_supported(int M, const TcOut* outs, int nout) {
     if (t.nseg != nseg || t.N <= 0 || !t.C) return false;
     if (t.mode == 0) {
       if (t.N % 8 || t.ldc % 8 || (reinterpret_cast<uintptr_t>(t.C) & 15u)) return false;
+      if (t.R && (t.ldr % 8 || (reinterpret_cast<uintptr_t>(t.R) & 15u))) return false;
     } else if (t.mode != 1 || (reinterpret_cast<uintptr_t>(t.C) & 3u)) {
       return false;
     }
@@ -625,6 +642,7 @@ cudaError_t launch_tc_gemm(int M, const TcOut* outs, int nout, int* status_word,
     p.C[o] = t.C; p.N[o] = t.N; p.tile_n[o] = tn;
     p.mode[o] = t.mode;
     p.ldc[o] = t.mode == 0 ? t.ldc : t.s_m;
+    p.R[o] = t.mode == 0 ? t.R : nullptr; p.ldr[o] = t.ldr;
     p.s_n[o] = t.s_n; p.s_blk[o] = t.s_blk; p.nb[o] = t.nb; p.alpha[o] = t.alpha; p.accumulate[o] = t.accumulate;
     p.tile_start[o] = tiles;
     tiles += p.m_tiles_o[o] * ((t.N + tn - 1) / tn);
