@@ -32,7 +32,8 @@ AUX_COEF = 0.01
 
 
 def workload_by_name(name: str) -> synth.Workload:
-    table = {"c1": synth.c1, "c2": synth.c2, "c3": synth.c3, "c4": synth.c4}
+    table = {"c1": synth.c1, "c2": synth.c2, "c3": synth.c3, "c4": synth.c4, "llama3-8b": synth.llama3_8b,
+             "wide-2b": synth.wide_2b}
     if name in table:
         return table[name]()
     if name.startswith("c5:"):                      # c5:N,k,r,T

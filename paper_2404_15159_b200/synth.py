@@ -63,6 +63,19 @@ def c5(n_experts: int, top_k: int, rank: int, tokens: int) -> Workload:
                     rank, 2.0 * rank, "bf16", 0.02, 1.0 / rank, 0.01, zipf_s=1.2, seed=BASE_SEED + 4)
 
 
+def llama3_8b(tokens: int = 8192) -> Workload:
+    """Second workload shape: LLaMA-3-8B's FFN (d = 4096, f = 14336), same adapter set-up as c3."""
+    return Workload(f"llama3-8b-T{tokens}", tokens, 4096, 14336, 8, 2, 16, 32.0, "bf16", 0.02, 1.0 / 16, 0.01,
+                    seed=BASE_SEED + 5)
+
+
+def wide_2b(tokens: int = 8192) -> Workload:
+    """Second workload shape: a 2B-class model with a wide FFN (d = 2048, f = 16384; the width ratio of Gemma-2B,
+    with the SwiGLU activation of this block)."""
+    return Workload(f"wide-2b-T{tokens}", tokens, 2048, 16384, 8, 2, 16, 32.0, "bf16", 0.02, 1.0 / 16, 0.01,
+                    seed=BASE_SEED + 6)
+
+
 def c5_grid():
     return [c5(n, k, r, t) for n in (8, 16) for k in (1, 2) for r in (8, 16, 64) for t in (512, 4096, 32768)]
 

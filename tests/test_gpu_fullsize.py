@@ -62,6 +62,12 @@ def test_c4_13b_shape_sampled_forward_at_8192_and_full_check_at_2048_tokens():
     full_check(synth.c4().with_(name="C4-2048", tokens=2048), aux_coef=0.01)
 
 
+@pytest.mark.parametrize("make", [synth.llama3_8b, synth.wide_2b])
+def test_second_workload_shapes_sampled_forward_at_4096_and_full_check_at_1024_tokens(make):
+    sampled_forward_check(make(4096), n_samples=12)
+    full_check(make(1024), aux_coef=0.01)
+
+
 @pytest.mark.parametrize("N,k,r", [(8, 1, 8), (8, 2, 16), (8, 2, 64), (16, 1, 16), (16, 2, 8), (16, 2, 64)])
 def test_c5_skew_sweep_512_tokens(N, k, r):
     w = synth.c5(N, k, r, 512)
