@@ -370,3 +370,22 @@ def layer_backward(z, params, w_norm, dh, saved, aux_coef=0.0, aux_f_mode=0):
     g = dict(g)
     g["d_x"] = dh + inv_rms[:, None] * (u - xh * np.mean(u * xh, axis=1, keepdims=True))
     return g
+
+
+# --------------------------------------------------------------------------- #
+# plain LoRA on a linear layer (Eq. 1), as MixLoRA puts it on the attention projections (Section 3.2)
+# --------------------------------------------------------------------------- #
+def lora_linear_forward(x, w, a, b, lora_alpha):
+    """`y = x W^T + s (x A^T) B^T`, `s = alpha / r`; W [out, in], A [r, in], B [out, r] (Eq. 1 applied to x)."""
+    x, w, a, b = (np.asarray(v, F64) for v in (x, w, a, b))
+    s = lora_alpha / a.shape[0]
+    return x @ w.T + s * ((x @ a.T) @ b.T)
+
+
+def lora_linear_backward(x, w, a, b, lora_alpha, dy):
+    """Gradients of `<dy, y>`: W is frozen.  Returns dict(d_x, d_a, d_b)."""
+    x, w, a, b, dy = (np.asarray(v, F64) for v in (x, w, a, b, dy))
+    s = lora_alpha / a.shape[0]
+    dz = s * (dy @ b)                       # [T, r]
+    return dict(d_x=dy @ w + dz @ a, d_a=dz.T @ x, d_b=s * (dy.T @ (x @ a.T)))
+

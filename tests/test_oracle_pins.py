@@ -415,3 +415,33 @@ def test_layer_pins_catch_a_dropped_projection_term_in_the_norm_gradient(monkeyp
     h, saved = orc.layer_forward(z, p, w, 0.0, **kw)
     g = orc.layer_backward(z, p, w, dh, saved)
     np.testing.assert_allclose(np.sum((g["d_x"] - dh) * z, axis=1), 0.0, atol=1e-10)
+
+
+# ---- plain LoRA linear (Eq. 1) -------------------------------------------------
+def test_lora_linear_equals_the_merged_weight_of_eq_1():
+    rng = np.random.default_rng(12)
+    x, w = rng.normal(size=(9, 6)), rng.normal(size=(5, 6))
+    a, b = rng.normal(size=(3, 6)), rng.normal(size=(5, 3))
+    y = orc.lora_linear_forward(x, w, a, b, 6.0)
+    np.testing.assert_allclose(y, x @ (w + (6.0 / 3) * b @ a).T, rtol=1e-12, atol=1e-12)
+    np.testing.assert_allclose(orc.lora_linear_forward(x, w, a, np.zeros_like(b), 6.0), x @ w.T, rtol=1e-13)
+
+
+def test_lora_linear_backward_matches_central_differences():
+    rng = np.random.default_rng(13)
+    x, w = rng.normal(size=(7, 5)), rng.normal(size=(4, 5))
+    a, b = rng.normal(size=(2, 5)), rng.normal(size=(4, 2))
+    dy = rng.normal(size=(7, 4))
+    g = orc.lora_linear_backward(x, w, a, b, 3.0, dy)
+    step = 1e-6
+    for name, arr in (("d_x", x), ("d_a", a), ("d_b", b)):
+        flat = arr.reshape(-1)
+        for i in range(flat.size):
+            old = flat[i]
+            flat[i] = old + step
+            lp = np.sum(dy * orc.lora_linear_forward(x, w, a, b, 3.0))
+            flat[i] = old - step
+            lm = np.sum(dy * orc.lora_linear_forward(x, w, a, b, 3.0))
+            flat[i] = old
+            assert g[name].reshape(-1)[i] == pytest.approx((lp - lm) / (2 * step), rel=1e-6, abs=1e-8), (name, i)
+
