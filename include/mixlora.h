@@ -167,6 +167,31 @@ mixlora_status_t mixlora_layer_backward(const mixlora_shape_t *shape /* host */,
                                         const void *dh, float aux_coef, void *workspace, size_t workspace_bytes,
                                         const mixlora_grads_t *grads /* host struct of device ptrs */, void *stream);
 
+/* Plain LoRA on a linear layer (Eq. 1, W' = W + B A, applied as in Section 3.2 to the attention projections of
+ * a MixLoRA model): y = x W^T + s (x A^T) B^T with s = lora_alpha / rank.  x [T, d_in], W [d_out, d_in] (frozen),
+ * A [rank, d_in], B [d_out, rank], y and dy [T, d_out], all device arrays of shape.dtype; d_in, d_out and rank are
+ * multiples of 8, rank <= MIXLORA_MAX_RANK.  The low-rank term is computed as `rank` extra reduction columns of the
+ * frozen product (forward) and of the input-gradient product (backward).  The workspace (256-byte aligned, caller-
+ * owned, mixlora_lora_linear_workspace_bytes) keeps s x A^T between the forward and the backward call of the same
+ * input.  The backward call writes d_a [rank, d_in] and d_b [d_out, rank] in fp32 (added to the old contents if
+ * accumulate = 1) and d_x [T, d_in] in shape.dtype; each may be NULL.  mixlora_lora_linear_status reads back the
+ * device status word of the last calls on this workspace (0 = ok; it synchronises the stream). */
+typedef struct {
+  uint32_t struct_size; /* = sizeof(mixlora_linear_shape_t) */
+  int32_t tokens, d_in, d_out, rank;
+  float lora_alpha;
+  int32_t dtype;        /* MIXLORA_DTYPE_* */
+} mixlora_linear_shape_t;
+size_t mixlora_lora_linear_workspace_bytes(const mixlora_linear_shape_t *shape /* host */);
+mixlora_status_t mixlora_lora_linear_forward(const mixlora_linear_shape_t *shape /* host */, const void *x,
+                                             const void *w, const void *a, const void *b, void *y, void *workspace,
+                                             size_t workspace_bytes, void *stream);
+mixlora_status_t mixlora_lora_linear_backward(const mixlora_linear_shape_t *shape /* host */, const void *x,
+                                              const void *w, const void *a, const void *b, const void *dy,
+                                              void *workspace, size_t workspace_bytes, float *d_a, float *d_b,
+                                              void *d_x, int32_t accumulate, void *stream);
+int32_t mixlora_lora_linear_status(const void *workspace, void *stream);
+
 /* Device pointers into the workspace, for inspection after a forward call:
  * expert_idx [T, k] (descending logit), gates [T, k], perm [T*k] (slot id at each position
  * of the order "expert ascending, token ascending"), seg_off [N+1] (first position of each

@@ -24,7 +24,13 @@ EXPORTS = ("mixlora_limits", "mixlora_workspace_bytes", "mixlora_ffn_forward", "
            "mixlora_status_string", "mixlora_stage_timing", "mixlora_stage_timing_read",
            "mixlora_dispatch_static", "mixlora_dispatch_static_max_tokens",
            "mixlora_multi_ffn_forward", "mixlora_multi_ffn_backward", "mixlora_layer_forward",
-           "mixlora_layer_backward")
+           "mixlora_layer_backward", "mixlora_lora_linear_workspace_bytes", "mixlora_lora_linear_forward",
+           "mixlora_lora_linear_backward", "mixlora_lora_linear_status")
+
+
+class mixlora_linear_shape_t(C.Structure):
+    _fields_ = [("struct_size", C.c_uint32), ("tokens", C.c_int32), ("d_in", C.c_int32), ("d_out", C.c_int32),
+                ("rank", C.c_int32), ("lora_alpha", C.c_float), ("dtype", C.c_int32)]
 
 
 class mixlora_shape_t(C.Structure):
@@ -103,6 +109,16 @@ def _load() -> C.CDLL:
                                            C.c_float, C.c_void_p, C.c_void_p, C.c_void_p, C.c_float, C.c_void_p,
                                            C.c_size_t, C.POINTER(mixlora_grads_t), C.c_void_p]
     lib.mixlora_layer_backward.restype = C.c_int
+    lib.mixlora_lora_linear_workspace_bytes.argtypes = [C.POINTER(mixlora_linear_shape_t)]
+    lib.mixlora_lora_linear_workspace_bytes.restype = C.c_size_t
+    lib.mixlora_lora_linear_forward.argtypes = [C.POINTER(mixlora_linear_shape_t)] + [C.c_void_p] * 6 + [C.c_size_t,
+                                                                                                          C.c_void_p]
+    lib.mixlora_lora_linear_forward.restype = C.c_int
+    lib.mixlora_lora_linear_backward.argtypes = ([C.POINTER(mixlora_linear_shape_t)] + [C.c_void_p] * 6 +
+                                                 [C.c_size_t, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p])
+    lib.mixlora_lora_linear_backward.restype = C.c_int
+    lib.mixlora_lora_linear_status.argtypes = [C.c_void_p, C.c_void_p]
+    lib.mixlora_lora_linear_status.restype = C.c_int32
     lib.mixlora_status_string.argtypes = [C.c_int]
     lib.mixlora_status_string.restype = C.c_char_p
     return lib
@@ -281,3 +297,33 @@ def mixlora_layer_backward(shape, params, norm_weight, eps, xn, inv_rms, dh, aux
                                       _ptr(inv_rms), _ptr(dh), float(aux_coef), _ptr(workspace),
                                       workspace.numel() if workspace is not None else 0, C.byref(grads),
                                       _stream(stream)), "mixlora_layer_backward")
+
+
+def make_linear_shape(tokens, d_in, d_out, rank, lora_alpha, dtype=MIXLORA_DTYPE_BF16) -> mixlora_linear_shape_t:
+    return mixlora_linear_shape_t(C.sizeof(mixlora_linear_shape_t), tokens, d_in, d_out, rank, float(lora_alpha), dtype)
+
+
+def alloc_linear_workspace(shape) -> torch.Tensor:
+    n = lib.mixlora_lora_linear_workspace_bytes(C.byref(shape))
+    if n == 0:
+        raise MixLoraError(1, "mixlora_lora_linear_workspace_bytes")
+    return torch.empty(n, dtype=torch.uint8, device="cuda")
+
+
+def mixlora_lora_linear_forward(shape, x, w, a, b, y, workspace, stream=None) -> None:
+    """y = x W^T + s (x A^T) B^T (plain LoRA on a linear layer)."""
+    _check(lib.mixlora_lora_linear_forward(C.byref(shape), _ptr(x), _ptr(w), _ptr(a), _ptr(b), _ptr(y), _ptr(workspace),
+                                           workspace.numel() if workspace is not None else 0, _stream(stream)),
+           "mixlora_lora_linear_forward")
+
+
+def mixlora_lora_linear_backward(shape, x, w, a, b, dy, workspace, d_a=None, d_b=None, d_x=None, accumulate=0,
+                                 stream=None) -> None:
+    _check(lib.mixlora_lora_linear_backward(C.byref(shape), _ptr(x), _ptr(w), _ptr(a), _ptr(b), _ptr(dy),
+                                            _ptr(workspace), workspace.numel() if workspace is not None else 0,
+                                            _ptr(d_a), _ptr(d_b), _ptr(d_x), int(accumulate), _stream(stream)),
+           "mixlora_lora_linear_backward")
+
+
+def mixlora_lora_linear_status(workspace, stream=None) -> int:
+    return int(lib.mixlora_lora_linear_status(_ptr(workspace), _stream(stream)))

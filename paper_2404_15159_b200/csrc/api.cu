@@ -195,7 +195,8 @@ cudaError_t dense_product(const Ctx& c, int M, const TcOut* outs, int nout, cons
     const TcOut& t = outs[o];
     const int Mo = t.M > 0 ? t.M : M;
     SGemm g = t.mode == 0 ? sgemm_base(c, t.C, t.ldc, 1, c.bf16, Mo, t.N) : sgemm_base(c, t.C, t.s_m, t.s_n, 0, Mo, t.N);
-    if (t.mode == 1) { g.c_nb = t.nb; g.c_sblk = t.s_blk; g.alpha = t.alpha; g.accumulate = t.accumulate; }
+    g.alpha = t.alpha;
+    if (t.mode == 1) { g.c_nb = t.nb; g.c_sblk = t.s_blk; g.accumulate = t.accumulate; }
     for (int i = 0; i < t.nseg; ++i) {
       const TcSeg& sg = t.seg[i];
       SOperand A = sg.a_mn ? soperand(sg.A, 1, sg.lda, c.bf16) : soperand(sg.A, sg.lda, 1, c.bf16);
@@ -757,6 +758,132 @@ int32_t mixlora_stage_timing_read(int32_t max_stages, const char** names, float*
     if (launches) launches[i] = g_prof.launches[i];
   }
   return ST_COUNT;
+}
+
+// ---- plain LoRA on a linear layer (Eq. 1; the attention projections of Section 3.2) ----
+namespace {
+struct LinearLayout { size_t status, zs, dzs, total; };
+LinearLayout linear_layout(const mixlora_linear_shape_t& s) {
+  const size_t el = s.dtype == MIXLORA_DTYPE_BF16 ? 2 : 4;
+  LinearLayout L;
+  size_t off = 0;
+  auto take = [&](size_t bytes) { size_t o = off; off += (bytes + 255) / 256 * 256; return o; };
+  L.status = take(256);
+  L.zs = take((size_t)(s.tokens > 0 ? s.tokens : 1) * s.rank * el);
+  L.dzs = take((size_t)(s.tokens > 0 ? s.tokens : 1) * s.rank * el);
+  L.total = off;
+  return L;
+}
+bool linear_shape_ok(const mixlora_linear_shape_t* s) {
+  return s && s->struct_size == sizeof(mixlora_linear_shape_t) && s->tokens >= 0 && s->d_in > 0 && s->d_out > 0 &&
+         s->rank > 0 && s->rank <= MIXLORA_MAX_RANK && s->d_in % 8 == 0 && s->d_out % 8 == 0 && s->rank % 8 == 0 &&
+         (s->dtype == MIXLORA_DTYPE_BF16 || s->dtype == MIXLORA_DTYPE_FP32) && s->lora_alpha == s->lora_alpha;
+}
+// the dense-product helpers only need the type, the stream and a status word from the context
+Ctx linear_ctx(const mixlora_linear_shape_t& s, void* workspace, void* stream) {
+  Ctx c;
+  memset(&c.s, 0, sizeof(c.s));
+  memset(&c.p, 0, sizeof(c.p));
+  memset(&c.L, 0, sizeof(c.L));
+  c.s.dtype = s.dtype;
+  c.s.tokens = s.tokens;
+  c.ws = reinterpret_cast<char*>(workspace);
+  c.st = reinterpret_cast<cudaStream_t>(stream);
+  c.bf16 = s.dtype == MIXLORA_DTYPE_BF16;
+  c.scale = s.lora_alpha / (float)s.rank;
+  return c;
+}
+}  // namespace
+
+size_t mixlora_lora_linear_workspace_bytes(const mixlora_linear_shape_t* shape) {
+  return linear_shape_ok(shape) ? linear_layout(*shape).total : 0;
+}
+
+mixlora_status_t mixlora_lora_linear_forward(const mixlora_linear_shape_t* shape, const void* x, const void* w,
+                                             const void* a, const void* b, void* y, void* workspace,
+                                             size_t workspace_bytes, void* stream) {
+  if (!linear_shape_ok(shape)) return MIXLORA_ERR_INVALID_ARG;
+  const void* req[] = {x, w, a, b, y};
+  for (const void* q : req)
+    if (!q || !aligned16(q)) return MIXLORA_ERR_INVALID_ARG;
+  const LinearLayout L = linear_layout(*shape);
+  if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255u) || workspace_bytes < L.total)
+    return MIXLORA_ERR_WORKSPACE;
+  const Ctx c = linear_ctx(*shape, workspace, stream);
+  const int T = shape->tokens, din = shape->d_in, dout = shape->d_out, r = shape->rank;
+  MIXLORA_CUDA(cudaMemsetAsync(c.ws + L.status, 0, 256, c.st));
+  if (T == 0) return MIXLORA_OK;
+  {   // zs = s x A^T
+    TcOut z = tc_out(c.ws + L.zs, r, r);
+    z.alpha = c.scale;
+    tc_add(z, x, din, din, a, din, 0);
+    MIXLORA_CUDA(dense_product(c, T, &z, 1));
+  }
+  // y = [x | zs] [W | B]^T : the low-rank term rides along as r extra reduction columns of the frozen product
+  TcOut out = tc_out(y, dout, dout);
+  tc_add(out, x, din, din, w, din, 0);
+  tc_add(out, c.ws + L.zs, r, r, b, r, 0);
+  MIXLORA_CUDA(dense_product(c, T, &out, 1));
+  return MIXLORA_OK;
+}
+
+mixlora_status_t mixlora_lora_linear_backward(const mixlora_linear_shape_t* shape, const void* x, const void* w,
+                                              const void* a, const void* b, const void* dy, void* workspace,
+                                              size_t workspace_bytes, float* d_a, float* d_b, void* d_x,
+                                              int32_t accumulate, void* stream) {
+  if (!linear_shape_ok(shape)) return MIXLORA_ERR_INVALID_ARG;
+  const void* req[] = {x, w, a, b, dy};
+  for (const void* q : req)
+    if (!q || !aligned16(q)) return MIXLORA_ERR_INVALID_ARG;
+  const void* opt[] = {d_a, d_b, d_x};
+  for (const void* q : opt)
+    if (q && !aligned16(q)) return MIXLORA_ERR_INVALID_ARG;
+  if (accumulate != 0 && accumulate != 1) return MIXLORA_ERR_INVALID_ARG;
+  const LinearLayout L = linear_layout(*shape);
+  if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255u) || workspace_bytes < L.total)
+    return MIXLORA_ERR_WORKSPACE;
+  const Ctx c = linear_ctx(*shape, workspace, stream);
+  const int T = shape->tokens, din = shape->d_in, dout = shape->d_out, r = shape->rank;
+  if (T == 0) {
+    if (!accumulate) {
+      if (d_a) MIXLORA_CUDA(cudaMemsetAsync(d_a, 0, sizeof(float) * (size_t)r * din, c.st));
+      if (d_b) MIXLORA_CUDA(cudaMemsetAsync(d_b, 0, sizeof(float) * (size_t)dout * r, c.st));
+    }
+    return MIXLORA_OK;
+  }
+  {   // dzs = s dy B
+    TcOut z = tc_out(c.ws + L.dzs, r, r);
+    z.alpha = c.scale;
+    tc_add(z, dy, dout, dout, b, r, 1);
+    MIXLORA_CUDA(dense_product(c, T, &z, 1));
+  }
+  if (d_x) {   // dx = [dy | dzs] [W ; A]
+    TcOut out = tc_out(d_x, din, din);
+    tc_add(out, dy, dout, dout, w, din, 1);
+    tc_add(out, c.ws + L.dzs, r, r, a, din, 1);
+    MIXLORA_CUDA(dense_product(c, T, &out, 1));
+  }
+  if (d_a) {   // dA[rr][c] = sum_t dzs[t][rr] x[t][c]
+    TcOut out = tc_out_f32(d_a, r, 1, din, 0, 0, 1.f, accumulate);
+    tc_add(out, x, din, T, c.ws + L.dzs, r, 1, 1);
+    MIXLORA_CUDA(dense_product(c, din, &out, 1));
+  }
+  if (d_b) {   // dB[c][rr] = sum_t dy[t][c] zs[t][rr]   (zs carries the scale s)
+    TcOut out = tc_out_f32(d_b, r, r, 1, 0, 0, 1.f, accumulate);
+    tc_add(out, dy, dout, T, c.ws + L.zs, r, 1, 1);
+    MIXLORA_CUDA(dense_product(c, dout, &out, 1));
+  }
+  return MIXLORA_OK;
+}
+
+int32_t mixlora_lora_linear_status(const void* workspace, void* stream) {
+  int v = 0;
+  if (!workspace) return (int32_t)MIXLORA_ERR_INVALID_ARG;
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+  if (cudaMemcpyAsync(&v, workspace, sizeof(int), cudaMemcpyDeviceToHost, st) != cudaSuccess ||
+      cudaStreamSynchronize(st) != cudaSuccess)
+    return (int32_t)MIXLORA_ERR_CUDA;
+  return v;
 }
 
 mixlora_status_t mixlora_gemm_bf16(const void* A, const void* B, void* C, int32_t M, int32_t N, int32_t K,

@@ -114,6 +114,7 @@ __device__ __forceinline__ void store_chunk32(const TcParams& p, int o, int row,
     }
   } else {
     bf16* crow = reinterpret_cast<bf16*>(p.C[o]) + (size_t)row * p.ldc[o];
+    const float alpha0 = p.alpha[o];
     const bf16* rrow = p.R[o] ? reinterpret_cast<const bf16*>(p.R[o]) + (size_t)row * p.ldr[o] : nullptr;
 #pragma unroll
     for (int g8 = 0; g8 < 4; ++g8) {
@@ -122,7 +123,7 @@ __device__ __forceinline__ void store_chunk32(const TcParams& p, int o, int row,
         uint4 q4;
         float w[8];
 #pragma unroll
-        for (int j = 0; j < 8; ++j) w[j] = __uint_as_float(v[g8 * 8 + j]);
+        for (int j = 0; j < 8; ++j) w[j] = alpha0 * __uint_as_float(v[g8 * 8 + j]);
         if (rrow) {                                   // fused residual add, in fp32 before the one rounding
           const uint4 r4 = *reinterpret_cast<const uint4*>(rrow + col);
           const __nv_bfloat162* rp = reinterpret_cast<const __nv_bfloat162*>(&r4);
