@@ -192,8 +192,12 @@ def run_cuda(args):
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device (the library has no CPU path)")
     torch.cuda.set_device(local)
+    use_dist = world > 1 or args.force_dist
     if world > 1:
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    elif use_dist:      # one rank going through the collective path (checks the stream and event plumbing on one GPU)
+        dist.init_process_group("nccl", init_method="tcp://127.0.0.1:29541", rank=0, world_size=1,
+                                device_id=torch.device("cuda", local))
 
     w = workload_by_name(args.workload)
     want_dx = not args.no_dx
@@ -231,8 +235,22 @@ def run_cuda(args):
         B.mixlora_ffn_forward(shape, params, y, ws)
         B.mixlora_aux_loss(shape, ws, AUX_COEF, loss)
         B.mixlora_ffn_backward(shape, params, dev["dy"], AUX_COEF, ws, grads)
-        if world > 1:
-            dist.all_reduce(flat)          # data-parallel sum of the LoRA and router gradients
+
+    if use_dist:
+        # data-parallel sum of the LoRA and router gradients (one flat buffer, one NCCL all-reduce) on a second
+        # stream: it starts when the parameter gradients are enqueued and runs beside the input-gradient product
+        comm = torch.cuda.Stream()
+        ev_ready = torch.cuda.Event()
+        ev_ready.record()
+
+        def step():                        # noqa: F811
+            B.mixlora_ffn_forward(shape, params, y, ws)
+            B.mixlora_aux_loss(shape, ws, AUX_COEF, loss)
+            B.mixlora_ffn_backward_overlap(shape, params, dev["dy"], AUX_COEF, ws, grads, ev_ready)
+            comm.wait_event(ev_ready)
+            with torch.cuda.stream(comm):
+                dist.all_reduce(flat)
+            torch.cuda.current_stream().wait_stream(comm)
 
     M = max(1, args.models)
     if M > 1:
@@ -262,7 +280,7 @@ def run_cuda(args):
             for m in range(M):
                 B.mixlora_aux_loss(m_shapes[m], m_ws[m], AUX_COEF, loss)
             B.mixlora_multi_ffn_backward(m_shapes, m_params, m_dys, [AUX_COEF] * M, m_ws, m_grads)
-            if world > 1:
+            if use_dist:
                 for fl, _ in m_keep:
                     dist.all_reduce(fl)
 
@@ -276,11 +294,11 @@ def run_cuda(args):
             B.mixlora_layer_forward(shape, params, wn, 1e-5, xn, inv_rms, y, ws)
             B.mixlora_aux_loss(shape, ws, AUX_COEF, loss)
             B.mixlora_layer_backward(shape, params, wn, 1e-5, xn, inv_rms, dev["dy"], AUX_COEF, ws, grads)
-            if world > 1:
+            if use_dist:
                 dist.all_reduce(flat)
 
     def barrier():
-        if world > 1:
+        if use_dist:
             dist.barrier()
         torch.cuda.synchronize()
 
@@ -297,7 +315,7 @@ def run_cuda(args):
         barrier()
         t1 = time.time()
         ms = torch.tensor([e0.elapsed_time(e1)], dtype=torch.float64, device="cuda")
-        if world > 1:
+        if use_dist:
             dist.all_reduce(ms, op=dist.ReduceOp.MAX)
         return float(ms.item()), t0, t1
 
@@ -356,7 +374,7 @@ def run_cuda(args):
             B.mixlora_ffn_forward(shape, pb[bi], yb[bi], ws)
             B.mixlora_aux_loss(shape, ws, AUX_COEF, loss)
             B.mixlora_ffn_backward(shape, pb[bi], dyb[bi], AUX_COEF, ws, grads)
-            if world > 1:
+            if use_dist:
                 dist.all_reduce(flat)
             ev_done[bi].record(main)
             with torch.cuda.stream(d2h):
@@ -374,7 +392,7 @@ def run_cuda(args):
     e1.record()
     barrier()
     e2e_t = torch.tensor([e0.elapsed_time(e1)], dtype=torch.float64, device="cuda")
-    if world > 1:
+    if use_dist:
         dist.all_reduce(e2e_t, op=dist.ReduceOp.MAX)
     e2e_ms = float(e2e_t.item())
     e2e_value = world * w.tokens / (e2e_ms / args.steps * 1e-3)
@@ -382,7 +400,7 @@ def run_cuda(args):
     d2h_bytes = hy.numel() * hy.element_size() + 4
 
     if rank != 0:
-        if world > 1:
+        if use_dist:
             dist.destroy_process_group()
         return
 
@@ -434,7 +452,7 @@ def run_cuda(args):
         "config": {"workload": w.name, "tokens_per_gpu": w.tokens, "d_model": w.d_model, "d_ff": w.d_ff,
                    "n_experts": w.n_experts, "top_k": w.top_k, "rank": w.rank, "lora_alpha": w.lora_alpha,
                    "backward_dx": want_dx, "aux_coef": AUX_COEF, "adapters": M, "layer_slice": bool(args.layer and M == 1 and want_dx),
-                   "parallelism": f"dp{world} over tokens" + (", NCCL all-reduce of LoRA/router grads" if world > 1 else ""),
+                   "parallelism": f"dp{world} over tokens" + (", NCCL all-reduce of LoRA/router grads beside the dx product" if use_dist else ""),
                    "l2": "inputs larger than L2 (weights 270 MB + activations > 126 MB), no flush"},
         "roofline": roofline, "cpu_baseline": cpu_baseline,
         "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d_bytes, "d2h_bytes_per_step": d2h_bytes,
@@ -444,7 +462,7 @@ def run_cuda(args):
         "stage_ms": {n: round(v, 4) for n, v in stage_ms.items()}, "device_status": status, "clocks": clocks,
     }
     print(json.dumps(line))
-    if world > 1:
+    if use_dist:
         dist.destroy_process_group()
 
 
@@ -456,6 +474,8 @@ def main():
     ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
     ap.add_argument("--workload", default="c3")
     ap.add_argument("--no-dx", action="store_true")
+    ap.add_argument("--force-dist", action="store_true",
+                    help="with one rank, still go through the NCCL gradient all-reduce path (plumbing check)")
     ap.add_argument("--layer", action="store_true",
                     help="time the block inside its layer (RMSNorm in front, residual behind) instead of the block alone")
     ap.add_argument("--models", type=int, default=1,

@@ -128,6 +128,19 @@ mixlora_status_t mixlora_ffn_backward(const mixlora_shape_t *shape /* host */,
                                       const void *dy, float aux_coef, void *workspace, size_t workspace_bytes,
                                       const mixlora_grads_t *grads /* host struct of device ptrs */, void *stream);
 
+/* mixlora_ffn_backward for data-parallel training (the paper trains on one GPU; the block is independent per token
+ * except for the sums over tokens in the LoRA / router gradients, so replicas hold their own tokens and sum those
+ * gradients).  Same arguments and results; in addition `param_grads_ready` (a cudaEvent_t created by the caller, or
+ * NULL) is recorded on `stream` as soon as every LoRA and router gradient has been enqueued, which is before the
+ * input-gradient product (the longest launch of the backward pass, and it writes no parameter gradient).  A caller
+ * that waits for the event on a second stream and all-reduces the gradients there overlaps the collective with that
+ * product. */
+mixlora_status_t mixlora_ffn_backward_overlap(const mixlora_shape_t *shape /* host */,
+                                              const mixlora_params_t *params /* host struct of device ptrs */,
+                                              const void *dy, float aux_coef, void *workspace, size_t workspace_bytes,
+                                              const mixlora_grads_t *grads /* host struct of device ptrs */,
+                                              void *param_grads_ready /* cudaEvent_t or NULL */, void *stream);
+
 /* Multi-model forward and backward (Section 3.3 (II), the task loop of Algorithm 1): n_models MixLoRA adapters,
  * each with its own tokens, router, experts, rank and workspace, share ONE frozen FFN (same w_gate, w_up, w_down
  * pointers, same d_model, d_ff and dtype; anything else returns MIXLORA_ERR_INVALID_ARG).  The frozen weights are

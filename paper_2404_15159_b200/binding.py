@@ -25,7 +25,7 @@ EXPORTS = ("mixlora_limits", "mixlora_workspace_bytes", "mixlora_ffn_forward", "
            "mixlora_dispatch_static", "mixlora_dispatch_static_max_tokens",
            "mixlora_multi_ffn_forward", "mixlora_multi_ffn_backward", "mixlora_layer_forward",
            "mixlora_layer_backward", "mixlora_lora_linear_workspace_bytes", "mixlora_lora_linear_forward",
-           "mixlora_lora_linear_backward", "mixlora_lora_linear_status")
+           "mixlora_lora_linear_backward", "mixlora_lora_linear_status", "mixlora_ffn_backward_overlap")
 
 
 class mixlora_linear_shape_t(C.Structure):
@@ -109,6 +109,10 @@ def _load() -> C.CDLL:
                                            C.c_float, C.c_void_p, C.c_void_p, C.c_void_p, C.c_float, C.c_void_p,
                                            C.c_size_t, C.POINTER(mixlora_grads_t), C.c_void_p]
     lib.mixlora_layer_backward.restype = C.c_int
+    lib.mixlora_ffn_backward_overlap.argtypes = [C.POINTER(mixlora_shape_t), C.POINTER(mixlora_params_t), C.c_void_p,
+                                                 C.c_float, C.c_void_p, C.c_size_t, C.POINTER(mixlora_grads_t),
+                                                 C.c_void_p, C.c_void_p]
+    lib.mixlora_ffn_backward_overlap.restype = C.c_int
     lib.mixlora_lora_linear_workspace_bytes.argtypes = [C.POINTER(mixlora_linear_shape_t)]
     lib.mixlora_lora_linear_workspace_bytes.restype = C.c_size_t
     lib.mixlora_lora_linear_forward.argtypes = [C.POINTER(mixlora_linear_shape_t)] + [C.c_void_p] * 6 + [C.c_size_t,
@@ -327,3 +331,13 @@ def mixlora_lora_linear_backward(shape, x, w, a, b, dy, workspace, d_a=None, d_b
 
 def mixlora_lora_linear_status(workspace, stream=None) -> int:
     return int(lib.mixlora_lora_linear_status(_ptr(workspace), _stream(stream)))
+
+
+def mixlora_ffn_backward_overlap(shape, params, dy, aux_coef, workspace, grads, ready_event, stream=None) -> None:
+    """mixlora_ffn_backward that records `ready_event` (a torch.cuda.Event that has been recorded at least once, so
+    that its handle exists) when the LoRA / router gradients are enqueued, before the input-gradient product."""
+    handle = ready_event.cuda_event if ready_event is not None else None
+    _check(lib.mixlora_ffn_backward_overlap(C.byref(shape), C.byref(params), _ptr(dy), float(aux_coef), _ptr(workspace),
+                                            workspace.numel() if workspace is not None else 0, C.byref(grads),
+                                            C.c_void_p(handle) if handle else None, _stream(stream)),
+           "mixlora_ffn_backward_overlap")

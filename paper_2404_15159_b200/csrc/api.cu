@@ -519,13 +519,21 @@ static mixlora_status_t bwd_zero_tokens(const Ctx& c, const mixlora_grads_t* gra
   return MIXLORA_OK;
 }
 
-static mixlora_status_t bwd_experts(const Ctx& c, const void* dy, float aux_coef, const mixlora_grads_t* grads) {
+// `param_grads_ready` (optional cudaEvent_t) is recorded once every LoRA / router gradient has been enqueued, before
+// the input-gradient product: a caller's gradient all-reduce can then overlap that product.
+static mixlora_status_t bwd_experts(const Ctx& c, const void* dy, float aux_coef, const mixlora_grads_t* grads,
+                                    void* param_grads_ready = nullptr) {
   const mixlora_params_t* params = &c.p;
   const int T = c.s.tokens, d = c.s.d_model, f = c.s.d_ff, N = c.s.n_experts, r = c.s.rank, k = c.s.top_k;
   const int Nr = N * r, NP = round_up8(N);
   const int acc = grads->accumulate;
   const int want_dx = grads->d_x != nullptr;
-  if (T == 0) return bwd_zero_tokens(c, grads);
+  if (T == 0) {
+    mixlora_status_t zs = bwd_zero_tokens(c, grads);
+    if (zs == MIXLORA_OK && param_grads_ready)
+      MIXLORA_CUDA(cudaEventRecord(reinterpret_cast<cudaEvent_t>(param_grads_ready), c.st));
+    return zs;
+  }
   {
     StageScope ss(ST_SWIGLU_BWD, c.st, 3);
     MIXLORA_CUDA(launch_slot_prep_bwd(c));
@@ -606,6 +614,7 @@ static mixlora_status_t bwd_experts(const Ctx& c, const void* dy, float aux_coef
     StageScope ss(ST_LORA_WGRAD, c.st, dense_launches(c, d, outs, n));
     MIXLORA_CUDA(dense_product(c, d, outs, n));
   }
+  if (param_grads_ready) MIXLORA_CUDA(cudaEventRecord(reinterpret_cast<cudaEvent_t>(param_grads_ready), c.st));
   if (want_dx) {
     // dx = [dabar | dbbar | dZg | dZu | dl] [W_g ; W_u ; A_g ; A_u ; W_r]
     TcOut out = tc_out(grads->d_x, d, d);
@@ -628,6 +637,16 @@ mixlora_status_t mixlora_ffn_backward(const mixlora_shape_t* shape, const mixlor
   if (st != MIXLORA_OK) return st;
   if ((st = bwd_shared_dgrad(&c, &dy, 1)) != MIXLORA_OK) return st;
   return bwd_experts(c, dy, aux_coef, grads);
+}
+
+mixlora_status_t mixlora_ffn_backward_overlap(const mixlora_shape_t* shape, const mixlora_params_t* params,
+                                              const void* dy, float aux_coef, void* workspace, size_t workspace_bytes,
+                                              const mixlora_grads_t* grads, void* param_grads_ready, void* stream) {
+  Ctx c;
+  mixlora_status_t st = bwd_check(shape, params, dy, workspace, workspace_bytes, grads, stream, &c);
+  if (st != MIXLORA_OK) return st;
+  if ((st = bwd_shared_dgrad(&c, &dy, 1)) != MIXLORA_OK) return st;
+  return bwd_experts(c, dy, aux_coef, grads, param_grads_ready);
 }
 
 mixlora_status_t mixlora_multi_ffn_backward(int32_t n_models, const mixlora_shape_t* shapes,

@@ -21,7 +21,7 @@ def rel_err(got, ref) -> float:
 
 
 def gpu_run(w: synth.Workload, tensors: dict, backward=True, want_dx=True, aux_coef=0.01, renormalize=1,
-            aux_f_mode=0, accumulate=0, grads_init=None, repeats=1):
+            aux_f_mode=0, accumulate=0, grads_init=None, repeats=1, overlap=False):
     """Forward (+ aux loss, + backward) on the GPU through the C ABI.  Returns numpy arrays."""
     import torch
     from paper_2404_15159_b200 import binding as B
@@ -63,8 +63,22 @@ def gpu_run(w: synth.Workload, tensors: dict, backward=True, want_dx=True, aux_c
                 g["d_x"] = torch.full((max(w.tokens, 1), w.d_model), float("nan"), dtype=act, device="cuda")[: w.tokens]
             grads = B.make_grads(accumulate=accumulate, **{n: (v if v.numel() else torch.empty(8, device="cuda"))
                                                            for n, v in g.items()})
-            B.mixlora_ffn_backward(shape, params, dev["dy"] if w.tokens else torch.empty(8, dtype=act, device="cuda"),
-                                   aux_coef, ws, grads)
+            dy_dev = dev["dy"] if w.tokens else torch.empty(8, dtype=act, device="cuda")
+            if overlap:
+                # the variant that signals when the parameter gradients are enqueued: a second stream copies them
+                # at that point, while the input-gradient product is still to run
+                ev = torch.cuda.Event()
+                ev.record()
+                side = torch.cuda.Stream()
+                B.mixlora_ffn_backward_overlap(shape, params, dy_dev, aux_coef, ws, grads, ev)
+                side.wait_event(ev)
+                with torch.cuda.stream(side):
+                    snap = {n: v.clone() for n, v in g.items() if n != "d_x"}
+                torch.cuda.current_stream().wait_stream(side)
+                for n, v in snap.items():
+                    out["snap_" + n] = v
+            else:
+                B.mixlora_ffn_backward(shape, params, dy_dev, aux_coef, ws, grads)
     torch.cuda.synchronize()
     out["status"] = B.mixlora_device_status(ws)
     out["y"] = y.float().cpu().numpy()
@@ -76,6 +90,8 @@ def gpu_run(w: synth.Workload, tensors: dict, backward=True, want_dx=True, aux_c
         out[n] = v.cpu().numpy().copy()
     for n, v in g.items():
         out[n] = v.float().cpu().numpy()
+    for n in [n for n in out if n.startswith("snap_")]:
+        out[n] = out[n].float().cpu().numpy()
     return out
 
 

@@ -82,3 +82,18 @@ def test_multi_call_rejects_adapters_with_different_frozen_weights():
     with pytest.raises(B.MixLoraError) as err:
         B.mixlora_multi_ffn_forward([shape, shape], ps, ys, wss)
     assert err.value.status == 1
+
+
+def test_backward_overlap_signals_after_the_parameter_gradients_and_changes_no_result():
+    # data-parallel replicas all-reduce the LoRA / router gradients while the input-gradient product still runs:
+    # what a second stream reads at the signal must already be the final gradients
+    w = adapters()[0]
+    t = synth.generate(w)
+    plain = helpers.gpu_run(w, t, aux_coef=0.01)
+    over = helpers.gpu_run(w, t, aux_coef=0.01, overlap=True)
+    assert over["status"] == 0
+    for n in GRADS:
+        np.testing.assert_array_equal(over[n], plain[n])
+        np.testing.assert_array_equal(over["snap_" + n], plain[n])
+    np.testing.assert_array_equal(over["d_x"], plain["d_x"])
+
