@@ -3,6 +3,7 @@
 #include <stdio.h>
 #include <string.h>
 
+#include <mutex>
 #include <vector>
 
 #include "common.cuh"
@@ -124,6 +125,62 @@ struct StageScope {
     }
   }
 };
+
+// ---- side streams for the per-adapter parts of the multi-model calls ----
+// The per-adapter steps of several adapters are independent and, at a few thousand tokens each, many of their
+// launches fill only part of the GPU; they are spread over a few library-owned streams between two points where
+// everything is back on the caller's stream.  Created on first use, one set per device, kept until exit.
+constexpr int kSideStreams = 4;
+struct SidePool {
+  cudaStream_t s[kSideStreams];
+  cudaEvent_t fork, join[kSideStreams];
+  bool ok = false, tried = false;
+};
+SidePool g_side[16];
+std::mutex g_side_mu;
+
+SidePool* side_pool() {
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 16) return nullptr;
+  std::lock_guard<std::mutex> lock(g_side_mu);
+  SidePool& p = g_side[dev];
+  if (!p.tried) {
+    p.tried = true;
+    bool ok = cudaEventCreateWithFlags(&p.fork, cudaEventDisableTiming) == cudaSuccess;
+    for (int i = 0; i < kSideStreams && ok; ++i)
+      ok = cudaStreamCreateWithFlags(&p.s[i], cudaStreamNonBlocking) == cudaSuccess &&
+           cudaEventCreateWithFlags(&p.join[i], cudaEventDisableTiming) == cudaSuccess;
+    p.ok = ok;
+  }
+  return p.ok ? &p : nullptr;
+}
+
+// Runs fn(adapter context, index) for every adapter, on the side streams when there are several adapters (and no
+// stage timing is being taken, which needs one stream), else in turn on the caller's stream.
+template <typename F>
+mixlora_status_t for_each_adapter(const Ctx* cs, int n, F fn) {
+  SidePool* pool = (n > 1 && !g_prof.on) ? side_pool() : nullptr;
+  mixlora_status_t st = MIXLORA_OK;
+  if (!pool) {
+    for (int m = 0; m < n && st == MIXLORA_OK; ++m) st = fn(cs[m], m);
+    return st;
+  }
+  cudaStream_t main_st = cs[0].st;
+  if (cudaEventRecord(pool->fork, main_st) != cudaSuccess) return MIXLORA_ERR_CUDA;
+  const int used = n < kSideStreams ? n : kSideStreams;
+  for (int j = 0; j < used; ++j)
+    if (cudaStreamWaitEvent(pool->s[j], pool->fork, 0) != cudaSuccess) st = MIXLORA_ERR_CUDA;
+  for (int m = 0; m < n && st == MIXLORA_OK; ++m) {
+    Ctx c = cs[m];
+    c.st = pool->s[m % kSideStreams];
+    st = fn(c, m);
+  }
+  for (int j = 0; j < used; ++j)   // always rejoin, also after an error, so that no stream is left dangling
+    if (cudaEventRecord(pool->join[j], pool->s[j]) != cudaSuccess ||
+        cudaStreamWaitEvent(main_st, pool->join[j], 0) != cudaSuccess)
+      st = st == MIXLORA_OK ? MIXLORA_ERR_CUDA : st;
+  return st;
+}
 
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
@@ -414,13 +471,10 @@ mixlora_status_t mixlora_multi_ffn_forward(int32_t n_models, const mixlora_shape
       if (workspaces[o] == workspaces[m] || y[o] == y[m]) return MIXLORA_ERR_INVALID_ARG;
   }
   mixlora_status_t st;
-  for (int m = 0; m < n_models; ++m)
-    if ((st = fwd_route(cs[m])) != MIXLORA_OK) return st;
+  if ((st = for_each_adapter(cs, n_models, [&](const Ctx& c, int) { return fwd_route(c); })) != MIXLORA_OK) return st;
   for (int m = 0; m < n_models; m += 2)
     if ((st = fwd_shared_projections(&cs[m], n_models - m >= 2 ? 2 : 1)) != MIXLORA_OK) return st;
-  for (int m = 0; m < n_models; ++m)
-    if ((st = fwd_experts(cs[m], y[m])) != MIXLORA_OK) return st;
-  return MIXLORA_OK;
+  return for_each_adapter(cs, n_models, [&](const Ctx& c, int m) { return fwd_experts(c, y[m]); });
 }
 
 mixlora_status_t mixlora_aux_loss(const mixlora_shape_t* shape, const void* workspace, float coef, float* loss,
@@ -668,9 +722,8 @@ mixlora_status_t mixlora_multi_ffn_backward(int32_t n_models, const mixlora_shap
   mixlora_status_t st;
   for (int m = 0; m < n_models; m += 2)
     if ((st = bwd_shared_dgrad(&cs[m], &dy[m], n_models - m >= 2 ? 2 : 1)) != MIXLORA_OK) return st;
-  for (int m = 0; m < n_models; ++m)
-    if ((st = bwd_experts(cs[m], dy[m], aux_coef[m], &grads[m])) != MIXLORA_OK) return st;
-  return MIXLORA_OK;
+  return for_each_adapter(cs, n_models,
+                          [&](const Ctx& c, int m) { return bwd_experts(c, dy[m], aux_coef[m], &grads[m]); });
 }
 
 
