@@ -148,7 +148,10 @@ mixlora_status_t mixlora_ffn_backward_overlap(const mixlora_shape_t *shape /* ho
  * every other step runs per adapter exactly as in the single-model calls, so each adapter's results equal those of
  * mixlora_ffn_forward / mixlora_ffn_backward on it alone, bit for bit.  All arrays are HOST arrays of n_models
  * entries (of structs / device pointers / sizes); workspaces and outputs must be distinct per adapter.
- * mixlora_aux_loss and mixlora_routing_view are called per adapter on its own workspace. */
+ * mixlora_aux_loss and mixlora_routing_view are called per adapter on its own workspace.
+ * The per-adapter steps of different adapters are enqueued on a few streams that the library creates on first use
+ * (one set per device, kept until exit); they start after everything enqueued on `stream` before the call, and work
+ * enqueued on `stream` after the call starts after them. */
 mixlora_status_t mixlora_multi_ffn_forward(int32_t n_models, const mixlora_shape_t *shapes /* host [n] */,
                                            const mixlora_params_t *params /* host [n] */, void *const *y /* host [n] */,
                                            void *const *workspaces /* host [n] */,
