@@ -108,7 +108,11 @@ size_t mixlora_workspace_bytes(const mixlora_shape_t *shape /* host */, int for_
  * prefix scan and stable permutation by expert; shared W1/W3 projections once per token
  * (Section 3.3 (I)); per-expert LoRA deltas; SwiGLU; down projection plus its LoRA; gate-
  * weighted combine.  `y` is [T, d] in shape.dtype.  The routing, the probabilities and the
- * activations that the backward pass re-uses are left in `workspace` (256-byte aligned). */
+ * activations that the backward pass re-uses are left in `workspace` (256-byte aligned).
+ * The router and the dispatch are enqueued on a stream that the library creates on first use (one set per device,
+ * kept until exit) so that they run beside the shared projections; they start after everything enqueued on
+ * `stream` before the call, and the rest of the call, like later work on `stream`, starts after them.
+ * MIXLORA_SERIAL=1 in the environment (read once) keeps every launch on `stream`. */
 mixlora_status_t mixlora_ffn_forward(const mixlora_shape_t *shape /* host */,
                                      const mixlora_params_t *params /* host struct of device ptrs */,
                                      void *y, void *workspace, size_t workspace_bytes, void *stream);

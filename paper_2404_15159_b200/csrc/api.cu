@@ -1,6 +1,7 @@
 // C ABI of the MixLoRA FFN library: argument checks, workspace layout, and the sequence of
 // kernel launches of the forward and backward passes.
 #include <stdio.h>
+#include <stdlib.h>
 #include <string.h>
 
 #include <mutex>
@@ -140,6 +141,8 @@ SidePool g_side[16];
 std::mutex g_side_mu;
 
 SidePool* side_pool() {
+  static const bool serial = [] { const char* e = getenv("MIXLORA_SERIAL"); return e && e[0] == '1'; }();
+  if (serial) return nullptr;                          // everything on the caller's stream, for measurements
   int dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 16) return nullptr;
   std::lock_guard<std::mutex> lock(g_side_mu);
@@ -155,11 +158,25 @@ SidePool* side_pool() {
   return p.ok ? &p : nullptr;
 }
 
-// Runs fn(adapter context, index) for every adapter, on the side streams when there are several adapters (and no
-// stage timing is being taken, which needs one stream), else in turn on the caller's stream.
+// Runs fn(adapter context, index) for every adapter, on the side streams when `spread` holds (and no stage timing
+// is being taken, which needs one stream), else in turn on the caller's stream.  With join = false the caller's
+// stream is not made to wait yet: join_adapters() does that later, so that work enqueued on the caller's stream in
+// between runs beside the adapters' steps.
+struct Forked { SidePool* pool = nullptr; int used = 0; };
+
+mixlora_status_t join_adapters(cudaStream_t main_st, Forked& fk) {
+  mixlora_status_t st = MIXLORA_OK;
+  for (int j = 0; fk.pool && j < fk.used; ++j)
+    if (cudaEventRecord(fk.pool->join[j], fk.pool->s[j]) != cudaSuccess ||
+        cudaStreamWaitEvent(main_st, fk.pool->join[j], 0) != cudaSuccess)
+      st = MIXLORA_ERR_CUDA;
+  fk.pool = nullptr;
+  return st;
+}
+
 template <typename F>
-mixlora_status_t for_each_adapter(const Ctx* cs, int n, F fn) {
-  SidePool* pool = (n > 1 && !g_prof.on) ? side_pool() : nullptr;
+mixlora_status_t for_each_adapter(const Ctx* cs, int n, bool spread, F fn, Forked* later = nullptr) {
+  SidePool* pool = (spread && !g_prof.on) ? side_pool() : nullptr;
   mixlora_status_t st = MIXLORA_OK;
   if (!pool) {
     for (int m = 0; m < n && st == MIXLORA_OK; ++m) st = fn(cs[m], m);
@@ -167,19 +184,23 @@ mixlora_status_t for_each_adapter(const Ctx* cs, int n, F fn) {
   }
   cudaStream_t main_st = cs[0].st;
   if (cudaEventRecord(pool->fork, main_st) != cudaSuccess) return MIXLORA_ERR_CUDA;
-  const int used = n < kSideStreams ? n : kSideStreams;
-  for (int j = 0; j < used; ++j)
+  Forked fk;
+  fk.pool = pool;
+  fk.used = n < kSideStreams ? n : kSideStreams;
+  for (int j = 0; j < fk.used; ++j)
     if (cudaStreamWaitEvent(pool->s[j], pool->fork, 0) != cudaSuccess) st = MIXLORA_ERR_CUDA;
   for (int m = 0; m < n && st == MIXLORA_OK; ++m) {
     Ctx c = cs[m];
     c.st = pool->s[m % kSideStreams];
     st = fn(c, m);
   }
-  for (int j = 0; j < used; ++j)   // always rejoin, also after an error, so that no stream is left dangling
-    if (cudaEventRecord(pool->join[j], pool->s[j]) != cudaSuccess ||
-        cudaStreamWaitEvent(main_st, pool->join[j], 0) != cudaSuccess)
-      st = st == MIXLORA_OK ? MIXLORA_ERR_CUDA : st;
-  return st;
+  if (later && st == MIXLORA_OK) {
+    *later = fk;
+    return st;
+  }
+  // rejoin at once (always after an error, so that no stream is left dangling)
+  mixlora_status_t js = join_adapters(main_st, fk);
+  return st == MIXLORA_OK ? js : st;
 }
 
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
@@ -345,8 +366,11 @@ static mixlora_status_t fwd_check(const mixlora_shape_t* shape, const mixlora_pa
 }
 
 // router (Eq. 7) and dispatch
-static mixlora_status_t fwd_route(const Ctx& c) {
+static mixlora_status_t fwd_clear_status(const Ctx& c) {
   MIXLORA_CUDA(cudaMemsetAsync(c.ws + c.L.status, 0, 256, c.st));
+  return MIXLORA_OK;
+}
+static mixlora_status_t fwd_route(const Ctx& c) {
   if (c.s.tokens == 0) return MIXLORA_OK;
   { StageScope ss(ST_ROUTER, c.st, 2); MIXLORA_CUDA(launch_router(c)); }
   { StageScope ss(ST_DISPATCH, c.st, 3); MIXLORA_CUDA(launch_dispatch(c)); }
@@ -447,8 +471,14 @@ mixlora_status_t mixlora_ffn_forward(const mixlora_shape_t* shape, const mixlora
   Ctx c;
   mixlora_status_t st = fwd_check(shape, params, y, workspace, workspace_bytes, stream, &c);
   if (st != MIXLORA_OK) return st;
-  if ((st = fwd_route(c)) != MIXLORA_OK) return st;
-  if ((st = fwd_shared_projections(&c, 1)) != MIXLORA_OK) return st;
+  if ((st = fwd_clear_status(c)) != MIXLORA_OK) return st;
+  // the router and the dispatch need only x: they run on a side stream beside the shared projections
+  Forked fk;
+  if ((st = for_each_adapter(&c, 1, true, [&](const Ctx& cc, int) { return fwd_route(cc); }, &fk)) != MIXLORA_OK)
+    return st;
+  st = fwd_shared_projections(&c, 1);
+  mixlora_status_t js = join_adapters(c.st, fk);
+  if (st != MIXLORA_OK || js != MIXLORA_OK) return st != MIXLORA_OK ? st : js;
   return fwd_experts(c, y);
 }
 
@@ -471,10 +501,16 @@ mixlora_status_t mixlora_multi_ffn_forward(int32_t n_models, const mixlora_shape
       if (workspaces[o] == workspaces[m] || y[o] == y[m]) return MIXLORA_ERR_INVALID_ARG;
   }
   mixlora_status_t st;
-  if ((st = for_each_adapter(cs, n_models, [&](const Ctx& c, int) { return fwd_route(c); })) != MIXLORA_OK) return st;
-  for (int m = 0; m < n_models; m += 2)
-    if ((st = fwd_shared_projections(&cs[m], n_models - m >= 2 ? 2 : 1)) != MIXLORA_OK) return st;
-  return for_each_adapter(cs, n_models, [&](const Ctx& c, int m) { return fwd_experts(c, y[m]); });
+  for (int m = 0; m < n_models; ++m)
+    if ((st = fwd_clear_status(cs[m])) != MIXLORA_OK) return st;
+  Forked fk;
+  if ((st = for_each_adapter(cs, n_models, true, [&](const Ctx& c, int) { return fwd_route(c); }, &fk)) != MIXLORA_OK)
+    return st;
+  for (int m = 0; m < n_models && st == MIXLORA_OK; m += 2)
+    st = fwd_shared_projections(&cs[m], n_models - m >= 2 ? 2 : 1);
+  mixlora_status_t js = join_adapters(cs[0].st, fk);
+  if (st != MIXLORA_OK || js != MIXLORA_OK) return st != MIXLORA_OK ? st : js;
+  return for_each_adapter(cs, n_models, n_models > 1, [&](const Ctx& c, int m) { return fwd_experts(c, y[m]); });
 }
 
 mixlora_status_t mixlora_aux_loss(const mixlora_shape_t* shape, const void* workspace, float coef, float* loss,
@@ -722,7 +758,7 @@ mixlora_status_t mixlora_multi_ffn_backward(int32_t n_models, const mixlora_shap
   mixlora_status_t st;
   for (int m = 0; m < n_models; m += 2)
     if ((st = bwd_shared_dgrad(&cs[m], &dy[m], n_models - m >= 2 ? 2 : 1)) != MIXLORA_OK) return st;
-  return for_each_adapter(cs, n_models,
+  return for_each_adapter(cs, n_models, n_models > 1,
                           [&](const Ctx& c, int m) { return bwd_experts(c, dy[m], aux_coef[m], &grads[m]); });
 }
 
@@ -755,8 +791,13 @@ mixlora_status_t mixlora_layer_forward(const mixlora_shape_t* shape, const mixlo
     StageScope ss(ST_NORM, c.st, shape->tokens > 0 ? 1 : 0);
     MIXLORA_CUDA(launch_rmsnorm_fwd(c, params->x, norm_weight, eps, xn, inv_rms));
   }
-  if ((st = fwd_route(c)) != MIXLORA_OK) return st;
-  if ((st = fwd_shared_projections(&c, 1)) != MIXLORA_OK) return st;
+  if ((st = fwd_clear_status(c)) != MIXLORA_OK) return st;
+  Forked fk;
+  if ((st = for_each_adapter(&c, 1, true, [&](const Ctx& cc, int) { return fwd_route(cc); }, &fk)) != MIXLORA_OK)
+    return st;
+  st = fwd_shared_projections(&c, 1);
+  mixlora_status_t js = join_adapters(c.st, fk);
+  if (st != MIXLORA_OK || js != MIXLORA_OK) return st != MIXLORA_OK ? st : js;
   return fwd_experts(c, h, params->x);
 }
 
