@@ -55,6 +55,9 @@ struct alignas(64) TcParams {
   int kblocks[kMaxSeg];
   int Mo[kMaxOut];                 // rows of each output (outputs of one launch may differ in rows)
   int m_tiles_o[kMaxOut];
+  int n_tiles_o[kMaxOut];          // column tiles of each output
+  int row_group;                   // > 0: tiles are handed out row group by row group (see tile_coord)
+  int nt_total;                    // column tiles of all outputs together
   int nseg, nout, total_tiles, tile_m;
   // Optional device-built work list (block-sparse schedule over the sorted slots): item = 8 ints
   // {output, m0, n0, first k-block, end k-block, first stored column, end stored column, 0}; *work_count items.
@@ -79,6 +82,28 @@ __device__ __forceinline__ TileCoord tile_coord(const TcParams& p, int tile) {
     t.o = a.x; t.m0 = a.y; t.n0 = a.z; t.kb0 = a.w; t.kb1 = b.x; t.n_lo = b.y; t.n_hi = b.z;
     return t;
   }
+  t.kb0 = 0; t.kb1 = -1;                  // all k-blocks of every segment
+  if (p.row_group > 0) {
+    // Row groups (all outputs have the same rows): inside a group of row_group row tiles, rows fastest, then the
+    // column tiles of every output in turn.  The CTAs that run together then cover a near-square patch of the
+    // output (few distinct A and B tiles per step of the reduction), and when the A rows of one group fit in L2
+    // they stay there while the group sweeps every column: DRAM sees A about once and B once per group.
+    const int m_tiles = p.m_tiles_o[0];
+    const int per_group = p.row_group * p.nt_total;
+    const int g = tile / per_group, rem = tile - g * per_group;
+    const int rows = min(p.row_group, m_tiles - g * p.row_group);
+    int cidx = rem / rows;
+    const int mloc = rem - cidx * rows;
+    int o = 0;
+#pragma unroll
+    for (int i = 0; i < kMaxOut - 1; ++i)
+      if (o == i && i + 1 < p.nout && cidx >= p.n_tiles_o[i]) { cidx -= p.n_tiles_o[i]; o = i + 1; }
+    t.o = o;
+    t.m0 = (g * p.row_group + mloc) * p.tile_m;
+    t.n0 = cidx * p.tile_n[o];
+    t.n_lo = 0; t.n_hi = p.N[o];
+    return t;
+  }
   int o = 0;
 #pragma unroll
   for (int i = 1; i < kMaxOut; ++i)
@@ -87,7 +112,6 @@ __device__ __forceinline__ TileCoord tile_coord(const TcParams& p, int tile) {
   t.o = o;
   t.m0 = (local % p.m_tiles_o[o]) * p.tile_m;  // rows fastest: neighbouring CTAs share the B tile
   t.n0 = (local / p.m_tiles_o[o]) * p.tile_n[o];
-  t.kb0 = 0; t.kb1 = -1;                  // all k-blocks of every segment
   t.n_lo = 0; t.n_hi = p.N[o];
   return t;
 }
@@ -646,7 +670,9 @@ cudaError_t launch_tc_gemm(int M, const TcOut* outs, int nout, int* status_word,
     p.R[o] = t.mode == 0 ? t.R : nullptr; p.ldr[o] = t.ldr;
     p.s_n[o] = t.s_n; p.s_blk[o] = t.s_blk; p.nb[o] = t.nb; p.alpha[o] = t.alpha; p.accumulate[o] = t.accumulate;
     p.tile_start[o] = tiles;
-    tiles += p.m_tiles_o[o] * ((t.N + tn - 1) / tn);
+    p.n_tiles_o[o] = (t.N + tn - 1) / tn;
+    p.nt_total += p.n_tiles_o[o];
+    tiles += p.m_tiles_o[o] * p.n_tiles_o[o];
     const int b_rows = pair ? tn / 2 : tn;               // rows of a K-major B tile held by one CTA
     for (int s = 0; s < nseg; ++s) {
       const TcSeg& g = t.seg[s];
@@ -659,6 +685,25 @@ cudaError_t launch_tc_gemm(int M, const TcOut* outs, int nout, int* status_word,
     }
   }
   for (int o = nout; o <= kMaxOut; ++o) p.tile_start[o] = tiles;
+  if (!wl) {
+    bool uniform = true;
+    for (int o = 1; o < nout; ++o) uniform = uniform && p.m_tiles_o[o] == p.m_tiles_o[0];
+    const int m_tiles = p.m_tiles_o[0];
+    long long k_total = 0;
+    for (int s = 0; s < nseg; ++s) k_total += outs[0].seg[s].K;
+    const long long slice = (long long)tile_m * k_total * 2;          // bytes of A behind one row tile
+    if (uniform && m_tiles > 1 && slice * m_tiles > (24ll << 20)) {   // A does not simply stay in L2
+      const long long resident = (40ll << 20) / slice;                // row tiles whose A rows fit in L2 together
+      int rg;
+      if (resident >= 8) {
+        const int groups = (int)((m_tiles + resident - 1) / resident);
+        rg = (m_tiles + groups - 1) / groups;                         // balanced groups
+      } else {
+        rg = 8;                                                        // deep reductions: near-square waves of CTAs
+      }
+      if (rg < m_tiles) p.row_group = rg;
+    }
+  }
   p.total_tiles = wl ? wl->max_items : tiles;
   tiles = p.total_tiles;
 
