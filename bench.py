@@ -434,8 +434,19 @@ def run_cuda(args):
            for n, bts in hbm_bytes.items() if bts and stage_ms.get(n)}
     roofline["hbm_stages"] = hbm
     roofline["hbm_peak_gbs"] = peaks["hbm_gbs"]
-    roofline["traffic_note"] = ("null: the DRAM counters were taken on a 2048-token case (gate/up launch: 199.7 MB read "
-                                "against 199.3 MB algorithmic) and do not scale with tokens, the weights being fixed")
+    # DRAM bytes (read + write) of the frozen-projection launches, from one single-pass ncu capture of this command's
+    # workload at full size (profiles/tc_gemm_pair_kernel_c3_dram.md); other workloads have no capture
+    measured_dram = {"gemm_gate_up": 905.3e6, "gemm_down": 905.9e6, "gemm_dgrad_down": 463.9e6, "gemm_dx": 2110.0e6}
+    algorithmic_dram = {"gemm_gate_up": (T_ * d_ + 2 * f_ * d_ + 2 * T_ * f_) * E,
+                        "gemm_down": (T_ * f_ + f_ * d_ + T_ * d_) * E,
+                        "gemm_dgrad_down": (T_ * d_ + f_ * d_ + T_ * f_) * E,
+                        "gemm_dx": (2 * T_ * f_ + 2 * f_ * d_ + T_ * d_) * E}
+    if w.name == synth.c3().name and want_dx and M == 1 and not args.layer and bf16:
+        roofline["traffic"] = measured_dram[dom]
+        roofline["traffic_note"] = ("dram__bytes_read.sum + dram__bytes_write.sum of the %s launch at this size; its "
+                                    "operands and result are %.1f MB" % (dom, algorithmic_dram[dom] / 1e6))
+    else:
+        roofline["traffic_note"] = "null: the DRAM counters were taken on the default workload only"
 
     cpu_baseline = None
     if world == 1 and not args.no_cpu_baseline:
