@@ -435,7 +435,7 @@ def run_cuda(args):
     roofline["hbm_stages"] = hbm
     roofline["hbm_peak_gbs"] = peaks["hbm_gbs"]
     # DRAM bytes (read + write) of the frozen-projection launches, from one single-pass ncu capture of this command's
-    # workload at full size (profiles/tc_gemm_pair_kernel_c3_dram.md); other workloads have no capture
+    # workload at full size (summary under profiles/); other workloads have no capture
     measured_dram = {"gemm_gate_up": 905.3e6, "gemm_down": 905.9e6, "gemm_dgrad_down": 463.9e6, "gemm_dx": 2110.0e6}
     algorithmic_dram = {"gemm_gate_up": (T_ * d_ + 2 * f_ * d_ + 2 * T_ * f_) * E,
                         "gemm_down": (T_ * f_ + f_ * d_ + T_ * d_) * E,
