@@ -374,6 +374,9 @@ static mixlora_status_t fwd_route(const Ctx& c) {
   if (c.s.tokens == 0) return MIXLORA_OK;
   { StageScope ss(ST_ROUTER, c.st, 2); MIXLORA_CUDA(launch_router(c)); }
   { StageScope ss(ST_DISPATCH, c.st, 3); MIXLORA_CUDA(launch_dispatch(c)); }
+  // repacks that depend on the parameters only (s B_d, s B_g, s B_u with all experts' blocks side by side); the
+  // backward pass finds them in the workspace
+  { StageScope ss(ST_DISPATCH, c.st, 3); MIXLORA_CUDA(launch_bd_cat(c)); MIXLORA_CUDA(launch_bgu_cat(c)); }
   return MIXLORA_OK;
 }
 
@@ -428,8 +431,7 @@ static mixlora_status_t fwd_experts(const Ctx& c, void* y, const void* residual 
   if (T == 0) return MIXLORA_OK;
   // per-slot LoRA-B expansion + SwiGLU
   {
-    StageScope ss(ST_LORA_B_SWIGLU, c.st, 5);
-    MIXLORA_CUDA(launch_bgu_cat(c));
+    StageScope ss(ST_LORA_B_SWIGLU, c.st, 3);
     MIXLORA_CUDA(launch_zpos(c));
     if (grouped_swiglu_supported(c)) {
       MIXLORA_CUDA(launch_zcompact(c));
@@ -452,7 +454,7 @@ static mixlora_status_t fwd_experts(const Ctx& c, void* y, const void* residual 
                                         c.at<int>(c.L.work_count) + 0));
     MIXLORA_CUDA(dense_product(c, T * k, &out, 1, block_sparse(c) ? &wl : nullptr));
   }
-  { StageScope ss(ST_COMBINE_H, c.st, c.bf16 ? 3 : 2); MIXLORA_CUDA(launch_combine_h(c)); MIXLORA_CUDA(launch_bd_cat(c)); }
+  { StageScope ss(ST_COMBINE_H, c.st, c.bf16 ? 2 : 1); MIXLORA_CUDA(launch_combine_h(c)); }
   // y = [hbar | Zs] [W_d | s B_d]^T : the frozen down projection acts once on the gate-weighted sum of a
   // token's slots (W_d is linear and shared), its LoRA rides along as extra reduction columns
   {
@@ -562,9 +564,8 @@ static mixlora_status_t bwd_shared_dgrad(const Ctx* cs, const void* const* dys, 
     TcOut outs[2];
     outs[0] = tc_out(c.ws + c.L.D, f, f);      tc_add(outs[0], dys[0], d, d, c.p.w_down, f, 1);
     outs[1] = tc_out(c.ws + c.L.spd, Nr, Nr);  tc_add(outs[1], dys[0], d, d, c.ws + c.L.bd_cat, Nr, 1);
-    StageScope ss(ST_GEMM_DGRAD_DOWN, c.st, 1 + dense_launches(c, T, outs, 2));
-    MIXLORA_CUDA(launch_bd_cat(c));
-    MIXLORA_CUDA(dense_product(c, T, outs, 2));
+    StageScope ss(ST_GEMM_DGRAD_DOWN, c.st, dense_launches(c, T, outs, 2));
+    MIXLORA_CUDA(dense_product(c, T, outs, 2));   // bd_cat is the forward pass's
     return MIXLORA_OK;
   }
   TcOut outs[2];
@@ -589,8 +590,7 @@ static mixlora_status_t bwd_shared_dgrad(const Ctx* cs, const void* const* dys, 
     if (T == 0) continue;
     TcOut z = tc_out(c.ws + c.L.spd, Nr, Nr);
     tc_add(z, dys[i], d, d, c.ws + c.L.bd_cat, Nr, 1);
-    StageScope ss(ST_GEMM_DGRAD_DOWN, c.st, 1 + dense_launches(c, T, &z, 1));
-    MIXLORA_CUDA(launch_bd_cat(c));
+    StageScope ss(ST_GEMM_DGRAD_DOWN, c.st, dense_launches(c, T, &z, 1));
     MIXLORA_CUDA(dense_product(c, T, &z, 1));
   }
   return MIXLORA_OK;
