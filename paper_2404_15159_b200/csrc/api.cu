@@ -162,7 +162,10 @@ SidePool* side_pool() {
 // is being taken, which needs one stream), else in turn on the caller's stream.  With join = false the caller's
 // stream is not made to wait yet: join_adapters() does that later, so that work enqueued on the caller's stream in
 // between runs beside the adapters' steps.
-struct Forked { SidePool* pool = nullptr; int used = 0; };
+// The pool's streams and events are shared by every caller on the device: `busy` is held from the fork to the join so
+// that two host threads cannot interleave their records and waits on the same events.
+std::mutex g_side_busy;
+struct Forked { SidePool* pool = nullptr; int used = 0; std::unique_lock<std::mutex> busy; };
 
 mixlora_status_t join_adapters(cudaStream_t main_st, Forked& fk) {
   mixlora_status_t st = MIXLORA_OK;
@@ -171,6 +174,7 @@ mixlora_status_t join_adapters(cudaStream_t main_st, Forked& fk) {
         cudaStreamWaitEvent(main_st, fk.pool->join[j], 0) != cudaSuccess)
       st = MIXLORA_ERR_CUDA;
   fk.pool = nullptr;
+  if (fk.busy.owns_lock()) fk.busy.unlock();
   return st;
 }
 
@@ -183,8 +187,9 @@ mixlora_status_t for_each_adapter(const Ctx* cs, int n, bool spread, F fn, Forke
     return st;
   }
   cudaStream_t main_st = cs[0].st;
-  if (cudaEventRecord(pool->fork, main_st) != cudaSuccess) return MIXLORA_ERR_CUDA;
   Forked fk;
+  fk.busy = std::unique_lock<std::mutex>(g_side_busy);
+  if (cudaEventRecord(pool->fork, main_st) != cudaSuccess) return MIXLORA_ERR_CUDA;
   fk.pool = pool;
   fk.used = n < kSideStreams ? n : kSideStreams;
   for (int j = 0; j < fk.used; ++j)
@@ -195,7 +200,7 @@ mixlora_status_t for_each_adapter(const Ctx* cs, int n, bool spread, F fn, Forke
     st = fn(c, m);
   }
   if (later && st == MIXLORA_OK) {
-    *later = fk;
+    *later = std::move(fk);
     return st;
   }
   // rejoin at once (always after an error, so that no stream is left dangling)
