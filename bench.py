@@ -297,6 +297,12 @@ def run_cuda(args):
             if use_dist:
                 dist.all_reduce(flat)
 
+    if args.forward_only:
+        # the forward-only configuration: no backward pass, no gradient exchange
+        def step():                        # noqa: F811
+            B.mixlora_ffn_forward(shape, params, y, ws)
+            B.mixlora_aux_loss(shape, ws, AUX_COEF, loss)
+
     def barrier():
         if use_dist:
             dist.barrier()
@@ -373,9 +379,10 @@ def run_cuda(args):
                 upload(bi ^ 1)
             B.mixlora_ffn_forward(shape, pb[bi], yb[bi], ws)
             B.mixlora_aux_loss(shape, ws, AUX_COEF, loss)
-            B.mixlora_ffn_backward(shape, pb[bi], dyb[bi], AUX_COEF, ws, grads)
-            if use_dist:
-                dist.all_reduce(flat)
+            if not args.forward_only:
+                B.mixlora_ffn_backward(shape, pb[bi], dyb[bi], AUX_COEF, ws, grads)
+                if use_dist:
+                    dist.all_reduce(flat)
             ev_done[bi].record(main)
             with torch.cuda.stream(d2h):
                 d2h.wait_event(ev_done[bi])
@@ -406,7 +413,7 @@ def run_cuda(args):
 
     peaks = load_peaks()
     fl = stage_flops(w, want_dx)
-    gemm_names = [n for n in fl if fl[n] > 0]
+    gemm_names = [n for n in fl if fl[n] > 0 and stage_ms.get(n, 0.0) > 0]
     dom = max(gemm_names, key=lambda n: stage_ms.get(n, 0.0))
     gemm_ms = sum(stage_ms.get(n, 0.0) for n in gemm_names)
     gemm_fl = sum(fl[n] for n in gemm_names)
@@ -441,7 +448,7 @@ def run_cuda(args):
                         "gemm_down": (T_ * f_ + f_ * d_ + T_ * d_) * E,
                         "gemm_dgrad_down": (T_ * d_ + f_ * d_ + T_ * f_) * E,
                         "gemm_dx": (2 * T_ * f_ + 2 * f_ * d_ + T_ * d_) * E}
-    if w.name == synth.c3().name and want_dx and M == 1 and not args.layer and bf16:
+    if w.name == synth.c3().name and want_dx and M == 1 and not args.layer and bf16 and not args.forward_only:
         roofline["traffic"] = measured_dram[dom]
         roofline["traffic_note"] = ("dram__bytes_read.sum + dram__bytes_write.sum of the %s launch at this size; its "
                                     "operands and result are %.1f MB" % (dom, algorithmic_dram[dom] / 1e6))
@@ -457,7 +464,8 @@ def run_cuda(args):
                                   f"workload at full d_model/d_ff, {sec:.1f} s"}
 
     line = {
-        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+        "metric": METRIC if not args.forward_only else "mixlora_ffn_fwd_tokens_per_s", "value": value, "unit": UNIT,
+        "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "bf16" if bf16 else "f32", "data": "synthetic",
         "config": {"workload": w.name, "tokens_per_gpu": w.tokens, "d_model": w.d_model, "d_ff": w.d_ff,
@@ -485,6 +493,9 @@ def main():
     ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
     ap.add_argument("--workload", default="c3")
     ap.add_argument("--no-dx", action="store_true")
+    ap.add_argument("--forward-only", action="store_true",
+                    help="time the forward pass and the aux loss only (the forward-only configuration); the metric is "
+                         "then named mixlora_ffn_fwd_tokens_per_s")
     ap.add_argument("--force-dist", action="store_true",
                     help="with one rank, still go through the NCCL gradient all-reduce path (plumbing check)")
     ap.add_argument("--layer", action="store_true",
