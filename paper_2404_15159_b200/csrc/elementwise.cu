@@ -125,10 +125,13 @@ combine_h_kernel(const T* __restrict__ h_sorted, const T* __restrict__ zd, const
   }
 }
 
-// bf16 version of the f-wide part of combine_h, 8 values per thread per step
+// bf16 version of the f-wide part of combine_h, 8 values per thread per step.  K = top-k when it is at most 4
+// (all of a chunk's loads are then issued before the first use), else 0 = any k.
+template <int K>
 __global__ void __launch_bounds__(ENT)
 combine_h_vec_kernel(const bf16* __restrict__ h_sorted, const float* __restrict__ gates, const int* __restrict__ inv,
-                     bf16* __restrict__ hbar, int f, int k) {
+                     bf16* __restrict__ hbar, int f, int k_any) {
+  const int k = K > 0 ? K : k_any;
   const int t = blockIdx.x;
   __shared__ int pos[MIXLORA_MAX_TOP_K];
   __shared__ float g[MIXLORA_MAX_TOP_K];
@@ -139,14 +142,30 @@ combine_h_vec_kernel(const bf16* __restrict__ h_sorted, const float* __restrict_
   __syncthreads();
   for (int c = threadIdx.x * 8; c < f; c += ENT * 8) {
     float acc[8] = {0, 0, 0, 0, 0, 0, 0, 0};
-    for (int j = 0; j < k; ++j) {
-      const uint4 raw = __ldg(reinterpret_cast<const uint4*>(h_sorted + (size_t)pos[j] * f + c));
-      const __nv_bfloat162* pr = reinterpret_cast<const __nv_bfloat162*>(&raw);
+    if (K > 0) {
+      uint4 raw[K > 0 ? K : 1];
 #pragma unroll
-      for (int i = 0; i < 4; ++i) {
-        const float2 v = __bfloat1622float2(pr[i]);
-        acc[2 * i] = fmaf(g[j], v.x, acc[2 * i]);
-        acc[2 * i + 1] = fmaf(g[j], v.y, acc[2 * i + 1]);
+      for (int j = 0; j < K; ++j) raw[j] = __ldg(reinterpret_cast<const uint4*>(h_sorted + (size_t)pos[j] * f + c));
+#pragma unroll
+      for (int j = 0; j < K; ++j) {                    // slot order, as in the generic loop: the same bits
+        const __nv_bfloat162* pr = reinterpret_cast<const __nv_bfloat162*>(&raw[j]);
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          const float2 v = __bfloat1622float2(pr[i]);
+          acc[2 * i] = fmaf(g[j], v.x, acc[2 * i]);
+          acc[2 * i + 1] = fmaf(g[j], v.y, acc[2 * i + 1]);
+        }
+      }
+    } else {
+      for (int j = 0; j < k; ++j) {
+        const uint4 raw = __ldg(reinterpret_cast<const uint4*>(h_sorted + (size_t)pos[j] * f + c));
+        const __nv_bfloat162* pr = reinterpret_cast<const __nv_bfloat162*>(&raw);
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          const float2 v = __bfloat1622float2(pr[i]);
+          acc[2 * i] = fmaf(g[j], v.x, acc[2 * i]);
+          acc[2 * i + 1] = fmaf(g[j], v.y, acc[2 * i + 1]);
+        }
       }
     }
     uint4 o;
@@ -728,8 +747,17 @@ cudaError_t launch_bd_cat(const Ctx& c) { return c.bf16 ? bd_cat_t<bf16>(c) : bd
 cudaError_t launch_lora_b_swiglu(const Ctx& c) { return c.bf16 ? lora_b_swiglu_t<bf16>(c) : lora_b_swiglu_t<float>(c); }
 cudaError_t launch_combine_h(const Ctx& c) {
   if (!c.bf16) return combine_h_t<float>(c);
-  combine_h_vec_kernel<<<c.s.tokens, ENT, 0, c.st>>>(c.at<bf16>(c.L.h_sorted), c.at<float>(c.L.gates), c.at<int>(c.L.inv),
-                                                    c.at<bf16>(c.L.hbar), c.s.d_ff, c.s.top_k);
+#define MIXLORA_COMBINE_H(KK)                                                                                      \
+  combine_h_vec_kernel<KK><<<c.s.tokens, ENT, 0, c.st>>>(c.at<bf16>(c.L.h_sorted), c.at<float>(c.L.gates),          \
+                                                        c.at<int>(c.L.inv), c.at<bf16>(c.L.hbar), c.s.d_ff, c.s.top_k)
+  switch (c.s.top_k) {
+    case 1: MIXLORA_COMBINE_H(1); break;
+    case 2: MIXLORA_COMBINE_H(2); break;
+    case 3: MIXLORA_COMBINE_H(3); break;
+    case 4: MIXLORA_COMBINE_H(4); break;
+    default: MIXLORA_COMBINE_H(0); break;
+  }
+#undef MIXLORA_COMBINE_H
   return combine_h_t<bf16>(c);
 }
 cudaError_t launch_swiglu_bwd(const Ctx& c) { return c.bf16 ? swiglu_bwd_t<bf16>(c) : swiglu_bwd_t<float>(c); }
