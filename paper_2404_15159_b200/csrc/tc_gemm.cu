@@ -340,10 +340,10 @@ __global__ void __launch_bounds__(kThreads, 1) tc_gemm_kernel(const __grid_const
 // ---- CTA-pair variant ------------------------------------------------------------------------
 // Two CTAs of a cluster work on one 256 x tile_n output tile with cta_group::2 MMAs: each CTA stages its own 128 rows
 // of A and HALF of the B tile, so the operand bytes per CTA and k-block drop from 48 KB to 32 KB and the same shared
-// memory holds a 6-stage ring.  Protocol (no TMA multicast anywhere):
+// memory holds a 6-stage ring.  Protocol (every CTA issues its own loads):
 //   - both CTAs allocate TMEM (cta_group::2) and run a producer warp; every load signals the LEADER's full barrier,
 //     on which the leader's producer has posted the byte count of both CTAs;
-//   - the leader's MMA thread issues the MMAs for the pair and multicast-commits onto both CTAs' empty barriers
+//   - the leader's MMA thread issues the MMAs for the pair and commits onto both CTAs' empty barriers at once
 //     (stage free) and accumulator-full barriers;
 //   - each CTA's epilogue warps drain that CTA's 128 accumulator rows and arrive on the leader's accumulator-empty
 //     barrier through its cluster address;

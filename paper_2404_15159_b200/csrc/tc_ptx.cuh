@@ -186,7 +186,7 @@ __device__ __forceinline__ void cluster_sync_all() {
 __device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
   asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
 }
-// TMA tile load into this CTA's smem that signals a barrier living in the pair's leader CTA (no multicast)
+// TMA tile load into this CTA's smem that signals a barrier living in the pair's leader CTA (each CTA issues its own loads)
 __device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap* map, uint32_t bar_cluster_addr, int c0,
                                                  int c1) {
   asm volatile(
