@@ -131,6 +131,8 @@ __global__ void __launch_bounds__(kThreads, 1) grouped_swiglu_kernel(const __gri
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * kMaxStages + 6 + 2 * kMaxSets);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
   int* out_hdr = reinterpret_cast<int*>(tmem_slot + 4);   // [2][4]: first slot, rows, column tile of the item in each output tile's turn
+  // [2], by item parity: a warp that runs ahead and gives up on the next item cannot change what the others read
+  // after this item's barrier
   volatile int* epi_stop = reinterpret_cast<volatile int*>(tmem_slot + 2);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -153,7 +155,8 @@ __global__ void __launch_bounds__(kThreads, 1) grouped_swiglu_kernel(const __gri
     // is written (one plain arrival each); it is empty again when every epilogue warp has read it
     for (int b = 0; b < kMaxSets; ++b) { mbar_init(gfull_bar(b), 2 * NGT); mbar_init(gempty_bar(b), 4 * kSplit); }
     *abort_flag = 0;
-    *epi_stop = 0;
+    epi_stop[0] = 0;
+    epi_stop[1] = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 1) {
@@ -260,7 +263,7 @@ __global__ void __launch_bounds__(kThreads, 1) grouped_swiglu_kernel(const __gri
     uint32_t n = 0;
     for (int w = blockIdx.x; w < total; w += gridDim.x, ++n) {
       named_barrier(1, NET + 32);                      // the item's results are complete in its output tile
-      if (*epi_stop) break;
+      if (epi_stop[n & 1u]) break;
       if (lane == 0) {
         // every epilogue thread is past the previous item (also past copying a short tile out), and that item's
         // TMA stores have read its tile (waited for below): the tile may be written again
@@ -461,10 +464,13 @@ __global__ void __launch_bounds__(kThreads, 1) grouped_swiglu_kernel(const __gri
         if (p.status) atomicExch(p.status, (int)MIXLORA_ERR_DEVICE_TIMEOUT);
       }
       fence_proxy_async_smem();                        // the tile written above is read by the TMA unit
-      if (!got) *epi_stop = 1;
+      if (!got) epi_stop[wcount & 1u] = 1;
       // the one CTA-wide barrier of an item (with the store warp): the results are complete in the output tile
       named_barrier(1, NET + 32);
-      if (got && rows < BM) {
+      // every thread sees the same value after the barrier: all of them (and the store warp) leave together, before
+      // the second barrier below, if any warp gave up on this item
+      if (epi_stop[wcount & 1u]) break;
+      if (rows < BM) {
         // a segment's last, shorter tile: the rows behind it belong to the next expert, so the valid rows are
         // copied out of the smem tile one 16-byte chunk per thread and turn
         const uint8_t* otile = out_smem + oidx * kOutBytes;
@@ -479,14 +485,13 @@ __global__ void __launch_bounds__(kThreads, 1) grouped_swiglu_kernel(const __gri
           }
         }
       }
-      if (p.out_sets == 1 && got && rows < BM) named_barrier(2, NET + 32);
-      if (BWD && got && part == 0 && row < rows) {     // the row's partial <Dt, h> over this column tile, fixed order
+      if (p.out_sets == 1 && rows < BM) named_barrier(2, NET + 32);
+      if (BWD && part == 0 && row < rows) {     // the row's partial <Dt, h> over this column tile, fixed order
         float sdg = 0.f;
 #pragma unroll
         for (int pp = 0; pp < kSplit; ++pp) sdg += dg_smem[(wcount & 1u) * (kSplit * BM) + pp * BM + row];
         p.dgate_part[(size_t)ct * p.slots + pos] = sdg;
       }
-      if (*epi_stop) break;                            // same value for every thread after the barrier
       if (++set == p.nsets) { set = 0; ++set_use; }
     }
   }
