@@ -616,8 +616,10 @@ static mixlora_status_t bwd_zero_tokens(const Ctx& c, const mixlora_grads_t* gra
 
 // `param_grads_ready` (optional cudaEvent_t) is recorded once every LoRA / router gradient has been enqueued, before
 // the input-gradient product: a caller's gradient all-reduce can then overlap that product.
+// `may_fork`: the gate-gradient reduction and the router's backward step may go to a side stream beside the dense
+// products that do not need them (not when this call already runs on a side stream).
 static mixlora_status_t bwd_experts(const Ctx& c, const void* dy, float aux_coef, const mixlora_grads_t* grads,
-                                    void* param_grads_ready = nullptr) {
+                                    void* param_grads_ready = nullptr, bool may_fork = true) {
   const mixlora_params_t* params = &c.p;
   const int T = c.s.tokens, d = c.s.d_model, f = c.s.d_ff, N = c.s.n_experts, r = c.s.rank, k = c.s.top_k;
   const int Nr = N * r, NP = round_up8(N);
@@ -629,19 +631,46 @@ static mixlora_status_t bwd_experts(const Ctx& c, const void* dy, float aux_coef
       MIXLORA_CUDA(cudaEventRecord(reinterpret_cast<cudaEvent_t>(param_grads_ready), c.st));
     return zs;
   }
+  int dgate_tiles = 0;                                 // > 0: the per-column-tile partial sums still have to be added
   {
-    StageScope ss(ST_SWIGLU_BWD, c.st, 3);
+    StageScope ss(ST_SWIGLU_BWD, c.st, 2);
     MIXLORA_CUDA(launch_slot_prep_bwd(c));
     if (grouped_swiglu_supported(c)) {
       MIXLORA_CUDA(launch_grouped_swiglu_bwd(c));
-      MIXLORA_CUDA(launch_dgate_reduce(c, grouped_swiglu_bwd_col_tiles(f)));
+      dgate_tiles = grouped_swiglu_bwd_col_tiles(f);
     } else if (fused_swiglu_supported(c)) {
       MIXLORA_CUDA(launch_fused_swiglu_bwd(c));
-      MIXLORA_CUDA(launch_dgate_reduce(c, fused_swiglu_bwd_col_tiles(f)));
+      dgate_tiles = fused_swiglu_bwd_col_tiles(f);
     } else {
       MIXLORA_CUDA(launch_swiglu_bwd(c));
     }
   }
+  // router: gate gradients -> probabilities -> logits.  Nothing before the d-sized weight gradients needs the
+  // result, so these small launches run beside the dense products below.
+  Forked router_fk;
+  {
+    mixlora_status_t st = for_each_adapter(
+        &c, 1, may_fork,
+        [&](const Ctx& cc, int) {
+          if (dgate_tiles > 0) {
+            StageScope ss(ST_SWIGLU_BWD, cc.st, 1);
+            MIXLORA_CUDA(launch_dgate_reduce(cc, dgate_tiles));
+          }
+          StageScope ss(ST_ROUTER_BWD, cc.st, 1 + (grads->d_router_bias ? 1 : 0) + (want_dx ? 1 : 0));
+          MIXLORA_CUDA(launch_router_bwd(cc, aux_coef, grads->d_router_bias, acc, want_dx));
+          return MIXLORA_OK;
+        },
+        &router_fk);
+    if (st != MIXLORA_OK) return st;
+  }
+  // from here to the join every early return has to hand the side stream back
+#define MIXLORA_CUDA_FK(expr)                                   \
+  do {                                                          \
+    if ((expr) != cudaSuccess) {                                \
+      join_adapters(c.st, router_fk);                           \
+      return MIXLORA_ERR_CUDA;                                  \
+    }                                                           \
+  } while (0)
   // dzg = da (s B_g), dzu = db (s B_u), against every expert (the slot's own block is used)
   {
     TcOut outs[2];
@@ -650,16 +679,11 @@ static mixlora_status_t bwd_experts(const Ctx& c, const void* dy, float aux_coef
     StageScope ss(ST_LORA_DZ, c.st, (block_sparse(c) ? 1 : 0) + dense_launches(c, T * k, outs, 2));
     TcWork wl = {c.at<int>(c.L.work_rows2), c.at<int>(c.L.work_count) + 1, rows_worklist_max(T * k, N, 2), r};
     if (block_sparse(c))
-      MIXLORA_CUDA(launch_rows_worklist(c, tc_gemm_tile_rows(T * k), 2, (f + 63) / 64, c.at<int>(c.L.work_rows2),
-                                        c.at<int>(c.L.work_count) + 1));
-    MIXLORA_CUDA(dense_product(c, T * k, outs, 2, block_sparse(c) ? &wl : nullptr));
+      MIXLORA_CUDA_FK(launch_rows_worklist(c, tc_gemm_tile_rows(T * k), 2, (f + 63) / 64, c.at<int>(c.L.work_rows2),
+                                           c.at<int>(c.L.work_count) + 1));
+    MIXLORA_CUDA_FK(dense_product(c, T * k, outs, 2, block_sparse(c) ? &wl : nullptr));
   }
-  // router: gates -> probabilities -> logits
-  {
-    StageScope ss(ST_ROUTER_BWD, c.st, 1 + (grads->d_router_bias ? 1 : 0) + (want_dx ? 1 : 0));
-    MIXLORA_CUDA(launch_router_bwd(c, aux_coef, grads->d_router_bias, acc, want_dx));
-  }
-  { StageScope ss(ST_COMBINE_BWD, c.st, (c.bf16 && want_dx) ? 2 : 1); MIXLORA_CUDA(launch_combine_bwd(c, want_dx)); }
+  { StageScope ss(ST_COMBINE_BWD, c.st, (c.bf16 && want_dx) ? 2 : 1); MIXLORA_CUDA_FK(launch_combine_bwd(c, want_dx)); }
   // LoRA and router weight gradients.  Reduction over the sorted slots (f-sized matrices) ...
   {
     TcOut outs[3];
@@ -681,11 +705,13 @@ static mixlora_status_t bwd_experts(const Ctx& c, const void* dy, float aux_coef
       // each expert's block is a sum over that expert's segment of sorted slots only
       TcWork wl = {c.at<int>(c.L.work_red), c.at<int>(c.L.work_count) + 2, reduce_worklist_max(f, N, n), r};
       if (block_sparse(c))
-        MIXLORA_CUDA(launch_reduce_worklist(c, f, tc_gemm_tile_rows(f), n, c.at<int>(c.L.work_red),
-                                            c.at<int>(c.L.work_count) + 2));
-      MIXLORA_CUDA(dense_product(c, f, outs, n, block_sparse(c) ? &wl : nullptr));
+        MIXLORA_CUDA_FK(launch_reduce_worklist(c, f, tc_gemm_tile_rows(f), n, c.at<int>(c.L.work_red),
+                                               c.at<int>(c.L.work_count) + 2));
+      MIXLORA_CUDA_FK(dense_product(c, f, outs, n, block_sparse(c) ? &wl : nullptr));
     }
   }
+#undef MIXLORA_CUDA_FK
+  if (join_adapters(c.st, router_fk) != MIXLORA_OK) return MIXLORA_ERR_CUDA;   // dl and the router terms are needed now
   // ... and over the tokens (d-sized matrices and the router weight)
   {
     TcOut outs[4];
@@ -764,7 +790,9 @@ mixlora_status_t mixlora_multi_ffn_backward(int32_t n_models, const mixlora_shap
   for (int m = 0; m < n_models; m += 2)
     if ((st = bwd_shared_dgrad(&cs[m], &dy[m], n_models - m >= 2 ? 2 : 1)) != MIXLORA_OK) return st;
   return for_each_adapter(cs, n_models, n_models > 1,
-                          [&](const Ctx& c, int m) { return bwd_experts(c, dy[m], aux_coef[m], &grads[m]); });
+                          [&](const Ctx& c, int m) {
+                            return bwd_experts(c, dy[m], aux_coef[m], &grads[m], nullptr, n_models == 1);
+                          });
 }
 
 
