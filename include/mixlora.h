@@ -126,7 +126,9 @@ mixlora_status_t mixlora_aux_loss(const mixlora_shape_t *shape /* host */, const
 /* Backward pass of L = <dy, y> + aux_coef * N * sum_i F_i P_i with respect to the LoRA
  * matrices, the router and, if grads->d_x is not NULL, x (chain rule on Algorithm 1; the
  * paper prints no backward).  Needs the workspace exactly as the forward call for the same
- * shape and params left it (size for_backward = 1).  `dy` is [T, d] in shape.dtype. */
+ * shape and params left it (size for_backward = 1).  `dy` is [T, d] in shape.dtype.  As in the forward call, a few
+ * small launches (the gate-gradient sums, the router's backward step) go to a library-owned stream that forks from
+ * and joins `stream` inside the call. */
 mixlora_status_t mixlora_ffn_backward(const mixlora_shape_t *shape /* host */,
                                       const mixlora_params_t *params /* host struct of device ptrs */,
                                       const void *dy, float aux_coef, void *workspace, size_t workspace_bytes,
