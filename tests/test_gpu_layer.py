@@ -164,3 +164,35 @@ def test_layer_rejects_aliased_buffers_and_wide_models():
     with pytest.raises(B.MixLoraError) as e:
         B.mixlora_layer_forward(wide, params, wn, EPS, h, inv, torch.zeros_like(h), ws)
     assert e.value.status == 2          # MIXLORA_ERR_UNSUPPORTED: wider than the norm kernels take
+
+
+def test_layer_with_no_tokens_returns_zero_gradients():
+    import torch
+    from paper_2404_15159_b200 import binding as B
+
+    w = synth.Workload("layer-empty", tokens=0, d_model=256, d_ff=512, n_experts=4, top_k=2, rank=8, lora_alpha=16.0,
+                       dtype="bf16", seed=synth.BASE_SEED + 602, std_frozen=0.03, std_a=0.06, std_b=0.03)
+    t = synth.generate(w.with_(tokens=8))
+    act = torch.bfloat16
+    dev = {n: (torch.from_numpy(np.ascontiguousarray(v)).cuda().to(act) if n in helpers.ACT_NAMES
+               else torch.from_numpy(np.ascontiguousarray(v, np.float32)).cuda())
+           for n, v in t.items() if v is not None}
+    dev["router_bias"] = None
+    shape = B.make_shape(0, w.d_model, w.d_ff, w.n_experts, w.top_k, w.rank, w.lora_alpha)
+    params = B.make_params(**{n: dev[n] for n in synth.PARAM_NAMES}, x=dev["x"])
+    ws = B.alloc_workspace(shape, True)
+    wn = torch.ones(w.d_model, dtype=act, device="cuda")
+    xn = torch.zeros(8, w.d_model, dtype=act, device="cuda")
+    inv = torch.zeros(8, dtype=torch.float32, device="cuda")
+    h = torch.zeros(8, w.d_model, dtype=act, device="cuda")
+    g = {}
+    for n in helpers.GRAD_NAMES:
+        shp = (w.n_experts,) if n == "d_router_bias" else tuple(np.shape(t[n[2:]]))
+        g[n] = torch.full(shp, float("nan"), dtype=torch.float32, device="cuda")
+    g["d_x"] = torch.zeros(8, w.d_model, dtype=act, device="cuda")
+    B.mixlora_layer_forward(shape, params, wn, EPS, xn, inv, h, ws)
+    B.mixlora_layer_backward(shape, params, wn, EPS, xn, inv, dev["dy"], 0.01, ws, B.make_grads(accumulate=0, **g))
+    torch.cuda.synchronize()
+    assert B.mixlora_device_status(ws) == 0
+    for n in helpers.GRAD_NAMES:
+        assert not g[n].cpu().numpy().any(), n
