@@ -504,7 +504,7 @@ def main():
                     help="split the batch over this many adapters sharing the frozen FFN (multi-model calls); the "
                          "end-to-end leg still runs the single-model calls")
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--cpu-sample", type=int, default=512, help="tokens of the oracle's timed sample")
+    ap.add_argument("--cpu-sample", type=int, default=4096, help="tokens of the oracle's timed sample")
     ap.add_argument("--ref-sample", type=int, default=256, help="tokens per step of --impl reference")
     args = ap.parse_args()
     if args.impl == "reference":
