@@ -196,3 +196,27 @@ def test_layer_with_no_tokens_returns_zero_gradients():
     assert B.mixlora_device_status(ws) == 0
     for n in helpers.GRAD_NAMES:
         assert not g[n].cpu().numpy().any(), n
+
+
+def test_layer_full_size_sampled_tokens():
+    # the 7B-shaped training configuration through the layer calls: forward output on sampled tokens that the oracle
+    # evaluates one by one (with the GPU's routing), and the norm's saved statistics for every token
+    w = synth.c3()
+    t = synth.generate(w)
+    t["x"] = synth.round_to_bf16(t["x"] * 1.5)
+    wn = norm_weight(w)
+    gpu = gpu_layer(w, t, wn)
+    assert gpu["status"] == 0
+    xn64, inv64 = orc.rmsnorm(t["x"], wn, EPS)
+    assert helpers.rel_err(gpu["inv_rms"], inv64) < 1e-5
+    assert helpers.rel_err(gpu["xn"], xn64) < 2e-2
+    params = synth.params_of(t)
+    xn_r = synth.round_to_bf16(xn64)
+    rng = np.random.default_rng(1)
+    toks = np.unique(np.concatenate([rng.integers(0, w.tokens, 16), [0, w.tokens - 1]]))
+    ref = np.stack([t["x"][i] + orc.token_forward(xn_r[i], params, w.top_k, w.lora_alpha,
+                                                  forced_experts=gpu["expert_idx"][i])[0] for i in toks])
+    err = np.abs(gpu["h"][toks] - ref).max() / np.abs(ref).max()
+    assert err < 2e-2, f"sampled h error {err:.3e}"
+    # the gradient with respect to the residual stream contains dh itself
+    assert np.isfinite(gpu["d_x"]).all()
