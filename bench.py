@@ -154,6 +154,13 @@ def run_reference(args):
         return
     w = workload_by_name(args.workload)
     sample = args.ref_sample
+    if sample <= 0:
+        # size the per-step sample so that the whole run (warm-up + timed steps) takes about two minutes: one
+        # calibration pass over 64 tokens gives the oracle's time per token on this host
+        probe = synth.generate(w.with_(tokens=64))
+        per_token = oracle_sample(w, probe, 64, True) / 64
+        sample = int(120.0 / ((args.warmup + args.steps) * per_token))
+        sample = max(16, min(256, sample))
     tensors = synth.generate(w.with_(tokens=sample))
     times = []
     for i in range(args.warmup + args.steps):
@@ -505,7 +512,8 @@ def main():
                          "end-to-end leg still runs the single-model calls")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--cpu-sample", type=int, default=4096, help="tokens of the oracle's timed sample")
-    ap.add_argument("--ref-sample", type=int, default=256, help="tokens per step of --impl reference")
+    ap.add_argument("--ref-sample", type=int, default=0,
+                    help="tokens per step of --impl reference (0 = sized so that the run takes about two minutes)")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
