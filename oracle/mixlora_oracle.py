@@ -24,9 +24,14 @@ Readings of the paper where it is silent or inconsistent:
     Norm(Top2(Softmax(.))); Eq. 7 omits the Norm);
   * selection is on the logits (monotone in the softmax), ties go to the lower
     expert index;
-  * F_i of Eq. 9 counts the arg-max expert only; P_i is the mean of the full
-    softmax probability.  PARITY UNPINNED for the choice of P_i (full softmax
-    versus re-normalised gate): no identity in the paper tells them apart.
+  * F_i of Eq. 9 counts the arg-max expert only (f_mode 1: every selection, the
+    reading of the sentence under Eq. 9; both are pinned by a hand-worked
+    example in which they differ); P_i is the mean of the full softmax
+    probability.  PARITY UNPINNED for the choice of P_i (full softmax versus
+    re-normalised gate): no identity in the paper tells them apart.
+  * F_i and P_i are fractions of the whole batch: when the batch is split over
+    data-parallel shards, the shards' sums are added before Eq. 8 is evaluated
+    (`aux_sums`, `aux_loss_from_sums`, `aux_batch=` of the backward pass).
   * the LoRA scale is s = alpha / r (Table 3 lists alpha; Eq. 1 has no scale).
 """
 from __future__ import annotations
@@ -150,6 +155,30 @@ def aux_loss(probs, expert_idx, coef, f_mode=0):
     return loss, F, P
 
 
+def aux_sums(probs, expert_idx, f_mode=0):
+    """The two sums over tokens that Eq. 9 is built from, un-normalised, for one batch or one shard of it:
+    count[i] = tokens whose arg-max expert is i (f_mode 1: selections that went to i), prob_sum[i] = sum over
+    tokens of the softmax probability of expert i.  Sums of shards add up to the sums of the whole batch."""
+    T, N = probs.shape
+    count = np.zeros(N, F64)
+    if f_mode == 0:
+        for t in range(T):
+            count[expert_idx[t, 0]] += 1.0
+    else:
+        for e in expert_idx.reshape(-1):
+            count[e] += 1.0
+    return count, probs.sum(axis=0)
+
+
+def aux_loss_from_sums(count, prob_sum, total_tokens, top_k, coef, f_mode=0):
+    """Eq. 8-9 from the sums of `aux_sums` taken over ALL `total_tokens` tokens of the batch (F_i and P_i are
+    fractions of the whole batch, so under data parallelism the shard sums are added first)."""
+    N = len(count)
+    F = np.asarray(count, F64) / (total_tokens * (top_k if f_mode == 1 else 1))
+    P = np.asarray(prob_sum, F64) / total_tokens
+    return coef * N * float(np.dot(F, P)), F, P
+
+
 # --------------------------------------------------------------------------- #
 # forward, optimised form (Algorithm 1: shared W1/W3 results, per-expert slices)
 # --------------------------------------------------------------------------- #
@@ -234,9 +263,12 @@ def ffn_forward_vanilla(x, params, top_k, lora_alpha, renormalize=True):
 # --------------------------------------------------------------------------- #
 # backward (chain rule on the forward above; the paper prints none)
 # --------------------------------------------------------------------------- #
-def ffn_backward(x, params, dy, saved, aux_coef=0.0, aux_f_mode=0, want_dx=True):
+def ffn_backward(x, params, dy, saved, aux_coef=0.0, aux_f_mode=0, want_dx=True, aux_batch=None):
     """Gradients of L = sum(dy * y) + L_aux with respect to the LoRA matrices,
     the router and (optionally) x.  The frozen weights get no gradient.
+
+    `aux_batch` = (F [N], total_tokens): when x is one shard of a larger batch, L_aux of Eq. 8 is the loss of
+    the whole batch, so its gradient uses the batch's F_i and token count instead of the shard's.
 
     Returns a dict: d_a_gate, d_b_gate, d_a_up, d_b_up, d_a_down, d_b_down,
     d_w_router, d_router_bias, d_x (or None), d_gates [T,k], d_logits [T,N].
@@ -291,8 +323,12 @@ def ffn_backward(x, params, dy, saved, aux_coef=0.0, aux_f_mode=0, want_dx=True)
     else:
         np.put_along_axis(dp, idx, dgate, axis=1)
     if aux_coef != 0.0:
-        _, F, _ = aux_loss(probs, route["expert_idx"], aux_coef, aux_f_mode)
-        dp += (aux_coef * N / T) * F[None, :]                 # F_i is piecewise constant
+        if aux_batch is None:
+            _, F, _ = aux_loss(probs, route["expert_idx"], aux_coef, aux_f_mode)
+            T_all = T
+        else:
+            F, T_all = np.asarray(aux_batch[0], F64), aux_batch[1]
+        dp += (aux_coef * N / T_all) * F[None, :]             # F_i is piecewise constant; P_i = sum_t p_ti / T_all
     dl = probs * (dp - np.sum(probs * dp, axis=1, keepdims=True))
     g_wr = dl.T @ x
     g_br = dl.sum(axis=0)
@@ -357,13 +393,14 @@ def layer_forward(z, params, w_norm, eps, top_k, lora_alpha, renormalize=True, f
     return np.asarray(z, F64) + y, saved
 
 
-def layer_backward(z, params, w_norm, dh, saved, aux_coef=0.0, aux_f_mode=0):
+def layer_backward(z, params, w_norm, dh, saved, aux_coef=0.0, aux_f_mode=0, aux_batch=None):
     """Chain rule through Eq. 6.  `dh` = dL/dh.  The LoRA and router gradients are those of `ffn_backward` at the
     normalised input; `d_x` becomes dL/dz = dh (residual path) + the normalisation's Jacobian applied to dL/dxn:
     with `xh = z * inv_rms`, `u = dL/dxn * w_norm`:  `inv_rms * (u - xh * mean(u * xh))`."""
     z = np.asarray(z, F64)
     dh = np.asarray(dh, F64)
-    g = ffn_backward(saved["xn"], params, dh, saved, aux_coef=aux_coef, aux_f_mode=aux_f_mode, want_dx=True)
+    g = ffn_backward(saved["xn"], params, dh, saved, aux_coef=aux_coef, aux_f_mode=aux_f_mode, want_dx=True,
+                     aux_batch=aux_batch)
     inv_rms = saved["inv_rms"]
     xh = z * inv_rms[:, None]
     u = g["d_x"] * np.asarray(w_norm, F64)[None, :]

@@ -134,6 +134,47 @@ def test_aux_loss_worked_example():
     assert loss == pytest.approx(g["loss"], rel=1e-14)
 
 
+def test_aux_loss_worked_example_where_the_two_counting_modes_differ():
+    # Eq. 9 counts the arg-max expert; the sentence under it speaks of the tokens dispatched to expert i, which
+    # with top-2 is every selection.  Worked by hand for N = 3, T = 4: the two readings give different F and loss.
+    with open(os.path.join(HERE, "golden", "aux_loss_n3_t4_k2.json")) as fh:
+        g = json.load(fh)
+    probs = np.array(g["probs"])
+    idx = np.array(g["expert_idx"], np.int32)
+    for mode in (0, 1):
+        loss, F, P = orc.aux_loss(probs, idx, g["coef"], f_mode=mode)
+        np.testing.assert_allclose(F, g[f"mode{mode}"]["F"], rtol=1e-15, atol=0)
+        np.testing.assert_allclose(P, g["P"], rtol=1e-15)
+        assert loss == pytest.approx(g[f"mode{mode}"]["loss"], rel=1e-14)
+        count, psum = orc.aux_sums(probs, idx, f_mode=mode)
+        assert list(count) == g[f"counts_mode{mode}"]
+        np.testing.assert_allclose(psum, g["prob_sums"], rtol=1e-15)
+    assert g["mode0"]["loss"] != g["mode1"]["loss"]
+
+
+@pytest.mark.parametrize("mode", [0, 1])
+def test_aux_sums_of_shards_add_up_to_the_loss_of_the_whole_batch(mode):
+    # Eq. 8-9 are fractions of the whole batch: the loss is NOT the mean of the shards' losses, but the shards'
+    # un-normalised sums add, and the loss from the added sums is the loss of the concatenated batch
+    x, p, _, kw = make_case(T=37, N=5, seed=3)
+    r = orc.router_forward(x, p["w_router"], None, 2)
+    full, F, P = orc.aux_loss(r["probs"], r["expert_idx"], 0.3, f_mode=mode)
+    cuts = [0, 9, 10, 30, 37]
+    count = np.zeros(5)
+    psum = np.zeros(5)
+    shard_losses = []
+    for a, b in zip(cuts[:-1], cuts[1:]):
+        c, s = orc.aux_sums(r["probs"][a:b], r["expert_idx"][a:b], f_mode=mode)
+        count += c
+        psum += s
+        shard_losses.append(orc.aux_loss(r["probs"][a:b], r["expert_idx"][a:b], 0.3, f_mode=mode)[0])
+    loss, F2, P2 = orc.aux_loss_from_sums(count, psum, 37, 2, 0.3, f_mode=mode)
+    assert loss == pytest.approx(full, rel=1e-13)
+    np.testing.assert_allclose(F2, F, rtol=1e-13)
+    np.testing.assert_allclose(P2, P, rtol=1e-13)
+    assert abs(np.mean(shard_losses) - full) > 1e-4          # the per-shard loss is a different quantity
+
+
 @pytest.mark.parametrize("N", [2, 4, 8, 16])
 def test_aux_loss_is_one_under_uniform_routing(N):
     # (i) F uniform through cyclic arg-max, P arbitrary-but-summing-to-one
@@ -250,13 +291,22 @@ def total_loss(x, p, dy, kw, coef, f_mode=0, renormalize=True):
     return float(np.sum(dy * y)) + la
 
 
-@pytest.mark.parametrize("k,N,renorm,coef", [(2, 3, True, 0.7), (3, 3, True, 0.0), (2, 4, False, 0.3), (1, 3, True, 0.5)])
-def test_identity_d_finite_differences(k, N, renorm, coef):
+@pytest.mark.parametrize("k,N,renorm,coef,f_mode", [(2, 3, True, 0.7, 0), (3, 3, True, 0.0, 0), (2, 4, False, 0.3, 0),
+                                                    (1, 3, True, 0.5, 0), (2, 4, True, 0.9, 1), (2, 3, False, 0.4, 1)])
+def test_identity_d_finite_differences(k, N, renorm, coef, f_mode):
     x, p, dy, kw = make_case(T=5, d=8, f=12, N=N, k=k, r=2, alpha=4.0, seed=11 + k, bias=True)
     # keep routing margins far above the step so the discrete choice is constant
     assert orc.router_forward(x, p["w_router"], p["router_bias"], k)["margin"].min() > 1e-3
     y, saved = orc.ffn_forward(x, p, renormalize=renorm, **kw)
-    g = orc.ffn_backward(x, p, dy, saved, aux_coef=coef)
+    g = orc.ffn_backward(x, p, dy, saved, aux_coef=coef, aux_f_mode=f_mode)
+    if f_mode == 1:
+        # the case must tell the two counting modes apart: P is not uniform, the two F differ, and so do the
+        # router gradients (a mode 1 that silently computed mode 0 would pass a comparison with itself)
+        _, F0, P = orc.aux_loss(saved["route"]["probs"], saved["route"]["expert_idx"], coef, 0)
+        _, F1, _ = orc.aux_loss(saved["route"]["probs"], saved["route"]["expert_idx"], coef, 1)
+        assert np.abs(P - 1.0 / N).max() > 0.02 and np.abs(F0 - F1).max() > 0.05
+        g0 = orc.ffn_backward(x, p, dy, saved, aux_coef=coef, aux_f_mode=0)
+        assert np.abs(g0["d_w_router"] - g["d_w_router"]).max() > 1e-4
     step = 1e-6
     rng = np.random.default_rng(5)
 
@@ -266,9 +316,9 @@ def test_identity_d_finite_differences(k, N, renorm, coef):
         for i in picks:
             old = flat[i]
             flat[i] = old + step
-            lp = total_loss(x, p, dy, kw, coef, renormalize=renorm)
+            lp = total_loss(x, p, dy, kw, coef, f_mode=f_mode, renormalize=renorm)
             flat[i] = old - step
-            lm = total_loss(x, p, dy, kw, coef, renormalize=renorm)
+            lm = total_loss(x, p, dy, kw, coef, f_mode=f_mode, renormalize=renorm)
             flat[i] = old
             fd = (lp - lm) / (2 * step)
             assert grad.reshape(-1)[i] == pytest.approx(fd, rel=2e-5, abs=2e-7), (name, i)
@@ -278,6 +328,41 @@ def test_identity_d_finite_differences(k, N, renorm, coef):
     check("w_router", p["w_router"], g["d_w_router"])
     check("router_bias", p["router_bias"], g["d_router_bias"])
     check("x", x, g["d_x"])
+
+
+@pytest.mark.parametrize("mode", [0, 1])
+def test_shard_gradients_with_the_batch_statistics_add_up_to_the_full_batch_gradient(mode):
+    # data parallel over tokens: every term of the backward pass is a sum over tokens once the aux term uses the
+    # whole batch's F_i and token count (Eq. 8-9), so the shards' gradients add up to the full-batch gradient
+    x, p, dy, kw = make_case(T=12, d=8, f=10, N=4, k=2, r=2, seed=21, bias=True)
+    coef = 0.8
+    _, saved = orc.ffn_forward(x, p, **kw)
+    full = orc.ffn_backward(x, p, dy, saved, aux_coef=coef, aux_f_mode=mode)
+    cuts = [0, 5, 12]
+    count = np.zeros(4)
+    psum = np.zeros(4)
+    shards = []
+    for a, b in zip(cuts[:-1], cuts[1:]):
+        _, sv = orc.ffn_forward(x[a:b], p, **kw)
+        c, s = orc.aux_sums(sv["route"]["probs"], sv["route"]["expert_idx"], f_mode=mode)
+        count += c
+        psum += s
+        shards.append((a, b, sv))
+    _, F, _ = orc.aux_loss_from_sums(count, psum, 12, 2, coef, f_mode=mode)
+    total = None
+    dx = np.zeros_like(x)
+    for a, b, sv in shards:
+        g = orc.ffn_backward(x[a:b], p, dy[a:b], sv, aux_coef=coef, aux_f_mode=mode, aux_batch=(F, 12))
+        dx[a:b] = g["d_x"]
+        part = {n: g[n] for n in g if n.startswith("d_") and n not in ("d_x", "d_gates", "d_logits")}
+        total = part if total is None else {n: total[n] + part[n] for n in part}
+    for n in total:
+        np.testing.assert_allclose(total[n], full[n], rtol=1e-11, atol=1e-13, err_msg=n)
+    np.testing.assert_allclose(dx, full["d_x"], rtol=1e-11, atol=1e-13)
+    # with the shards' own statistics instead, the router gradient is a different one
+    g_local = orc.ffn_backward(x[:5], p, dy[:5], shards[0][2], aux_coef=coef, aux_f_mode=mode)
+    g_batch = orc.ffn_backward(x[:5], p, dy[:5], shards[0][2], aux_coef=coef, aux_f_mode=mode, aux_batch=(F, 12))
+    assert np.abs(g_local["d_w_router"] - g_batch["d_w_router"]).max() > 1e-3
 
 
 def test_backward_without_dx_leaves_other_gradients_unchanged():
