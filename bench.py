@@ -26,6 +26,7 @@ import numpy as np
 
 from paper_2404_15159_b200 import synth
 
+DRAM_CAPTURE = "profiles/tc_gemm_pair_kernel_c3_dram.md"
 METRIC = "mixlora_ffn_fwd_bwd_tokens_per_s"
 UNIT = "tokens/s"
 AUX_COEF = 0.01
@@ -42,19 +43,37 @@ def workload_by_name(name: str) -> synth.Workload:
     raise SystemExit(f"unknown workload {name}")
 
 
+def config_of(w: synth.Workload, args, world: int, use_dist: bool) -> dict:
+    """The `config` object of the JSON line; both arms (the CUDA library and the CPU oracle) print the same keys."""
+    want_dx = not args.no_dx
+    M = max(1, args.models)
+    return {"workload": w.name, "tokens_per_gpu": w.tokens, "d_model": w.d_model, "d_ff": w.d_ff,
+            "n_experts": w.n_experts, "top_k": w.top_k, "rank": w.rank, "lora_alpha": w.lora_alpha,
+            "backward_dx": want_dx, "aux_coef": AUX_COEF, "adapters": M,
+            "layer_slice": bool(args.layer and M == 1 and want_dx),
+            "parallelism": f"dp{world} over tokens" + (", aux statistics (2N floats) and LoRA/router gradients "
+                                                        "all-reduced over NCCL, the latter beside the dx product"
+                                                        if use_dist else ""),
+            "l2": "inputs larger than L2 (weights 270 MB + activations > 126 MB), no flush; a flushed variant is "
+                  "reported in step_ms_l2_flushed"}
+
+
 # ----------------------------------------------------------------------------------------
-# flop / byte model of the stages (algorithmic, per step)
+# flop / byte model of the stages (per step)
 # ----------------------------------------------------------------------------------------
-def stage_flops(w: synth.Workload, want_dx: bool) -> dict:
+def stage_flops(w: synth.Workload, want_dx: bool, executed: bool = False) -> dict:
+    """Flops of the four frozen-projection launches.  Algorithmic: what the step needs, a slot's low-rank terms
+    counted for its own expert only (k r columns per token).  Executed: what the launches compute, with the low-rank
+    columns of every expert riding along (N r per token)."""
     T, d, f, N, k, r = w.tokens, w.d_model, w.d_ff, w.n_experts, w.top_k, w.rank
     U = 2.0 * T * d * f
-    Nr = N * r
-    NP = (N + 7) // 8 * 8
+    cols = (N if executed else k) * r
+    NR = ((N + 7) // 8 * 8) if executed else N
     fl = {
-        "gemm_gate_up": 2 * U + 2 * 2.0 * T * d * Nr,          # W1, W3 once per token + LoRA-A of every expert
-        "gemm_down": U + 2.0 * T * Nr * d,                     # W2 on the gate-weighted sum + LoRA-B down
-        "gemm_dgrad_down": U + 2.0 * T * d * Nr,               # dy W2 + B_d^T dy
-        "gemm_dx": (2 * U + 2 * 2.0 * T * Nr * d + 2.0 * T * NP * d) if want_dx else 0.0,
+        "gemm_gate_up": 2 * U + 2 * 2.0 * T * d * cols,        # W1, W3 once per token + LoRA-A
+        "gemm_down": U + 2.0 * T * cols * d,                   # W2 on the gate-weighted sum + LoRA-B down
+        "gemm_dgrad_down": U + 2.0 * T * d * cols,             # dy W2 + B_d^T dy
+        "gemm_dx": (2 * U + 2 * 2.0 * T * cols * d + 2.0 * T * NR * d) if want_dx else 0.0,
     }
     return fl
 
@@ -174,11 +193,13 @@ def run_reference(args):
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": per_step * 1e3, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": w.name, "tokens_per_gpu": w.tokens, "d_model": w.d_model, "d_ff": w.d_ff,
-                   "n_experts": w.n_experts, "top_k": w.top_k, "rank": w.rank},
+        "config": config_of(w, args, 1, False),
         "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle",
                          "sample": f"first {sample} tokens of the workload per step, full d_model/d_ff, forward + aux + "
-                                   f"backward with dx, float64 numpy"},
+                                   f"backward with dx, float64 numpy",
+                         "role": "this run (the reference arm: a bounded sample per step so that any --steps ends in "
+                                 "minutes); the stated CPU baseline is the cpu_baseline of the CUDA arm's line, one "
+                                 "oracle pass over 4096 tokens"},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
     }
@@ -198,6 +219,9 @@ def run_cuda(args):
     local = int(os.environ.get("LOCAL_RANK", "0"))
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device (the library has no CPU path)")
+    if world != max(1, args.gpus) and rank == 0:
+        print(f"bench.py: --gpus {args.gpus} but the launcher started {world} rank(s); reporting n_gpus = {world}",
+              file=sys.stderr)
     torch.cuda.set_device(local)
     use_dist = world > 1 or args.force_dist
     if world > 1:
@@ -238,10 +262,10 @@ def run_cuda(args):
         g["d_x"] = torch.empty(w.tokens, w.d_model, dtype=act, device="cuda")
     grads = B.make_grads(accumulate=0, **g)
 
-    def step():
-        B.mixlora_ffn_forward(shape, params, y, ws)
+    def compute(params_, y_, dy_):
+        B.mixlora_ffn_forward(shape, params_, y_, ws)
         B.mixlora_aux_loss(shape, ws, AUX_COEF, loss)
-        B.mixlora_ffn_backward(shape, params, dev["dy"], AUX_COEF, ws, grads)
+        B.mixlora_ffn_backward(shape, params_, dy_, AUX_COEF, ws, grads)
 
     if use_dist:
         # data-parallel sum of the LoRA and router gradients (one flat buffer, one NCCL all-reduce) on a second
@@ -250,14 +274,23 @@ def run_cuda(args):
         ev_ready = torch.cuda.Event()
         ev_ready.record()
 
-        def step():                        # noqa: F811
-            B.mixlora_ffn_forward(shape, params, y, ws)
-            B.mixlora_aux_loss(shape, ws, AUX_COEF, loss)
-            B.mixlora_ffn_backward_overlap(shape, params, dev["dy"], AUX_COEF, ws, grads, ev_ready)
+        aux_sums = torch.zeros(2 * w.n_experts, dtype=torch.float32, device="cuda")   # probability sums, counts
+
+        def compute(params_, y_, dy_):     # noqa: F811
+            B.mixlora_ffn_forward(shape, params_, y_, ws)
+            # Eq. 8-9 are fractions of the whole batch: the shards' sums are added (2N floats) before the loss
+            B.mixlora_aux_stats(shape, ws, aux_sums[:w.n_experts], aux_sums[w.n_experts:])
+            dist.all_reduce(aux_sums)
+            B.mixlora_aux_loss_global(shape, ws, AUX_COEF, aux_sums[:w.n_experts], aux_sums[w.n_experts:],
+                                      world * w.tokens, loss)
+            B.mixlora_ffn_backward_overlap(shape, params_, dy_, AUX_COEF, ws, grads, ev_ready)
             comm.wait_event(ev_ready)
             with torch.cuda.stream(comm):
                 dist.all_reduce(flat)
             torch.cuda.current_stream().wait_stream(comm)
+
+    def step():
+        compute(params, y, dev["dy"])
 
     M = max(1, args.models)
     if M > 1:
@@ -353,6 +386,26 @@ def run_cuda(args):
     B.mixlora_stage_timing(False)
     stage_ms = {n: v[0] / args.steps for n, v in stages.items()}
 
+    # every step with its own pair of events: median and minimum beside the mean of the headline loop; then the same
+    # with L2 flushed before each step (a buffer larger than L2 is overwritten outside the timed pair)
+    def per_step_times(flush):
+        scratch = torch.empty(256 << 20, dtype=torch.uint8, device="cuda") if flush else None
+        evs = []
+        for _ in range(args.steps):
+            if flush:
+                scratch.fill_(1)
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record()
+            step()
+            b.record()
+            evs.append((a, b))
+        torch.cuda.synchronize()
+        ts = sorted(a.elapsed_time(b) for a, b in evs)
+        return {"median": round(ts[len(ts) // 2], 4), "min": round(ts[0], 4), "mean": round(sum(ts) / len(ts), 4)}
+
+    step_ms = per_step_times(False)
+    step_ms_flushed = per_step_times(True)
+
     # End to end through the same C-ABI calls with HOST buffers: every step's x and dy come from pinned host
     # memory and its y and loss go back to the host, all inside the timed region.  The copies of step i+1 run on
     # their own stream while step i computes (two device buffers per input), as a training loop would prefetch.
@@ -384,12 +437,11 @@ def run_cuda(args):
             main.wait_event(ev_in[bi])
             if i + 1 < steps:
                 upload(bi ^ 1)
-            B.mixlora_ffn_forward(shape, pb[bi], yb[bi], ws)
-            B.mixlora_aux_loss(shape, ws, AUX_COEF, loss)
-            if not args.forward_only:
-                B.mixlora_ffn_backward(shape, pb[bi], dyb[bi], AUX_COEF, ws, grads)
-                if use_dist:
-                    dist.all_reduce(flat)
+            if args.forward_only:
+                B.mixlora_ffn_forward(shape, pb[bi], yb[bi], ws)
+                B.mixlora_aux_loss(shape, ws, AUX_COEF, loss)
+            else:
+                compute(pb[bi], yb[bi], dyb[bi])
             ev_done[bi].record(main)
             with torch.cuda.stream(d2h):
                 d2h.wait_event(ev_done[bi])
@@ -420,18 +472,31 @@ def run_cuda(args):
 
     peaks = load_peaks()
     fl = stage_flops(w, want_dx)
+    fl_exec = stage_flops(w, want_dx, executed=True)
     gemm_names = [n for n in fl if fl[n] > 0 and stage_ms.get(n, 0.0) > 0]
     dom = max(gemm_names, key=lambda n: stage_ms.get(n, 0.0))
     gemm_ms = sum(stage_ms.get(n, 0.0) for n in gemm_names)
     gemm_fl = sum(fl[n] for n in gemm_names)
-    peak_tf = peaks["bf16_tflops_sustained"]       # the kernel is timed inside a long step
+    # The peak that applies depends on how long the GPU has been under load: a timed region well under a second
+    # runs at the boost clock (the burst figure), a seconds-long one under the power cap (the sustained figure).
+    # The stage timing above runs right after the headline loop and is as long, so it is judged the same way.
+    burst = total_ms < 1000.0
+    peak_tf = peaks["bf16_tflops"] if burst else peaks["bf16_tflops_sustained"]
     dom_tf = fl[dom] / (stage_ms[dom] * 1e-3) / 1e12 if stage_ms.get(dom) else 0.0
+    gemm_tf = gemm_fl / (gemm_ms * 1e-3) / 1e12 if gemm_ms else 0.0
     roofline = {"bound": "tensor", "kernel": dom, "achieved": dom_tf, "peak": peak_tf, "unit": "TFLOP/s",
-                "frac": dom_tf / peak_tf, "peak_source": peaks["source"] + " (sustained bf16)",
-                "flops_per_launch": fl[dom], "ms_per_launch": stage_ms.get(dom), "traffic": None,
-                "gemm_phases": {"tflops": gemm_fl / (gemm_ms * 1e-3) / 1e12 if gemm_ms else 0.0,
-                                "frac": (gemm_fl / (gemm_ms * 1e-3) / 1e12 / peak_tf) if gemm_ms else 0.0,
+                "frac": dom_tf / peak_tf,
+                "peak_source": "%s (%s bf16: the timed region is %.2f s)" % (peaks["source"], "burst" if burst else "sustained",
+                                                                             total_ms * 1e-3),
+                "frac_of_burst": dom_tf / peaks["bf16_tflops"], "frac_of_sustained": dom_tf / peaks["bf16_tflops_sustained"],
+                "sm_mhz_median": clocks.get("sm_mhz") if clocks else None,
+                "flops_per_launch": fl[dom], "flops_executed_per_launch": fl_exec[dom],
+                "ms_per_launch": stage_ms.get(dom), "traffic": None,
+                "gemm_phases": {"tflops": gemm_tf, "frac": gemm_tf / peak_tf,
+                                "frac_of_burst": gemm_tf / peaks["bf16_tflops"],
+                                "frac_of_sustained": gemm_tf / peaks["bf16_tflops_sustained"],
                                 "ms": gemm_ms, "share_of_step": gemm_ms / sum(stage_ms.values())}}
+    roofline["check"] = "ok" if roofline["frac"] <= 1.02 else "frac above 1.02: the peak and the timed region do not match"
 
     # HBM-bound stages: algorithmic bytes / stage time against the measured copy bandwidth
     T_, d_, f_, k_, N_, r_ = w.tokens, w.d_model, w.d_ff, w.top_k, w.n_experts, w.rank
@@ -457,8 +522,10 @@ def run_cuda(args):
                         "gemm_dx": (2 * T_ * f_ + 2 * f_ * d_ + T_ * d_) * E}
     if w.name == synth.c3().name and want_dx and M == 1 and not args.layer and bf16 and not args.forward_only:
         roofline["traffic"] = measured_dram[dom]
-        roofline["traffic_note"] = ("dram__bytes_read.sum + dram__bytes_write.sum of the %s launch at this size; its "
-                                    "operands and result are %.1f MB" % (dom, algorithmic_dram[dom] / 1e6))
+        roofline["traffic_note"] = ("constant from %s (one single-pass ncu capture of this command's workload, not "
+                                    "measured in this run): dram__bytes_read.sum + dram__bytes_write.sum of the %s "
+                                    "launch; its operands and result are %.1f MB"
+                                    % (DRAM_CAPTURE, dom, algorithmic_dram[dom] / 1e6))
     else:
         roofline["traffic_note"] = "null: the DRAM counters were taken on the default workload only"
 
@@ -468,27 +535,96 @@ def run_cuda(args):
         sec = oracle_sample(w, tensors, sample, want_dx)
         cpu_baseline = {"value": sample / sec, "unit": UNIT, "cores": threads_used(), "kind": "oracle",
                         "sample": f"one oracle pass (forward + aux + backward) over the first {sample} tokens of the "
-                                  f"workload at full d_model/d_ff, {sec:.1f} s"}
+                                  f"workload at full d_model/d_ff, {sec:.1f} s",
+                        "role": "the stated CPU baseline (the line of --impl reference times the same oracle on a "
+                                "smaller per-step sample)"}
 
     line = {
         "metric": METRIC if not args.forward_only else "mixlora_ffn_fwd_tokens_per_s", "value": value, "unit": UNIT,
         "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "bf16" if bf16 else "f32", "data": "synthetic",
-        "config": {"workload": w.name, "tokens_per_gpu": w.tokens, "d_model": w.d_model, "d_ff": w.d_ff,
-                   "n_experts": w.n_experts, "top_k": w.top_k, "rank": w.rank, "lora_alpha": w.lora_alpha,
-                   "backward_dx": want_dx, "aux_coef": AUX_COEF, "adapters": M, "layer_slice": bool(args.layer and M == 1 and want_dx),
-                   "parallelism": f"dp{world} over tokens" + (", NCCL all-reduce of LoRA/router grads beside the dx product" if use_dist else ""),
-                   "l2": "inputs larger than L2 (weights 270 MB + activations > 126 MB), no flush"},
+        "config": config_of(w, args, world, use_dist),
         "roofline": roofline, "cpu_baseline": cpu_baseline,
         "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d_bytes, "d2h_bytes_per_step": d2h_bytes,
                 "ms_per_step": e2e_ms / args.steps,
                 "note": "x, dy from pinned host memory and y, loss back to it every step; copies of step i+1 overlap step i"},
         "gpu_launches": launches_per_step * args.steps, "gpu_launches_per_step": launches_per_step,
-        "stage_ms": {n: round(v, 4) for n, v in stage_ms.items()}, "device_status": status, "clocks": clocks,
+        "stage_ms": {n: round(v, 4) for n, v in stage_ms.items()}, "step_ms": step_ms,
+        "step_ms_l2_flushed": step_ms_flushed, "device_status": status, "clocks": clocks,
     }
     print(json.dumps(line))
     if use_dist:
+        dist.destroy_process_group()
+
+
+# ----------------------------------------------------------------------------------------
+# --gpus N without a launcher: start the ranks here
+# ----------------------------------------------------------------------------------------
+def spawn_ranks(args) -> int:
+    """Re-runs this script as `args.gpus` ranks under torch.distributed.run (one process per GPU, rendezvous on
+    127.0.0.1) and returns the launcher's exit code.  Rank 0 prints the JSON line."""
+    if not args.stub:
+        import torch
+        seen = torch.cuda.device_count()
+        if args.gpus > seen:
+            raise SystemExit(f"--gpus {args.gpus}, but {seen} CUDA device(s) are visible")
+    import socket
+    with socket.socket() as sk:
+        sk.bind(("127.0.0.1", 0))
+        port = sk.getsockname()[1]
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={args.gpus}",
+           "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__)] + sys.argv[1:]
+    env = dict(os.environ)
+    env.setdefault("NCCL_DEBUG", "INFO")            # the communicator's rank count can be read from its log (stderr)
+    env.setdefault("NCCL_DEBUG_SUBSYS", "INIT")
+    env.setdefault("OMP_NUM_THREADS", "4")
+    return subprocess.call(cmd, env=env)
+
+
+def run_stub(args):
+    """Host-only check of the multi-rank plumbing (no GPU, gloo): the same rendezvous, barriers, max-over-ranks
+    timing and rank-0 JSON line as the CUDA leg around a stand-in step that only does the step's two exchanges
+    (2N floats of auxiliary statistics, the flat gradient buffer).  It measures nothing."""
+    import torch
+    import torch.distributed as dist
+    from paper_2404_15159_b200 import dp
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    if world > 1:
+        dist.init_process_group("gloo")
+    w = workload_by_name(args.workload)
+    offsets, total = dp.flat_grad_layout(64, 96, w.n_experts, 8)
+    flat = torch.full((total,), float(rank + 1), dtype=torch.float32)
+    aux = torch.full((2 * w.n_experts,), 1.0, dtype=torch.float32)
+
+    def step():
+        time.sleep(0.001)
+        if world > 1:
+            dist.all_reduce(aux)
+            dist.all_reduce(flat)
+
+    for _ in range(args.warmup):
+        step()
+    if world > 1:
+        dist.barrier()
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        step()
+    if world > 1:
+        dist.barrier()
+    ms = torch.tensor([(time.perf_counter() - t0) * 1e3], dtype=torch.float64)
+    if world > 1:
+        dist.all_reduce(ms, op=dist.ReduceOp.MAX)
+    if rank == 0:
+        per = float(ms.item()) / args.steps
+        print(json.dumps({"impl": "stub", "metric": METRIC, "value": world * w.tokens / (per * 1e-3), "unit": UNIT,
+                          "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": per,
+                          "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "none",
+                          "data": "none", "config": config_of(w, args, world, world > 1), "gpu_launches": 0,
+                          "note": "plumbing check on CPU ranks; not a measurement"}))
+    if world > 1:
         dist.destroy_process_group()
 
 
@@ -514,9 +650,17 @@ def main():
     ap.add_argument("--cpu-sample", type=int, default=4096, help="tokens of the oracle's timed sample")
     ap.add_argument("--ref-sample", type=int, default=0,
                     help="tokens per step of --impl reference (0 = sized so that the run takes about two minutes)")
+    ap.add_argument("--stub", action="store_true",
+                    help="host-only check of the multi-rank plumbing: gloo ranks on CPU around a stand-in step")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
+        return
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        # started without a launcher: become the launcher (one rank per GPU), the ranks print the line
+        raise SystemExit(spawn_ranks(args))
+    if args.stub:
+        run_stub(args)
     else:
         run_cuda(args)
 

@@ -10,9 +10,11 @@
  * Conventions
  *   - Every tensor pointer is a DEVICE pointer unless marked "host".  All tensors are
  *     dense, row-major, 16-byte aligned and owned by the caller, including the workspace.
- *     The library allocates no device memory in these calls and keeps no state between
- *     calls other than what it writes into the caller's workspace (the opt-in measurement
- *     bookkeeping of mixlora_stage_timing excepted).
+ *     The library allocates no device memory in these calls.  What a call computes depends only on its
+ *     arguments and the workspace; the process-wide state the library keeps is scheduling plumbing: a few streams
+ *     and events per device that calls borrow between a fork and a join (see mixlora_ffn_forward), a table of
+ *     encoded tensor maps, the switches of mixlora_set_option and the opt-in bookkeeping of mixlora_stage_timing.
+ *     Calls may be made from several host threads (different workspaces).
  *   - Weights are stored [out, in] as in Eq. 1 (W in R^{d1 x d2}).
  *   - T tokens, d = d_model, f = d_ff, N experts, k = top_k, r = rank, s = lora_alpha / r.
  *     A slot is one (token, selected expert) pair; slot id = t * k + j, j = 0 for the
@@ -112,7 +114,7 @@ size_t mixlora_workspace_bytes(const mixlora_shape_t *shape /* host */, int for_
  * The router and the dispatch are enqueued on a stream that the library creates on first use (one set per device,
  * kept until exit) so that they run beside the shared projections; they start after everything enqueued on
  * `stream` before the call, and the rest of the call, like later work on `stream`, starts after them.
- * MIXLORA_SERIAL=1 in the environment (read once) keeps every launch on `stream`. */
+ * mixlora_set_option(MIXLORA_OPT_SERIAL, 1) keeps every launch on `stream`. */
 mixlora_status_t mixlora_ffn_forward(const mixlora_shape_t *shape /* host */,
                                      const mixlora_params_t *params /* host struct of device ptrs */,
                                      void *y, void *workspace, size_t workspace_bytes, void *stream);
@@ -122,6 +124,24 @@ mixlora_status_t mixlora_ffn_forward(const mixlora_shape_t *shape /* host */,
  * are device arrays of N floats or NULL. */
 mixlora_status_t mixlora_aux_loss(const mixlora_shape_t *shape /* host */, const void *workspace, float coef,
                                   float *loss, float *F, float *P, void *stream);
+
+/* Eq. 8-9 when the batch is spread over data-parallel shards (the paper trains on one GPU; F_i and P_i are
+ * fractions of the WHOLE batch, so the loss of the batch is not the mean of the shards' losses, but the sums over
+ * tokens that F_i and P_i are built from add up over shards).
+ * mixlora_aux_stats copies, from the routing that the last forward call left in `workspace`, the un-normalised sums
+ * of this call's tokens into two device arrays of N floats: prob_sum[i] = sum_t p_t[i], count[i] = tokens whose
+ * arg-max expert is i (aux_f_mode 1: selections that went to i).  The caller adds both over its shards (one
+ * all-reduce of 2N floats) and hands the totals, with the token count of the whole batch, to
+ * mixlora_aux_loss_global, which returns loss = coef * N * sum_i F_i P_i of the whole batch (`loss` device scalar,
+ * `F`, `P` device [N] or NULL) and leaves F_i and the batch's token count in `workspace`: a backward call that
+ * follows then differentiates the batch's loss (d L_aux / d p_t[i] = coef N F_i / total_tokens), so that the shards'
+ * gradients add up to the gradient of the whole batch.  Without this call the backward pass uses this call's own
+ * tokens, as mixlora_aux_loss does.  total_tokens >= shape->tokens. */
+mixlora_status_t mixlora_aux_stats(const mixlora_shape_t *shape /* host */, const void *workspace, float *prob_sum,
+                                   float *count, void *stream);
+mixlora_status_t mixlora_aux_loss_global(const mixlora_shape_t *shape /* host */, void *workspace, float coef,
+                                         const float *prob_sum, const float *count, int64_t total_tokens,
+                                         float *loss, float *F, float *P, void *stream);
 
 /* Backward pass of L = <dy, y> + aux_coef * N * sum_i F_i P_i with respect to the LoRA
  * matrices, the router and, if grads->d_x is not NULL, x (chain rule on Algorithm 1; the
@@ -244,7 +264,10 @@ mixlora_status_t mixlora_gemm_bf16(const void *A, const void *B, void *C, int32_
  * process with a memory budget fixed at start-up.  The per-block count tables that the
  * dispatch kernels need between their three launches sit in a 64 KiB array that is part of
  * the library image on every GPU that loads it (held until the process exits).
- *   expert_idx [tokens, top_k] int32 device, values in [0, n_experts), distinct per token.
+ *   expert_idx [tokens, top_k] int32 device, values in [0, n_experts), distinct per token.  An entry outside
+ *         [0, n_experts) is skipped (it is counted nowhere and leaves one trailing position of perm unwritten); an
+ *         expert repeated within a token makes that token's slots share a position.  Neither reads or writes
+ *         outside the arrays.
  *   perm  [tokens * top_k] int32 device out: slot id (t * top_k + j) at each position of the
  *         order "expert ascending, token ascending".
  *   seg_off [n_experts + 1] int32 device out: first position of each expert.
@@ -260,7 +283,23 @@ mixlora_status_t mixlora_dispatch_static(const int32_t *expert_idx, int32_t toke
                                          int32_t top_k, int32_t *perm, int32_t *seg_off, void *stream);
 int32_t mixlora_dispatch_static_max_tokens(void);
 
-/* Opt-in bookkeeping for measurements (host side, process-wide, not thread-safe).
+/* Process-wide switches (they change how work is scheduled, never a result).  value is 0 or 1.
+ *   MIXLORA_OPT_SERIAL    1: every launch goes to the caller's stream; the library uses no stream of its own.
+ *                         Default 0, or 1 when MIXLORA_SERIAL=1 is in the environment at the first call.
+ *   MIXLORA_OPT_TC_SINGLE 1: the dense products use the single-CTA tensor-core kernel for every shape instead of
+ *                         CTA pairs (a measurement switch).  Default 0, or 1 with MIXLORA_TC_SINGLE=1. */
+#define MIXLORA_OPT_SERIAL 0
+#define MIXLORA_OPT_TC_SINGLE 1
+mixlora_status_t mixlora_set_option(int32_t option, int32_t value);
+
+/* Failure-path check that faults nothing: launches one thread that waits, for at most `wait_rounds` polls
+ * (1 .. 2^20), on a barrier nothing ever signals - the bounded wait every kernel of this library uses - and then
+ * records MIXLORA_ERR_DEVICE_TIMEOUT in the status word at the start of `workspace` (256-byte aligned device
+ * memory, at least 256 bytes), exactly as a production kernel does when one of its waits runs out.
+ * mixlora_device_status then reads 5; the context stays usable. */
+mixlora_status_t mixlora_selftest_wait_timeout(void *workspace, uint32_t wait_rounds, void *stream);
+
+/* Opt-in bookkeeping for measurements (host side, process-wide).
  * mixlora_stage_timing(1) clears the counters and makes every later forward / backward /
  * aux_loss call bracket each stage of the path (router, dispatch, the dense products, the
  * LoRA stages, ...) with CUDA events on the caller's stream; mixlora_stage_timing(0) clears

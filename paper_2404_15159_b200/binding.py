@@ -25,7 +25,11 @@ EXPORTS = ("mixlora_limits", "mixlora_workspace_bytes", "mixlora_ffn_forward", "
            "mixlora_dispatch_static", "mixlora_dispatch_static_max_tokens",
            "mixlora_multi_ffn_forward", "mixlora_multi_ffn_backward", "mixlora_layer_forward",
            "mixlora_layer_backward", "mixlora_lora_linear_workspace_bytes", "mixlora_lora_linear_forward",
-           "mixlora_lora_linear_backward", "mixlora_lora_linear_status", "mixlora_ffn_backward_overlap")
+           "mixlora_lora_linear_backward", "mixlora_lora_linear_status", "mixlora_ffn_backward_overlap",
+           "mixlora_aux_stats", "mixlora_aux_loss_global", "mixlora_set_option", "mixlora_selftest_wait_timeout")
+
+MIXLORA_OPT_SERIAL = 0
+MIXLORA_OPT_TC_SINGLE = 1
 
 
 class mixlora_linear_shape_t(C.Structure):
@@ -123,6 +127,15 @@ def _load() -> C.CDLL:
     lib.mixlora_lora_linear_backward.restype = C.c_int
     lib.mixlora_lora_linear_status.argtypes = [C.c_void_p, C.c_void_p]
     lib.mixlora_lora_linear_status.restype = C.c_int32
+    lib.mixlora_aux_stats.argtypes = [C.POINTER(mixlora_shape_t), C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
+    lib.mixlora_aux_stats.restype = C.c_int
+    lib.mixlora_aux_loss_global.argtypes = [C.POINTER(mixlora_shape_t), C.c_void_p, C.c_float, C.c_void_p, C.c_void_p,
+                                            C.c_int64, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
+    lib.mixlora_aux_loss_global.restype = C.c_int
+    lib.mixlora_set_option.argtypes = [C.c_int32, C.c_int32]
+    lib.mixlora_set_option.restype = C.c_int
+    lib.mixlora_selftest_wait_timeout.argtypes = [C.c_void_p, C.c_uint32, C.c_void_p]
+    lib.mixlora_selftest_wait_timeout.restype = C.c_int
     lib.mixlora_status_string.argtypes = [C.c_int]
     lib.mixlora_status_string.restype = C.c_char_p
     return lib
@@ -201,6 +214,29 @@ def mixlora_ffn_forward(shape, params, y, workspace, stream=None) -> None:
 def mixlora_aux_loss(shape, workspace, coef, loss, F=None, P=None, stream=None) -> None:
     _check(lib.mixlora_aux_loss(C.byref(shape), _ptr(workspace), float(coef), _ptr(loss), _ptr(F), _ptr(P),
                                 _stream(stream)), "mixlora_aux_loss")
+
+
+def mixlora_aux_stats(shape, workspace, prob_sum, count, stream=None) -> None:
+    """Un-normalised sums of Eq. 9 over this call's tokens (to be added over data-parallel shards)."""
+    _check(lib.mixlora_aux_stats(C.byref(shape), _ptr(workspace), _ptr(prob_sum), _ptr(count), _stream(stream)),
+           "mixlora_aux_stats")
+
+
+def mixlora_aux_loss_global(shape, workspace, coef, prob_sum, count, total_tokens, loss, F=None, P=None,
+                            stream=None) -> None:
+    """Eq. 8-9 of the whole batch from the shards' added sums; the backward call that follows uses them too."""
+    _check(lib.mixlora_aux_loss_global(C.byref(shape), _ptr(workspace), float(coef), _ptr(prob_sum), _ptr(count),
+                                       int(total_tokens), _ptr(loss), _ptr(F), _ptr(P), _stream(stream)),
+           "mixlora_aux_loss_global")
+
+
+def mixlora_set_option(option: int, value: int) -> None:
+    _check(lib.mixlora_set_option(int(option), int(value)), "mixlora_set_option")
+
+
+def mixlora_selftest_wait_timeout(workspace, wait_rounds: int, stream=None) -> None:
+    _check(lib.mixlora_selftest_wait_timeout(_ptr(workspace), int(wait_rounds), _stream(stream)),
+           "mixlora_selftest_wait_timeout")
 
 
 def mixlora_ffn_backward(shape, params, dy, aux_coef, workspace, grads, stream=None) -> None:

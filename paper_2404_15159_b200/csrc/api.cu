@@ -4,6 +4,7 @@
 #include <stdlib.h>
 #include <string.h>
 
+#include <atomic>
 #include <mutex>
 #include <vector>
 
@@ -40,6 +41,8 @@ WsLayout ws_layout(const mixlora_shape_t& s) {
   L.blk_off = take(nblk * N * 4);
   L.stat_F = take(N * 4);
   L.stat_P = take(N * 4);
+  L.stat_raw = take(2 * N * 4);
+  L.stat_part = take((size_t)router_part_blocks(s.tokens) * 2 * N * 4);
   L.tile_info = take((mt * 4 + 4) * 4);
   L.G = take(T * f * E);
   L.U = take(T * f * E);
@@ -52,12 +55,14 @@ WsLayout ws_layout(const mixlora_shape_t& s) {
   L.bu_cat = take(f * N * r * E);
   L.Zg_pos = take(T * k * N * r * E);
   L.Zu_pos = take(T * k * N * r * E);
+  const size_t rp = (size_t)pad_rank(s.rank);
   {
-    const size_t rp = r < 16 ? 16 : r;
     L.zg_s = take(T * k * rp * E);
     L.zu_s = take(T * k * rp * E);
-    L.bgp = take(N * f * 16 * E);
-    L.bup = take(N * f * 16 * E);
+    const size_t padded = rp != r ? N * f * rp * E : 0;
+    L.bgp = take(padded);
+    L.bup = take(padded);
+    L.adp = take(padded);
   }
   L.h_sorted = take(T * k * f * E);
   L.hbar = take(T * f * E);
@@ -71,12 +76,9 @@ WsLayout ws_layout(const mixlora_shape_t& s) {
   L.dabar = take(T * f * E);
   L.dbbar = take(T * f * E);
   L.P_pos = take(T * k * N * r * E);
-  L.p_s = take(T * k * (r < 16 ? 16 : r) * E);
+  L.p_s = take(T * k * rp * E);
   L.dZd_pos = take(T * k * N * r * E);
-  {
-    const int a = fused_swiglu_bwd_col_tiles(s.d_ff), b = grouped_swiglu_bwd_col_tiles(s.d_ff);
-    L.dgate_part = take((size_t)(a > b ? a : b) * T * k * 4);
-  }
+  L.dgate_part = take((size_t)grouped_swiglu_bwd_col_tiles(s.d_ff) * T * k * 4);
   L.dzg_all = take(T * k * N * r * E);
   L.dzu_all = take(T * k * N * r * E);
   L.dZg = take(T * N * r * E);
@@ -105,6 +107,7 @@ const char* const kStageNames[ST_COUNT] = {
 struct StageRec { int stage; cudaEvent_t a, b; };
 struct Profiler {
   bool on = false;
+  std::mutex mu;                                       // host threads may call into the library side by side
   std::vector<StageRec> recs;
   long long launches[ST_COUNT] = {0};
 };
@@ -113,7 +116,7 @@ Profiler g_prof;
 struct StageScope {
   int stage; cudaStream_t st; cudaEvent_t a = nullptr, b = nullptr; bool on;
   StageScope(int stage_, cudaStream_t st_, int launches) : stage(stage_), st(st_), on(g_prof.on) {
-    g_prof.launches[stage] += launches;
+    { std::lock_guard<std::mutex> lock(g_prof.mu); g_prof.launches[stage] += launches; }
     if (on) {
       if (cudaEventCreate(&a) != cudaSuccess || cudaEventCreate(&b) != cudaSuccess) { on = false; return; }
       cudaEventRecord(a, st);
@@ -122,50 +125,83 @@ struct StageScope {
   ~StageScope() {
     if (on) {
       cudaEventRecord(b, st);
+      std::lock_guard<std::mutex> lock(g_prof.mu);
       g_prof.recs.push_back({stage, a, b});
     }
   }
 };
 
-// ---- side streams for the per-adapter parts of the multi-model calls ----
-// The per-adapter steps of several adapters are independent and, at a few thousand tokens each, many of their
-// launches fill only part of the GPU; they are spread over a few library-owned streams between two points where
-// everything is back on the caller's stream.  Created on first use, one set per device, kept until exit.
+// ---- side streams ----
+// Steps that do not depend on each other (the router and the dispatch beside the shared projections; the per-adapter
+// steps of different adapters) are spread over a few library-owned streams between two points where everything is
+// back on the caller's stream.  A call borrows a set of streams and events from a per-device list for the time
+// between its fork and its join; the list's lock is held only while a set is picked or handed back, never across
+// launches, so host threads that drive different layers or devices do not wait for each other.  Sets are created on
+// first need (up to kMaxSideSets per device, kept until exit); with none free the call runs on the caller's stream.
 constexpr int kSideStreams = 4;
-struct SidePool {
+constexpr int kMaxSideSets = 8;
+constexpr int kMaxDevices = 64;
+struct SideSet {
   cudaStream_t s[kSideStreams];
   cudaEvent_t fork, join[kSideStreams];
-  bool ok = false, tried = false;
+  bool busy = false;
 };
-SidePool g_side[16];
-std::mutex g_side_mu;
+struct DeviceSides {
+  std::mutex mu;
+  std::vector<SideSet*> sets;
+};
+DeviceSides g_sides[kMaxDevices];
+std::atomic<int> g_serial{-1};                          // MIXLORA_OPT_SERIAL; -1 = take the default from the environment
 
-SidePool* side_pool() {
-  static const bool serial = [] { const char* e = getenv("MIXLORA_SERIAL"); return e && e[0] == '1'; }();
-  if (serial) return nullptr;                          // everything on the caller's stream, for measurements
-  int dev = 0;
-  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 16) return nullptr;
-  std::lock_guard<std::mutex> lock(g_side_mu);
-  SidePool& p = g_side[dev];
-  if (!p.tried) {
-    p.tried = true;
-    bool ok = cudaEventCreateWithFlags(&p.fork, cudaEventDisableTiming) == cudaSuccess;
-    for (int i = 0; i < kSideStreams && ok; ++i)
-      ok = cudaStreamCreateWithFlags(&p.s[i], cudaStreamNonBlocking) == cudaSuccess &&
-           cudaEventCreateWithFlags(&p.join[i], cudaEventDisableTiming) == cudaSuccess;
-    p.ok = ok;
+bool serial_mode() {
+  int v = g_serial.load(std::memory_order_relaxed);
+  if (v < 0) {
+    const char* e = getenv("MIXLORA_SERIAL");
+    v = (e && e[0] == '1') ? 1 : 0;
+    g_serial.store(v, std::memory_order_relaxed);
   }
-  return p.ok ? &p : nullptr;
+  return v != 0;
 }
 
-// Runs fn(adapter context, index) for every adapter, on the side streams when `spread` holds (and no stage timing
-// is being taken, which needs one stream), else in turn on the caller's stream.  With join = false the caller's
+SideSet* acquire_side_set(int* dev_out) {
+  if (serial_mode()) return nullptr;                   // everything on the caller's stream, for measurements
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return nullptr;
+  *dev_out = dev;
+  DeviceSides& D = g_sides[dev];
+  std::lock_guard<std::mutex> lock(D.mu);
+  for (SideSet* p : D.sets)
+    if (!p->busy) { p->busy = true; return p; }
+  if ((int)D.sets.size() >= kMaxSideSets) return nullptr;
+  SideSet* p = new SideSet();
+  bool ok = cudaEventCreateWithFlags(&p->fork, cudaEventDisableTiming) == cudaSuccess;
+  int made = 0;
+  for (int i = 0; i < kSideStreams && ok; ++i) {
+    ok = cudaStreamCreateWithFlags(&p->s[i], cudaStreamNonBlocking) == cudaSuccess &&
+         cudaEventCreateWithFlags(&p->join[i], cudaEventDisableTiming) == cudaSuccess;
+    if (ok) ++made;
+  }
+  if (!ok) {                                           // nothing half-made stays behind
+    for (int i = 0; i < made; ++i) { cudaStreamDestroy(p->s[i]); cudaEventDestroy(p->join[i]); }
+    delete p;
+    return nullptr;
+  }
+  p->busy = true;
+  D.sets.push_back(p);
+  return p;
+}
+
+void release_side_set(SideSet* p, int dev) {
+  if (!p) return;
+  std::lock_guard<std::mutex> lock(g_sides[dev].mu);
+  p->busy = false;
+}
+
+// Runs fn(adapter context, index) for every adapter, on side streams when `spread` holds (and no stage timing
+// is being taken, which needs one stream), else in turn on the caller's stream.  With `later` set the caller's
 // stream is not made to wait yet: join_adapters() does that later, so that work enqueued on the caller's stream in
 // between runs beside the adapters' steps.
-// The pool's streams and events are shared by every caller on the device: `busy` is held from the fork to the join so
-// that two host threads cannot interleave their records and waits on the same events.
-std::mutex g_side_busy;
-struct Forked { SidePool* pool = nullptr; int used = 0; std::unique_lock<std::mutex> busy; };
+struct Forked { SideSet* pool = nullptr; int used = 0; int dev = 0; };
 
 mixlora_status_t join_adapters(cudaStream_t main_st, Forked& fk) {
   mixlora_status_t st = MIXLORA_OK;
@@ -173,23 +209,26 @@ mixlora_status_t join_adapters(cudaStream_t main_st, Forked& fk) {
     if (cudaEventRecord(fk.pool->join[j], fk.pool->s[j]) != cudaSuccess ||
         cudaStreamWaitEvent(main_st, fk.pool->join[j], 0) != cudaSuccess)
       st = MIXLORA_ERR_CUDA;
+  // the waits above are enqueued: later users of the set are ordered behind this call's work on its streams
+  release_side_set(fk.pool, fk.dev);
   fk.pool = nullptr;
-  if (fk.busy.owns_lock()) fk.busy.unlock();
   return st;
 }
 
 template <typename F>
 mixlora_status_t for_each_adapter(const Ctx* cs, int n, bool spread, F fn, Forked* later = nullptr) {
-  SidePool* pool = (spread && !g_prof.on) ? side_pool() : nullptr;
+  Forked fk;
+  SideSet* pool = (spread && !g_prof.on) ? acquire_side_set(&fk.dev) : nullptr;
   mixlora_status_t st = MIXLORA_OK;
   if (!pool) {
     for (int m = 0; m < n && st == MIXLORA_OK; ++m) st = fn(cs[m], m);
     return st;
   }
   cudaStream_t main_st = cs[0].st;
-  Forked fk;
-  fk.busy = std::unique_lock<std::mutex>(g_side_busy);
-  if (cudaEventRecord(pool->fork, main_st) != cudaSuccess) return MIXLORA_ERR_CUDA;
+  if (cudaEventRecord(pool->fork, main_st) != cudaSuccess) {
+    release_side_set(pool, fk.dev);
+    return MIXLORA_ERR_CUDA;
+  }
   fk.pool = pool;
   fk.used = n < kSideStreams ? n : kSideStreams;
   for (int j = 0; j < fk.used; ++j)
@@ -200,7 +239,7 @@ mixlora_status_t for_each_adapter(const Ctx* cs, int n, bool spread, F fn, Forke
     st = fn(c, m);
   }
   if (later && st == MIXLORA_OK) {
-    *later = std::move(fk);
+    *later = fk;
     return st;
   }
   // rejoin at once (always after an error, so that no stream is left dangling)
@@ -441,8 +480,6 @@ static mixlora_status_t fwd_experts(const Ctx& c, void* y, const void* residual 
     if (grouped_swiglu_supported(c)) {
       MIXLORA_CUDA(launch_zcompact(c));
       MIXLORA_CUDA(launch_grouped_swiglu_fwd(c));
-    } else if (fused_swiglu_supported(c)) {
-      MIXLORA_CUDA(launch_fused_swiglu_fwd(c));
     } else {
       MIXLORA_CUDA(launch_lora_b_swiglu(c));
     }
@@ -534,6 +571,37 @@ mixlora_status_t mixlora_aux_loss(const mixlora_shape_t* shape, const void* work
     return MIXLORA_OK;
   }
   { StageScope ss(ST_ROUTER, c.st, 1); MIXLORA_CUDA(launch_aux_loss(c, coef, loss, F, P)); }
+  return MIXLORA_OK;
+}
+
+mixlora_status_t mixlora_aux_stats(const mixlora_shape_t* shape, const void* workspace, float* prob_sum, float* count,
+                                   void* stream) {
+  mixlora_status_t st = check_shape(shape);
+  if (st != MIXLORA_OK) return st;
+  if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255u)) return MIXLORA_ERR_WORKSPACE;
+  if (!prob_sum || !count) return MIXLORA_ERR_INVALID_ARG;
+  Ctx c = make_ctx(shape, nullptr, const_cast<void*>(workspace), stream);
+  const size_t nb = sizeof(float) * shape->n_experts;
+  if (shape->tokens == 0) {
+    MIXLORA_CUDA(cudaMemsetAsync(prob_sum, 0, nb, c.st));
+    MIXLORA_CUDA(cudaMemsetAsync(count, 0, nb, c.st));
+    return MIXLORA_OK;
+  }
+  const float* raw = c.at<float>(c.L.stat_raw);
+  MIXLORA_CUDA(cudaMemcpyAsync(prob_sum, raw, nb, cudaMemcpyDeviceToDevice, c.st));
+  MIXLORA_CUDA(cudaMemcpyAsync(count, raw + shape->n_experts, nb, cudaMemcpyDeviceToDevice, c.st));
+  return MIXLORA_OK;
+}
+
+mixlora_status_t mixlora_aux_loss_global(const mixlora_shape_t* shape, void* workspace, float coef,
+                                         const float* prob_sum, const float* count, int64_t total_tokens, float* loss,
+                                         float* F, float* P, void* stream) {
+  mixlora_status_t st = check_shape(shape);
+  if (st != MIXLORA_OK) return st;
+  if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255u)) return MIXLORA_ERR_WORKSPACE;
+  if (!loss || !prob_sum || !count || total_tokens < shape->tokens || total_tokens <= 0) return MIXLORA_ERR_INVALID_ARG;
+  Ctx c = make_ctx(shape, nullptr, workspace, stream);
+  { StageScope ss(ST_ROUTER, c.st, 1); MIXLORA_CUDA(launch_aux_loss_global(c, coef, prob_sum, count, total_tokens, loss, F, P)); }
   return MIXLORA_OK;
 }
 
@@ -638,9 +706,6 @@ static mixlora_status_t bwd_experts(const Ctx& c, const void* dy, float aux_coef
     if (grouped_swiglu_supported(c)) {
       MIXLORA_CUDA(launch_grouped_swiglu_bwd(c));
       dgate_tiles = grouped_swiglu_bwd_col_tiles(f);
-    } else if (fused_swiglu_supported(c)) {
-      MIXLORA_CUDA(launch_fused_swiglu_bwd(c));
-      dgate_tiles = fused_swiglu_bwd_col_tiles(f);
     } else {
       MIXLORA_CUDA(launch_swiglu_bwd(c));
     }
@@ -883,7 +948,25 @@ mixlora_status_t mixlora_device_status(const void* workspace, int32_t* code, voi
   return MIXLORA_OK;
 }
 
+mixlora_status_t mixlora_set_option(int32_t option, int32_t value) {
+  if (value != 0 && value != 1) return MIXLORA_ERR_INVALID_ARG;
+  switch (option) {
+    case MIXLORA_OPT_SERIAL: g_serial.store(value, std::memory_order_relaxed); return MIXLORA_OK;
+    case MIXLORA_OPT_TC_SINGLE: tc_set_force_single(value); return MIXLORA_OK;
+  }
+  return MIXLORA_ERR_INVALID_ARG;
+}
+
+mixlora_status_t mixlora_selftest_wait_timeout(void* workspace, uint32_t wait_rounds, void* stream) {
+  if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255u)) return MIXLORA_ERR_WORKSPACE;
+  if (wait_rounds == 0 || wait_rounds > (1u << 20)) return MIXLORA_ERR_INVALID_ARG;
+  MIXLORA_CUDA(launch_wait_timeout_selftest(reinterpret_cast<int*>(workspace), wait_rounds,
+                                            reinterpret_cast<cudaStream_t>(stream)));
+  return MIXLORA_OK;
+}
+
 mixlora_status_t mixlora_stage_timing(int32_t enable) {
+  std::lock_guard<std::mutex> lock(g_prof.mu);
   for (auto& r : g_prof.recs) { cudaEventDestroy(r.a); cudaEventDestroy(r.b); }
   g_prof.recs.clear();
   for (int i = 0; i < ST_COUNT; ++i) g_prof.launches[i] = 0;
@@ -892,6 +975,7 @@ mixlora_status_t mixlora_stage_timing(int32_t enable) {
 }
 
 int32_t mixlora_stage_timing_read(int32_t max_stages, const char** names, float* ms, int64_t* launches) {
+  std::lock_guard<std::mutex> lock(g_prof.mu);
   float acc[ST_COUNT] = {0};
   for (auto& r : g_prof.recs) {
     float t = 0.f;

@@ -18,7 +18,8 @@ typedef __nv_bfloat16 bf16;
 // The regions up to total_fwd are what a forward call needs; the rest is backward scratch.
 // ---------------------------------------------------------------------------------------
 struct WsLayout {
-  size_t status;      // int32[64]; [0] = device status word
+  size_t status;      // int32[64]; [0] = device status word; bytes 8..15: int64 token count of the whole batch when
+                      //            the auxiliary loss was evaluated over data-parallel shards (0 = this call's tokens)
   size_t probs;       // f32 [T, N]        softmax probabilities (Eq. 7)
   size_t expert_idx;  // i32 [T, k]
   size_t gates;       // f32 [T, k]
@@ -32,6 +33,8 @@ struct WsLayout {
   size_t blk_off;     // i32 [nblk, N]
   size_t stat_F;      // f32 [N]           F_i of Eq. 9
   size_t stat_P;      // f32 [N]           P_i of Eq. 9
+  size_t stat_raw;    // f32 [2N]          un-normalised sums of Eq. 9: probability per expert, then selections per expert
+  size_t stat_part;   // f32 [router blocks, 2N]  the same sums per block of the router kernel
   size_t tile_info;   // i32 [max_tiles, 4] (expert, first position, rows, 0) of kSegTile-row segment tiles;
                       //                    the int after the table holds the tile count
   size_t G, U;        // act [T, f]        shared W1 / W3 projections (Section 3.3 (I))
@@ -41,8 +44,9 @@ struct WsLayout {
   size_t bd_cat;      // act [d, N*r]      s * B_d laid out [c][e*r + rr]
   size_t bg_cat, bu_cat;  // act [f, N*r]  s * B_g, s * B_u laid out [f'][e*r + rr]
   size_t Zg_pos, Zu_pos;  // act [T*k, N*r]  zg / zu of the slot in its expert block, zero elsewhere
-  size_t zg_s, zu_s;  // act [T*k, max(r,16)]  s * zg, s * zu of the slot's own expert, zero padded
-  size_t bgp, bup;    // act [N*f, 16]     B_g, B_u zero padded to 16 columns (used when r < 16)
+  size_t zg_s, zu_s;  // act [T*k, pad_rank(r)]  s * zg, s * zu of the slot's own expert, zero padded
+  size_t bgp, bup;    // act [N*f, pad_rank(r)]  B_g, B_u zero padded (used when pad_rank(r) != r)
+  size_t adp;         // act [N*pad_rank(r), f]  A_d with each expert's rows zero padded (same condition)
   size_t h_sorted;    // act [T*k, f]
   size_t hbar;        // act [T, f]        sum_j g_j h_j
   size_t work_count;  // i32 [8]  item counts of the work lists below
@@ -53,7 +57,7 @@ struct WsLayout {
   size_t da_sorted, db_sorted;  // act [T*k, f]
   size_t dabar, dbbar;          // act [T, f]
   size_t P_pos;                 // act [T*k, N*r]  s * pd of the slot in its expert block, zero elsewhere
-  size_t p_s;                   // act [T*k, max(r,16)]  s * pd of the slot's own expert, zero padded
+  size_t p_s;                   // act [T*k, pad_rank(r)]  s * pd of the slot's own expert, zero padded
   size_t dZd_pos;               // act [T*k, N*r]  gate * P_pos
   size_t dgate_part;            // f32 [ceil(f/64), T*k]  per column tile partial <Dt, h> of the fused backward
   size_t dzg_all, dzu_all;      // act [T*k, N*r]  da (s B_g) and db (s B_u) against every expert
@@ -75,6 +79,9 @@ static const int kSegTile = 128;           // rows of a segment tile
 static inline int route_blocks(int T) { return (T + kRouteBlockTokens - 1) / kRouteBlockTokens; }
 static inline int max_seg_tiles(int T, int k, int N) { return (int)(((long long)T * k + kSegTile - 1) / kSegTile) + N; }
 static inline int round_up8(int v) { return (v + 7) / 8 * 8; }
+// rank-r operands of the grouped SwiGLU kernels are rows of 32, 64 or 128 bytes (or two 128-byte blocks): other
+// ranks are zero-padded to the next of these widths
+static inline int pad_rank(int r) { return r <= 16 ? 16 : (r <= 32 ? 32 : (r <= 64 ? 64 : 128)); }
 
 WsLayout ws_layout(const mixlora_shape_t& s);
 
@@ -141,19 +148,18 @@ struct Ctx {
 cudaError_t launch_router(const Ctx& c);              // probs, expert_idx, gates, low_margin, stats
 cudaError_t launch_dispatch(const Ctx& c);            // perm, inv, pos_token, pos_expert, seg_off, tile_info
 cudaError_t launch_aux_loss(const Ctx& c, float coef, float* loss, float* F, float* P);
+cudaError_t launch_aux_loss_global(const Ctx& c, float coef, const float* prob_sum, const float* count,
+                                   long long total_tokens, float* loss, float* F, float* P);
+int router_part_blocks(int tokens);                   // upper bound of the router kernel's blocks
 cudaError_t launch_bd_cat(const Ctx& c);
 cudaError_t launch_bgu_cat(const Ctx& c);              // bg_cat, bu_cat
 cudaError_t launch_zpos(const Ctx& c);                 // Zg_pos, Zu_pos
 cudaError_t launch_dgate_reduce(const Ctx& c, int col_tiles);   // dgate from dgate_part
-cudaError_t launch_zcompact(const Ctx& c);             // zg_s, zu_s (and bgp, bup when r < 16)
+cudaError_t launch_zcompact(const Ctx& c);             // zg_s, zu_s (and bgp, bup, adp when the rank is padded)
 bool grouped_swiglu_supported(const Ctx& c);
 int grouped_swiglu_bwd_col_tiles(int f);
 cudaError_t launch_grouped_swiglu_fwd(const Ctx& c);   // per-expert tiles, K = r (grouped_swiglu.cu)
 cudaError_t launch_grouped_swiglu_bwd(const Ctx& c);
-bool fused_swiglu_supported(const Ctx& c);
-int fused_swiglu_bwd_col_tiles(int f);
-cudaError_t launch_fused_swiglu_fwd(const Ctx& c);     // tensor-core version of lora_b_swiglu
-cudaError_t launch_fused_swiglu_bwd(const Ctx& c);     // tensor-core version of swiglu_bwd (writes dgate_part)
 cudaError_t launch_lora_b_swiglu(const Ctx& c);       // h_sorted from G, U, zga, zua, B_g, B_u
 cudaError_t launch_combine_h(const Ctx& c);           // hbar, Zs
 cudaError_t launch_swiglu_bwd(const Ctx& c);          // h_sorted, da_sorted, db_sorted, dgate, Zg_pos, Zu_pos
@@ -197,6 +203,8 @@ struct TcWork {
   int block_cols;     // columns of one block (the LoRA rank)
 };
 bool tc_gemm_supported(int M, const TcOut* outs, int nout);
+void tc_set_force_single(int v);   // 1: single-CTA tensor-core kernel for every shape (measurement switch)
+cudaError_t launch_wait_timeout_selftest(int* status, unsigned limit, cudaStream_t st);
 int tc_gemm_tile_rows(int M);   // rows of the tiles the tensor-core kernel will use for a problem with M rows
 cudaError_t launch_tc_gemm(int M, const TcOut* outs, int nout, int* status_word, cudaStream_t st,
                            const TcWork* wl = nullptr);

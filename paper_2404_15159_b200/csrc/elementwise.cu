@@ -375,14 +375,26 @@ __global__ void zcompact_kernel(const T* __restrict__ zga, const T* __restrict__
   }
 }
 
-// out[row][c] = in[row][c] for c < r, zero up to 16 columns (rows = N * f)
+// out[row][c] = in[row][c] for c < r, zero up to rp columns
 template <typename T>
-__global__ void pad16_kernel(const T* __restrict__ in, T* __restrict__ out, long long rows, int r) {
-  const long long n = rows * 16;
+__global__ void pad_cols_kernel(const T* __restrict__ in, T* __restrict__ out, long long rows, int r, int rp) {
+  const long long n = rows * rp;
   for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < n; i += (long long)gridDim.x * blockDim.x) {
-    const long long row = i / 16;
-    const int cidx = (int)(i % 16);
+    const long long row = i / rp;
+    const int cidx = (int)(i % rp);
     out[i] = cidx < r ? in[row * r + cidx] : from_f<T>(0.f);
+  }
+}
+
+// out[e][rr][c] = in[e][rr][c] for rr < r, zero rows up to rp per expert (A_d is [N, r, f])
+template <typename T>
+__global__ void pad_rows_kernel(const T* __restrict__ in, T* __restrict__ out, int N, int r, int rp, int f) {
+  const long long n = (long long)N * rp * f;
+  for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < n; i += (long long)gridDim.x * blockDim.x) {
+    const int col = (int)(i % f);
+    const int rr = (int)((i / f) % rp);
+    const int e = (int)(i / ((long long)f * rp));
+    out[i] = rr < r ? in[((long long)e * r + rr) * f + col] : from_f<T>(0.f);
   }
 }
 
@@ -439,9 +451,14 @@ template <typename T>
 __global__ void router_bwd_kernel(const float* __restrict__ probs, const float* __restrict__ gates,
                                   const int* __restrict__ expert_idx, const float* __restrict__ dgate,
                                   const float* __restrict__ F, float* __restrict__ dlogits, T* __restrict__ dl_act,
-                                  int tokens, int N, int NP, int k, int renorm, float aux_scale) {
+                                  int tokens, int N, int NP, int k, int renorm, float aux_coef,
+                                  const long long* __restrict__ batch_tokens) {
   const int t = blockIdx.x * blockDim.x + threadIdx.x;
   if (t >= tokens) return;
+  // d L_aux / d p_ti = coef N F_i / T with T the tokens of the whole batch (Eq. 8-9): this call's, unless the
+  // auxiliary loss was evaluated over data-parallel shards, which leaves the batch's count (and F) in the workspace
+  const long long bt = *batch_tokens;
+  const float aux_scale = aux_coef * (float)N / (float)(bt > 0 ? bt : (long long)tokens);
   float dp[MIXLORA_MAX_EXPERTS];
 #pragma unroll
   for (int e = 0; e < MIXLORA_MAX_EXPERTS; ++e) dp[e] = (e < N) ? aux_scale * F[e] : 0.f;
@@ -533,16 +550,18 @@ cudaError_t zpos_t(const Ctx& c) {
 
 template <typename T>
 cudaError_t zcompact_t(const Ctx& c) {
-  const int slots = c.s.tokens * c.s.top_k, r = c.s.rank, rp = r < 16 ? 16 : r;
+  const int slots = c.s.tokens * c.s.top_k, r = c.s.rank, rp = pad_rank(r);
   zcompact_kernel<T><<<grid_for((long long)slots * rp, 256), 256, 0, c.st>>>(
       c.at<T>(c.L.zga), c.at<T>(c.L.zua), c.at<int>(c.L.pos_token), c.at<int>(c.L.pos_expert), c.at<T>(c.L.zg_s),
       c.at<T>(c.L.zu_s), slots, c.s.n_experts, r, rp, c.scale);
-  if (r < 16) {
+  if (rp != r) {   // parameter-only repacks for the grouped kernels; the backward pass finds them in the workspace
     const long long rows = (long long)c.s.n_experts * c.s.d_ff;
-    pad16_kernel<T><<<grid_for(rows * 16, 256), 256, 0, c.st>>>(reinterpret_cast<const T*>(c.p.b_gate),
-                                                               c.at<T>(c.L.bgp), rows, r);
-    pad16_kernel<T><<<grid_for(rows * 16, 256), 256, 0, c.st>>>(reinterpret_cast<const T*>(c.p.b_up), c.at<T>(c.L.bup),
-                                                               rows, r);
+    pad_cols_kernel<T><<<grid_for(rows * rp, 256), 256, 0, c.st>>>(reinterpret_cast<const T*>(c.p.b_gate),
+                                                                  c.at<T>(c.L.bgp), rows, r, rp);
+    pad_cols_kernel<T><<<grid_for(rows * rp, 256), 256, 0, c.st>>>(reinterpret_cast<const T*>(c.p.b_up),
+                                                                  c.at<T>(c.L.bup), rows, r, rp);
+    pad_rows_kernel<T><<<grid_for(rows * rp, 256), 256, 0, c.st>>>(reinterpret_cast<const T*>(c.p.a_down),
+                                                                  c.at<T>(c.L.adp), c.s.n_experts, r, rp, c.s.d_ff);
   }
   return cudaGetLastError();
 }
@@ -590,7 +609,7 @@ cudaError_t slot_prep_bwd_t(const Ctx& c) {
   slot_prep_bwd_kernel<T><<<grid_for((long long)slots * c.s.rank * c.s.n_experts, 256), 256, 0, c.st>>>(
       c.at<T>(c.L.spd), c.at<float>(c.L.gates), c.at<int>(c.L.perm), c.at<int>(c.L.pos_token),
       c.at<int>(c.L.pos_expert), c.at<T>(c.L.P_pos), c.at<T>(c.L.dZd_pos), c.at<T>(c.L.p_s), slots, c.s.n_experts,
-      c.s.rank, c.s.rank < 16 ? 16 : c.s.rank);
+      c.s.rank, pad_rank(c.s.rank));
   return cudaGetLastError();
 }
 
@@ -607,11 +626,10 @@ cudaError_t combine_bwd_t(const Ctx& c, int want_dx) {
 template <typename T>
 cudaError_t router_bwd_t(const Ctx& c, float aux_coef, float* d_bias, int accumulate, int want_dx) {
   const int T_ = c.s.tokens, N = c.s.n_experts, NP = round_up8(N);
-  const float aux_scale = (T_ > 0) ? aux_coef * (float)N / (float)T_ : 0.f;
   router_bwd_kernel<T><<<(T_ + 127) / 128, 128, 0, c.st>>>(
       c.at<float>(c.L.probs), c.at<float>(c.L.gates), c.at<int>(c.L.expert_idx), c.at<float>(c.L.dgate),
       c.at<float>(c.L.stat_F), c.at<float>(c.L.dlogits), c.at<T>(c.L.dl_act), T_, N, NP, c.s.top_k,
-      c.s.renormalize, aux_scale);
+      c.s.renormalize, aux_coef, reinterpret_cast<const long long*>(c.ws + c.L.status + 8));
   if (d_bias) colsum_kernel<<<N, 256, 0, c.st>>>(c.at<float>(c.L.dlogits), d_bias, T_, N, accumulate);
   if (want_dx)
     wr_act_kernel<T><<<grid_for((long long)NP * c.s.d_model, 256), 256, 0, c.st>>>(c.p.w_router, c.at<T>(c.L.wr_act), N,

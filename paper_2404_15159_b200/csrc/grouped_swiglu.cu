@@ -513,7 +513,7 @@ cudaError_t launch_t(const Ctx& c) {
   constexpr int CB = COLS / 64;
   constexpr int NMAT = BWD ? 3 : 2;
   const int slots = c.s.tokens * c.s.top_k, f = c.s.d_ff, r = c.s.rank, N = c.s.n_experts;
-  const int rp = r < 16 ? 16 : r;
+  const int rp = pad_rank(r);
   GsParams p;
   memset(&p, 0, sizeof(p));
   p.row_bytes = rp >= 64 ? 128 : rp * 2;               // bytes of one operand row per k-block
@@ -544,8 +544,10 @@ cudaError_t launch_t(const Ctx& c) {
   const uint32_t smem_bytes = fixed + nst * p.stage_bytes;
 
   const int kbc = p.row_bytes / 2;
-  const void* bg = r < 16 ? (const void*)(c.ws + c.L.bgp) : c.p.b_gate;
-  const void* bu = r < 16 ? (const void*)(c.ws + c.L.bup) : c.p.b_up;
+  // ranks between the native widths work on zero-padded copies of B_g, B_u and A_d (built with the compact z)
+  const void* bg = rp != r ? (const void*)(c.ws + c.L.bgp) : c.p.b_gate;
+  const void* bu = rp != r ? (const void*)(c.ws + c.L.bup) : c.p.b_up;
+  const void* ad = rp != r ? (const void*)(c.ws + c.L.adp) : c.p.a_down;
   bool ok = tc_encode_2d(&p.a_map[0], c.ws + c.L.zg_s, slots, rp, rp, BM, kbc, p.row_bytes) &&
             tc_encode_2d(&p.a_map[1], c.ws + c.L.zu_s, slots, rp, rp, BM, kbc, p.row_bytes) &&
             tc_encode_2d(&p.b_map[0], bg, (long long)N * f, rp, rp, COLS, kbc, p.row_bytes) &&
@@ -553,7 +555,7 @@ cudaError_t launch_t(const Ctx& c) {
             tc_encode_2d(&p.o_map[0], c.ws + c.L.h_sorted, slots, f, f, BM, 64, 128);
   if (BWD)
     ok = ok && tc_encode_2d(&p.a_map[2], c.ws + c.L.p_s, slots, rp, rp, BM, kbc, p.row_bytes) &&
-         tc_encode_2d(&p.b_map[2], c.p.a_down, (long long)N * r, f, f, p.krows, 64, 128) &&
+         tc_encode_2d(&p.b_map[2], ad, (long long)N * rp, f, f, p.krows, 64, 128) &&
          tc_encode_2d(&p.o_map[0], c.ws + c.L.da_sorted, slots, f, f, BM, 64, 128) &&
          tc_encode_2d(&p.o_map[1], c.ws + c.L.db_sorted, slots, f, f, BM, 64, 128);
   if (!ok) return cudaErrorInvalidValue;
@@ -563,7 +565,7 @@ cudaError_t launch_t(const Ctx& c) {
   p.h = c.at<bf16>(c.L.h_sorted); p.da = c.at<bf16>(c.L.da_sorted); p.db = c.at<bf16>(c.L.db_sorted);
   p.dgate_part = c.at<float>(c.L.dgate_part);
   p.max_tiles = max_seg_tiles(c.s.tokens, c.s.top_k, N);
-  p.slots = slots; p.f = f; p.r = r;
+  p.slots = slots; p.f = f; p.r = rp;                  // rows per expert in the A_d operand
   p.col_tiles = (f + COLS - 1) / COLS;
   // columns per group: the group's pieces of the gathered matrices (tokens x columns x NMAT) stay well inside L2
   const long long group_cols = (32ll << 20) / ((long long)c.s.tokens * 2 * NMAT);
@@ -581,10 +583,10 @@ cudaError_t launch_t(const Ctx& c) {
 
 }  // namespace
 
-// ranks this kernel takes: the operand rows must be 32, 64 or 128 bytes, or two 128-byte blocks
+// every bf16 rank (a multiple of 8 up to 128): the operand rows are 32, 64 or 128 bytes, or two 128-byte blocks,
+// other ranks zero-padded to the next of these
 bool grouped_swiglu_supported(const Ctx& c) {
-  const int r = c.s.rank;
-  return c.bf16 && c.s.tokens > 0 && (r == 8 || r == 16 || r == 32 || r == 64 || r == 128);
+  return c.bf16 && c.s.tokens > 0 && c.s.rank % 8 == 0 && c.s.rank <= 128;
 }
 int grouped_swiglu_bwd_col_tiles(int f) { return (f + 63) / 64; }
 cudaError_t launch_grouped_swiglu_fwd(const Ctx& c) { return launch_t<0>(c); }

@@ -6,44 +6,54 @@ namespace mixlora {
 
 namespace {
 
-constexpr int kWarpsPerBlock = 4;
+constexpr int kRWarps = 8;            // warps per block of the router kernel
+constexpr int kRCols = 256;           // features per step: 32 lanes x 8
 constexpr float kMarginFlag = 1e-4f;
 
-// VEC consecutive features of one row as floats (16-byte load)
-template <int VEC> struct FeatVec { float v[VEC]; };
-__device__ __forceinline__ FeatVec<4> ld_feat(const float* p) {
-  const float4 r = *reinterpret_cast<const float4*>(p);
-  FeatVec<4> o; o.v[0] = r.x; o.v[1] = r.y; o.v[2] = r.z; o.v[3] = r.w;
-  return o;
+// 8 consecutive features of one row, as loaded (16 bytes of bf16, 32 bytes of fp32) and as floats
+template <typename T> struct Raw8;
+template <> struct Raw8<bf16> { uint4 v; };
+template <> struct Raw8<float> { float4 lo, hi; };
+__device__ __forceinline__ void ld_raw8(const bf16* p, Raw8<bf16>& r) { r.v = __ldg(reinterpret_cast<const uint4*>(p)); }
+__device__ __forceinline__ void ld_raw8(const float* p, Raw8<float>& r) {
+  r.lo = __ldg(reinterpret_cast<const float4*>(p));
+  r.hi = __ldg(reinterpret_cast<const float4*>(p) + 1);
 }
-__device__ __forceinline__ FeatVec<8> ld_feat(const bf16* p) {
-  const uint4 raw = *reinterpret_cast<const uint4*>(p);
-  const __nv_bfloat162* h = reinterpret_cast<const __nv_bfloat162*>(&raw);
-  FeatVec<8> o;
+__device__ __forceinline__ void zero_raw8(Raw8<bf16>& r) { r.v = make_uint4(0u, 0u, 0u, 0u); }
+__device__ __forceinline__ void zero_raw8(Raw8<float>& r) { r.lo = r.hi = make_float4(0.f, 0.f, 0.f, 0.f); }
+__device__ __forceinline__ void cvt_raw8(const Raw8<bf16>& r, float (&o)[8]) {
+  const uint32_t w[4] = {r.v.x, r.v.y, r.v.z, r.v.w};
 #pragma unroll
-  for (int i = 0; i < 4; ++i) {
-    const float2 f = __bfloat1622float2(h[i]);
-    o.v[2 * i] = f.x; o.v[2 * i + 1] = f.y;
+  for (int i = 0; i < 4; ++i) {                     // a bf16 is the upper half of the fp32 with the same value
+    o[2 * i] = __uint_as_float(w[i] << 16);
+    o[2 * i + 1] = __uint_as_float(w[i] & 0xffff0000u);
   }
-  return o;
 }
-template <typename T> struct VecOf;
-template <> struct VecOf<float> { static constexpr int value = 4; };
-template <> struct VecOf<bf16> { static constexpr int value = 8; };
+__device__ __forceinline__ void cvt_raw8(const Raw8<float>& r, float (&o)[8]) {
+  o[0] = r.lo.x; o[1] = r.lo.y; o[2] = r.lo.z; o[3] = r.lo.w;
+  o[4] = r.hi.x; o[5] = r.hi.y; o[6] = r.hi.z; o[7] = r.hi.w;
+}
 
-// One warp handles TOK tokens at a time and NE (>= N) logits per token, TOK * NE = 32
-// accumulators per lane.  Each lane covers VEC consecutive features (one 16-byte load of x)
-// per step of 32 * VEC features.
+// Router (Eq. 7).  A block of kRWarps warps handles kRWarps * TOK tokens; a warp handles TOK tokens and NE (>= N)
+// logits per token, TOK * NE accumulators per lane, and each lane covers 8 consecutive features per step of 256.
+// x is read once, 16 bytes per lane and token, one step ahead of its use.  The router weight goes through shared
+// memory in chunks of 256 features (staged by all threads, laid out so that a lane's two 16-byte pieces of an
+// expert's row are read without bank conflicts), so a block reads W_r once for all its tokens and each weight
+// register serves TOK tokens.  The block also leaves the sums over its tokens that Eq. 9 needs (probability per
+// expert, selections per expert) in `part`, in a fixed order.
 template <typename T, int NE, int TOK>
-__global__ void __launch_bounds__(kWarpsPerBlock * 32)
+__global__ void __launch_bounds__(kRWarps * 32)
 router_kernel(const T* __restrict__ x, const float* __restrict__ w_router, const float* __restrict__ bias,
               float* __restrict__ probs, int* __restrict__ expert_idx, float* __restrict__ gates,
-              uint8_t* __restrict__ low_margin, int tokens, int d, int N, int k, int renorm) {
-  constexpr int VEC = VecOf<T>::value;
-  const int lane = threadIdx.x & 31;
-  const int warp = (blockIdx.x * kWarpsPerBlock) + (threadIdx.x >> 5);
-  const int t0 = warp * TOK;
-  if (t0 >= tokens) return;
+              uint8_t* __restrict__ low_margin, float* __restrict__ part, int tokens, int d, int N, int k,
+              int renorm, int f_mode) {
+  constexpr int WPT = NE / 4;                          // 16-byte pieces of a weight chunk staged per thread
+  constexpr int BT = kRWarps * TOK;                    // tokens per block
+  __shared__ float4 wsm[NE * 2 * 32];                  // [expert][half of the lane's 8 features][lane]
+  __shared__ float sp[BT][NE];                         // probabilities of the block's tokens
+  __shared__ unsigned ssel[BT];                        // bit e set: expert e counts for F_i of this token
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int t0 = (blockIdx.x * kRWarps + warp) * TOK;
 
   float acc[TOK][NE];
 #pragma unroll
@@ -51,26 +61,48 @@ router_kernel(const T* __restrict__ x, const float* __restrict__ w_router, const
 #pragma unroll
     for (int e = 0; e < NE; ++e) acc[a][e] = 0.f;
 
-  for (int c = lane * VEC; c < d; c += 32 * VEC) {
-    FeatVec<VEC> xv[TOK];
+  float4 wn[WPT];
+  Raw8<T> xr[TOK];
+  auto load_w = [&](int ch) {
+#pragma unroll
+    for (int i = 0; i < WPT; ++i) {
+      const int j = threadIdx.x + i * (kRWarps * 32), e = j >> 6, c = ch * kRCols + (j & 63) * 4;
+      wn[i] = (e < N && c < d) ? __ldg(reinterpret_cast<const float4*>(w_router + (size_t)e * d + c))
+                               : make_float4(0.f, 0.f, 0.f, 0.f);
+    }
+  };
+  auto load_x = [&](int ch) {
+    const int c = ch * kRCols + lane * 8;
 #pragma unroll
     for (int a = 0; a < TOK; ++a) {
-      const int t = min(t0 + a, tokens - 1);       // rows past the end repeat the last token; never written
-      xv[a] = ld_feat(x + (size_t)t * d + c);
+      const int t = min(t0 + a, tokens - 1);           // rows past the end repeat the last token; never written
+      if (c < d) ld_raw8(x + (size_t)t * d + c, xr[a]); else zero_raw8(xr[a]);
     }
+  };
+  const int nchunk = (d + kRCols - 1) / kRCols;
+  load_w(0);
+  load_x(0);
+  for (int ch = 0; ch < nchunk; ++ch) {
+    __syncthreads();                                   // the previous chunk has been read by every warp
+#pragma unroll
+    for (int i = 0; i < WPT; ++i) {
+      const int j = threadIdx.x + i * (kRWarps * 32), e = j >> 6, q = j & 63;
+      wsm[(e * 2 + (q & 1)) * 32 + (q >> 1)] = wn[i];
+    }
+    __syncthreads();
+    float xv[TOK][8];
+#pragma unroll
+    for (int a = 0; a < TOK; ++a) cvt_raw8(xr[a], xv[a]);
+    if (ch + 1 < nchunk) { load_w(ch + 1); load_x(ch + 1); }
 #pragma unroll
     for (int e = 0; e < NE; ++e) {
       if (e < N) {
-        float w[VEC];
-#pragma unroll
-        for (int i = 0; i < VEC; i += 4) {
-          const float4 r = __ldg(reinterpret_cast<const float4*>(w_router + (size_t)e * d + c + i));
-          w[i] = r.x; w[i + 1] = r.y; w[i + 2] = r.z; w[i + 3] = r.w;
-        }
+        const float4 w0 = wsm[(e * 2) * 32 + lane], w1 = wsm[(e * 2 + 1) * 32 + lane];
+        const float w[8] = {w0.x, w0.y, w0.z, w0.w, w1.x, w1.y, w1.z, w1.w};
 #pragma unroll
         for (int a = 0; a < TOK; ++a)
 #pragma unroll
-          for (int i = 0; i < VEC; ++i) acc[a][e] = fmaf(xv[a].v[i], w[i], acc[a][e]);
+          for (int i = 0; i < 8; ++i) acc[a][e] = fmaf(xv[a][i], w[i], acc[a][e]);
       }
     }
   }
@@ -88,7 +120,14 @@ router_kernel(const T* __restrict__ x, const float* __restrict__ w_router, const
 #pragma unroll
   for (int a = 0; a < TOK; ++a) {
     const int t = t0 + a;
-    if (t >= tokens || lane != a) continue;
+    if (lane != a) continue;
+    const int bt = warp * TOK + a;
+    if (t >= tokens) {
+      ssel[bt] = 0u;
+#pragma unroll
+      for (int e = 0; e < NE; ++e) sp[bt][e] = 0.f;
+      continue;
+    }
     float l[NE];
     float mx = -INFINITY;
 #pragma unroll
@@ -107,9 +146,13 @@ router_kernel(const T* __restrict__ x, const float* __restrict__ w_router, const
 #pragma unroll
     for (int e = 0; e < NE; ++e) {
       p[e] *= inv_sum;
+      sp[bt][e] = p[e];
       if (e < N) probs[(size_t)t * N + e] = p[e];
     }
-    // top-k on the logits, ties to the lower index
+    // top-k on the logits, ties to the lower index.  Each round starts from the lowest expert not taken yet, so
+    // the k choices are distinct whatever the logits are (NaN or -inf rows included: those show up in the
+    // values, never as a repeated index)
+    const unsigned all = (N >= 32) ? 0xffffffffu : ((1u << N) - 1u);
     unsigned taken = 0;
     float qsum = 0.f, first = 0.f, second = 0.f, last = 0.f;
     int sel[MIXLORA_MAX_TOP_K];
@@ -117,12 +160,14 @@ router_kernel(const T* __restrict__ x, const float* __restrict__ w_router, const
 #pragma unroll
     for (int j = 0; j < MIXLORA_MAX_TOP_K; ++j) {
       if (j < k) {
-        float best = -INFINITY;
-        int bi = 0;
-        float bp = 0.f;
+        int bi = __ffs(~taken & all) - 1;
+        float best = -INFINITY, bp = 0.f;
+#pragma unroll
+        for (int e = 0; e < NE; ++e)
+          if (e == bi) { best = l[e]; bp = p[e]; }
 #pragma unroll
         for (int e = 0; e < NE; ++e) {
-          bool free_e = !((taken >> e) & 1u) && e < N;
+          const bool free_e = !((taken >> e) & 1u) && e < N;
           if (free_e && l[e] > best) { best = l[e]; bi = e; bp = p[e]; }
         }
         taken |= 1u << bi;
@@ -137,14 +182,14 @@ router_kernel(const T* __restrict__ x, const float* __restrict__ w_router, const
     float next = -INFINITY;  // largest logit left out
 #pragma unroll
     for (int e = 0; e < NE; ++e) {
-      bool free_e = !((taken >> e) & 1u) && e < N;
+      const bool free_e = !((taken >> e) & 1u) && e < N;
       if (free_e && l[e] > next) next = l[e];
     }
     float margin = INFINITY;
     if (k < N) margin = fminf(margin, last - next);
     if (N > 1) margin = fminf(margin, first - ((k >= 2) ? second : next));
     low_margin[t] = (margin < kMarginFlag) ? 1 : 0;
-    
+    ssel[bt] = f_mode == 0 ? (1u << sel[0]) : taken;
 #pragma unroll
     for (int j = 0; j < MIXLORA_MAX_TOP_K; ++j) {
       if (j < k) {
@@ -153,39 +198,43 @@ router_kernel(const T* __restrict__ x, const float* __restrict__ w_router, const
       }
     }
   }
+  __syncthreads();
+  if (threadIdx.x < N) {                                // the block's sums for Eq. 9, tokens in order
+    const int e = threadIdx.x;
+    float ps = 0.f, cnt = 0.f;
+    for (int i = 0; i < BT; ++i) {
+      ps += sp[i][e];
+      cnt += (float)((ssel[i] >> e) & 1u);
+    }
+    part[(size_t)blockIdx.x * 2 * N + e] = ps;
+    part[(size_t)blockIdx.x * 2 * N + N + e] = cnt;
+  }
 }
 
-// F_i and P_i of Eq. 9, one block per expert, fixed summation order (deterministic).
+// F_i and P_i of Eq. 9 from the blocks' partial sums: warp e adds expert e's entries in a fixed order.  Also keeps
+// the un-normalised sums (for callers that add them over data-parallel shards first).
 __global__ void __launch_bounds__(1024)
-router_stats_kernel(const float* __restrict__ probs, const int* __restrict__ expert_idx, float* __restrict__ F,
-                    float* __restrict__ P, int tokens, int N, int k, int f_mode) {
-  __shared__ float sp[1024];
-  __shared__ int sc[1024];
-  const int e = blockIdx.x;
-  float ps = 0.f;
-  int cnt = 0;
-  for (int t = threadIdx.x; t < tokens; t += 1024) {
-    ps += probs[(size_t)t * N + e];
-    if (f_mode == 0) {
-      cnt += (expert_idx[(size_t)t * k] == e);
-    } else {
-      for (int j = 0; j < k; ++j) cnt += (expert_idx[(size_t)t * k + j] == e);
-    }
+router_stats_kernel(const float* __restrict__ part, int nblocks, float* __restrict__ F, float* __restrict__ P,
+                    float* __restrict__ raw /* [2N]: probability sums, then counts */, int tokens, int N, int k,
+                    int f_mode) {
+  const int e = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  if (e >= N) return;
+  float ps = 0.f, cnt = 0.f;
+  for (int b = lane; b < nblocks; b += 32) {
+    ps += part[(size_t)b * 2 * N + e];
+    cnt += part[(size_t)b * 2 * N + N + e];
   }
-  sp[threadIdx.x] = ps;
-  sc[threadIdx.x] = cnt;
-  __syncthreads();
-  for (int o = 512; o > 0; o >>= 1) {
-    if (threadIdx.x < o) {
-      sp[threadIdx.x] += sp[threadIdx.x + o];
-      sc[threadIdx.x] += sc[threadIdx.x + o];
-    }
-    __syncthreads();
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    ps += __shfl_xor_sync(0xffffffffu, ps, o);
+    cnt += __shfl_xor_sync(0xffffffffu, cnt, o);
   }
-  if (threadIdx.x == 0) {
+  if (lane == 0) {
     const float denom = (f_mode == 0) ? (float)tokens : (float)tokens * (float)k;
-    F[e] = tokens > 0 ? (float)sc[0] / denom : 0.f;
-    P[e] = tokens > 0 ? sp[0] / (float)tokens : 0.f;
+    F[e] = tokens > 0 ? cnt / denom : 0.f;
+    P[e] = tokens > 0 ? ps / (float)tokens : 0.f;
+    raw[e] = ps;
+    raw[N + e] = cnt;
   }
 }
 
@@ -202,6 +251,29 @@ __global__ void aux_loss_kernel(const float* __restrict__ Fs, const float* __res
   }
 }
 
+// Eq. 8-9 over a batch that is spread over several shards: `psum`, `count` are the shards' sums added up,
+// `total_tokens` the size of the whole batch.  Leaves F, P of the whole batch and its token count in the workspace,
+// where the backward pass picks them up for the gradient of the auxiliary loss.
+__global__ void aux_loss_global_kernel(const float* __restrict__ psum, const float* __restrict__ count,
+                                       long long total_tokens, int N, int k, int f_mode, float coef, float* ws_F,
+                                       float* ws_P, long long* ws_tokens, float* loss, float* F, float* P) {
+  if (threadIdx.x == 0 && blockIdx.x == 0) {
+    const float tt = (float)total_tokens;
+    const float denom = f_mode == 0 ? tt : tt * (float)k;
+    float acc = 0.f;
+    for (int e = 0; e < N; ++e) {
+      const float fe = count[e] / denom, pe = psum[e] / tt;
+      acc += fe * pe;
+      ws_F[e] = fe;
+      ws_P[e] = pe;
+      if (F) F[e] = fe;
+      if (P) P[e] = pe;
+    }
+    *ws_tokens = total_tokens;
+    *loss = coef * (float)N * acc;
+  }
+}
+
 // ---- dispatch ---------------------------------------------------------------------------
 // Step 1: slots per expert inside each block of kRouteBlockTokens tokens.
 __global__ void __launch_bounds__(kRouteBlockTokens)
@@ -211,7 +283,7 @@ dispatch_count_kernel(const int* __restrict__ expert_idx, int* __restrict__ blk_
   __syncthreads();
   const int t = blockIdx.x * kRouteBlockTokens + threadIdx.x;
   if (t < tokens)
-    for (int j = 0; j < k; ++j) atomicAdd(&cnt[expert_idx[(size_t)t * k + j]], 1);
+    for (int j = 0; j < k; ++j) atomicAdd(&cnt[expert_idx[(size_t)t * k + j]], 1);   // the router's indices: valid, distinct
   __syncthreads();
   if (threadIdx.x < N) blk_counts[blockIdx.x * N + threadIdx.x] = cnt[threadIdx.x];
 }
@@ -346,31 +418,31 @@ cudaError_t launch_router_t(const Ctx& c) {
   int* idx = c.at<int>(c.L.expert_idx);
   float* gates = c.at<float>(c.L.gates);
   uint8_t* flags = c.at<uint8_t>(c.L.low_margin);
+  int blocks = 0;
 #define MIXLORA_ROUTER_LAUNCH(NE, TOK)                                                                         \
   {                                                                                                            \
-    int warps = (s.tokens + TOK - 1) / TOK;                                                                    \
-    int blocks = (warps + kWarpsPerBlock - 1) / kWarpsPerBlock;                                                \
-    router_kernel<T, NE, TOK><<<blocks, kWarpsPerBlock * 32, 0, c.st>>>(                                       \
-        x, c.p.w_router, c.p.router_bias, probs, idx, gates, flags, s.tokens, s.d_model, s.n_experts, s.top_k, \
-        s.renormalize);                                                                                        \
+    blocks = (s.tokens + kRWarps * TOK - 1) / (kRWarps * TOK);                                                 \
+    router_kernel<T, NE, TOK><<<blocks, kRWarps * 32, 0, c.st>>>(                                              \
+        x, c.p.w_router, c.p.router_bias, probs, idx, gates, flags, c.at<float>(c.L.stat_part), s.tokens,      \
+        s.d_model, s.n_experts, s.top_k, s.renormalize, s.aux_f_mode);                                         \
   }
-  if (s.n_experts <= 8) MIXLORA_ROUTER_LAUNCH(8, 2)
-  else if (s.n_experts <= 16) MIXLORA_ROUTER_LAUNCH(16, 2)
-  else MIXLORA_ROUTER_LAUNCH(32, 1)
+  if (s.n_experts <= 8) MIXLORA_ROUTER_LAUNCH(8, 4)
+  else if (s.n_experts <= 16) MIXLORA_ROUTER_LAUNCH(16, 4)
+  else MIXLORA_ROUTER_LAUNCH(32, 2)
 #undef MIXLORA_ROUTER_LAUNCH
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return e;
+  router_stats_kernel<<<1, 1024, 0, c.st>>>(c.at<float>(c.L.stat_part), blocks, c.at<float>(c.L.stat_F),
+                                            c.at<float>(c.L.stat_P), c.at<float>(c.L.stat_raw), s.tokens, s.n_experts,
+                                            s.top_k, s.aux_f_mode);
   return cudaGetLastError();
 }
 
 }  // namespace
 
-cudaError_t launch_router(const Ctx& c) {
-  cudaError_t e = c.bf16 ? launch_router_t<bf16>(c) : launch_router_t<float>(c);
-  if (e != cudaSuccess) return e;
-  router_stats_kernel<<<c.s.n_experts, 1024, 0, c.st>>>(c.at<float>(c.L.probs), c.at<int>(c.L.expert_idx),
-                                                       c.at<float>(c.L.stat_F), c.at<float>(c.L.stat_P), c.s.tokens,
-                                                       c.s.n_experts, c.s.top_k, c.s.aux_f_mode);
-  return cudaGetLastError();
-}
+int router_part_blocks(int tokens) { return (tokens + kRWarps * 2 - 1) / (kRWarps * 2); }   // the smallest block
+
+cudaError_t launch_router(const Ctx& c) { return c.bf16 ? launch_router_t<bf16>(c) : launch_router_t<float>(c); }
 
 cudaError_t launch_dispatch(const Ctx& c) {
   const mixlora_shape_t& s = c.s;
@@ -410,6 +482,14 @@ cudaError_t launch_reduce_worklist(const Ctx& c, int out_rows, int tile_rows, in
 cudaError_t launch_aux_loss(const Ctx& c, float coef, float* loss, float* F, float* P) {
   aux_loss_kernel<<<1, 32, 0, c.st>>>(c.at<float>(c.L.stat_F), c.at<float>(c.L.stat_P), coef, c.s.n_experts, loss, F,
                                       P);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_aux_loss_global(const Ctx& c, float coef, const float* prob_sum, const float* count,
+                                   long long total_tokens, float* loss, float* F, float* P) {
+  aux_loss_global_kernel<<<1, 32, 0, c.st>>>(prob_sum, count, total_tokens, c.s.n_experts, c.s.top_k, c.s.aux_f_mode,
+                                             coef, c.at<float>(c.L.stat_F), c.at<float>(c.L.stat_P),
+                                             reinterpret_cast<long long*>(c.ws + c.L.status + 8), loss, F, P);
   return cudaGetLastError();
 }
 

@@ -55,7 +55,10 @@ static_count_kernel(const int* __restrict__ expert_idx, int* __restrict__ blk_co
   __syncthreads();
   const int t = blockIdx.x * kStaticBlockTokens + threadIdx.x;
   if (t < tokens)
-    for (int j = 0; j < k; ++j) atomicAdd(&cnt[expert_idx[(size_t)t * k + j]], 1);
+    for (int j = 0; j < k; ++j) {
+      const int e = expert_idx[(size_t)t * k + j];
+      if ((unsigned)e < (unsigned)N) atomicAdd(&cnt[e], 1);   // an index outside [0, N) is skipped, never followed
+    }
   __syncthreads();
   if (threadIdx.x < N) blk_counts[blockIdx.x * N + threadIdx.x] = cnt[threadIdx.x];
 }
@@ -101,6 +104,7 @@ static_scatter_kernel(const int* __restrict__ expert_idx, const int* __restrict_
 #pragma unroll
   for (int j = 0; j < MIXLORA_MAX_TOP_K; ++j) {
     mine[j] = (t < tokens && j < k) ? expert_idx[(size_t)t * k + j] : -1;
+    if ((unsigned)mine[j] >= (unsigned)N) mine[j] = -1;        // skipped, as in the count kernel
     rank[j] = 0;
   }
   for (int e = 0; e < N; ++e) {

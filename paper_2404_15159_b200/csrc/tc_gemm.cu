@@ -15,7 +15,9 @@
 
 #include <stdlib.h>
 
+#include <atomic>
 #include <mutex>
+#include <unordered_map>
 
 #include "common.cuh"
 #include "tc_ptx.cuh"
@@ -543,10 +545,37 @@ EncodeFn get_encode() {
 }
 
 // 2-D bf16 tensor [rows, cols] row-major with leading dimension ld (elements); box = [box_rows, box_cols].
+// A tensor map is a pure function of the address and the geometry, and the same few dozen (frozen weights, workspace
+// regions) come back on every call, so encoded maps are kept in a small table keyed by exactly those arguments.
+struct MapKey {
+  const void* ptr; long long rows, cols, ld; int box_rows, box_cols, swizzle;
+  bool operator==(const MapKey& o) const {
+    return ptr == o.ptr && rows == o.rows && cols == o.cols && ld == o.ld && box_rows == o.box_rows &&
+           box_cols == o.box_cols && swizzle == o.swizzle;
+  }
+};
+struct MapKeyHash {
+  size_t operator()(const MapKey& k) const {
+    size_t h = reinterpret_cast<size_t>(k.ptr) * 0x9E3779B97F4A7C15ull;
+    auto mix = [&](long long v) { h ^= (size_t)v + 0x9E3779B97F4A7C15ull + (h << 6) + (h >> 2); };
+    mix(k.rows); mix(k.cols); mix(k.ld); mix(k.box_rows); mix(k.box_cols); mix(k.swizzle);
+    return h;
+  }
+};
+std::mutex g_map_mu;
+std::unordered_map<MapKey, CUtensorMap, MapKeyHash> g_map_cache;
+constexpr size_t kMapCacheMax = 4096;
+
 bool encode_2d(CUtensorMap* map, const void* ptr, long long rows, long long cols, long long ld, int box_rows,
                int box_cols, int swizzle_bytes = 128) {
   EncodeFn fn = get_encode();
   if (!fn) return false;
+  const MapKey key{ptr, rows, cols, ld, box_rows, box_cols, swizzle_bytes};
+  {
+    std::lock_guard<std::mutex> lock(g_map_mu);
+    auto it = g_map_cache.find(key);
+    if (it != g_map_cache.end()) { *map = it->second; return true; }
+  }
   cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
   cuuint64_t strides[1] = {(cuuint64_t)ld * 2};
   cuuint32_t box[2] = {(cuuint32_t)box_cols, (cuuint32_t)box_rows};
@@ -557,7 +586,24 @@ bool encode_2d(CUtensorMap* map, const void* ptr, long long rows, long long cols
                                        : (swizzle_bytes == 64 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_32B),
                   CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-  return r == CUDA_SUCCESS;
+  if (r != CUDA_SUCCESS) return false;
+  std::lock_guard<std::mutex> lock(g_map_mu);
+  if (g_map_cache.size() >= kMapCacheMax) g_map_cache.clear();
+  g_map_cache.emplace(key, *map);
+  return true;
+}
+
+// cudaFuncSetAttribute(MaxDynamicSharedMemorySize) once per kernel and device
+constexpr int kMaxDev = 64;
+template <typename K>
+cudaError_t ensure_smem_attr(K kernel, bool (&done)[kMaxDev], uint32_t bytes) {
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  if (dev >= 0 && dev < kMaxDev && done[dev]) return cudaSuccess;
+  e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+  if (e == cudaSuccess && dev >= 0 && dev < kMaxDev) done[dev] = true;   // a race only repeats the call
+  return e;
 }
 
 int round_up(int v, int a) { return (v + a - 1) / a * a; }
@@ -596,10 +642,12 @@ bool tc_gemm_supported(int M, const TcOut* outs, int nout) {
   return true;
 }
 
+namespace {
+
 template <int A_MN, int B_KN>
 cudaError_t launch_variant(const TcParams& p, int grid, cudaStream_t st) {
-  // the attribute is per function and per device; cheap enough to repeat on every launch
-  cudaError_t e = cudaFuncSetAttribute(tc_gemm_kernel<A_MN, B_KN>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+  static bool done[kMaxDev] = {false};
+  cudaError_t e = ensure_smem_attr(tc_gemm_kernel<A_MN, B_KN>, done, kSmemBytes);
   if (e != cudaSuccess) return e;
   tc_gemm_kernel<A_MN, B_KN><<<grid, kThreads, kSmemBytes, st>>>(p);
   return cudaGetLastError();
@@ -607,7 +655,8 @@ cudaError_t launch_variant(const TcParams& p, int grid, cudaStream_t st) {
 
 template <int A_MN, int B_KN>
 cudaError_t launch_pair_variant(const TcParams& p, int grid, cudaStream_t st) {
-  cudaError_t e = cudaFuncSetAttribute(tc_gemm_pair_kernel<A_MN, B_KN>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes2);
+  static bool done[kMaxDev] = {false};
+  cudaError_t e = ensure_smem_attr(tc_gemm_pair_kernel<A_MN, B_KN>, done, kSmemBytes2);
   if (e != cudaSuccess) return e;
   cudaLaunchConfig_t cfg;
   memset(&cfg, 0, sizeof(cfg));
@@ -625,14 +674,40 @@ cudaError_t launch_pair_variant(const TcParams& p, int grid, cudaStream_t st) {
   return cudaLaunchKernelEx(&cfg, tc_gemm_pair_kernel<A_MN, B_KN>, p);
 }
 
-// CTA pairs are used whenever the problem has at least 256 rows; MIXLORA_TC_SINGLE=1 in the environment keeps the
-// single-CTA kernel for every shape (a measurement switch, read once)
+// CTA pairs are used whenever the problem has at least 256 rows; the option MIXLORA_OPT_TC_SINGLE keeps the
+// single-CTA kernel for every shape (a measurement switch; MIXLORA_TC_SINGLE=1 in the environment sets its default)
+std::atomic<int> g_force_single{-1};
 bool tc_force_single() {
-  static const bool v = [] {
+  int v = g_force_single.load(std::memory_order_relaxed);
+  if (v < 0) {
     const char* e = getenv("MIXLORA_TC_SINGLE");
-    return e && e[0] == '1';
-  }();
-  return v;
+    v = (e && e[0] == '1') ? 1 : 0;
+    g_force_single.store(v, std::memory_order_relaxed);
+  }
+  return v != 0;
+}
+
+// A kernel whose only job is to let a bounded wait run out: one thread waits, with the given limit, on an mbarrier
+// that nothing arrives on (no copy is in flight, nothing else is touched) and records the status the production
+// kernels record in that case.
+__global__ void wait_timeout_selftest_kernel(int* status, uint32_t limit) {
+  __shared__ uint64_t bar;
+  __shared__ int abort_flag;
+  if (threadIdx.x == 0) {
+    abort_flag = 0;
+    mbar_init(smem_u32(&bar), 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    if (!mbar_wait_limit(smem_u32(&bar), 0, &abort_flag, limit)) atomicExch(status, (int)MIXLORA_ERR_DEVICE_TIMEOUT);
+  }
+}
+
+}  // namespace
+
+void tc_set_force_single(int v) { g_force_single.store(v ? 1 : 0, std::memory_order_relaxed); }
+
+cudaError_t launch_wait_timeout_selftest(int* status, unsigned limit, cudaStream_t st) {
+  wait_timeout_selftest_kernel<<<1, 32, 0, st>>>(status, limit);
+  return cudaGetLastError();
 }
 
 int tc_gemm_tile_rows(int M) { return (!tc_force_single() && M >= 2 * BM) ? 2 * BM : BM; }

@@ -12,6 +12,7 @@ import ctypes as C
 import numpy as np
 import pytest
 
+from oracle import mixlora_oracle as orc
 from paper_2404_15159_b200 import synth
 
 pytestmark = pytest.mark.gpu
@@ -50,6 +51,52 @@ def test_static_dispatch_matches_the_workspace_path_on_two_calls_in_a_row():
         assert torch.equal(perm, ref["perm"]), w.name
         assert torch.equal(seg_off, ref["seg_off"]), w.name
         assert sorted(perm.cpu().tolist()) == list(range(w.tokens * w.top_k))
+        want = orc.dispatch(ref["expert_idx"].cpu().numpy(), w.n_experts)        # and the oracle's dispatch directly
+        np.testing.assert_array_equal(perm.cpu().numpy(), want["perm"])
+        np.testing.assert_array_equal(seg_off.cpu().numpy(), want["seg_off"])
+
+
+def test_static_dispatch_at_its_stated_maximum_and_with_the_larger_problem_second():
+    # 65536 tokens, 32 experts, top-8: the whole fixed scratch is in use (256 blocks x 32 experts, both tables).
+    # A small problem runs first on the same stream, so the large one starts from a scratch that holds leftovers.
+    import torch
+    from paper_2404_15159_b200 import binding as B
+
+    rng = np.random.default_rng(7)
+    cases = []
+    for tokens, N, k in ((700, 6, 3), (B.mixlora_dispatch_static_max_tokens(), 32, 8)):
+        keys = rng.random((tokens, N))
+        idx = np.argsort(keys, axis=1)[:, :k].astype(np.int32)                  # k distinct experts per token
+        cases.append((tokens, N, k, idx))
+    outs = []
+    for tokens, N, k, idx in cases:
+        dev_idx = torch.from_numpy(idx).cuda()
+        perm = torch.full((tokens * k,), -1, dtype=torch.int32, device="cuda")
+        seg = torch.full((N + 1,), -1, dtype=torch.int32, device="cuda")
+        outs.append((dev_idx, perm, seg))
+    for (tokens, N, k, idx), (dev_idx, perm, seg) in zip(cases, outs):
+        B.mixlora_dispatch_static(dev_idx, tokens, N, k, perm, seg)
+    torch.cuda.synchronize()
+    for (tokens, N, k, idx), (dev_idx, perm, seg) in zip(cases, outs):
+        flat = idx.reshape(-1)
+        want_perm = np.argsort(flat, kind="stable").astype(np.int32)            # expert ascending, slot ascending
+        want_seg = np.concatenate([[0], np.cumsum(np.bincount(flat, minlength=N))]).astype(np.int32)
+        np.testing.assert_array_equal(perm.cpu().numpy(), want_perm)
+        np.testing.assert_array_equal(seg.cpu().numpy(), want_seg)
+
+
+def test_static_dispatch_skips_indices_outside_the_expert_range():
+    import torch
+    from paper_2404_15159_b200 import binding as B
+
+    idx = np.array([[0, 1], [2, 9], [-3, 1], [1, 0]], np.int32)               # 9 and -3 are not experts of N = 3
+    dev_idx = torch.from_numpy(idx).cuda()
+    perm = torch.full((8,), -1, dtype=torch.int32, device="cuda")
+    seg = torch.full((4,), -1, dtype=torch.int32, device="cuda")
+    B.mixlora_dispatch_static(dev_idx, 4, 3, 2, perm, seg)
+    torch.cuda.synchronize()
+    assert seg.cpu().tolist() == [0, 2, 5, 6]
+    assert perm.cpu().tolist() == [0, 7, 1, 5, 6, 2, -1, -1]                   # skipped slots leave the tail untouched
 
 
 def test_static_dispatch_rejects_sizes_beyond_its_fixed_scratch():
