@@ -204,10 +204,6 @@ def test_auxiliary_loss_of_the_whole_batch_over_two_shards(f_mode):
     coef = 0.5
     t = synth.generate(w)
     params_np = synth.params_of(t)
-    y_ref, saved = orc.ffn_forward(t["x"], params_np, w.top_k, w.lora_alpha)
-    assert saved["route"]["margin"].min() > helpers.ROUTE_MARGIN
-    loss_ref, F_ref, P_ref = orc.aux_loss(saved["route"]["probs"], saved["route"]["expert_idx"], coef, f_mode)
-    g_ref = orc.ffn_backward(t["x"], params_np, t["dy"], saved, aux_coef=coef, aux_f_mode=f_mode)
     dev = {n: (None if v is None else torch.from_numpy(np.ascontiguousarray(v, np.float32)).cuda()) for n, v in t.items()}
     cuts = [(0, 113), (113, 300)]
     state = []
@@ -225,6 +221,19 @@ def test_auxiliary_loss_of_the_whole_batch_over_two_shards(f_mode):
         psum += ps
         cnt += c
         state.append((shape, params, ws, y))
+    torch.cuda.synchronize()
+    # the oracle on the whole batch; a token whose deciding logit gap is below the flag threshold may keep the
+    # library's choice when that choice is one the near tie allows
+    gpu_idx = np.concatenate([B.mixlora_routing_view(st[0], st[2])["expert_idx"].cpu().numpy() for st in state])
+    y_ref, saved = orc.ffn_forward(t["x"], params_np, w.top_k, w.lora_alpha)
+    route = saved["route"]
+    diff = (gpu_idx != route["expert_idx"]).any(axis=1)
+    assert not (diff & (route["margin"] >= helpers.ROUTE_MARGIN)).any()
+    if diff.any():
+        helpers.assert_near_tie(route["logits"], route["expert_idx"], gpu_idx, diff, helpers.ROUTE_MARGIN)
+        y_ref, saved = orc.ffn_forward(t["x"], params_np, w.top_k, w.lora_alpha, forced_expert_idx=gpu_idx)
+    loss_ref, F_ref, P_ref = orc.aux_loss(saved["route"]["probs"], saved["route"]["expert_idx"], coef, f_mode)
+    g_ref = orc.ffn_backward(t["x"], params_np, t["dy"], saved, aux_coef=coef, aux_f_mode=f_mode)
     total = {n: None for n in helpers.GRAD_NAMES}
     dx = np.zeros_like(t["x"], dtype=np.float32)
     for (b, e), (shape, params, ws, y) in zip(cuts, state):
