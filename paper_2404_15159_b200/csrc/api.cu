@@ -79,8 +79,10 @@ WsLayout ws_layout(const mixlora_shape_t& s) {
   L.p_s = take(T * k * rp * E);
   L.dZd_pos = take(T * k * N * r * E);
   L.dgate_part = take((size_t)grouped_swiglu_bwd_col_tiles(s.d_ff) * T * k * 4);
-  L.dzg_all = take(T * k * N * r * E);
-  L.dzu_all = take(T * k * N * r * E);
+  const bool fold_dz = grouped_bwd_folds_dz(s);
+  L.dzg_all = take(fold_dz ? 0 : T * k * N * r * E);
+  L.dzu_all = take(fold_dz ? 0 : T * k * N * r * E);
+  L.dz_part = take(fold_dz ? (size_t)grouped_bwd_max_groups(s.tokens, s.d_ff) * T * k * 2 * r * 4 : 0);
   L.dZg = take(T * N * r * E);
   L.dZu = take(T * N * r * E);
   L.dgate = take(T * k * 4);
@@ -736,8 +738,9 @@ static mixlora_status_t bwd_experts(const Ctx& c, const void* dy, float aux_coef
       return MIXLORA_ERR_CUDA;                                  \
     }                                                           \
   } while (0)
-  // dzg = da (s B_g), dzu = db (s B_u), against every expert (the slot's own block is used)
-  {
+  // dzg = da (s B_g), dzu = db (s B_u), against every expert (the slot's own block is used); not when the grouped
+  // kernel above has formed them from the tiles it held
+  if (!grouped_bwd_folds_dz(c.s)) {
     TcOut outs[2];
     outs[0] = tc_out(c.ws + c.L.dzg_all, Nr, Nr); tc_add(outs[0], c.ws + c.L.da_sorted, f, f, c.ws + c.L.bg_cat, Nr, 1);
     outs[1] = tc_out(c.ws + c.L.dzu_all, Nr, Nr); tc_add(outs[1], c.ws + c.L.db_sorted, f, f, c.ws + c.L.bu_cat, Nr, 1);

@@ -49,7 +49,8 @@ struct WsLayout {
   size_t adp;         // act [N*pad_rank(r), f]  A_d with each expert's rows zero padded (same condition)
   size_t h_sorted;    // act [T*k, f]
   size_t hbar;        // act [T, f]        sum_j g_j h_j
-  size_t work_count;  // i32 [8]  item counts of the work lists below
+  size_t work_count;  // i32 [8]  item counts of the work lists below; [3] = column groups the backward grouped
+                      //          kernel used (rows of dz_part)
   size_t work_rows1;  // i32 [.., 8]  rows list with one output (A_d h)
   size_t total_fwd;
   size_t D;           // act [T, f]        dy W_d
@@ -60,7 +61,9 @@ struct WsLayout {
   size_t p_s;                   // act [T*k, pad_rank(r)]  s * pd of the slot's own expert, zero padded
   size_t dZd_pos;               // act [T*k, N*r]  gate * P_pos
   size_t dgate_part;            // f32 [ceil(f/64), T*k]  per column tile partial <Dt, h> of the fused backward
-  size_t dzg_all, dzu_all;      // act [T*k, N*r]  da (s B_g) and db (s B_u) against every expert
+  size_t dzg_all, dzu_all;      // act [T*k, N*r]  da (s B_g) and db (s B_u) against every expert (not when the
+                                //                 grouped kernel forms them, see dz_part)
+  size_t dz_part;               // f32 [groups, T*k, 2, r]  per column group: dzg, dzu of the slot's own expert
   size_t dZg, dZu;    // act [T, N*r]      dzg / dzu scattered dense
   size_t dgate;       // f32 [T*k]         by slot id
   size_t dlogits;     // f32 [T, N]
@@ -84,6 +87,28 @@ static inline int round_up8(int v) { return (v + 7) / 8 * 8; }
 static inline int pad_rank(int r) { return r <= 16 ? 16 : (r <= 32 ? 32 : (r <= 64 ? 64 : 128)); }
 
 WsLayout ws_layout(const mixlora_shape_t& s);
+
+// Column tiles of the backward grouped SwiGLU kernel (64 columns each) and the widest group of them whose pieces of
+// G, U and D (tokens x columns x 3 matrices) stay well inside L2 while every segment tile of the group is worked on.
+static inline int grouped_bwd_col_tiles(int f) { return (f + 63) / 64; }
+static inline int grouped_bwd_col_group_max(int tokens, int f) {
+  const long long cols = (32ll << 20) / ((long long)(tokens > 0 ? tokens : 1) * 2 * 3);
+  const long long g = cols / 64;
+  const int ct = grouped_bwd_col_tiles(f);
+  return (int)(g < 1 ? 1 : (g > ct ? ct : g));
+}
+// The backward grouped kernel also forms dzg = da (s B_g), dzu = db (s B_u) of a slot's own expert (summed over the
+// column tiles of a group in TMEM, one fp32 partial per group) when the rank divides a 64-column operand block and
+// the groups are wide enough for the partials to be small beside da, db themselves.
+static inline bool grouped_bwd_folds_dz(const mixlora_shape_t& s) {
+  return s.dtype == MIXLORA_DTYPE_BF16 && s.tokens > 0 && (s.rank == 8 || s.rank == 16 || s.rank == 32) &&
+         grouped_bwd_col_group_max(s.tokens, s.d_ff) >= 4 && (long long)s.tokens * s.d_ff < (1ll << 31);
+}
+// the kernel may narrow the groups down to half the widest to even out the CTAs' shares: bound of the group count
+static inline int grouped_bwd_max_groups(int tokens, int f) {
+  const int cg_min = (grouped_bwd_col_group_max(tokens, f) + 1) / 2;
+  return (grouped_bwd_col_tiles(f) + cg_min - 1) / cg_min;
+}
 
 static inline size_t act_size(const mixlora_shape_t& s) { return s.dtype == MIXLORA_DTYPE_BF16 ? 2 : 4; }
 

@@ -409,19 +409,44 @@ __global__ void dgate_reduce_kernel(const float* __restrict__ part, const int* _
 }
 
 // dabar_t = sum_j da_tj, dbbar_t = sum_j db_tj ; dZg / dZu = dzg / dzu scattered to the expert block
+// With `dz_part` (the grouped backward kernel's per-column-group partial sums [groups, slots, 2, r] of the slot's
+// own expert) dzg / dzu are those partials added up in group order; else they are read from dzg_sorted / dzu_sorted.
 template <typename T>
 __global__ void __launch_bounds__(ENT)
 combine_bwd_kernel(const T* __restrict__ da_sorted, const T* __restrict__ db_sorted, const T* __restrict__ dzg_sorted,
-                   const T* __restrict__ dzu_sorted, const int* __restrict__ inv, const int* __restrict__ expert_idx,
-                   T* __restrict__ dabar, T* __restrict__ dbbar, T* __restrict__ dZg, T* __restrict__ dZu, int f, int N,
-                   int r, int k, int want_dx) {
+                   const T* __restrict__ dzu_sorted, const float* __restrict__ dz_part,
+                   const int* __restrict__ dz_groups, int slots, const int* __restrict__ inv,
+                   const int* __restrict__ expert_idx, T* __restrict__ dabar, T* __restrict__ dbbar,
+                   T* __restrict__ dZg, T* __restrict__ dZu, int f, int N, int r, int k, int want_dx) {
   const int t = blockIdx.x;
   __shared__ int pos[MIXLORA_MAX_TOP_K], ex[MIXLORA_MAX_TOP_K];
+  __shared__ float dzs[MIXLORA_MAX_TOP_K * 2 * 32];    // fold mode (r <= 32): [slot of the token][dzg, dzu][r]
   if (threadIdx.x < k) {
     pos[threadIdx.x] = inv[(size_t)t * k + threadIdx.x];
     ex[threadIdx.x] = expert_idx[(size_t)t * k + threadIdx.x];
   }
   __syncthreads();
+  if (dz_part) {
+    // one thread per value of the token's slots; a warp's loads of one group are contiguous
+    const int groups = *dz_groups;
+    const size_t gstride = (size_t)slots * 2 * r;
+    for (int i = threadIdx.x; i < k * 2 * r; i += blockDim.x) {
+      const int j = i / (2 * r);
+      const float* src = dz_part + (size_t)pos[j] * 2 * r + (i - j * 2 * r);
+      float sum = 0.f;
+      int g = 0;
+      for (; g + 8 <= groups; g += 8) {                // eight groups' loads in flight; the sum keeps group order
+        float tv[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) tv[u] = __ldg(src + (size_t)(g + u) * gstride);
+#pragma unroll
+        for (int u = 0; u < 8; ++u) sum += tv[u];
+      }
+      for (; g < groups; ++g) sum += __ldg(src + (size_t)g * gstride);
+      dzs[i] = sum;
+    }
+    __syncthreads();
+  }
   for (int c = threadIdx.x; want_dx && c < f; c += ENT) {
     float sa = 0.f, sb = 0.f;
     for (int j = 0; j < k; ++j) {
@@ -437,8 +462,13 @@ combine_bwd_kernel(const T* __restrict__ da_sorted, const T* __restrict__ db_sor
     T vg = from_f<T>(0.f), vu = from_f<T>(0.f);
     for (int j = 0; j < k; ++j)
       if (ex[j] == e) {
-        vg = dzg_sorted[(size_t)pos[j] * nr + q];
-        vu = dzu_sorted[(size_t)pos[j] * nr + q];
+        if (dz_part) {
+          vg = from_f<T>(dzs[j * 2 * r + rr]);
+          vu = from_f<T>(dzs[j * 2 * r + r + rr]);
+        } else {
+          vg = dzg_sorted[(size_t)pos[j] * nr + q];
+          vu = dzu_sorted[(size_t)pos[j] * nr + q];
+        }
       }
     dZg[(size_t)t * nr + q] = vg;
     dZu[(size_t)t * nr + q] = vu;
@@ -618,7 +648,8 @@ cudaError_t combine_bwd_t(const Ctx& c, int want_dx) {
   constexpr bool vec = sizeof(T) == 2;
   combine_bwd_kernel<T><<<c.s.tokens, vec ? 128 : ENT, 0, c.st>>>(
       c.at<T>(c.L.da_sorted), c.at<T>(c.L.db_sorted), c.at<T>(c.L.dzg_all), c.at<T>(c.L.dzu_all),
-      c.at<int>(c.L.inv), c.at<int>(c.L.expert_idx), c.at<T>(c.L.dabar), c.at<T>(c.L.dbbar), c.at<T>(c.L.dZg),
+      grouped_bwd_folds_dz(c.s) ? c.at<float>(c.L.dz_part) : nullptr, c.at<int>(c.L.work_count) + 3,
+      c.s.tokens * c.s.top_k, c.at<int>(c.L.inv), c.at<int>(c.L.expert_idx), c.at<T>(c.L.dabar), c.at<T>(c.L.dbbar), c.at<T>(c.L.dZg),
       c.at<T>(c.L.dZu), c.s.d_ff, c.s.n_experts, c.s.rank, c.s.top_k, vec ? 0 : want_dx);
   return cudaGetLastError();
 }

@@ -17,7 +17,16 @@
 // The TMA stores of these 128-byte-wide boxes drain at about 15 cycles per row and SM, which paces the kernel; both
 // other ways out (coalesced stores from the smem tile, 32-byte stores straight from the registers) measured slower.
 // All waits are bounded as in the dense product.
+//
+// Backward with FOLD: the kernel also forms the rank-r gradients dzg = da (s B_g[e]), dzu = db (s B_u[e]) of every
+// slot.  A CTA then takes units of work (one segment tile x one group of column tiles) instead of single items and
+// walks the unit's column tiles in turn; after the barrier of an item the store warp's thread multiplies the da and
+// db tiles, still in shared memory, with the matching 64 x 64 blocks of s B_g, s B_u (all experts' blocks side by
+// side, so the block holds the tile's expert) into two accumulators of 64 TMEM columns that live for the whole unit.
+// At the unit's end eight epilogue warps write the expert's own r columns as one fp32 partial per column group; a
+// later kernel adds the groups in a fixed order.  da and db are then not read again for this product.
 #include <algorithm>
+#include <type_traits>
 
 #include "common.cuh"
 #include "tc_ptx.cuh"
@@ -44,6 +53,8 @@ constexpr int kMaxStages = 4;
 constexpr int kMaxSets = 4;               // gathered tiles in flight per CTA
 constexpr int kHdrFloats = 128 + 4;       // per set: gates of the 128 rows, first slot, row count, column tile
 constexpr uint32_t kBlockBytes = 128 * 128;   // one 64-column block of a 128-row tile
+constexpr uint32_t kDzbBytes = 64 * 128;      // one 64 x 64 block of s B_g or s B_u
+constexpr int kUnitsAlways = 0;               // 1: whole (segment tile, column group) units without the rank-r products too (measured: no gain)
 
 struct alignas(64) GsParams {
   CUtensorMap a_map[3];    // zg_s, zu_s, p_s : [slots, RP]
@@ -56,7 +67,67 @@ struct alignas(64) GsParams {
   int max_tiles, slots, f, r, row_bytes, kblocks, ksteps, krows, col_tiles, col_group, nstages, nsets, out_sets;
   uint32_t stage_bytes, a_bytes;
   int* status;
+  // FOLD only
+  CUtensorMap z_map[2];    // s B_g, s B_u with all experts' blocks side by side: [f, N r], boxes of 64 x 64
+  float* dz_part;          // [groups, slots, 2, r_true]
+  int* groups_used;        // the number of column groups the kernel settled on
+  int r_true, cg_min;
 };
+
+// The order in which a CTA takes (segment tile, column tile) items; every role of the CTA walks it the same way.
+//   items : groups of col_group column tiles; inside a group every segment tile in turn, its column tiles innermost;
+//           consecutive items go to consecutive CTAs.  The slots of a token (they sit in different experts' segments)
+//           are then worked on while the token's piece of G / U / D is still in L2, so DRAM sees each piece once.
+//   units : the same groups, but a CTA takes a whole (segment tile, group) and walks its column tiles itself.
+template <int UNITS>
+struct Walk {
+  int w;                                    // next item or unit of this CTA
+  int tile, ct, ct_end, group;              // units: the unit being walked
+  __device__ Walk() : w(blockIdx.x), tile(0), ct(0), ct_end(0), group(0) {}
+  // the next item: its segment tile and column tile, and whether it opens / closes a unit
+  __device__ __forceinline__ bool next(int ntiles, int col_tiles, int col_group, int& tile_o, int& ct_o, bool& first,
+                                       bool& last) {
+    if (!UNITS) {
+      if (w >= ntiles * col_tiles) return false;
+      const int per_group = ntiles * col_group;
+      const int g = w / per_group, rem = w - g * per_group;
+      const int gw = min(col_group, col_tiles - g * col_group);   // the last group may be narrower
+      tile_o = rem / gw;
+      ct_o = g * col_group + rem % gw;
+      first = last = false;
+      w += gridDim.x;
+      return true;
+    }
+    if (ct >= ct_end) {
+      const int groups = (col_tiles + col_group - 1) / col_group;
+      if (w >= ntiles * groups) return false;
+      group = w / ntiles;
+      tile = w - group * ntiles;
+      ct = group * col_group;
+      ct_end = min(ct + col_group, col_tiles);
+      w += gridDim.x;
+    }
+    tile_o = tile;
+    ct_o = ct;
+    first = ct == group * col_group;
+    last = ct == ct_end - 1;
+    ++ct;
+    return true;
+  }
+};
+
+// Width of the column groups in units mode: between cg_min and cg_max, the one that leaves the busiest CTA the
+// fewest items (a pure function of its arguments: every thread of every CTA gets the same answer).
+__device__ __forceinline__ int choose_col_group(int ntiles, int col_tiles, int cg_min, int cg_max, int ctas) {
+  int best = cg_max, best_cost = 0x7fffffff;
+  for (int cg = cg_max; cg >= cg_min && cg >= 1; --cg) {
+    const int groups = (col_tiles + cg - 1) / cg;
+    const int rounds = (ntiles * groups + ctas - 1) / ctas;
+    const int cost = rounds * cg;
+    if (cost < best_cost) { best_cost = cost; best = cg; }
+  }
+  return best;
+}
 
 // Packed fp32 pairs: one add / mul / fma instruction works on both halves of a 64-bit register pair, which halves
 // the issue slots of the element-wise math (the kernel is bound by instruction issue, not by a pipe).
@@ -108,7 +179,7 @@ __device__ __forceinline__ uint64_t sigmoid2(uint64_t a) {
   asm("tanh.approx.f32 %0, %1;" : "=f"(th) : "f"(hi));
   return fma2(pk2(tl, th), kHalf2, kHalf2);
 }
-template <int BWD>
+template <int BWD, int FOLD, int UNITS>
 __global__ void __launch_bounds__(kThreads, 1) grouped_swiglu_kernel(const __grid_constant__ GsParams p) {
   constexpr int COLS = BWD ? 64 : 128;
   constexpr int CB = COLS / 64;                        // 64-column blocks per tile
@@ -119,21 +190,30 @@ __global__ void __launch_bounds__(kThreads, 1) grouped_swiglu_kernel(const __gri
   constexpr uint32_t kSetBytes = NMAT * CB * kBlockBytes;
   constexpr uint32_t kOutBytes = NOUT * CB * kBlockBytes;
   constexpr int WCOLS = COLS / kSplit;                 // columns per epilogue thread
+  constexpr uint32_t kDzCol0 = 192, kDzCol1 = 448;     // TMEM columns of the dzg / dzu accumulators (64 each): the
+                                                       // backward's two buffers use columns 0-191 and 256-447
+                                                       // (dz_readout reads them back)
+  static_assert(!FOLD || (BWD && UNITS), "the rank-r gradients belong to the backward kernel and need units of work");
 
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   uint8_t* gather_smem = smem;                                    // nsets sets
   uint8_t* out_smem = gather_smem + p.nsets * kSetBytes;           // one or two output tiles
-  uint8_t* stage_smem = out_smem + p.out_sets * kOutBytes;
+  uint8_t* dzb_smem = out_smem + p.out_sets * kOutBytes;           // FOLD: the 64 x 64 blocks of s B_g, s B_u
+  uint8_t* stage_smem = dzb_smem + (FOLD ? 2 * kDzbBytes : 0);
   float* dg_smem = reinterpret_cast<float*>(stage_smem + p.nstages * p.stage_bytes);   // [2][kSplit][128]
   float* hdr_smem = dg_smem + (BWD ? 2 * kSplit * BM : 0);                              // [nsets][kHdrFloats]
   uint64_t* bars = reinterpret_cast<uint64_t*>(hdr_smem + p.nsets * kHdrFloats);
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * kMaxStages + 6 + 2 * kMaxSets);
+  constexpr int kNumBars = 2 * kMaxStages + 6 + 2 * kMaxSets + 4;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + kNumBars);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
   int* out_hdr = reinterpret_cast<int*>(tmem_slot + 4);   // [2][4]: first slot, rows, column tile of the item in each output tile's turn
   // [2], by item parity: a warp that runs ahead and gives up on the next item cannot change what the others read
   // after this item's barrier
   volatile int* epi_stop = reinterpret_cast<volatile int*>(tmem_slot + 2);
+  // FOLD: [gather warp][set][4]: each gather warp's own note of the item it put into a set (closes a unit / column
+  // group / expert's column offset, first slot, rows), read back by the same warp when the set returns
+  int* gnote = reinterpret_cast<int*>(tmem_slot + 12);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t stage_base = smem_u32(stage_smem);
@@ -145,6 +225,13 @@ __global__ void __launch_bounds__(kThreads, 1) grouped_swiglu_kernel(const __gri
   auto gfull_bar = [&](int b) { return bar_base + 8u * (2 * kMaxStages + 4 + b); };
   auto gempty_bar = [&](int b) { return bar_base + 8u * (2 * kMaxStages + 4 + kMaxSets + b); };
   auto ofree_bar = [&](int b) { return bar_base + 8u * (2 * kMaxStages + 4 + 2 * kMaxSets + b); };
+  // FOLD: the s B blocks of an item have landed; the item's rank-r products are done (they have read the output tile
+  // and the blocks); the accumulators of the finished unit have been read out
+  const uint32_t dzb_full_bar = bar_base + 8u * (2 * kMaxStages + 6 + 2 * kMaxSets);
+  const uint32_t dzdone_bar = dzb_full_bar + 8u, dzfree_bar = dzb_full_bar + 16u;
+  // FOLD: a unit's last rank-r products are done.  One arrival per unit, and the next unit cannot get there before
+  // this one's accumulators have been read out (dzfree), so a waiter that counts units never sees a later phase.
+  const uint32_t dzunit_bar = dzb_full_bar + 24u;
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < kMaxStages; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
@@ -154,6 +241,7 @@ __global__ void __launch_bounds__(kThreads, 1) grouped_swiglu_kernel(const __gri
     // a set is full when every gather thread's copies have landed (one asynchronous arrival each) and its header
     // is written (one plain arrival each); it is empty again when every epilogue warp has read it
     for (int b = 0; b < kMaxSets; ++b) { mbar_init(gfull_bar(b), 2 * NGT); mbar_init(gempty_bar(b), 4 * kSplit); }
+    mbar_init(dzb_full_bar, 1); mbar_init(dzdone_bar, 1); mbar_init(dzfree_bar, kGatherWarps); mbar_init(dzunit_bar, 1);
     *abort_flag = 0;
     epi_stop[0] = 0;
     epi_stop[1] = 0;
@@ -168,18 +256,12 @@ __global__ void __launch_bounds__(kThreads, 1) grouped_swiglu_kernel(const __gri
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
   const int ntiles = min(p.tile_info[p.max_tiles * 4], p.max_tiles);
-  const int total = ntiles * p.col_tiles;
   const int kb_cols = p.row_bytes / 2;                 // K elements per k-block (16, 32 or 64)
-  // Item order: groups of col_group column tiles, inside a group every segment tile in turn.  The slots of a token
-  // (they sit in different experts' segments) are then worked on while the token's piece of G / U / D is still in
-  // L2, so DRAM sees each piece once; inside a group the CTAs still sweep col_group tiles of the same rows together.
-  const int per_group = ntiles * p.col_group;
-  auto item_at = [&](int w, int& tile, int& ct) {
-    const int g = w / per_group, rem = w - g * per_group;
-    const int gw = min(p.col_group, p.col_tiles - g * p.col_group);   // the last group may be narrower
-    tile = rem / gw;
-    ct = g * p.col_group + rem % gw;
-  };
+  const int col_group = UNITS ? choose_col_group(ntiles, p.col_tiles, p.cg_min, p.col_group, (int)gridDim.x) : p.col_group;
+  if (FOLD && blockIdx.x == 0 && threadIdx.x == 0) *p.groups_used = (p.col_tiles + col_group - 1) / col_group;
+  Walk<UNITS> walk;
+  int tile, ct;
+  bool first, last;
 
   if (warp == 0) {
     // ---------------- producer: rank-r operands ----------------
@@ -187,9 +269,7 @@ __global__ void __launch_bounds__(kThreads, 1) grouped_swiglu_kernel(const __gri
       for (int s = 0; s < NSUB; ++s) { prefetch_tmap(&p.a_map[s]); prefetch_tmap(&p.b_map[s]); }
       uint32_t it = 0;
       bool ok = true;
-      for (int w = blockIdx.x; w < total && ok; w += gridDim.x) {
-        int tile, ct;
-        item_at(w, tile, ct);
+      while (ok && walk.next(ntiles, p.col_tiles, col_group, tile, ct, first, last)) {
         const int col0 = ct * COLS;
         const int e = p.tile_info[tile * 4 + 0], p0 = p.tile_info[tile * 4 + 1];
         for (int sub = 0; sub < NSUB && ok; ++sub) {
@@ -224,7 +304,7 @@ __global__ void __launch_bounds__(kThreads, 1) grouped_swiglu_kernel(const __gri
       uint32_t it = 0, wcount = 0;
       bool ok = true;
       const uint32_t idesc_k = make_idesc(COLS, 0, 0), idesc_n = make_idesc(COLS, 0, 1);
-      for (int w = blockIdx.x; w < total && ok; w += gridDim.x, ++wcount) {
+      for (; ok && walk.next(ntiles, p.col_tiles, col_group, tile, ct, first, last); ++wcount) {
         const uint32_t buf = wcount & 1u, use = wcount >> 1;
         if (!mbar_wait(tempty_bar(buf), (use & 1u) ^ 1u, abort_flag)) { ok = false; break; }
         tc_fence_after();
@@ -257,16 +337,34 @@ __global__ void __launch_bounds__(kThreads, 1) grouped_swiglu_kernel(const __gri
     // ---------------- store warp ----------------
     if (lane == 0) {
       for (int m = 0; m < NOUT; ++m) prefetch_tmap(&p.o_map[m]);
+      if (FOLD) { prefetch_tmap(&p.z_map[0]); prefetch_tmap(&p.z_map[1]); }
     }
     const uint32_t out_base = smem_u32(out_smem);
+    const uint32_t dzb_base = smem_u32(dzb_smem);
+    // FOLD: fetches the item's 64 x 64 blocks of s B_g, s B_u (rows = the tile's columns of the FFN width, columns =
+    // the 64-column block of the N r experts' columns that holds the tile's expert)
+    auto load_dzb = [&](int tile_, int ct_) {
+      const int e = p.tile_info[tile_ * 4 + 0];
+      const int zc = (e * p.r_true) / 64 * 64;
+      mbar_expect_tx(dzb_full_bar, 2 * kDzbBytes);
+      tma_load_2d(dzb_base, &p.z_map[0], dzb_full_bar, zc, ct_ * COLS);
+      tma_load_2d(dzb_base + kDzbBytes, &p.z_map[1], dzb_full_bar, zc, ct_ * COLS);
+    };
     int prev_o = -1;
-    uint32_t n = 0;
-    for (int w = blockIdx.x; w < total; w += gridDim.x, ++n) {
+    uint32_t n = 0, units_done = 0;
+    bool have = walk.next(ntiles, p.col_tiles, col_group, tile, ct, first, last);
+    bool dz_ok = true;                                 // lane 0 only: no bounded wait of the rank-r products gave up
+    if (FOLD && have && lane == 0) load_dzb(tile, ct);
+    for (; have; ++n) {
       named_barrier(1, NET + 32);                      // the item's results are complete in its output tile
       if (epi_stop[n & 1u]) break;
+      const bool cur_first = first, cur_last = last;
+      int ntile = 0, nct = 0;
+      have = walk.next(ntiles, p.col_tiles, col_group, ntile, nct, first, last);        // the item after this one (its s B blocks are fetched below)
       if (lane == 0) {
-        // every epilogue thread is past the previous item (also past copying a short tile out), and that item's
-        // TMA stores have read its tile (waited for below): the tile may be written again
+        // every epilogue thread is past the previous item (also past copying a short tile out), that item's
+        // TMA stores have read its tile and, with FOLD, so have its rank-r products (both waited for below):
+        // the tile may be written again
         if (prev_o >= 0) mbar_arrive(ofree_bar(prev_o));
         const int o = p.out_sets == 2 ? (int)(n & 1u) : 0;
         const int* hdr = reinterpret_cast<const int*>(out_hdr + 4 * (n & 1u));
@@ -279,9 +377,42 @@ __global__ void __launch_bounds__(kThreads, 1) grouped_swiglu_kernel(const __gri
               tma_store_2d(&p.o_map[m], out_base + o * kOutBytes + (m * CB + j) * kBlockBytes, col0 + j * 64, p0);
         }
         tma_store_commit();
+        if (FOLD && dz_ok) {
+          // dzg += da_tile (s B_g block), dzu += db_tile (s B_u block): A = the 128 x 64 tile just written (K-major,
+          // K = the tile's 64 columns), B = the 64 x 64 block as fetched ([K, N] row-major), four K-steps of 16
+          dz_ok = mbar_wait(dzb_full_bar, n & 1u, abort_flag);
+          if (dz_ok && cur_first) dz_ok = mbar_wait(dzfree_bar, (units_done & 1u) ^ 1u, abort_flag);
+          if (dz_ok) {
+            tc_fence_after();
+            const uint32_t idesc = make_idesc(64, 0, 1);
+#pragma unroll
+            for (int m = 0; m < 2; ++m) {
+              const uint32_t a_addr = out_base + o * kOutBytes + m * kBlockBytes;
+              const uint32_t b_addr = dzb_base + m * kDzbBytes;
+              const uint32_t d_tmem = tmem_base + (m == 0 ? kDzCol0 : kDzCol1);
+#pragma unroll
+              for (int k = 0; k < 4; ++k)
+                umma_bf16(d_tmem, make_desc_kmajor_rows(a_addr + k * 32, 128), make_desc(b_addr + k * 2048, 8192, 1024),
+                          idesc, (cur_first && k == 0) ? 0u : 1u);
+            }
+            umma_commit(dzdone_bar);
+          }
+        }
         tma_store_wait_read<0>();
+        if (FOLD) {
+          if (dz_ok) dz_ok = mbar_wait(dzdone_bar, n & 1u, abort_flag);
+          if (dz_ok && cur_last) mbar_arrive(dzunit_bar);   // the gather warps may read the unit's accumulators
+          if (dz_ok && have) load_dzb(ntile, nct);
+          if (!dz_ok) {
+            // everyone leaves at the next item's barrier (this warp still arrives there)
+            *abort_flag = 1;
+            if (p.status) atomicExch(p.status, (int)MIXLORA_ERR_DEVICE_TIMEOUT);
+            epi_stop[(n + 1) & 1u] = 1;
+          }
+        }
         prev_o = o;
       }
+      if (cur_last) ++units_done;
       if (p.out_sets == 1) {
         // a single output tile is handed back at once: after the copy has read it or, for a short tile, after
         // the epilogue threads have copied it out (they meet the store warp once more)
@@ -303,20 +434,53 @@ __global__ void __launch_bounds__(kThreads, 1) grouped_swiglu_kernel(const __gri
     const uint32_t g_dst0 = smem_u32(gather_smem) + g_r0 * 128 + ((g_cb ^ (g_r0 & 7)) << 4);
     int set = 0;
     uint32_t set_use = 0;                              // times the ring has wrapped
+    uint32_t gitem = 0;                                // items gathered so far
     bool ok = true;
-    for (int w = blockIdx.x; w < total; w += gridDim.x) {
+    // FOLD: the accumulators of a finished unit go out as that column group's partial: the expert's own r columns
+    // of dzg and dzu for this thread's row of the tile, then the accumulators are handed back to the store warp.
+    // `info`, `zp0`, `zrows` are the note of the unit's last item.  The wait is short: the store warp issues the
+    // item's rank-r products right behind the item's barrier, which the epilogue warps have reached (or are about
+    // to reach) when the item's gathered set comes back.
+    uint32_t gunits = 0;                               // units read out so far
+    auto dz_readout = [&](int info, int zp0, int zrows) {
+      if (!__all_sync(0xffffffffu, mbar_wait(dzunit_bar, gunits & 1u, abort_flag))) return false;
+      ++gunits;
+      tc_fence_after();
+      const int r = p.r_true;
+      const int zrow = (warp & 3) * 32 + lane;         // the TMEM lanes this warp may read
+      const uint32_t z_addr = tmem_base + ((uint32_t)((warp & 3) * 32) << 16) + (uint32_t)(info >> 16);
+      float* dst = p.dz_part + ((size_t)((info >> 1) & 0x7fff) * p.slots + zp0 + zrow) * 2 * r;
+      // 8 columns at a time: the expert's columns may end with the accumulator's (and TMEM's) last column
+      for (int m = 0; m < 2; ++m)
+        for (int c = 0; c < r; c += 8) {
+          uint32_t v[8];
+          tmem_ld8(z_addr + (m == 0 ? kDzCol0 : kDzCol1) + c, v);
+          tmem_ld_wait();
+          if (zrow < zrows) {
+            *reinterpret_cast<float4*>(dst + m * r + c) = make_float4(__uint_as_float(v[0]), __uint_as_float(v[1]),
+                                                                      __uint_as_float(v[2]), __uint_as_float(v[3]));
+            *reinterpret_cast<float4*>(dst + m * r + c + 4) = make_float4(__uint_as_float(v[4]), __uint_as_float(v[5]),
+                                                                          __uint_as_float(v[6]), __uint_as_float(v[7]));
+          }
+        }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(dzfree_bar);
+      return true;
+    };
+    while (walk.next(ntiles, p.col_tiles, col_group, tile, ct, first, last)) {
       // everything the item needs from global memory besides the rows themselves is fetched before the wait for
       // a free set, so those dependent loads never delay the copies
-      int tile, ct;
-      item_at(w, tile, ct);
       const int col0 = ct * COLS;
       const int p0 = p.tile_info[tile * 4 + 1], rows = p.tile_info[tile * 4 + 2];
       // rows past the tile's end and columns past f are clamped to valid data: what is computed from them is
       // never stored (kRowsPerPass is a multiple of 8, so the swizzle term of a thread's rows is constant)
-      size_t roff[kPasses];
+      // (with FOLD the element offsets fit 32 bits: the groups are only wide enough for it at modest token counts)
+      typename std::conditional<FOLD != 0, uint32_t, size_t>::type roff[kPasses];
 #pragma unroll
       for (int ps = 0; ps < kPasses; ++ps)
-        roff[ps] = (size_t)p.pos_token[p0 + min(g_r0 + kRowsPerPass * ps, rows - 1)] * p.f;
+        roff[ps] = (typename std::conditional<FOLD != 0, uint32_t, size_t>::type)
+                       p.pos_token[p0 + min(g_r0 + kRowsPerPass * ps, rows - 1)] * p.f;
       float gate0 = 0.f, gate1 = 0.f;                  // gates of rows gt and (fewer than 128 gather threads) gt + NGT
       if (BWD) {
         if (gt < rows) gate0 = p.gates[p.perm[p0 + gt]];
@@ -324,6 +488,21 @@ __global__ void __launch_bounds__(kThreads, 1) grouped_swiglu_kernel(const __gri
       }
       if (!mbar_wait(gempty_bar(set), (set_use & 1u) ^ 1u, abort_flag)) { ok = false; break; }
       float* hdr = hdr_smem + set * kHdrFloats;
+      // FOLD: the set that has just come back held the item nsets items ago, which is finished; this warp's note of
+      // it is still there.  If that item closed a unit, the unit's accumulators are read out below, once this
+      // item's copies are on their way.
+      int old_info = 0, old_p0 = 0, old_rows = 0;
+      int* note = gnote + ((warp - kFirstGatherWarp) * kMaxSets + set) * 4;
+      if (FOLD) {
+        if (gitem >= (uint32_t)p.nsets) { old_info = note[0]; old_p0 = note[1]; old_rows = note[2]; }
+        __syncwarp();
+        if (lane == 0) {
+          note[0] = (last ? 1 : 0) | (walk.group << 1) | (((p.tile_info[tile * 4 + 0] * p.r_true) & 63) << 16);
+          note[1] = p0;
+          note[2] = rows;
+        }
+        __syncwarp();
+      }
       if (BWD) {
         hdr[gt] = gate0;
         if (NGT < 128) hdr[gt + NGT] = gate1;
@@ -337,7 +516,8 @@ __global__ void __launch_bounds__(kThreads, 1) grouped_swiglu_kernel(const __gri
 #pragma unroll
       for (int j = 0; j < CB; ++j) {
         const int col = min(col0 + j * 64 + g_cb * 8, p.f - 8);
-        // D is zero-filled past column f: those columns must not add to the row's <Dt, h>
+        // D is zero-filled past column f: those columns must not add to the row's <Dt, h> (and, with D and the
+        // A_d product zero there, da and db come out as zero, so they add nothing to the rank-r products either)
         const uint32_t d_bytes = col0 + j * 64 + g_cb * 8 < p.f ? 16u : 0u;
 #pragma unroll
         for (int m = 0; m < NMAT; ++m) {
@@ -358,7 +538,19 @@ __global__ void __launch_bounds__(kThreads, 1) grouped_swiglu_kernel(const __gri
       }
       asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];" ::"r"(gfull_bar(set)) : "memory");
       mbar_arrive(gfull_bar(set));                     // publishes the header
+      if (FOLD && (old_info & 1) && !dz_readout(old_info, old_p0, old_rows)) { ok = false; break; }
+      if (FOLD) ++gitem;
       if (++set == p.nsets) { set = 0; ++set_use; }
+    }
+    if (FOLD && ok) {
+      // the last nsets items (fewer if the CTA had fewer): their records are still in the ring, oldest first
+      const uint32_t left = gitem < (uint32_t)p.nsets ? gitem : (uint32_t)p.nsets;
+      if (gitem < (uint32_t)p.nsets) set = 0;
+      for (uint32_t i = gitem - left; i < gitem && ok; ++i) {
+        const int* note = gnote + ((warp - kFirstGatherWarp) * kMaxSets + set) * 4;
+        if ((note[0] & 1) && !dz_readout(note[0], note[1], note[2])) ok = false;
+        if (++set == p.nsets) set = 0;
+      }
     }
     asm volatile("cp.async.wait_all;" ::: "memory");
     if (!ok && lane == 0) {
@@ -375,17 +567,26 @@ __global__ void __launch_bounds__(kThreads, 1) grouped_swiglu_kernel(const __gri
     const int jblk = (part * (WCOLS / 8)) >> 3, cb0 = (part * (WCOLS / 8)) & 7, rx = row & 7;
     const uint32_t row_off = jblk * kBlockBytes + row * 128;
 
-    uint32_t wcount = 0;
+    // the items of this CTA are only counted here: what an item is comes with its gathered set's header
+    uint32_t n_items = 0;
+    if (UNITS) {
+      const int groups = (p.col_tiles + col_group - 1) / col_group;
+      for (int u = blockIdx.x; u < ntiles * groups; u += gridDim.x)
+        n_items += min(col_group, p.col_tiles - (u / ntiles) * col_group);
+    } else {
+      const int total = ntiles * p.col_tiles;
+      n_items = (int)blockIdx.x < total ? (total - blockIdx.x + gridDim.x - 1) / gridDim.x : 0;
+    }
     int set = 0;
     uint32_t set_use = 0;
-    for (int w = blockIdx.x; w < total; w += gridDim.x, ++wcount) {
+    for (uint32_t wcount = 0; wcount < n_items; ++wcount) {
       const uint32_t buf = wcount & 1u, use = wcount >> 1;
       const int oidx = p.out_sets == 2 ? (int)buf : 0;  // output tile of this item
       const uint32_t o_use = p.out_sets == 2 ? use : wcount;
       const bool got = __all_sync(0xffffffffu, mbar_wait(gfull_bar(set), set_use & 1u, abort_flag) &&
                                                    mbar_wait(tfull_bar(buf), use & 1u, abort_flag) &&
                                                    mbar_wait(ofree_bar(oidx), (o_use & 1u) ^ 1u, abort_flag));
-      int ct = 0, pos = 0, p0 = 0, rows = 0;
+      int pos = 0, p0 = 0, rows = 0, ct = 0;
       if (got) {
         tc_fence_after();
         const float* hdr = hdr_smem + set * kHdrFloats;
@@ -463,7 +664,7 @@ __global__ void __launch_bounds__(kThreads, 1) grouped_swiglu_kernel(const __gri
         *abort_flag = 1;
         if (p.status) atomicExch(p.status, (int)MIXLORA_ERR_DEVICE_TIMEOUT);
       }
-      fence_proxy_async_smem();                        // the tile written above is read by the TMA unit
+      fence_proxy_async_smem();                        // the tile written above is read by the TMA unit (and the MMA)
       if (!got) epi_stop[wcount & 1u] = 1;
       // the one CTA-wide barrier of an item (with the store warp): the results are complete in the output tile
       named_barrier(1, NET + 32);
@@ -514,6 +715,7 @@ cudaError_t launch_t(const Ctx& c) {
   constexpr int NMAT = BWD ? 3 : 2;
   const int slots = c.s.tokens * c.s.top_k, f = c.s.d_ff, r = c.s.rank, N = c.s.n_experts;
   const int rp = pad_rank(r);
+  const bool fold = BWD && grouped_bwd_folds_dz(c.s);
   GsParams p;
   memset(&p, 0, sizeof(p));
   p.row_bytes = rp >= 64 ? 128 : rp * 2;               // bytes of one operand row per k-block
@@ -528,11 +730,12 @@ cudaError_t launch_t(const Ctx& c) {
   // wide operands), then as many operand stages as fit
   constexpr int NOUT = BWD ? 2 : 1;
   const uint32_t set_bytes = NMAT * CB * kBlockBytes, out_bytes = NOUT * CB * kBlockBytes;
-  const uint32_t base = (BWD ? 2 * kSplit * BM * 4 : 0) + 1024 + 256;
+  const uint32_t base = (BWD ? 2 * kSplit * BM * 4 : 0) + 1024 + 640 + (fold ? 2 * kDzbBytes : 0);
   auto need = [&](int ns, int os) { return ns * (set_bytes + kHdrFloats * 4) + os * out_bytes + base + 2 * p.stage_bytes; };
   int nsets = kMaxSets, out_sets = 2;
   while (nsets > 2 && need(nsets, out_sets) > budget) --nsets;
   if (need(nsets, out_sets) > budget) out_sets = 1;
+  if (fold && out_sets != 2) return cudaErrorInvalidConfiguration;   // ranks up to 32 always leave room for two
   const uint32_t other = base + nsets * kHdrFloats * 4;
   const uint32_t fixed = nsets * set_bytes + out_sets * out_bytes + other;
   if (fixed + 2 * p.stage_bytes > budget) return cudaErrorInvalidConfiguration;
@@ -558,6 +761,9 @@ cudaError_t launch_t(const Ctx& c) {
          tc_encode_2d(&p.b_map[2], ad, (long long)N * rp, f, f, p.krows, 64, 128) &&
          tc_encode_2d(&p.o_map[0], c.ws + c.L.da_sorted, slots, f, f, BM, 64, 128) &&
          tc_encode_2d(&p.o_map[1], c.ws + c.L.db_sorted, slots, f, f, BM, 64, 128);
+  if (fold)
+    ok = ok && tc_encode_2d(&p.z_map[0], c.ws + c.L.bg_cat, f, (long long)N * r, (long long)N * r, 64, 64, 128) &&
+         tc_encode_2d(&p.z_map[1], c.ws + c.L.bu_cat, f, (long long)N * r, (long long)N * r, 64, 64, 128);
   if (!ok) return cudaErrorInvalidValue;
   p.G = c.at<bf16>(c.L.G); p.U = c.at<bf16>(c.L.U); p.D = c.at<bf16>(c.L.D);
   p.pos_token = c.at<int>(c.L.pos_token); p.perm = c.at<int>(c.L.perm); p.gates = c.at<float>(c.L.gates);
@@ -570,14 +776,29 @@ cudaError_t launch_t(const Ctx& c) {
   // columns per group: the group's pieces of the gathered matrices (tokens x columns x NMAT) stay well inside L2
   const long long group_cols = (32ll << 20) / ((long long)c.s.tokens * 2 * NMAT);
   p.col_group = (int)std::min<long long>(std::max<long long>(group_cols / COLS, 1), p.col_tiles);
+  p.cg_min = (p.col_group + 1) / 2;                    // units of work: the kernel may settle on narrower groups
+  if (fold) {
+    p.col_group = grouped_bwd_col_group_max(c.s.tokens, f);
+    p.cg_min = (p.col_group + 1) / 2;
+    p.dz_part = c.at<float>(c.L.dz_part);
+    p.groups_used = c.at<int>(c.L.work_count) + 3;
+    p.r_true = r;
+  }
   p.status = c.at<int>(c.L.status);
   int dev = 0, sms = 148;
   cudaGetDevice(&dev);
   cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-  cudaError_t e = cudaFuncSetAttribute(grouped_swiglu_kernel<BWD>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes);
-  if (e != cudaSuccess) return e;
   // the number of segment tiles is only known on the device; every CTA reads it and idles if it has no item
-  grouped_swiglu_kernel<BWD><<<sms, kThreads, smem_bytes, c.st>>>(p);
+  cudaError_t e;
+  if (fold) {
+    e = cudaFuncSetAttribute(grouped_swiglu_kernel<BWD, BWD, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes);
+    if (e != cudaSuccess) return e;
+    grouped_swiglu_kernel<BWD, BWD, 1><<<sms, kThreads, smem_bytes, c.st>>>(p);
+  } else {
+    e = cudaFuncSetAttribute(grouped_swiglu_kernel<BWD, 0, kUnitsAlways>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes);
+    if (e != cudaSuccess) return e;
+    grouped_swiglu_kernel<BWD, 0, kUnitsAlways><<<sms, kThreads, smem_bytes, c.st>>>(p);
+  }
   return cudaGetLastError();
 }
 
