@@ -209,6 +209,41 @@ mixlora_status_t mixlora_layer_backward(const mixlora_shape_t *shape /* host */,
                                         const void *dh, float aux_coef, void *workspace, size_t workspace_bytes,
                                         const mixlora_grads_t *grads /* host struct of device ptrs */, void *stream);
 
+/* MixDoRA (Section 4.1 and Table 1 name the variant: MixLoRA with every expert's LoRA replaced by DoRA; the paper
+ * prints no formula, so this is the weight-decomposed form as it is commonly applied to a linear layer).  Each of
+ * an expert's three projections becomes
+ *     W'_e = diag(m_e / n_e) (W + s B_e A_e),   n_e[o] = || W[o, :] + s B_e[o, :] A_e ||_2,
+ * with one trainable magnitude per output feature and expert (m_gate, m_up [N, f], m_down [N, d], fp32) and the
+ * norm n_e, recomputed from the current weights in every forward call, treated as a constant by the backward pass.
+ * With m = n the block is MixLoRA; with B = 0 and m = the row norms of W it is the frozen FFN.  Router, gates,
+ * dispatch and auxiliary loss are those of mixlora_ffn_forward; W1 x and W3 x are still computed once per token
+ * (the scale acts on output rows), while W2 is applied per slot, because the scale of its output differs between
+ * a token's experts.  The workspace has its own size (mixlora_dora_workspace_bytes) and layout; mixlora_aux_loss,
+ * mixlora_routing_view and mixlora_device_status work on it as after mixlora_ffn_forward.  The backward call needs
+ * the workspace as the forward call for the same arguments left it and returns, besides the gradients of
+ * mixlora_ffn_backward, those of the magnitudes (fp32, same shapes; NULL skips one; `accumulate` of `grads`
+ * applies to them too).  Every step runs on `stream`. */
+typedef struct {
+  const float *m_gate, *m_up; /* [N, f] */
+  const float *m_down;        /* [N, d] */
+} mixlora_dora_t;
+typedef struct {
+  float *d_m_gate, *d_m_up;   /* [N, f] or NULL */
+  float *d_m_down;            /* [N, d] or NULL */
+} mixlora_dora_grads_t;
+size_t mixlora_dora_workspace_bytes(const mixlora_shape_t *shape /* host */, int for_backward);
+mixlora_status_t mixlora_dora_ffn_forward(const mixlora_shape_t *shape /* host */,
+                                          const mixlora_params_t *params /* host struct of device ptrs */,
+                                          const mixlora_dora_t *magnitudes /* host struct of device ptrs */, void *y,
+                                          void *workspace, size_t workspace_bytes, void *stream);
+mixlora_status_t mixlora_dora_ffn_backward(const mixlora_shape_t *shape /* host */,
+                                           const mixlora_params_t *params /* host struct of device ptrs */,
+                                           const mixlora_dora_t *magnitudes /* host struct of device ptrs */,
+                                           const void *dy, float aux_coef, void *workspace, size_t workspace_bytes,
+                                           const mixlora_grads_t *grads /* host struct of device ptrs */,
+                                           const mixlora_dora_grads_t *magnitude_grads /* host struct of device ptrs */,
+                                           void *stream);
+
 /* Plain LoRA on a linear layer (Eq. 1, W' = W + B A, applied as in Section 3.2 to the attention projections of
  * a MixLoRA model): y = x W^T + s (x A^T) B^T with s = lora_alpha / rank.  x [T, d_in], W [d_out, d_in] (frozen),
  * A [rank, d_in], B [d_out, rank], y and dy [T, d_out], all device arrays of shape.dtype; d_in, d_out and rank are

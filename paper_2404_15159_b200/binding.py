@@ -26,7 +26,8 @@ EXPORTS = ("mixlora_limits", "mixlora_workspace_bytes", "mixlora_ffn_forward", "
            "mixlora_multi_ffn_forward", "mixlora_multi_ffn_backward", "mixlora_layer_forward",
            "mixlora_layer_backward", "mixlora_lora_linear_workspace_bytes", "mixlora_lora_linear_forward",
            "mixlora_lora_linear_backward", "mixlora_lora_linear_status", "mixlora_ffn_backward_overlap",
-           "mixlora_aux_stats", "mixlora_aux_loss_global", "mixlora_set_option", "mixlora_selftest_wait_timeout")
+           "mixlora_aux_stats", "mixlora_aux_loss_global", "mixlora_set_option", "mixlora_selftest_wait_timeout",
+           "mixlora_dora_workspace_bytes", "mixlora_dora_ffn_forward", "mixlora_dora_ffn_backward")
 
 MIXLORA_OPT_SERIAL = 0
 MIXLORA_OPT_TC_SINGLE = 1
@@ -51,6 +52,14 @@ class mixlora_params_t(C.Structure):
 class mixlora_grads_t(C.Structure):
     _fields_ = [(n, C.c_void_p) for n in ("d_a_gate", "d_b_gate", "d_a_up", "d_b_up", "d_a_down", "d_b_down",
                                           "d_w_router", "d_router_bias", "d_x")] + [("accumulate", C.c_int32)]
+
+
+class mixlora_dora_t(C.Structure):
+    _fields_ = [(n, C.c_void_p) for n in ("m_gate", "m_up", "m_down")]
+
+
+class mixlora_dora_grads_t(C.Structure):
+    _fields_ = [(n, C.c_void_p) for n in ("d_m_gate", "d_m_up", "d_m_down")]
 
 
 class mixlora_limits_t(C.Structure):
@@ -136,6 +145,15 @@ def _load() -> C.CDLL:
     lib.mixlora_set_option.restype = C.c_int
     lib.mixlora_selftest_wait_timeout.argtypes = [C.c_void_p, C.c_uint32, C.c_void_p]
     lib.mixlora_selftest_wait_timeout.restype = C.c_int
+    lib.mixlora_dora_workspace_bytes.argtypes = [C.POINTER(mixlora_shape_t), C.c_int]
+    lib.mixlora_dora_workspace_bytes.restype = C.c_size_t
+    lib.mixlora_dora_ffn_forward.argtypes = [C.POINTER(mixlora_shape_t), C.POINTER(mixlora_params_t),
+                                             C.POINTER(mixlora_dora_t), C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p]
+    lib.mixlora_dora_ffn_forward.restype = C.c_int
+    lib.mixlora_dora_ffn_backward.argtypes = [C.POINTER(mixlora_shape_t), C.POINTER(mixlora_params_t),
+                                              C.POINTER(mixlora_dora_t), C.c_void_p, C.c_float, C.c_void_p, C.c_size_t,
+                                              C.POINTER(mixlora_grads_t), C.POINTER(mixlora_dora_grads_t), C.c_void_p]
+    lib.mixlora_dora_ffn_backward.restype = C.c_int
     lib.mixlora_status_string.argtypes = [C.c_int]
     lib.mixlora_status_string.restype = C.c_char_p
     return lib
@@ -243,6 +261,35 @@ def mixlora_ffn_backward(shape, params, dy, aux_coef, workspace, grads, stream=N
     _check(lib.mixlora_ffn_backward(C.byref(shape), C.byref(params), _ptr(dy), float(aux_coef), _ptr(workspace),
                                     workspace.numel() if workspace is not None else 0, C.byref(grads),
                                     _stream(stream)), "mixlora_ffn_backward")
+
+
+def make_dora(m_gate, m_up, m_down) -> mixlora_dora_t:
+    return mixlora_dora_t(_ptr(m_gate), _ptr(m_up), _ptr(m_down))
+
+
+def make_dora_grads(d_m_gate=None, d_m_up=None, d_m_down=None) -> mixlora_dora_grads_t:
+    return mixlora_dora_grads_t(_ptr(d_m_gate), _ptr(d_m_up), _ptr(d_m_down))
+
+
+def alloc_dora_workspace(shape: mixlora_shape_t, for_backward: bool, device="cuda") -> torch.Tensor:
+    n = int(lib.mixlora_dora_workspace_bytes(C.byref(shape), 1 if for_backward else 0))
+    if n == 0:
+        raise MixLoraError(1, "mixlora_dora_workspace_bytes")
+    return torch.empty(n, dtype=torch.uint8, device=device)
+
+
+def mixlora_dora_ffn_forward(shape, params, magnitudes, y, workspace, stream=None) -> None:
+    _check(lib.mixlora_dora_ffn_forward(C.byref(shape), C.byref(params), C.byref(magnitudes), _ptr(y), _ptr(workspace),
+                                        workspace.numel() if workspace is not None else 0, _stream(stream)),
+           "mixlora_dora_ffn_forward")
+
+
+def mixlora_dora_ffn_backward(shape, params, magnitudes, dy, aux_coef, workspace, grads, magnitude_grads,
+                              stream=None) -> None:
+    _check(lib.mixlora_dora_ffn_backward(C.byref(shape), C.byref(params), C.byref(magnitudes), _ptr(dy),
+                                         float(aux_coef), _ptr(workspace),
+                                         workspace.numel() if workspace is not None else 0, C.byref(grads),
+                                         C.byref(magnitude_grads), _stream(stream)), "mixlora_dora_ffn_backward")
 
 
 def mixlora_routing_view(shape, workspace) -> dict:

@@ -11,7 +11,7 @@ ROOT = os.path.dirname(PKG)
 CSRC = os.path.join(PKG, "csrc")
 LIB = os.path.join(PKG, "libmixlora.so")
 OBJ_DIR = os.path.join(PKG, "_build")
-SOURCES = ["api.cu", "router.cu", "simt_gemm.cu", "elementwise.cu", "tc_gemm.cu", "static_dispatch.cu", "grouped_swiglu.cu"]
+SOURCES = ["api.cu", "router.cu", "simt_gemm.cu", "elementwise.cu", "tc_gemm.cu", "static_dispatch.cu", "grouped_swiglu.cu", "dora.cu"]
 HEADERS = [os.path.join(CSRC, "common.cuh"), os.path.join(CSRC, "tc_ptx.cuh"), os.path.join(ROOT, "include", "mixlora.h")]
 
 NVCC_FLAGS = [

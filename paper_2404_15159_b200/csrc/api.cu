@@ -12,7 +12,7 @@
 
 namespace mixlora {
 
-WsLayout ws_layout(const mixlora_shape_t& s) {
+WsLayout ws_layout(const mixlora_shape_t& s, bool allow_fold) {
   WsLayout L;
   memset(&L, 0, sizeof(L));
   const size_t T = (size_t)s.tokens, d = (size_t)s.d_model, f = (size_t)s.d_ff, N = (size_t)s.n_experts,
@@ -79,7 +79,7 @@ WsLayout ws_layout(const mixlora_shape_t& s) {
   L.p_s = take(T * k * rp * E);
   L.dZd_pos = take(T * k * N * r * E);
   L.dgate_part = take((size_t)grouped_swiglu_bwd_col_tiles(s.d_ff) * T * k * 4);
-  const bool fold_dz = grouped_bwd_folds_dz(s);
+  const bool fold_dz = allow_fold && grouped_bwd_folds_dz(s);
   L.dzg_all = take(fold_dz ? 0 : T * k * N * r * E);
   L.dzu_all = take(fold_dz ? 0 : T * k * N * r * E);
   L.dz_part = take(fold_dz ? (size_t)grouped_bwd_max_groups(s.tokens, s.d_ff) * T * k * 2 * r * 4 : 0);
@@ -740,7 +740,7 @@ static mixlora_status_t bwd_experts(const Ctx& c, const void* dy, float aux_coef
   } while (0)
   // dzg = da (s B_g), dzu = db (s B_u), against every expert (the slot's own block is used); not when the grouped
   // kernel above has formed them from the tiles it held
-  if (!grouped_bwd_folds_dz(c.s)) {
+  if (!ctx_folds_dz(c)) {
     TcOut outs[2];
     outs[0] = tc_out(c.ws + c.L.dzg_all, Nr, Nr); tc_add(outs[0], c.ws + c.L.da_sorted, f, f, c.ws + c.L.bg_cat, Nr, 1);
     outs[1] = tc_out(c.ws + c.L.dzu_all, Nr, Nr); tc_add(outs[1], c.ws + c.L.db_sorted, f, f, c.ws + c.L.bu_cat, Nr, 1);
@@ -920,6 +920,226 @@ mixlora_status_t mixlora_layer_backward(const mixlora_shape_t* shape, const mixl
     // d_x holds dL/dxn now; the norm's Jacobian and the residual path turn it into dL/dz in place
     StageScope ss(ST_NORM, c.st, shape->tokens > 0 ? 1 : 0);
     MIXLORA_CUDA(launch_rmsnorm_bwd(c, params->x, norm_weight, inv_rms, grads->d_x, dh, grads->d_x));
+  }
+  return MIXLORA_OK;
+}
+
+// ---- MixDoRA (Section 4.1 / Table 1): every expert projection is diag(m / n) (W + s B A) ----
+namespace {
+struct DoraLayout {
+  size_t cg, cu, cd, inv_g, inv_u, inv_d, rowsq_g, rowsq_u, rowsq_d, wa_g, wa_u, wa_d, aat_g, aat_u, aat_d;
+  size_t Zd_pos, gZd_pos, o_pre, total_fwd;
+  size_t dO, D_s, spd_s, dmp_g, dmp_u, dmp_d, total_bwd;
+};
+// the MixLoRA layout (sized for both passes, without the grouped kernel's partial sums) followed by the extra regions
+DoraLayout dora_layout(const mixlora_shape_t& s, const WsLayout& L) {
+  DoraLayout D;
+  const size_t T = (size_t)s.tokens, d = (size_t)s.d_model, f = (size_t)s.d_ff, N = (size_t)s.n_experts,
+               k = (size_t)s.top_k, r = (size_t)s.rank, E = act_size(s);
+  const size_t mt = (size_t)max_seg_tiles(s.tokens, s.top_k, s.n_experts);
+  size_t off = L.total_bwd;
+  auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + (bytes ? bytes : 1), 256); return o; };
+  D.cg = take(N * f * 4); D.cu = take(N * f * 4); D.cd = take(N * d * 4);
+  D.inv_g = take(N * f * 4); D.inv_u = take(N * f * 4); D.inv_d = take(N * d * 4);
+  D.rowsq_g = take(f * 4); D.rowsq_u = take(f * 4); D.rowsq_d = take(d * 4);
+  D.wa_g = take(f * N * r * 4); D.wa_u = take(f * N * r * 4); D.wa_d = take(d * N * r * 4);
+  D.aat_g = take(N * r * N * r * 4); D.aat_u = take(N * r * N * r * 4); D.aat_d = take(N * r * N * r * 4);
+  D.Zd_pos = take(T * k * N * r * E); D.gZd_pos = take(T * k * N * r * E);
+  D.o_pre = take(T * k * d * E);
+  D.total_fwd = off;
+  D.dO = take(T * k * d * E);
+  D.D_s = take(T * k * f * E);
+  D.spd_s = take(T * k * N * r * E);
+  D.dmp_g = take(mt * f * 4); D.dmp_u = take(mt * f * 4); D.dmp_d = take(mt * d * 4);
+  D.total_bwd = off;
+  return D;
+}
+
+mixlora_status_t dora_setup(const mixlora_shape_t* shape, const mixlora_params_t* params,
+                            const mixlora_dora_t* magn, void* workspace, size_t workspace_bytes, int for_backward,
+                            void* stream, Ctx* c, DoraCtx* dc) {
+  mixlora_status_t st = check_shape(shape);
+  if (st != MIXLORA_OK) return st;
+  if ((st = check_params(params)) != MIXLORA_OK) return st;
+  if (!magn || !magn->m_gate || !magn->m_up || !magn->m_down) return MIXLORA_ERR_INVALID_ARG;
+  const void* mq[] = {magn->m_gate, magn->m_up, magn->m_down};
+  for (const void* q : mq)
+    if (reinterpret_cast<uintptr_t>(q) & 3u) return MIXLORA_ERR_INVALID_ARG;
+  *c = make_ctx(shape, params, workspace, stream);
+  c->L = ws_layout(*shape, false);
+  c->no_fold = 1;
+  const DoraLayout D = dora_layout(*shape, c->L);
+  if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255u) ||
+      workspace_bytes < (for_backward ? D.total_bwd : D.total_fwd))
+    return MIXLORA_ERR_WORKSPACE;
+  dc->m = *magn;
+  dc->cg = c->at<float>(D.cg); dc->cu = c->at<float>(D.cu); dc->cd = c->at<float>(D.cd);
+  dc->inv_g = c->at<float>(D.inv_g); dc->inv_u = c->at<float>(D.inv_u); dc->inv_d = c->at<float>(D.inv_d);
+  dc->rowsq_g = c->at<float>(D.rowsq_g); dc->rowsq_u = c->at<float>(D.rowsq_u); dc->rowsq_d = c->at<float>(D.rowsq_d);
+  dc->wa_g = c->at<float>(D.wa_g); dc->wa_u = c->at<float>(D.wa_u); dc->wa_d = c->at<float>(D.wa_d);
+  dc->aat_g = c->at<float>(D.aat_g); dc->aat_u = c->at<float>(D.aat_u); dc->aat_d = c->at<float>(D.aat_d);
+  dc->Zd_pos = c->ws + D.Zd_pos; dc->gZd_pos = c->ws + D.gZd_pos; dc->o_pre = c->ws + D.o_pre;
+  dc->dO = c->ws + D.dO; dc->D_s = c->ws + D.D_s; dc->spd_s = c->ws + D.spd_s;
+  dc->dmp_g = c->at<float>(D.dmp_g); dc->dmp_u = c->at<float>(D.dmp_u); dc->dmp_d = c->at<float>(D.dmp_d);
+  return MIXLORA_OK;
+}
+}  // namespace
+
+size_t mixlora_dora_workspace_bytes(const mixlora_shape_t* shape, int for_backward) {
+  if (check_shape(shape) != MIXLORA_OK) return 0;
+  const WsLayout L = ws_layout(*shape, false);
+  const DoraLayout D = dora_layout(*shape, L);
+  return for_backward ? D.total_bwd : D.total_fwd;
+}
+
+mixlora_status_t mixlora_dora_ffn_forward(const mixlora_shape_t* shape, const mixlora_params_t* params,
+                                          const mixlora_dora_t* magnitudes, void* y, void* workspace,
+                                          size_t workspace_bytes, void* stream) {
+  Ctx c;
+  DoraCtx dc;
+  mixlora_status_t st = dora_setup(shape, params, magnitudes, workspace, workspace_bytes, 0, stream, &c, &dc);
+  if (st != MIXLORA_OK) return st;
+  if (!y || !aligned16(y)) return MIXLORA_ERR_INVALID_ARG;
+  const int T = c.s.tokens, d = c.s.d_model, f = c.s.d_ff, N = c.s.n_experts, r = c.s.rank, k = c.s.top_k;
+  const int Nr = N * r;
+  if ((st = fwd_clear_status(c)) != MIXLORA_OK) return st;
+  if (T == 0) return MIXLORA_OK;
+  if ((st = fwd_route(c)) != MIXLORA_OK) return st;
+  // the scales c = m / n of the three projections: |W_o + s B_o A|^2 = |W_o|^2 + 2 s B_o . (W A^T)_o + s^2 B_o (A A^T) B_o^T
+  {
+    TcOut gu[2];
+    gu[0] = tc_out_f32(dc.wa_g, Nr, Nr, 1, 0, 0, 1.f, 0); tc_add(gu[0], params->w_gate, d, d, params->a_gate, d, 0);
+    gu[1] = tc_out_f32(dc.wa_u, Nr, Nr, 1, 0, 0, 1.f, 0); tc_add(gu[1], params->w_up, d, d, params->a_up, d, 0);
+    MIXLORA_CUDA(dense_product(c, f, gu, 2));
+    TcOut dn = tc_out_f32(dc.wa_d, Nr, Nr, 1, 0, 0, 1.f, 0);
+    tc_add(dn, params->w_down, f, f, params->a_down, f, 0);
+    MIXLORA_CUDA(dense_product(c, d, &dn, 1));
+    TcOut aa[2];
+    aa[0] = tc_out_f32(dc.aat_g, Nr, Nr, 1, 0, 0, 1.f, 0); tc_add(aa[0], params->a_gate, d, d, params->a_gate, d, 0);
+    aa[1] = tc_out_f32(dc.aat_u, Nr, Nr, 1, 0, 0, 1.f, 0); tc_add(aa[1], params->a_up, d, d, params->a_up, d, 0);
+    MIXLORA_CUDA(dense_product(c, Nr, aa, 2));
+    TcOut ad = tc_out_f32(dc.aat_d, Nr, Nr, 1, 0, 0, 1.f, 0);
+    tc_add(ad, params->a_down, f, f, params->a_down, f, 0);
+    MIXLORA_CUDA(dense_product(c, Nr, &ad, 1));
+    MIXLORA_CUDA(launch_dora_scales(c, dc));
+  }
+  if ((st = fwd_shared_projections(&c, 1)) != MIXLORA_OK) return st;   // W1 x, W3 x once per token, A_g x, A_u x
+  MIXLORA_CUDA(launch_dora_swiglu_fwd(c, dc));
+  {   // zd = A_d h against every expert, then the slot's own block (and gate times it)
+    TcOut out = tc_out(c.ws + c.L.zd_all, Nr, Nr);
+    tc_add(out, c.ws + c.L.h_sorted, f, f, params->a_down, f, 0);
+    MIXLORA_CUDA(dense_product(c, T * k, &out, 1));
+    MIXLORA_CUDA(launch_dora_own_block(c, c.ws + c.L.zd_all, dc.Zd_pos, dc.gZd_pos));
+  }
+  {   // o_pre = [h | Zd] [W2 | s B_d]^T per sorted slot: W2 cannot act on the gate-weighted sum of a token's slots
+      // here, because the scale of its output differs between the token's experts
+    TcOut out = tc_out(dc.o_pre, d, d);
+    tc_add(out, c.ws + c.L.h_sorted, f, f, params->w_down, f, 0);
+    tc_add(out, dc.Zd_pos, Nr, Nr, c.ws + c.L.bd_cat, Nr, 0);
+    MIXLORA_CUDA(dense_product(c, T * k, &out, 1));
+  }
+  MIXLORA_CUDA(launch_dora_combine_y(c, dc, y));
+  return MIXLORA_OK;
+}
+
+mixlora_status_t mixlora_dora_ffn_backward(const mixlora_shape_t* shape, const mixlora_params_t* params,
+                                           const mixlora_dora_t* magnitudes, const void* dy, float aux_coef,
+                                           void* workspace, size_t workspace_bytes, const mixlora_grads_t* grads,
+                                           const mixlora_dora_grads_t* mgrads, void* stream) {
+  Ctx c;
+  DoraCtx dc;
+  mixlora_status_t st = dora_setup(shape, params, magnitudes, workspace, workspace_bytes, 1, stream, &c, &dc);
+  if (st != MIXLORA_OK) return st;
+  if (!dy || !aligned16(dy) || !grads || !mgrads) return MIXLORA_ERR_INVALID_ARG;
+  {
+    const void* outs[] = {grads->d_a_gate, grads->d_b_gate, grads->d_a_up, grads->d_b_up, grads->d_a_down,
+                          grads->d_b_down, grads->d_w_router, grads->d_x};
+    for (const void* q : outs)
+      if (q && !aligned16(q)) return MIXLORA_ERR_INVALID_ARG;
+    if (grads->accumulate != 0 && grads->accumulate != 1) return MIXLORA_ERR_INVALID_ARG;
+  }
+  const int T = c.s.tokens, d = c.s.d_model, f = c.s.d_ff, N = c.s.n_experts, r = c.s.rank, k = c.s.top_k;
+  const int Nr = N * r, NP = round_up8(N), acc = grads->accumulate, want_dx = grads->d_x != nullptr;
+  if (T == 0) {
+    if ((st = bwd_zero_tokens(c, grads)) != MIXLORA_OK) return st;
+    if (!acc) {
+      if (mgrads->d_m_gate) MIXLORA_CUDA(cudaMemsetAsync(mgrads->d_m_gate, 0, sizeof(float) * N * f, c.st));
+      if (mgrads->d_m_up) MIXLORA_CUDA(cudaMemsetAsync(mgrads->d_m_up, 0, sizeof(float) * N * f, c.st));
+      if (mgrads->d_m_down) MIXLORA_CUDA(cudaMemsetAsync(mgrads->d_m_down, 0, sizeof(float) * N * d, c.st));
+    }
+    return MIXLORA_OK;
+  }
+  // dO = c_d * dy per sorted slot (and the down magnitude's shares), then D = dO W2 and s B_d^T dO per slot
+  MIXLORA_CUDA(launch_dora_dout(c, dc, dy));
+  {
+    TcOut outs[2];
+    outs[0] = tc_out(dc.D_s, f, f);      tc_add(outs[0], dc.dO, d, d, params->w_down, f, 1);
+    outs[1] = tc_out(dc.spd_s, Nr, Nr);  tc_add(outs[1], dc.dO, d, d, c.ws + c.L.bd_cat, Nr, 1);
+    MIXLORA_CUDA(dense_product(c, T * k, outs, 2));
+  }
+  MIXLORA_CUDA(launch_dora_swiglu_bwd(c, dc));
+  MIXLORA_CUDA(launch_dgate_reduce(c, dora_bwd_col_chunks(f)));
+  MIXLORA_CUDA(launch_router_bwd(c, aux_coef, grads->d_router_bias, acc, want_dx));
+  if (mgrads->d_m_gate) MIXLORA_CUDA(launch_dora_dm_reduce(c, dc.dmp_g, dc.inv_g, mgrads->d_m_gate, f, acc));
+  if (mgrads->d_m_up) MIXLORA_CUDA(launch_dora_dm_reduce(c, dc.dmp_u, dc.inv_u, mgrads->d_m_up, f, acc));
+  if (mgrads->d_m_down) MIXLORA_CUDA(launch_dora_dm_reduce(c, dc.dmp_d, dc.inv_d, mgrads->d_m_down, d, acc));
+  {   // dzg = da (s B_g), dzu = db (s B_u) with da, db the gradients of the pre-scale activations
+    TcOut outs[2];
+    outs[0] = tc_out(c.ws + c.L.dzg_all, Nr, Nr); tc_add(outs[0], c.ws + c.L.da_sorted, f, f, c.ws + c.L.bg_cat, Nr, 1);
+    outs[1] = tc_out(c.ws + c.L.dzu_all, Nr, Nr); tc_add(outs[1], c.ws + c.L.db_sorted, f, f, c.ws + c.L.bu_cat, Nr, 1);
+    MIXLORA_CUDA(dense_product(c, T * k, outs, 2));
+  }
+  MIXLORA_CUDA(launch_combine_bwd(c, want_dx));
+  MIXLORA_CUDA(launch_zpos(c));
+  // dZd_pos = gate * (s B_d^T dO) in the slot's own block
+  MIXLORA_CUDA(launch_dora_own_block(c, dc.spd_s, nullptr, c.ws + c.L.dZd_pos));
+  {
+    TcOut outs[3];
+    int n = 0;
+    if (grads->d_b_gate) {
+      outs[n] = tc_out_f32(grads->d_b_gate, Nr, r, 1, r, (long long)f * r, c.scale, acc);
+      tc_add(outs[n++], c.ws + c.L.da_sorted, f, T * k, c.ws + c.L.Zg_pos, Nr, 1, 1);
+    }
+    if (grads->d_b_up) {
+      outs[n] = tc_out_f32(grads->d_b_up, Nr, r, 1, r, (long long)f * r, c.scale, acc);
+      tc_add(outs[n++], c.ws + c.L.db_sorted, f, T * k, c.ws + c.L.Zu_pos, Nr, 1, 1);
+    }
+    if (grads->d_a_down) {
+      outs[n] = tc_out_f32(grads->d_a_down, Nr, 1, f, 0, 0, 1.f, acc);
+      tc_add(outs[n++], c.ws + c.L.h_sorted, f, T * k, c.ws + c.L.dZd_pos, Nr, 1, 1);
+    }
+    MIXLORA_CUDA(dense_product(c, f, outs, n));
+  }
+  if (grads->d_b_down) {   // dB_d[e][c][rr] = s sum over slots of dO[slot][c] (g zd)[slot][e r + rr]
+    TcOut out = tc_out_f32(grads->d_b_down, Nr, r, 1, r, (long long)d * r, c.scale, acc);
+    tc_add(out, dc.dO, d, T * k, dc.gZd_pos, Nr, 1, 1);
+    MIXLORA_CUDA(dense_product(c, d, &out, 1));
+  }
+  {
+    TcOut outs[3];
+    int n = 0;
+    if (grads->d_a_gate) {
+      outs[n] = tc_out_f32(grads->d_a_gate, Nr, 1, d, 0, 0, 1.f, acc);
+      tc_add(outs[n++], params->x, d, T, c.ws + c.L.dZg, Nr, 1, 1);
+    }
+    if (grads->d_a_up) {
+      outs[n] = tc_out_f32(grads->d_a_up, Nr, 1, d, 0, 0, 1.f, acc);
+      tc_add(outs[n++], params->x, d, T, c.ws + c.L.dZu, Nr, 1, 1);
+    }
+    if (grads->d_w_router) {
+      outs[n] = tc_out_f32(grads->d_w_router, N, 1, d, 0, 0, 1.f, acc);
+      tc_add(outs[n++], params->x, d, T, c.ws + c.L.dl_act, NP, 1, 1, NP);
+    }
+    MIXLORA_CUDA(dense_product(c, d, outs, n));
+  }
+  if (want_dx) {
+    TcOut out = tc_out(grads->d_x, d, d);
+    tc_add(out, c.ws + c.L.dabar, f, f, params->w_gate, d, 1);
+    tc_add(out, c.ws + c.L.dbbar, f, f, params->w_up, d, 1);
+    tc_add(out, c.ws + c.L.dZg, Nr, Nr, params->a_gate, d, 1);
+    tc_add(out, c.ws + c.L.dZu, Nr, Nr, params->a_up, d, 1);
+    tc_add(out, c.ws + c.L.dl_act, NP, NP, c.ws + c.L.wr_act, d, 1);
+    MIXLORA_CUDA(dense_product(c, T, &out, 1));
   }
   return MIXLORA_OK;
 }

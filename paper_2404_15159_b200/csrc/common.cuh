@@ -86,7 +86,8 @@ static inline int round_up8(int v) { return (v + 7) / 8 * 8; }
 // ranks are zero-padded to the next of these widths
 static inline int pad_rank(int r) { return r <= 16 ? 16 : (r <= 32 ? 32 : (r <= 64 ? 64 : 128)); }
 
-WsLayout ws_layout(const mixlora_shape_t& s);
+// `allow_fold` = false sizes every region for the path that does not form dzg / dzu inside the grouped kernel
+WsLayout ws_layout(const mixlora_shape_t& s, bool allow_fold = true);
 
 // Column tiles of the backward grouped SwiGLU kernel (64 columns each) and the widest group of them whose pieces of
 // G, U and D (tokens x columns x 3 matrices) stay well inside L2 while every segment tile of the group is worked on.
@@ -166,9 +167,12 @@ struct Ctx {
   char* ws;
   cudaStream_t st;
   int bf16;  // activation type is bf16
+  int no_fold = 0;   // 1: the workspace was laid out with allow_fold = false (MixDoRA path)
   float scale;
   template <typename T> T* at(size_t off) const { return reinterpret_cast<T*>(ws + off); }
 };
+
+static inline bool ctx_folds_dz(const Ctx& c) { return !c.no_fold && grouped_bwd_folds_dz(c.s); }
 
 cudaError_t launch_router(const Ctx& c);              // probs, expert_idx, gates, low_margin, stats
 cudaError_t launch_dispatch(const Ctx& c);            // perm, inv, pos_token, pos_expert, seg_off, tile_info
@@ -197,6 +201,31 @@ cudaError_t launch_rmsnorm_fwd(const Ctx& c, const void* z, const void* w_norm, 
 cudaError_t launch_rmsnorm_bwd(const Ctx& c, const void* z, const void* w_norm, const float* inv_rms, const void* dxn,
                                const void* dh, void* dz);
 cudaError_t launch_residual_add(const Ctx& c, void* C, long long ldc, const void* R, long long ldr, int M, int N);
+
+// MixDoRA (dora.cu): pointers into the extra regions of its workspace, and the launchers of its kernels
+struct DoraCtx {
+  mixlora_dora_t m;
+  float *cg, *cu, *cd;                 // [N, f], [N, f], [N, d]  c = m / n
+  float *inv_g, *inv_u, *inv_d;        // 1 / n
+  float *rowsq_g, *rowsq_u, *rowsq_d;  // [f], [f], [d]  squared row norms of the frozen weights
+  float *wa_g, *wa_u, *wa_d;           // [f, N r], [f, N r], [d, N r]  W times every expert's A^T
+  float *aat_g, *aat_u, *aat_d;        // [N r, N r]  A_cat A_cat^T (diagonal blocks used)
+  void *Zd_pos, *gZd_pos;              // act [T k, N r]  zd (and gate * zd) of the slot in its expert block
+  void *o_pre;                         // act [T k, d]   W2 h + s B_d zd per sorted slot, before the scale
+  void *dO;                            // act [T k, d]   c_d * dy per sorted slot
+  void *D_s;                           // act [T k, f]   dO W2 per sorted slot
+  void *spd_s;                         // act [T k, N r] s B_d^T dO for every expert, per sorted slot
+  float *dmp_g, *dmp_u, *dmp_d;        // [tiles, f], [tiles, f], [tiles, d]  per-tile shares of the magnitude gradients
+};
+int dora_bwd_col_chunks(int f);
+cudaError_t launch_dora_scales(const Ctx& c, const DoraCtx& dc);
+cudaError_t launch_dora_swiglu_fwd(const Ctx& c, const DoraCtx& dc);
+cudaError_t launch_dora_own_block(const Ctx& c, const void* in, void* own, void* gown);
+cudaError_t launch_dora_combine_y(const Ctx& c, const DoraCtx& dc, void* y);
+cudaError_t launch_dora_dout(const Ctx& c, const DoraCtx& dc, const void* dy);
+cudaError_t launch_dora_swiglu_bwd(const Ctx& c, const DoraCtx& dc);
+cudaError_t launch_dora_dm_reduce(const Ctx& c, const float* part, const float* inv_n, float* dm, int width,
+                                  int accumulate);
 
 // Dense product (tensor-core kernel in tc_gemm.cu, SIMT kernel otherwise), fp32 accumulation:
 //   C_o[M, N_o] = sum_seg op(A_o,seg) * op(B_o,seg)

@@ -648,7 +648,7 @@ cudaError_t combine_bwd_t(const Ctx& c, int want_dx) {
   constexpr bool vec = sizeof(T) == 2;
   combine_bwd_kernel<T><<<c.s.tokens, vec ? 128 : ENT, 0, c.st>>>(
       c.at<T>(c.L.da_sorted), c.at<T>(c.L.db_sorted), c.at<T>(c.L.dzg_all), c.at<T>(c.L.dzu_all),
-      grouped_bwd_folds_dz(c.s) ? c.at<float>(c.L.dz_part) : nullptr, c.at<int>(c.L.work_count) + 3,
+      ctx_folds_dz(c) ? c.at<float>(c.L.dz_part) : nullptr, c.at<int>(c.L.work_count) + 3,
       c.s.tokens * c.s.top_k, c.at<int>(c.L.inv), c.at<int>(c.L.expert_idx), c.at<T>(c.L.dabar), c.at<T>(c.L.dbbar), c.at<T>(c.L.dZg),
       c.at<T>(c.L.dZu), c.s.d_ff, c.s.n_experts, c.s.rank, c.s.top_k, vec ? 0 : want_dx);
   return cudaGetLastError();

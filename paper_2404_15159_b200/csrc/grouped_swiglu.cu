@@ -715,7 +715,7 @@ cudaError_t launch_t(const Ctx& c) {
   constexpr int NMAT = BWD ? 3 : 2;
   const int slots = c.s.tokens * c.s.top_k, f = c.s.d_ff, r = c.s.rank, N = c.s.n_experts;
   const int rp = pad_rank(r);
-  const bool fold = BWD && grouped_bwd_folds_dz(c.s);
+  const bool fold = BWD && ctx_folds_dz(c);
   GsParams p;
   memset(&p, 0, sizeof(p));
   p.row_bytes = rp >= 64 ? 128 : rp * 2;               // bytes of one operand row per k-block
