@@ -51,6 +51,7 @@ def config_of(w: synth.Workload, args, world: int, use_dist: bool) -> dict:
             "n_experts": w.n_experts, "top_k": w.top_k, "rank": w.rank, "lora_alpha": w.lora_alpha,
             "backward_dx": want_dx, "aux_coef": AUX_COEF, "adapters": M,
             "layer_slice": bool(args.layer and M == 1 and want_dx),
+            "variant": "mixdora" if getattr(args, "dora", False) else "mixlora",
             "parallelism": f"dp{world} over tokens" + (", aux statistics (2N floats) and LoRA/router gradients "
                                                         "all-reduced over NCCL, the latter beside the dx product"
                                                         if use_dist else ""),
@@ -337,6 +338,29 @@ def run_cuda(args):
             if use_dist:
                 dist.all_reduce(flat)
 
+    if args.dora:
+        # MixDoRA (Section 4.1 / Table 1): the same step with every expert's LoRA replaced by DoRA.  Magnitudes start,
+        # as DoRA's do, from the row norms of the frozen weights, here times a factor in [0.8, 1.2].
+        gen = torch.Generator(device="cuda").manual_seed(w.seed + 7)
+
+        def mag(wt):
+            base = wt.float().norm(dim=1)
+            return (base[None, :] * (0.8 + 0.4 * torch.rand(w.n_experts, base.numel(), generator=gen, device="cuda"))
+                    ).contiguous()
+
+        m_dev = [mag(dev["w_gate"]), mag(dev["w_up"]), mag(dev["w_down"])]
+        dm_dev = [torch.zeros_like(v) for v in m_dev]
+        magn, dmagn = B.make_dora(*m_dev), B.make_dora_grads(*dm_dev)
+        ws = B.alloc_dora_workspace(shape, True)
+
+        def compute(params_, y_, dy_):     # noqa: F811
+            B.mixlora_dora_ffn_forward(shape, params_, magn, y_, ws)
+            B.mixlora_aux_loss(shape, ws, AUX_COEF, loss)
+            B.mixlora_dora_ffn_backward(shape, params_, magn, dy_, AUX_COEF, ws, grads, dmagn)
+
+        def step():                        # noqa: F811
+            compute(params, y, dev["dy"])
+
     if args.forward_only:
         # the forward-only configuration: no backward pass, no gradient exchange
         def step():                        # noqa: F811
@@ -520,7 +544,8 @@ def run_cuda(args):
                         "gemm_down": (T_ * f_ + f_ * d_ + T_ * d_) * E,
                         "gemm_dgrad_down": (T_ * d_ + f_ * d_ + T_ * f_) * E,
                         "gemm_dx": (2 * T_ * f_ + 2 * f_ * d_ + T_ * d_) * E}
-    if w.name == synth.c3().name and want_dx and M == 1 and not args.layer and bf16 and not args.forward_only:
+    if (w.name == synth.c3().name and want_dx and M == 1 and not args.layer and bf16 and not args.forward_only
+            and not args.dora):
         roofline["traffic"] = measured_dram[dom]
         roofline["traffic_note"] = ("constant from %s (one single-pass ncu capture of this command's workload, not "
                                     "measured in this run): dram__bytes_read.sum + dram__bytes_write.sum of the %s "
@@ -646,6 +671,8 @@ def main():
     ap.add_argument("--models", type=int, default=1,
                     help="split the batch over this many adapters sharing the frozen FFN (multi-model calls); the "
                          "end-to-end leg still runs the single-model calls")
+    ap.add_argument("--dora", action="store_true",
+                    help="time the MixDoRA variant of the step (mixlora_dora_ffn_forward / _backward)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--cpu-sample", type=int, default=4096, help="tokens of the oracle's timed sample")
     ap.add_argument("--ref-sample", type=int, default=0,

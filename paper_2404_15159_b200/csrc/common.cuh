@@ -105,9 +105,14 @@ static inline bool grouped_bwd_folds_dz(const mixlora_shape_t& s) {
   return s.dtype == MIXLORA_DTYPE_BF16 && s.tokens > 0 && (s.rank == 8 || s.rank == 16 || s.rank == 32) &&
          grouped_bwd_col_group_max(s.tokens, s.d_ff) >= 4 && (long long)s.tokens * s.d_ff < (1ll << 31);
 }
-// the kernel may narrow the groups down to half the widest to even out the CTAs' shares: bound of the group count
+// the kernel may narrow the groups down to a quarter of the widest (not below 4 tiles) to even out the CTAs' shares:
+// narrowest width, and the bound of the group count that follows from it
+static inline int grouped_bwd_col_group_min(int tokens, int f) {
+  const int q = (grouped_bwd_col_group_max(tokens, f) + 3) / 4;
+  return q < 4 ? 4 : q;
+}
 static inline int grouped_bwd_max_groups(int tokens, int f) {
-  const int cg_min = (grouped_bwd_col_group_max(tokens, f) + 1) / 2;
+  const int cg_min = grouped_bwd_col_group_min(tokens, f);
   return (grouped_bwd_col_tiles(f) + cg_min - 1) / cg_min;
 }
 

@@ -779,7 +779,7 @@ cudaError_t launch_t(const Ctx& c) {
   p.cg_min = (p.col_group + 1) / 2;                    // units of work: the kernel may settle on narrower groups
   if (fold) {
     p.col_group = grouped_bwd_col_group_max(c.s.tokens, f);
-    p.cg_min = (p.col_group + 1) / 2;
+    p.cg_min = grouped_bwd_col_group_min(c.s.tokens, f);
     p.dz_part = c.at<float>(c.L.dz_part);
     p.groups_used = c.at<int>(c.L.work_count) + 3;
     p.r_true = r;

@@ -137,3 +137,9 @@ def test_zero_tokens_and_accumulation():
     b = gpu_dora(w, t, m, 0.01, accumulate=1, init=0.5)
     for n in helpers.GRAD_NAMES + tuple("d_m_" + k for k in MAG):
         np.testing.assert_allclose(b[n], a[n] + 0.5, rtol=1e-5, atol=1e-6)
+
+
+def test_llama2_7b_shape_1024_tokens_every_output():
+    # the 7B-shaped block (d = 4096, f = 11008, 8 experts, top-2, rank 16) on the tensor-core products
+    errs = check(synth.c3().with_(name="dora-7b-1024", tokens=1024), 2e-2)
+    print("MixDoRA 7B shape, 1024 tokens:", {k: f"{v:.2e}" for k, v in errs.items()})
