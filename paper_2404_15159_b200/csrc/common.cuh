@@ -105,11 +105,11 @@ static inline bool grouped_bwd_folds_dz(const mixlora_shape_t& s) {
   return s.dtype == MIXLORA_DTYPE_BF16 && s.tokens > 0 && (s.rank == 8 || s.rank == 16 || s.rank == 32) &&
          grouped_bwd_col_group_max(s.tokens, s.d_ff) >= 4 && (long long)s.tokens * s.d_ff < (1ll << 31);
 }
-// the kernel may narrow the groups down to a quarter of the widest (not below 4 tiles) to even out the CTAs' shares:
-// narrowest width, and the bound of the group count that follows from it
+// the kernel may narrow the groups down to 4 tiles to even out the CTAs' shares (with few tokens there are few segment
+// tiles, and wide groups would leave most CTAs without a unit): narrowest width, and the bound of the group count
 static inline int grouped_bwd_col_group_min(int tokens, int f) {
-  const int q = (grouped_bwd_col_group_max(tokens, f) + 3) / 4;
-  return q < 4 ? 4 : q;
+  (void)tokens; (void)f;
+  return 4;
 }
 static inline int grouped_bwd_max_groups(int tokens, int f) {
   const int cg_min = grouped_bwd_col_group_min(tokens, f);
