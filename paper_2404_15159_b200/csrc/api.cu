@@ -48,7 +48,9 @@ WsLayout ws_layout(const mixlora_shape_t& s, bool allow_fold) {
   L.U = take(T * f * E);
   L.zga = take(T * N * r * E);
   L.zua = take(T * N * r * E);
-  L.zd_all = take(T * k * N * r * E);
+  const bool fold_zd = allow_fold && grouped_fwd_folds_zd(s);
+  L.zd_all = take(fold_zd ? 0 : T * k * N * r * E);
+  L.zd_part = take(fold_zd ? (size_t)grouped_fwd_max_groups(s.d_ff) * T * k * r * 4 : 0);
   L.Zs = take(T * N * r * E);
   L.bd_cat = take(d * N * r * E);
   L.bg_cat = take(f * N * r * E);
@@ -486,8 +488,9 @@ static mixlora_status_t fwd_experts(const Ctx& c, void* y, const void* residual 
       MIXLORA_CUDA(launch_lora_b_swiglu(c));
     }
   }
-  // zd = A_d h per slot, against every expert's A_d (the slot's own block is picked up by the combine)
-  {
+  // zd = A_d h per slot, against every expert's A_d (the slot's own block is picked up by the combine); not when
+  // the grouped kernel above has formed it from the tiles it held
+  if (!ctx_folds_zd(c)) {
     TcOut out = tc_out(c.ws + c.L.zd_all, Nr, Nr);
     tc_add(out, c.ws + c.L.h_sorted, f, f, params->a_down, f, 0);
     StageScope ss(ST_LORA_A_DOWN, c.st, (block_sparse(c) ? 1 : 0) + dense_launches(c, T * k, &out, 1));

@@ -50,7 +50,7 @@ struct WsLayout {
   size_t h_sorted;    // act [T*k, f]
   size_t hbar;        // act [T, f]        sum_j g_j h_j
   size_t work_count;  // i32 [8]  item counts of the work lists below; [3] = column groups the backward grouped
-                      //          kernel used (rows of dz_part)
+                      //          kernel used (rows of dz_part); [4] = the same of the forward kernel (zd_part)
   size_t work_rows1;  // i32 [.., 8]  rows list with one output (A_d h)
   size_t total_fwd;
   size_t D;           // act [T, f]        dy W_d
@@ -64,6 +64,8 @@ struct WsLayout {
   size_t dzg_all, dzu_all;      // act [T*k, N*r]  da (s B_g) and db (s B_u) against every expert (not when the
                                 //                 grouped kernel forms them, see dz_part)
   size_t dz_part;               // f32 [groups, T*k, 2, r]  per column group: dzg, dzu of the slot's own expert
+  size_t zd_part;               // f32 [groups, T*k, r]  per column group: zd = A_d h of the slot's own expert (forward;
+                                //                 takes the place of zd_all where the grouped kernel forms it)
   size_t dZg, dZu;    // act [T, N*r]      dzg / dzu scattered dense
   size_t dgate;       // f32 [T*k]         by slot id
   size_t dlogits;     // f32 [T, N]
@@ -111,6 +113,19 @@ static inline int grouped_bwd_col_group_min(int tokens, int f) {
   (void)tokens; (void)f;
   return 4;
 }
+// The forward grouped kernel forms zd = h A_d[e]^T (the input of the LoRA of W2) the same way, on 64-column tiles,
+// for ranks up to 32: widest column group (tokens x columns x 2 matrices G, U inside L2) and the condition.
+static inline int grouped_fwd_col_group_max(int tokens, int f) {
+  const long long cols = (32ll << 20) / ((long long)(tokens > 0 ? tokens : 1) * 2 * 2);
+  const long long g = cols / 64;
+  const int ct = grouped_bwd_col_tiles(f);
+  return (int)(g < 1 ? 1 : (g > ct ? ct : g));
+}
+static inline bool grouped_fwd_folds_zd(const mixlora_shape_t& s) {
+  return s.dtype == MIXLORA_DTYPE_BF16 && s.tokens > 0 && s.rank % 8 == 0 && s.rank <= 32 &&
+         grouped_fwd_col_group_max(s.tokens, s.d_ff) >= 4 && (long long)s.tokens * s.d_ff < (1ll << 31);
+}
+static inline int grouped_fwd_max_groups(int f) { return (grouped_bwd_col_tiles(f) + 3) / 4; }
 static inline int grouped_bwd_max_groups(int tokens, int f) {
   const int cg_min = grouped_bwd_col_group_min(tokens, f);
   return (grouped_bwd_col_tiles(f) + cg_min - 1) / cg_min;
@@ -178,6 +193,7 @@ struct Ctx {
 };
 
 static inline bool ctx_folds_dz(const Ctx& c) { return !c.no_fold && grouped_bwd_folds_dz(c.s); }
+static inline bool ctx_folds_zd(const Ctx& c) { return !c.no_fold && grouped_fwd_folds_zd(c.s); }
 
 cudaError_t launch_router(const Ctx& c);              // probs, expert_idx, gates, low_margin, stats
 cudaError_t launch_dispatch(const Ctx& c);            // perm, inv, pos_token, pos_expert, seg_off, tile_info

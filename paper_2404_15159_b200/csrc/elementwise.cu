@@ -95,21 +95,45 @@ lora_b_swiglu_kernel(const T* __restrict__ G, const T* __restrict__ U, const T* 
   }
 }
 
-// hbar_t = sum_j g_tj h_tj ;  Zs[t, e_j*r + rr] = g_tj * zd_j[rr], zero elsewhere.
+// hbar_t = sum_j g_tj h_tj ;  Zs[t, e_j*r + rr] = g_tj * zd_j[rr], zero elsewhere.  With `zd_part` (the forward
+// grouped kernel's per-column-group partial sums [groups, slots, r] of the slot's own expert) zd is those partials
+// added up in group order; else it is read from zd [slots, N r].
 template <typename T>
 __global__ void __launch_bounds__(ENT)
-combine_h_kernel(const T* __restrict__ h_sorted, const T* __restrict__ zd, const float* __restrict__ gates,
+combine_h_kernel(const T* __restrict__ h_sorted, const T* __restrict__ zd, const float* __restrict__ zd_part,
+                 const int* __restrict__ zd_groups, int slots, const float* __restrict__ gates,
                  const int* __restrict__ inv, const int* __restrict__ expert_idx, T* __restrict__ hbar,
                  T* __restrict__ Zs, int f, int N, int r, int k, int do_wide) {
   const int t = blockIdx.x;
   __shared__ int pos[MIXLORA_MAX_TOP_K], ex[MIXLORA_MAX_TOP_K];
   __shared__ float g[MIXLORA_MAX_TOP_K];
+  __shared__ float zds[MIXLORA_MAX_TOP_K * 32];        // fold mode (r <= 32): [slot of the token][r]
   if (threadIdx.x < k) {
     pos[threadIdx.x] = inv[(size_t)t * k + threadIdx.x];
     ex[threadIdx.x] = expert_idx[(size_t)t * k + threadIdx.x];
     g[threadIdx.x] = gates[(size_t)t * k + threadIdx.x];
   }
   __syncthreads();
+  if (zd_part) {
+    const int groups = *zd_groups;
+    const size_t gstride = (size_t)slots * r;
+    for (int i = threadIdx.x; i < k * r; i += blockDim.x) {
+      const int j = i / r;
+      const float* src = zd_part + (size_t)pos[j] * r + (i - j * r);
+      float sum = 0.f;
+      int gi = 0;
+      for (; gi + 8 <= groups; gi += 8) {              // eight groups' loads in flight; the sum keeps group order
+        float tv[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) tv[u] = __ldg(src + (size_t)(gi + u) * gstride);
+#pragma unroll
+        for (int u = 0; u < 8; ++u) sum += tv[u];
+      }
+      for (; gi < groups; ++gi) sum += __ldg(src + (size_t)gi * gstride);
+      zds[i] = sum;
+    }
+    __syncthreads();
+  }
   for (int c = threadIdx.x; do_wide && c < f; c += ENT) {
     float acc = 0.f;
     for (int j = 0; j < k; ++j) acc = fmaf(g[j], to_f(h_sorted[(size_t)pos[j] * f + c]), acc);
@@ -120,7 +144,7 @@ combine_h_kernel(const T* __restrict__ h_sorted, const T* __restrict__ zd, const
     const int e = q / r, rr = q % r;
     float v = 0.f;
     for (int j = 0; j < k; ++j)
-      if (ex[j] == e) v = g[j] * to_f(zd[(size_t)pos[j] * nr + q]);
+      if (ex[j] == e) v = g[j] * (zd_part ? to_f(from_f<T>(zds[j * r + rr])) : to_f(zd[(size_t)pos[j] * nr + q]));
     Zs[(size_t)t * nr + q] = from_f<T>(v);
   }
 }
@@ -613,7 +637,9 @@ cudaError_t combine_h_t(const Ctx& c) {
   // with bf16 activations the f-wide sum runs in its own vectorised kernel; this one then only scatters Zs
   constexpr bool vec = sizeof(T) == 2;
   combine_h_kernel<T><<<c.s.tokens, vec ? 128 : ENT, 0, c.st>>>(
-      c.at<T>(c.L.h_sorted), c.at<T>(c.L.zd_all), c.at<float>(c.L.gates), c.at<int>(c.L.inv), c.at<int>(c.L.expert_idx),
+      c.at<T>(c.L.h_sorted), c.at<T>(c.L.zd_all), ctx_folds_zd(c) ? c.at<float>(c.L.zd_part) : nullptr,
+      c.at<int>(c.L.work_count) + 4, c.s.tokens * c.s.top_k, c.at<float>(c.L.gates), c.at<int>(c.L.inv),
+      c.at<int>(c.L.expert_idx),
       c.at<T>(c.L.hbar), c.at<T>(c.L.Zs), c.s.d_ff, c.s.n_experts, c.s.rank, c.s.top_k, vec ? 0 : 1);
   return cudaGetLastError();
 }

@@ -23,8 +23,10 @@
 // walks the unit's column tiles in turn; after the barrier of an item the store warp's thread multiplies the da and
 // db tiles, still in shared memory, with the matching 64 x 64 blocks of s B_g, s B_u (all experts' blocks side by
 // side, so the block holds the tile's expert) into two accumulators of 64 TMEM columns that live for the whole unit.
-// At the unit's end eight epilogue warps write the expert's own r columns as one fp32 partial per column group; a
+// At the unit's end the gather warps write the expert's own r columns as one fp32 partial per column group; a
 // later kernel adds the groups in a fixed order.  da and db are then not read again for this product.
+// Forward with FOLD: the same for zd = h A_d[e]^T (the input of the LoRA of W2): 64-column tiles like the backward
+// kernel's, which leaves TMEM columns for one accumulator of up to 128; B = the r x 64 block of A_d[e].
 #include <algorithm>
 #include <type_traits>
 
@@ -181,7 +183,7 @@ __device__ __forceinline__ uint64_t sigmoid2(uint64_t a) {
 }
 template <int BWD, int FOLD, int UNITS>
 __global__ void __launch_bounds__(kThreads, 1) grouped_swiglu_kernel(const __grid_constant__ GsParams p) {
-  constexpr int COLS = BWD ? 64 : 128;
+  constexpr int COLS = (BWD || FOLD) ? 64 : 128;
   constexpr int CB = COLS / 64;                        // 64-column blocks per tile
   constexpr int NSUB = BWD ? 3 : 2;                    // MMAs per item
   constexpr int NMAT = BWD ? 3 : 2;                    // gathered matrices G, U (, D)
@@ -193,7 +195,9 @@ __global__ void __launch_bounds__(kThreads, 1) grouped_swiglu_kernel(const __gri
   constexpr uint32_t kDzCol0 = 192, kDzCol1 = 448;     // TMEM columns of the dzg / dzu accumulators (64 each): the
                                                        // backward's two buffers use columns 0-191 and 256-447
                                                        // (dz_readout reads them back)
-  static_assert(!FOLD || (BWD && UNITS), "the rank-r gradients belong to the backward kernel and need units of work");
+  static_assert(!FOLD || UNITS, "the rank-r products accumulate over a unit of work");
+  constexpr uint32_t kZdCol = 128;                     // forward FOLD: TMEM columns of the zd accumulator (up to 128; the
+                                                       // forward's two 128-column buffers sit at 0 and 256)
 
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -337,7 +341,7 @@ __global__ void __launch_bounds__(kThreads, 1) grouped_swiglu_kernel(const __gri
     // ---------------- store warp ----------------
     if (lane == 0) {
       for (int m = 0; m < NOUT; ++m) prefetch_tmap(&p.o_map[m]);
-      if (FOLD) { prefetch_tmap(&p.z_map[0]); prefetch_tmap(&p.z_map[1]); }
+      if (FOLD) { prefetch_tmap(&p.z_map[0]); if (BWD) prefetch_tmap(&p.z_map[1]); }
     }
     const uint32_t out_base = smem_u32(out_smem);
     const uint32_t dzb_base = smem_u32(dzb_smem);
@@ -345,10 +349,15 @@ __global__ void __launch_bounds__(kThreads, 1) grouped_swiglu_kernel(const __gri
     // the 64-column block of the N r experts' columns that holds the tile's expert)
     auto load_dzb = [&](int tile_, int ct_) {
       const int e = p.tile_info[tile_ * 4 + 0];
-      const int zc = (e * p.r_true) / 64 * 64;
-      mbar_expect_tx(dzb_full_bar, 2 * kDzbBytes);
-      tma_load_2d(dzb_base, &p.z_map[0], dzb_full_bar, zc, ct_ * COLS);
-      tma_load_2d(dzb_base + kDzbBytes, &p.z_map[1], dzb_full_bar, zc, ct_ * COLS);
+      if (BWD) {
+        const int zc = (e * p.r_true) / 64 * 64;
+        mbar_expect_tx(dzb_full_bar, 2 * kDzbBytes);
+        tma_load_2d(dzb_base, &p.z_map[0], dzb_full_bar, zc, ct_ * COLS);
+        tma_load_2d(dzb_base + kDzbBytes, &p.z_map[1], dzb_full_bar, zc, ct_ * COLS);
+      } else {                                         // the r x 64 block of A_d[e] under the tile's columns
+        mbar_expect_tx(dzb_full_bar, (uint32_t)p.r * 128u);
+        tma_load_2d(dzb_base, &p.z_map[0], dzb_full_bar, ct_ * COLS, e * p.r);
+      }
     };
     int prev_o = -1;
     uint32_t n = 0, units_done = 0;
@@ -384,16 +393,26 @@ __global__ void __launch_bounds__(kThreads, 1) grouped_swiglu_kernel(const __gri
           if (dz_ok && cur_first) dz_ok = mbar_wait(dzfree_bar, (units_done & 1u) ^ 1u, abort_flag);
           if (dz_ok) {
             tc_fence_after();
-            const uint32_t idesc = make_idesc(64, 0, 1);
+            if (BWD) {
+              const uint32_t idesc = make_idesc(64, 0, 1);
 #pragma unroll
-            for (int m = 0; m < 2; ++m) {
-              const uint32_t a_addr = out_base + o * kOutBytes + m * kBlockBytes;
-              const uint32_t b_addr = dzb_base + m * kDzbBytes;
-              const uint32_t d_tmem = tmem_base + (m == 0 ? kDzCol0 : kDzCol1);
+              for (int m = 0; m < 2; ++m) {
+                const uint32_t a_addr = out_base + o * kOutBytes + m * kBlockBytes;
+                const uint32_t b_addr = dzb_base + m * kDzbBytes;
+                const uint32_t d_tmem = tmem_base + (m == 0 ? kDzCol0 : kDzCol1);
+#pragma unroll
+                for (int k = 0; k < 4; ++k)
+                  umma_bf16(d_tmem, make_desc_kmajor_rows(a_addr + k * 32, 128), make_desc(b_addr + k * 2048, 8192, 1024),
+                            idesc, (cur_first && k == 0) ? 0u : 1u);
+              }
+            } else {
+              // zd += h_tile A_d[e]^T over the tile's 64 columns: both operands K-major with 128-byte rows
+              const uint32_t idesc = make_idesc(p.r, 0, 0);
+              const uint32_t a_addr = out_base + o * kOutBytes;
 #pragma unroll
               for (int k = 0; k < 4; ++k)
-                umma_bf16(d_tmem, make_desc_kmajor_rows(a_addr + k * 32, 128), make_desc(b_addr + k * 2048, 8192, 1024),
-                          idesc, (cur_first && k == 0) ? 0u : 1u);
+                umma_bf16(tmem_base + kZdCol, make_desc_kmajor_rows(a_addr + k * 32, 128),
+                          make_desc_kmajor_rows(dzb_base + k * 32, 128), idesc, (cur_first && k == 0) ? 0u : 1u);
             }
             umma_commit(dzdone_bar);
           }
@@ -449,12 +468,13 @@ __global__ void __launch_bounds__(kThreads, 1) grouped_swiglu_kernel(const __gri
       const int r = p.r_true;
       const int zrow = (warp & 3) * 32 + lane;         // the TMEM lanes this warp may read
       const uint32_t z_addr = tmem_base + ((uint32_t)((warp & 3) * 32) << 16) + (uint32_t)(info >> 16);
-      float* dst = p.dz_part + ((size_t)((info >> 1) & 0x7fff) * p.slots + zp0 + zrow) * 2 * r;
+      constexpr int NZ = BWD ? 2 : 1;                  // accumulators: dzg, dzu backward; zd forward
+      float* dst = p.dz_part + ((size_t)((info >> 1) & 0x7fff) * p.slots + zp0 + zrow) * NZ * r;
       // 8 columns at a time: the expert's columns may end with the accumulator's (and TMEM's) last column
-      for (int m = 0; m < 2; ++m)
+      for (int m = 0; m < NZ; ++m)
         for (int c = 0; c < r; c += 8) {
           uint32_t v[8];
-          tmem_ld8(z_addr + (m == 0 ? kDzCol0 : kDzCol1) + c, v);
+          tmem_ld8(z_addr + (BWD ? (m == 0 ? kDzCol0 : kDzCol1) : kZdCol) + c, v);
           tmem_ld_wait();
           if (zrow < zrows) {
             *reinterpret_cast<float4*>(dst + m * r + c) = make_float4(__uint_as_float(v[0]), __uint_as_float(v[1]),
@@ -497,7 +517,8 @@ __global__ void __launch_bounds__(kThreads, 1) grouped_swiglu_kernel(const __gri
         if (gitem >= (uint32_t)p.nsets) { old_info = note[0]; old_p0 = note[1]; old_rows = note[2]; }
         __syncwarp();
         if (lane == 0) {
-          note[0] = (last ? 1 : 0) | (walk.group << 1) | (((p.tile_info[tile * 4 + 0] * p.r_true) & 63) << 16);
+          note[0] = (last ? 1 : 0) | (walk.group << 1) |
+                    ((BWD ? (p.tile_info[tile * 4 + 0] * p.r_true) & 63 : 0) << 16);
           note[1] = p0;
           note[2] = rows;
         }
@@ -710,12 +731,11 @@ __global__ void __launch_bounds__(kThreads, 1) grouped_swiglu_kernel(const __gri
 
 template <int BWD>
 cudaError_t launch_t(const Ctx& c) {
-  constexpr int COLS = BWD ? 64 : 128;
-  constexpr int CB = COLS / 64;
   constexpr int NMAT = BWD ? 3 : 2;
   const int slots = c.s.tokens * c.s.top_k, f = c.s.d_ff, r = c.s.rank, N = c.s.n_experts;
   const int rp = pad_rank(r);
-  const bool fold = BWD && ctx_folds_dz(c);
+  const bool fold = BWD ? ctx_folds_dz(c) : ctx_folds_zd(c);
+  const int COLS = (BWD || fold) ? 64 : 128, CB = COLS / 64;
   GsParams p;
   memset(&p, 0, sizeof(p));
   p.row_bytes = rp >= 64 ? 128 : rp * 2;               // bytes of one operand row per k-block
@@ -761,9 +781,11 @@ cudaError_t launch_t(const Ctx& c) {
          tc_encode_2d(&p.b_map[2], ad, (long long)N * rp, f, f, p.krows, 64, 128) &&
          tc_encode_2d(&p.o_map[0], c.ws + c.L.da_sorted, slots, f, f, BM, 64, 128) &&
          tc_encode_2d(&p.o_map[1], c.ws + c.L.db_sorted, slots, f, f, BM, 64, 128);
-  if (fold)
+  if (fold && BWD)
     ok = ok && tc_encode_2d(&p.z_map[0], c.ws + c.L.bg_cat, f, (long long)N * r, (long long)N * r, 64, 64, 128) &&
          tc_encode_2d(&p.z_map[1], c.ws + c.L.bu_cat, f, (long long)N * r, (long long)N * r, 64, 64, 128);
+  if (fold && !BWD)
+    ok = ok && tc_encode_2d(&p.z_map[0], ad, (long long)N * rp, f, f, rp, 64, 128);
   if (!ok) return cudaErrorInvalidValue;
   p.G = c.at<bf16>(c.L.G); p.U = c.at<bf16>(c.L.U); p.D = c.at<bf16>(c.L.D);
   p.pos_token = c.at<int>(c.L.pos_token); p.perm = c.at<int>(c.L.perm); p.gates = c.at<float>(c.L.gates);
@@ -777,11 +799,18 @@ cudaError_t launch_t(const Ctx& c) {
   const long long group_cols = (32ll << 20) / ((long long)c.s.tokens * 2 * NMAT);
   p.col_group = (int)std::min<long long>(std::max<long long>(group_cols / COLS, 1), p.col_tiles);
   p.cg_min = (p.col_group + 1) / 2;                    // units of work: the kernel may settle on narrower groups
-  if (fold) {
+  if (fold && BWD) {
     p.col_group = grouped_bwd_col_group_max(c.s.tokens, f);
     p.cg_min = grouped_bwd_col_group_min(c.s.tokens, f);
     p.dz_part = c.at<float>(c.L.dz_part);
     p.groups_used = c.at<int>(c.L.work_count) + 3;
+    p.r_true = r;
+  }
+  if (fold && !BWD) {
+    p.col_group = grouped_fwd_col_group_max(c.s.tokens, f);
+    p.cg_min = 4;
+    p.dz_part = c.at<float>(c.L.zd_part);
+    p.groups_used = c.at<int>(c.L.work_count) + 4;
     p.r_true = r;
   }
   p.status = c.at<int>(c.L.status);
@@ -791,9 +820,9 @@ cudaError_t launch_t(const Ctx& c) {
   // the number of segment tiles is only known on the device; every CTA reads it and idles if it has no item
   cudaError_t e;
   if (fold) {
-    e = cudaFuncSetAttribute(grouped_swiglu_kernel<BWD, BWD, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes);
+    e = cudaFuncSetAttribute(grouped_swiglu_kernel<BWD, 1, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes);
     if (e != cudaSuccess) return e;
-    grouped_swiglu_kernel<BWD, BWD, 1><<<sms, kThreads, smem_bytes, c.st>>>(p);
+    grouped_swiglu_kernel<BWD, 1, 1><<<sms, kThreads, smem_bytes, c.st>>>(p);
   } else {
     e = cudaFuncSetAttribute(grouped_swiglu_kernel<BWD, 0, kUnitsAlways>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes);
     if (e != cudaSuccess) return e;
