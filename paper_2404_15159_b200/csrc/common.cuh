@@ -114,7 +114,9 @@ static inline int grouped_bwd_col_group_min(int tokens, int f) {
   return 4;
 }
 // The forward grouped kernel forms zd = h A_d[e]^T (the input of the LoRA of W2) the same way, on 64-column tiles,
-// for ranks up to 32: widest column group (tokens x columns x 2 matrices G, U inside L2) and the condition.
+// for ranks up to 32: widest column group (tokens x columns x 2 matrices G, U inside L2) and the condition.  The
+// narrower tile costs the kernel about as much as the dense product it replaces at 8192 tokens of the 7B width
+// (measured), and less below, so the fold is taken up to 4096 tokens there (groups of at least 32 tiles).
 static inline int grouped_fwd_col_group_max(int tokens, int f) {
   const long long cols = (32ll << 20) / ((long long)(tokens > 0 ? tokens : 1) * 2 * 2);
   const long long g = cols / 64;
@@ -123,7 +125,7 @@ static inline int grouped_fwd_col_group_max(int tokens, int f) {
 }
 static inline bool grouped_fwd_folds_zd(const mixlora_shape_t& s) {
   return s.dtype == MIXLORA_DTYPE_BF16 && s.tokens > 0 && s.rank % 8 == 0 && s.rank <= 32 &&
-         grouped_fwd_col_group_max(s.tokens, s.d_ff) >= 4 && (long long)s.tokens * s.d_ff < (1ll << 31);
+         grouped_fwd_col_group_max(s.tokens, s.d_ff) >= 32 && (long long)s.tokens * s.d_ff < (1ll << 31);
 }
 static inline int grouped_fwd_max_groups(int f) { return (grouped_bwd_col_tiles(f) + 3) / 4; }
 static inline int grouped_bwd_max_groups(int tokens, int f) {
