@@ -71,7 +71,7 @@ WsLayout ws_layout(const mixlora_shape_t& s, bool allow_fold) {
   L.work_count = take(8 * 4);
   L.work_rows1 = take((size_t)rows_worklist_max(s.tokens * s.top_k, s.n_experts, 1) * 32);
   L.total_fwd = off;
-  L.D = take(T * f * E);
+  L.D = L.hbar;                      // hbar (forward scratch) is dead once y is written; D = dy W_d takes its place
   L.spd = take(T * N * r * E);
   L.da_sorted = take(T * k * f * E);
   L.db_sorted = take(T * k * f * E);
@@ -1010,6 +1010,7 @@ mixlora_status_t mixlora_dora_ffn_forward(const mixlora_shape_t* shape, const mi
   if ((st = fwd_route(c)) != MIXLORA_OK) return st;
   // the scales c = m / n of the three projections: |W_o + s B_o A|^2 = |W_o|^2 + 2 s B_o . (W A^T)_o + s^2 B_o (A A^T) B_o^T
   {
+    StageScope ss(ST_NORM, c.st, 12);
     TcOut gu[2];
     gu[0] = tc_out_f32(dc.wa_g, Nr, Nr, 1, 0, 0, 1.f, 0); tc_add(gu[0], params->w_gate, d, d, params->a_gate, d, 0);
     gu[1] = tc_out_f32(dc.wa_u, Nr, Nr, 1, 0, 0, 1.f, 0); tc_add(gu[1], params->w_up, d, d, params->a_up, d, 0);
@@ -1027,8 +1028,9 @@ mixlora_status_t mixlora_dora_ffn_forward(const mixlora_shape_t* shape, const mi
     MIXLORA_CUDA(launch_dora_scales(c, dc));
   }
   if ((st = fwd_shared_projections(&c, 1)) != MIXLORA_OK) return st;   // W1 x, W3 x once per token, A_g x, A_u x
-  MIXLORA_CUDA(launch_dora_swiglu_fwd(c, dc));
+  { StageScope ss(ST_LORA_B_SWIGLU, c.st, 1); MIXLORA_CUDA(launch_dora_swiglu_fwd(c, dc)); }
   {   // zd = A_d h against every expert, then the slot's own block (and gate times it)
+    StageScope ss(ST_LORA_A_DOWN, c.st, 2);
     TcOut out = tc_out(c.ws + c.L.zd_all, Nr, Nr);
     tc_add(out, c.ws + c.L.h_sorted, f, f, params->a_down, f, 0);
     MIXLORA_CUDA(dense_product(c, T * k, &out, 1));
@@ -1036,12 +1038,13 @@ mixlora_status_t mixlora_dora_ffn_forward(const mixlora_shape_t* shape, const mi
   }
   {   // o_pre = [h | Zd] [W2 | s B_d]^T per sorted slot: W2 cannot act on the gate-weighted sum of a token's slots
       // here, because the scale of its output differs between the token's experts
+    StageScope ss(ST_GEMM_DOWN, c.st, 1);
     TcOut out = tc_out(dc.o_pre, d, d);
     tc_add(out, c.ws + c.L.h_sorted, f, f, params->w_down, f, 0);
     tc_add(out, dc.Zd_pos, Nr, Nr, c.ws + c.L.bd_cat, Nr, 0);
     MIXLORA_CUDA(dense_product(c, T * k, &out, 1));
   }
-  MIXLORA_CUDA(launch_dora_combine_y(c, dc, y));
+  { StageScope ss(ST_COMBINE_H, c.st, 1); MIXLORA_CUDA(launch_dora_combine_y(c, dc, y)); }
   return MIXLORA_OK;
 }
 
@@ -1073,15 +1076,17 @@ mixlora_status_t mixlora_dora_ffn_backward(const mixlora_shape_t* shape, const m
     return MIXLORA_OK;
   }
   // dO = c_d * dy per sorted slot (and the down magnitude's shares), then D = dO W2 and s B_d^T dO per slot
-  MIXLORA_CUDA(launch_dora_dout(c, dc, dy));
+  { StageScope ss(ST_COMBINE_BWD, c.st, 1); MIXLORA_CUDA(launch_dora_dout(c, dc, dy)); }
   {
+    StageScope ss(ST_GEMM_DGRAD_DOWN, c.st, 1);
     TcOut outs[2];
     outs[0] = tc_out(dc.D_s, f, f);      tc_add(outs[0], dc.dO, d, d, params->w_down, f, 1);
     outs[1] = tc_out(dc.spd_s, Nr, Nr);  tc_add(outs[1], dc.dO, d, d, c.ws + c.L.bd_cat, Nr, 1);
     MIXLORA_CUDA(dense_product(c, T * k, outs, 2));
   }
-  MIXLORA_CUDA(launch_dora_swiglu_bwd(c, dc));
-  MIXLORA_CUDA(launch_dgate_reduce(c, dora_bwd_col_chunks(f)));
+  { StageScope ss(ST_SWIGLU_BWD, c.st, 2);
+    MIXLORA_CUDA(launch_dora_swiglu_bwd(c, dc));
+    MIXLORA_CUDA(launch_dgate_reduce(c, dora_bwd_col_chunks(f))); }
   MIXLORA_CUDA(launch_router_bwd(c, aux_coef, grads->d_router_bias, acc, want_dx));
   if (mgrads->d_m_gate) MIXLORA_CUDA(launch_dora_dm_reduce(c, dc.dmp_g, dc.inv_g, mgrads->d_m_gate, f, acc));
   if (mgrads->d_m_up) MIXLORA_CUDA(launch_dora_dm_reduce(c, dc.dmp_u, dc.inv_u, mgrads->d_m_up, f, acc));

@@ -18,6 +18,21 @@ __device__ __forceinline__ float sigmoidf_(float v) { return 1.f / (1.f + expf(-
 
 constexpr int kCols = 256;   // columns (threads) per block of the tile kernels
 
+// 8 consecutive values of a row as floats (16-byte loads; the row start is 16-byte aligned when r % 8 == 0)
+__device__ __forceinline__ void load8(const bf16* p, float (&o)[8]) {
+  const uint4 raw = __ldg(reinterpret_cast<const uint4*>(p));
+  const uint32_t w[4] = {raw.x, raw.y, raw.z, raw.w};
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    o[2 * i] = __uint_as_float(w[i] << 16);
+    o[2 * i + 1] = __uint_as_float(w[i] & 0xffff0000u);
+  }
+}
+__device__ __forceinline__ void load8(const float* p, float (&o)[8]) {
+  const float4 a = __ldg(reinterpret_cast<const float4*>(p)), b = __ldg(reinterpret_cast<const float4*>(p) + 1);
+  o[0] = a.x; o[1] = a.y; o[2] = a.z; o[3] = a.w; o[4] = b.x; o[5] = b.y; o[6] = b.z; o[7] = b.w;
+}
+
 // rowsq[o] = sum_c W[o, c]^2, one warp per row
 template <typename T>
 __global__ void rowsq_kernel(const T* __restrict__ w, float* __restrict__ rowsq, int rows, int cols) {
@@ -60,53 +75,77 @@ __global__ void dora_scale_kernel(const float* __restrict__ rowsq, const float* 
   }
 }
 
-// Forward, per sorted slot (blocks of 8 slots, a thread per column): a = c_g[e] (G_t + s B_g[e] zg),
+// Forward, per single-expert tile and chunk of 256 columns (a thread per column, 8 rows at a time in registers so
+// that a column's rows of B_g[e], B_u[e] are read once per 8 slots): a = c_g[e] (G_t + s B_g[e] zg),
 // b = c_u[e] (U_t + s B_u[e] zu), h = SiLU(a) b.
-constexpr int SL = 8;
 template <typename T>
 __global__ void __launch_bounds__(kCols)
 dora_swiglu_fwd_kernel(const T* __restrict__ G, const T* __restrict__ U, const T* __restrict__ zga,
                        const T* __restrict__ zua, const T* __restrict__ b_gate, const T* __restrict__ b_up,
                        const float* __restrict__ cg, const float* __restrict__ cu, const int* __restrict__ pos_token,
-                       const int* __restrict__ pos_expert, T* __restrict__ h_sorted, int slots, int f, int N, int r,
+                       const int* __restrict__ tile_info, int max_tiles, T* __restrict__ h_sorted, int f, int N, int r,
                        float s) {
+  constexpr int RB = 8;
   extern __shared__ float sm[];
-  float* zg = sm;              // [SL][r], already scaled by s
-  float* zu = sm + SL * r;
-  __shared__ int tok[SL], ex[SL];
-  const int base = blockIdx.x * SL;
-  const int ns = min(SL, slots - base);
-  if (threadIdx.x < SL) {
-    tok[threadIdx.x] = (threadIdx.x < ns) ? pos_token[base + threadIdx.x] : 0;
-    ex[threadIdx.x] = (threadIdx.x < ns) ? pos_expert[base + threadIdx.x] : 0;
-  }
-  __syncthreads();
-  for (int i = threadIdx.x; i < SL * r; i += kCols) {
-    const int sl = i / r, rr = i % r;
-    float vg = 0.f, vu = 0.f;
-    if (sl < ns) {
-      const size_t o = (size_t)tok[sl] * N * r + (size_t)ex[sl] * r + rr;
-      vg = s * to_f(zga[o]);
-      vu = s * to_f(zua[o]);
-    }
-    zg[i] = vg;
-    zu[i] = vu;
-  }
-  __syncthreads();
-  for (int c = threadIdx.x; c < f; c += kCols) {
-    for (int i = 0; i < ns; ++i) {
-      const int e = ex[i];
-      const T* bg = b_gate + ((size_t)e * f + c) * r;
-      const T* bu = b_up + ((size_t)e * f + c) * r;
-      float ea = 0.f, eb = 0.f;
-      for (int rr = 0; rr < r; ++rr) {
-        ea = fmaf(zg[i * r + rr], to_f(bg[rr]), ea);
-        eb = fmaf(zu[i * r + rr], to_f(bu[rr]), eb);
+  float* zg = sm;                                // [RB][r], already scaled by s
+  float* zu = zg + RB * r;
+  __shared__ int tok[kSegTile];
+  const int tile = blockIdx.x;
+  const int c = blockIdx.y * kCols + threadIdx.x;
+  if (tile >= min(tile_info[max_tiles * 4], max_tiles)) return;
+  const int e = tile_info[tile * 4 + 0], p0 = tile_info[tile * 4 + 1], rows = tile_info[tile * 4 + 2];
+  for (int i = threadIdx.x; i < rows; i += kCols) tok[i] = pos_token[p0 + i];
+  const bool live = c < f;
+  const int cc = live ? c : f - 1;               // threads past the width read valid data and store nothing
+  const T* bg = b_gate + ((size_t)e * f + cc) * r;
+  const T* bu = b_up + ((size_t)e * f + cc) * r;
+  const float cgv = cg[(size_t)e * f + cc], cuv = cu[(size_t)e * f + cc];
+  for (int i0 = 0; i0 < rows; i0 += RB) {
+    __syncthreads();                             // tok is set; the previous rows' vectors are no longer read
+    for (int i = threadIdx.x; i < RB * r; i += kCols) {
+      const int sl = i / r, rr = i % r;
+      float vg = 0.f, vu = 0.f;
+      if (i0 + sl < rows) {
+        const size_t o = ((size_t)tok[i0 + sl] * N + e) * r + rr;
+        vg = s * to_f(zga[o]);
+        vu = s * to_f(zua[o]);
       }
-      const size_t go = (size_t)tok[i] * f + c;
-      const float a = cg[(size_t)e * f + c] * (to_f(G[go]) + ea);
-      const float b = cu[(size_t)e * f + c] * (to_f(U[go]) + eb);
-      h_sorted[(size_t)(base + i) * f + c] = from_f<T>(a * sigmoidf_(a) * b);
+      zg[rr * RB + sl] = vg; zu[rr * RB + sl] = vu;      // [rr][row]: a step of the rank reads 8 rows as two float4
+    }
+    __syncthreads();
+    float ea[RB], eb[RB];
+#pragma unroll
+    for (int i = 0; i < RB; ++i) { ea[i] = 0.f; eb[i] = 0.f; }
+    auto rank_step = [&](int rr, float wg, float wu) {
+      const float4 g0 = *reinterpret_cast<const float4*>(zg + rr * RB), g1 = *reinterpret_cast<const float4*>(zg + rr * RB + 4);
+      const float4 u0 = *reinterpret_cast<const float4*>(zu + rr * RB), u1 = *reinterpret_cast<const float4*>(zu + rr * RB + 4);
+      const float zgv[RB] = {g0.x, g0.y, g0.z, g0.w, g1.x, g1.y, g1.z, g1.w};
+      const float zuv[RB] = {u0.x, u0.y, u0.z, u0.w, u1.x, u1.y, u1.z, u1.w};
+#pragma unroll
+      for (int i = 0; i < RB; ++i) {
+        ea[i] = fmaf(zgv[i], wg, ea[i]);
+        eb[i] = fmaf(zuv[i], wu, eb[i]);
+      }
+    };
+    if (r % 8 == 0) {
+      for (int r0 = 0; r0 < r; r0 += 8) {
+        float wg[8], wu[8];
+        load8(bg + r0, wg);
+        load8(bu + r0, wu);
+#pragma unroll
+        for (int q = 0; q < 8; ++q) rank_step(r0 + q, wg[q], wu[q]);
+      }
+    } else {
+      for (int rr = 0; rr < r; ++rr) rank_step(rr, to_f(bg[rr]), to_f(bu[rr]));
+    }
+#pragma unroll
+    for (int i = 0; i < RB; ++i) {
+      if (i0 + i < rows && live) {
+        const size_t go = (size_t)tok[i0 + i] * f + c;
+        const float a = cgv * (to_f(G[go]) + ea[i]);
+        const float b = cuv * (to_f(U[go]) + eb[i]);
+        h_sorted[(size_t)(p0 + i0 + i) * f + c] = from_f<T>(a * sigmoidf_(a) * b);
+      }
     }
   }
 }
@@ -229,20 +268,37 @@ dora_swiglu_bwd_kernel(const T* __restrict__ G, const T* __restrict__ U, const T
         vu = s * to_f(zua[o]);
         vp = to_f(spd[((size_t)(p0 + i0 + sl) * N + e) * r + rr]);
       }
-      zg[i] = vg; zu[i] = vu; pd[i] = vp;
+      zg[rr * RB + sl] = vg; zu[rr * RB + sl] = vu; pd[rr * RB + sl] = vp;   // [rr][row]
     }
     __syncthreads();
     float ea[RB], eb[RB], ed[RB];
 #pragma unroll
     for (int i = 0; i < RB; ++i) { ea[i] = 0.f; eb[i] = 0.f; ed[i] = 0.f; }
-    for (int rr = 0; rr < r; ++rr) {
-      const float wg = to_f(bg[rr]), wu = to_f(bu[rr]), wd = to_f(ad[(size_t)rr * f]);
+    auto rank_step = [&](int rr, float wg, float wu) {
+      const float wd = to_f(ad[(size_t)rr * f]);
+      const float4 g0 = *reinterpret_cast<const float4*>(zg + rr * RB), g1 = *reinterpret_cast<const float4*>(zg + rr * RB + 4);
+      const float4 u0 = *reinterpret_cast<const float4*>(zu + rr * RB), u1 = *reinterpret_cast<const float4*>(zu + rr * RB + 4);
+      const float4 d0 = *reinterpret_cast<const float4*>(pd + rr * RB), d1 = *reinterpret_cast<const float4*>(pd + rr * RB + 4);
+      const float zgv[RB] = {g0.x, g0.y, g0.z, g0.w, g1.x, g1.y, g1.z, g1.w};
+      const float zuv[RB] = {u0.x, u0.y, u0.z, u0.w, u1.x, u1.y, u1.z, u1.w};
+      const float pdv[RB] = {d0.x, d0.y, d0.z, d0.w, d1.x, d1.y, d1.z, d1.w};
 #pragma unroll
       for (int i = 0; i < RB; ++i) {
-        ea[i] = fmaf(zg[i * r + rr], wg, ea[i]);
-        eb[i] = fmaf(zu[i * r + rr], wu, eb[i]);
-        ed[i] = fmaf(pd[i * r + rr], wd, ed[i]);
+        ea[i] = fmaf(zgv[i], wg, ea[i]);
+        eb[i] = fmaf(zuv[i], wu, eb[i]);
+        ed[i] = fmaf(pdv[i], wd, ed[i]);
       }
+    };
+    if (r % 8 == 0) {
+      for (int r0 = 0; r0 < r; r0 += 8) {
+        float wg[8], wu[8];
+        load8(bg + r0, wg);
+        load8(bu + r0, wu);
+#pragma unroll
+        for (int q = 0; q < 8; ++q) rank_step(r0 + q, wg[q], wu[q]);
+      }
+    } else {
+      for (int rr = 0; rr < r; ++rr) rank_step(rr, to_f(bg[rr]), to_f(bu[rr]));
     }
 #pragma unroll
     for (int i = 0; i < RB; ++i) {
@@ -318,11 +374,12 @@ cudaError_t scales_t(const Ctx& c, const DoraCtx& dc) {
 
 template <typename T>
 cudaError_t swiglu_fwd_t(const Ctx& c, const DoraCtx& dc) {
-  const int slots = c.s.tokens * c.s.top_k;
-  dora_swiglu_fwd_kernel<T><<<(slots + SL - 1) / SL, kCols, 2 * SL * c.s.rank * sizeof(float), c.st>>>(
+  const int mt = max_seg_tiles(c.s.tokens, c.s.top_k, c.s.n_experts);
+  dim3 grid(mt, (c.s.d_ff + kCols - 1) / kCols);
+  dora_swiglu_fwd_kernel<T><<<grid, kCols, 2 * 8 * c.s.rank * sizeof(float), c.st>>>(
       c.at<T>(c.L.G), c.at<T>(c.L.U), c.at<T>(c.L.zga), c.at<T>(c.L.zua), reinterpret_cast<const T*>(c.p.b_gate),
-      reinterpret_cast<const T*>(c.p.b_up), dc.cg, dc.cu, c.at<int>(c.L.pos_token), c.at<int>(c.L.pos_expert),
-      c.at<T>(c.L.h_sorted), slots, c.s.d_ff, c.s.n_experts, c.s.rank, c.scale);
+      reinterpret_cast<const T*>(c.p.b_up), dc.cg, dc.cu, c.at<int>(c.L.pos_token), c.at<int>(c.L.tile_info), mt,
+      c.at<T>(c.L.h_sorted), c.s.d_ff, c.s.n_experts, c.s.rank, c.scale);
   return cudaGetLastError();
 }
 
