@@ -26,7 +26,7 @@ import numpy as np
 
 from paper_2404_15159_b200 import synth
 
-DRAM_CAPTURE = "profiles/tc_gemm_pair_kernel_c3_dram.md"
+DRAM_CAPTURE = "profiles/c3_step_dram_bytes.md"
 METRIC = "mixlora_ffn_fwd_bwd_tokens_per_s"
 UNIT = "tokens/s"
 AUX_COEF = 0.01
@@ -539,7 +539,7 @@ def run_cuda(args):
     roofline["hbm_peak_gbs"] = peaks["hbm_gbs"]
     # DRAM bytes (read + write) of the frozen-projection launches, from one single-pass ncu capture of this command's
     # workload at full size (summary under profiles/); other workloads have no capture
-    measured_dram = {"gemm_gate_up": 905.3e6, "gemm_down": 905.9e6, "gemm_dgrad_down": 463.9e6, "gemm_dx": 2110.0e6}
+    measured_dram = {"gemm_gate_up": 887.7e6, "gemm_down": 901.7e6, "gemm_dgrad_down": 460.7e6, "gemm_dx": 1798.2e6}
     algorithmic_dram = {"gemm_gate_up": (T_ * d_ + 2 * f_ * d_ + 2 * T_ * f_) * E,
                         "gemm_down": (T_ * f_ + f_ * d_ + T_ * d_) * E,
                         "gemm_dgrad_down": (T_ * d_ + f_ * d_ + T_ * f_) * E,
