@@ -77,7 +77,6 @@ WsLayout ws_layout(const mixlora_shape_t& s, bool allow_fold) {
   L.db_sorted = take(T * k * f * E);
   L.dabar = take(T * f * E);
   L.dbbar = take(T * f * E);
-  L.P_pos = take(T * k * N * r * E);
   L.p_s = take(T * k * rp * E);
   L.dZd_pos = take(T * k * N * r * E);
   L.dgate_part = take((size_t)grouped_swiglu_bwd_col_tiles(s.d_ff) * T * k * 4);

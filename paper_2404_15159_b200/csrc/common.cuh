@@ -57,9 +57,8 @@ struct WsLayout {
   size_t spd;         // act [T, N*r]      s * B_d^T dy for every expert
   size_t da_sorted, db_sorted;  // act [T*k, f]
   size_t dabar, dbbar;          // act [T, f]
-  size_t P_pos;                 // act [T*k, N*r]  s * pd of the slot in its expert block, zero elsewhere
   size_t p_s;                   // act [T*k, pad_rank(r)]  s * pd of the slot's own expert, zero padded
-  size_t dZd_pos;               // act [T*k, N*r]  gate * P_pos
+  size_t dZd_pos;               // act [T*k, N*r]  gate * s * pd of the slot in its expert block, zero elsewhere
   size_t dgate_part;            // f32 [ceil(f/64), T*k]  per column tile partial <Dt, h> of the fused backward
   size_t dzg_all, dzu_all;      // act [T*k, N*r]  da (s B_g) and db (s B_u) against every expert (not when the
                                 //                 grouped kernel forms them, see dz_part)
@@ -92,20 +91,21 @@ static inline int pad_rank(int r) { return r <= 16 ? 16 : (r <= 32 ? 32 : (r <= 
 WsLayout ws_layout(const mixlora_shape_t& s, bool allow_fold = true);
 
 // Column tiles of the backward grouped SwiGLU kernel (64 columns each) and the widest group of them whose pieces of
-// G, U and D (tokens x columns x 3 matrices) stay well inside L2 while every segment tile of the group is worked on.
+// G, U and D (tokens x columns x 3 matrices) stay well inside L2 while every segment tile of the group is worked on;
+// never narrower than 4 tiles (beyond about 14 000 tokens at the 7B width the group then outgrows that share of L2,
+// which measured cheaper than giving the fold up: 3.04 -> 2.64 ms for the three backward stages at 32768 tokens).
 static inline int grouped_bwd_col_tiles(int f) { return (f + 63) / 64; }
 static inline int grouped_bwd_col_group_max(int tokens, int f) {
   const long long cols = (32ll << 20) / ((long long)(tokens > 0 ? tokens : 1) * 2 * 3);
   const long long g = cols / 64;
   const int ct = grouped_bwd_col_tiles(f);
-  return (int)(g < 1 ? 1 : (g > ct ? ct : g));
+  return (int)(g < 4 ? 4 : (g > ct ? ct : g));
 }
 // The backward grouped kernel also forms dzg = da (s B_g), dzu = db (s B_u) of a slot's own expert (summed over the
-// column tiles of a group in TMEM, one fp32 partial per group) when the rank divides a 64-column operand block and
-// the groups are wide enough for the partials to be small beside da, db themselves.
+// column tiles of a group in TMEM, one fp32 partial per group) when the rank divides a 64-column operand block.
 static inline bool grouped_bwd_folds_dz(const mixlora_shape_t& s) {
   return s.dtype == MIXLORA_DTYPE_BF16 && s.tokens > 0 && (s.rank == 8 || s.rank == 16 || s.rank == 32) &&
-         grouped_bwd_col_group_max(s.tokens, s.d_ff) >= 4 && (long long)s.tokens * s.d_ff < (1ll << 31);
+         (long long)s.tokens * s.d_ff < (1ll << 31);
 }
 // the kernel may narrow the groups down to 4 tiles to even out the CTAs' shares (with few tokens there are few segment
 // tiles, and wide groups would leave most CTAs without a unit): narrowest width, and the bound of the group count
@@ -215,7 +215,7 @@ cudaError_t launch_grouped_swiglu_bwd(const Ctx& c);
 cudaError_t launch_lora_b_swiglu(const Ctx& c);       // h_sorted from G, U, zga, zua, B_g, B_u
 cudaError_t launch_combine_h(const Ctx& c);           // hbar, Zs
 cudaError_t launch_swiglu_bwd(const Ctx& c);          // h_sorted, da_sorted, db_sorted, dgate, Zg_pos, Zu_pos
-cudaError_t launch_slot_prep_bwd(const Ctx& c);       // P_pos, dZd_pos
+cudaError_t launch_slot_prep_bwd(const Ctx& c);       // dZd_pos, p_s
 cudaError_t launch_combine_bwd(const Ctx& c, int want_dx);  // dZg, dZu and, for dx, dabar, dbbar
 cudaError_t launch_router_bwd(const Ctx& c, float aux_coef, float* d_bias, int accumulate, int want_dx);
 // the block inside its layer (Eq. 5 / Eq. 6)

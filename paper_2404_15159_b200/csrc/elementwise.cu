@@ -341,19 +341,14 @@ swiglu_bwd_kernel(const T* __restrict__ G, const T* __restrict__ U, const T* __r
 template <typename T>
 __global__ void slot_prep_bwd_kernel(const T* __restrict__ spd, const float* __restrict__ gates,
                                      const int* __restrict__ perm, const int* __restrict__ pos_token,
-                                     const int* __restrict__ pos_expert, T* __restrict__ P_pos,
+                                     const int* __restrict__ pos_expert,
                                      T* __restrict__ dZd_pos, T* __restrict__ p_s, int slots, int N, int r, int rp) {
   const long long nr = (long long)N * r;
   const long long n = (long long)slots * nr;
   for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < n; i += (long long)gridDim.x * blockDim.x) {
     const int pos = (int)(i / nr), q = (int)(i % nr);
-    T pv = from_f<T>(0.f);
     float v = 0.f;
-    if (q / r == pos_expert[pos]) {
-      pv = spd[(size_t)pos_token[pos] * nr + q];
-      v = gates[perm[pos]] * to_f(pv);
-    }
-    P_pos[i] = pv;
+    if (q / r == pos_expert[pos]) v = gates[perm[pos]] * to_f(spd[(size_t)pos_token[pos] * nr + q]);
     dZd_pos[i] = from_f<T>(v);
   }
   // compact copy: the slot's own r values, zero padded to rp
@@ -664,7 +659,7 @@ cudaError_t slot_prep_bwd_t(const Ctx& c) {
   const int slots = c.s.tokens * c.s.top_k;
   slot_prep_bwd_kernel<T><<<grid_for((long long)slots * c.s.rank * c.s.n_experts, 256), 256, 0, c.st>>>(
       c.at<T>(c.L.spd), c.at<float>(c.L.gates), c.at<int>(c.L.perm), c.at<int>(c.L.pos_token),
-      c.at<int>(c.L.pos_expert), c.at<T>(c.L.P_pos), c.at<T>(c.L.dZd_pos), c.at<T>(c.L.p_s), slots, c.s.n_experts,
+      c.at<int>(c.L.pos_expert), c.at<T>(c.L.dZd_pos), c.at<T>(c.L.p_s), slots, c.s.n_experts,
       c.s.rank, pad_rank(c.s.rank));
   return cudaGetLastError();
 }
