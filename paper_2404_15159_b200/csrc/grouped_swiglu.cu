@@ -9,7 +9,7 @@
 //   gather warps  : fetch the shared projections G, U (and D = dy W_d) of the tile's tokens with cp.async, four
 //                   rows of 128 contiguous bytes per warp instruction, into a ring of 128B-swizzled smem tiles,
 //                   up to three items ahead of the epilogue; they also look up the item's slot range and gates
-//   16 epilogue warps: a = G + da, b = U + db, h = SiLU(a) b (backward: Dt = D + dd, dgate, d a, d b as well) in
+//   16 (8 backward) epilogue warps: a = G + da, b = U + db, h = SiLU(a) b (backward: Dt = D + dd, dgate, d a, d b as well) in
 //                   packed fp32 pairs, into one of two swizzled output tiles; one CTA-wide barrier per item
 //   store warp    : after that barrier, sends full tiles out by TMA, waits until the copy has read the tile and
 //                   hands it back; the last, shorter tile of a segment (whose remaining rows belong to the next
@@ -39,14 +39,19 @@ namespace {
 
 using namespace tc;
 
-constexpr int kSplit = 4;                 // epilogue warps per TMEM lane quarter
-constexpr int NET = 128 * kSplit;         // epilogue threads
+// epilogue warps per TMEM lane quarter: 4 forward (16 warps, 80 registers per thread); 2 backward, whose heavier
+// per-element arithmetic gains a little more from 128 registers per thread (8 warps) than from the extra warps
+// (measured at C3: forward 0.217 ms with 4 against 0.235 with 2, backward 0.472 with 4 against 0.456 with 2)
+template <int BWD> struct Epi {
+  static constexpr int kSplit = BWD ? 2 : 4;
+  static constexpr int NET = 128 * kSplit;   // epilogue threads
+};
 constexpr int kStoreWarp = 2;             // issues the TMA stores of the results
 constexpr int kGatherWarps = 4;           // warps that fetch the G / U / D rows
 constexpr int NGT = 32 * kGatherWarps;
 constexpr int kFirstGatherWarp = 3;
 constexpr int kFirstEpiWarp = kFirstGatherWarp + kGatherWarps;
-constexpr int kThreads = 32 * kFirstEpiWarp + NET;
+template <int BWD> constexpr int kThreadsOf = 32 * kFirstEpiWarp + Epi<BWD>::NET;
 constexpr int kRowsPerPass = NGT / 8;     // rows one pass of the gather threads covers
 constexpr int kPasses = 128 / kRowsPerPass;
 constexpr uint32_t kTmemCols = 512;
@@ -182,7 +187,8 @@ __device__ __forceinline__ uint64_t sigmoid2(uint64_t a) {
   return fma2(pk2(tl, th), kHalf2, kHalf2);
 }
 template <int BWD, int FOLD, int UNITS>
-__global__ void __launch_bounds__(kThreads, 1) grouped_swiglu_kernel(const __grid_constant__ GsParams p) {
+__global__ void __launch_bounds__(kThreadsOf<BWD>, 1) grouped_swiglu_kernel(const __grid_constant__ GsParams p) {
+  constexpr int kSplit = Epi<BWD>::kSplit, NET = Epi<BWD>::NET;
   constexpr int COLS = (BWD || FOLD) ? 64 : 128;
   constexpr int CB = COLS / 64;                        // 64-column blocks per tile
   constexpr int NSUB = BWD ? 3 : 2;                    // MMAs per item
@@ -750,6 +756,7 @@ cudaError_t launch_t(const Ctx& c) {
   // wide operands), then as many operand stages as fit
   constexpr int NOUT = BWD ? 2 : 1;
   const uint32_t set_bytes = NMAT * CB * kBlockBytes, out_bytes = NOUT * CB * kBlockBytes;
+  constexpr int kSplit = Epi<BWD>::kSplit;
   const uint32_t base = (BWD ? 2 * kSplit * BM * 4 : 0) + 1024 + 640 + (fold ? 2 * kDzbBytes : 0);
   auto need = [&](int ns, int os) { return ns * (set_bytes + kHdrFloats * 4) + os * out_bytes + base + 2 * p.stage_bytes; };
   int nsets = kMaxSets, out_sets = 2;
@@ -822,11 +829,11 @@ cudaError_t launch_t(const Ctx& c) {
   if (fold) {
     e = cudaFuncSetAttribute(grouped_swiglu_kernel<BWD, 1, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes);
     if (e != cudaSuccess) return e;
-    grouped_swiglu_kernel<BWD, 1, 1><<<sms, kThreads, smem_bytes, c.st>>>(p);
+    grouped_swiglu_kernel<BWD, 1, 1><<<sms, kThreadsOf<BWD>, smem_bytes, c.st>>>(p);
   } else {
     e = cudaFuncSetAttribute(grouped_swiglu_kernel<BWD, 0, kUnitsAlways>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes);
     if (e != cudaSuccess) return e;
-    grouped_swiglu_kernel<BWD, 0, kUnitsAlways><<<sms, kThreads, smem_bytes, c.st>>>(p);
+    grouped_swiglu_kernel<BWD, 0, kUnitsAlways><<<sms, kThreadsOf<BWD>, smem_bytes, c.st>>>(p);
   }
   return cudaGetLastError();
 }
