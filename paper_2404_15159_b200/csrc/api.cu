@@ -28,6 +28,7 @@ WsLayout ws_layout(const mixlora_shape_t& s, bool allow_fold) {
     return o;
   };
   L.status = take(64 * 4);
+  L.splitk_cnt = take(kSplitCounters * 4);
   L.probs = take(T * N * 4);
   L.expert_idx = take(T * k * 4);
   L.gates = take(T * k * 4);
@@ -70,6 +71,8 @@ WsLayout ws_layout(const mixlora_shape_t& s, bool allow_fold) {
   L.hbar = take(T * f * E);
   L.work_count = take(8 * 4);
   L.work_rows1 = take((size_t)rows_worklist_max(s.tokens * s.top_k, s.n_experts, 1) * 32);
+  L.splitk_bytes = s.dtype == MIXLORA_DTYPE_BF16 ? splitk_part_bytes(s.tokens, s.d_model) : 0;
+  L.splitk_part = take(L.splitk_bytes);
   L.total_fwd = off;
   L.D = L.hbar;                      // hbar (forward scratch) is dead once y is written; D = dy W_d takes its place
   L.spd = take(T * N * r * E);
@@ -312,10 +315,16 @@ void add_seg(SGemm& g, const SOperand& A, const SOperand& B, int K) {
 }
 
 // Dense product on the tensor-core kernel when it takes the shape, else on the SIMT kernel.
-cudaError_t dense_product(const Ctx& c, int M, const TcOut* outs, int nout, const TcWork* wl = nullptr) {
+// `split`: the launch may share each tile's reduction among idle CTA pairs through the workspace's split scratch
+// (the [T, d] products of a short batch: down projection and dx); one such launch at a time per workspace.
+cudaError_t dense_product(const Ctx& c, int M, const TcOut* outs, int nout, const TcWork* wl = nullptr,
+                          bool split = false) {
   if (nout == 0 || M <= 0) return cudaSuccess;
-  if (c.bf16 && tc_gemm_supported(M, outs, nout))
-    return launch_tc_gemm(M, outs, nout, c.at<int>(c.L.status), c.st, wl);   // the SIMT kernel below computes every block
+  if (c.bf16 && tc_gemm_supported(M, outs, nout)) {
+    TcSplit sp{c.at<float>(c.L.splitk_part), c.L.splitk_bytes, c.at<int>(c.L.splitk_cnt), kSplitCounters};
+    return launch_tc_gemm(M, outs, nout, c.at<int>(c.L.status), c.st, wl,   // the SIMT kernel below computes every block
+                          split && c.L.splitk_bytes ? &sp : nullptr);
+  }
   for (int o = 0; o < nout; ++o) {
     const TcOut& t = outs[o];
     const int Mo = t.M > 0 ? t.M : M;
@@ -414,7 +423,7 @@ static mixlora_status_t fwd_check(const mixlora_shape_t* shape, const mixlora_pa
 
 // router (Eq. 7) and dispatch
 static mixlora_status_t fwd_clear_status(const Ctx& c) {
-  MIXLORA_CUDA(cudaMemsetAsync(c.ws + c.L.status, 0, 256, c.st));
+  MIXLORA_CUDA(cudaMemsetAsync(c.ws + c.L.status, 0, 256 + kSplitCounters * 4, c.st));   // status, then the split counters
   return MIXLORA_OK;
 }
 static mixlora_status_t fwd_route(const Ctx& c) {
@@ -509,7 +518,7 @@ static mixlora_status_t fwd_experts(const Ctx& c, void* y, const void* residual 
     tc_add(out, c.ws + c.L.hbar, f, f, params->w_down, f, 0);
     tc_add(out, c.ws + c.L.Zs, Nr, Nr, c.ws + c.L.bd_cat, Nr, 0);
     StageScope ss(ST_GEMM_DOWN, c.st, dense_launches(c, T, &out, 1));
-    MIXLORA_CUDA(dense_product(c, T, &out, 1));
+    MIXLORA_CUDA(dense_product(c, T, &out, 1, nullptr, true));
   }
   return MIXLORA_OK;
 }
@@ -815,7 +824,7 @@ static mixlora_status_t bwd_experts(const Ctx& c, const void* dy, float aux_coef
     tc_add(out, c.ws + c.L.dZu, Nr, Nr, params->a_up, d, 1);
     tc_add(out, c.ws + c.L.dl_act, NP, NP, c.ws + c.L.wr_act, d, 1);
     StageScope ss(ST_GEMM_DX, c.st, dense_launches(c, T, &out, 1));
-    MIXLORA_CUDA(dense_product(c, T, &out, 1));
+    MIXLORA_CUDA(dense_product(c, T, &out, 1, nullptr, true));
   }
   return MIXLORA_OK;
 }
@@ -1146,7 +1155,7 @@ mixlora_status_t mixlora_dora_ffn_backward(const mixlora_shape_t* shape, const m
     tc_add(out, c.ws + c.L.dZg, Nr, Nr, params->a_gate, d, 1);
     tc_add(out, c.ws + c.L.dZu, Nr, Nr, params->a_up, d, 1);
     tc_add(out, c.ws + c.L.dl_act, NP, NP, c.ws + c.L.wr_act, d, 1);
-    MIXLORA_CUDA(dense_product(c, T, &out, 1));
+    MIXLORA_CUDA(dense_product(c, T, &out, 1, nullptr, true));
   }
   return MIXLORA_OK;
 }

@@ -20,6 +20,7 @@ typedef __nv_bfloat16 bf16;
 struct WsLayout {
   size_t status;      // int32[64]; [0] = device status word; bytes 8..15: int64 token count of the whole batch when
                       //            the auxiliary loss was evaluated over data-parallel shards (0 = this call's tokens)
+  size_t splitk_cnt;  // i32 [kSplitCounters]  arrival counters of a split reduction, zero between launches
   size_t probs;       // f32 [T, N]        softmax probabilities (Eq. 7)
   size_t expert_idx;  // i32 [T, k]
   size_t gates;       // f32 [T, k]
@@ -52,6 +53,8 @@ struct WsLayout {
   size_t work_count;  // i32 [8]  item counts of the work lists below; [3] = column groups the backward grouped
                       //          kernel used (rows of dz_part); [4] = the same of the forward kernel (zd_part)
   size_t work_rows1;  // i32 [.., 8]  rows list with one output (A_d h)
+  size_t splitk_part; // f32 partial tiles of a split reduction ([T, d] products of a short batch), splitk_bytes long
+  size_t splitk_bytes;
   size_t total_fwd;
   size_t D;           // act [T, f]        dy W_d
   size_t spd;         // act [T, N*r]      s * B_d^T dy for every expert
@@ -283,8 +286,27 @@ bool tc_gemm_supported(int M, const TcOut* outs, int nout);
 void tc_set_force_single(int v);   // 1: single-CTA tensor-core kernel for every shape (measurement switch)
 cudaError_t launch_wait_timeout_selftest(int* status, unsigned limit, cudaStream_t st);
 int tc_gemm_tile_rows(int M);   // rows of the tiles the tensor-core kernel will use for a problem with M rows
+// Optional scratch for a split reduction: when a launch has too few output tiles to occupy the CTA pairs (few rows,
+// deep reduction) and every output is of mode 0, the kernel gives each tile's reduction to 2..kSplitKMax pairs that
+// exchange fp32 partials through `part`; `counters` must be zero at the launch and are zero again after it.
+constexpr int kSplitKMax = 4;
+constexpr int kSplitCounters = 512;                          // ints; 8 per output tile
+constexpr size_t kSplitTileBytes = 256 * 256 * 4;            // one fp32 partial of a 256 x 256 tile
+struct TcSplit {
+  float* part; size_t part_bytes;
+  int* counters; int n_counters;
+};
+// Bytes of `part` that make the split possible for an output of [rows, cols] (0 where it would never be used).
+static inline size_t splitk_part_bytes(long long rows, long long cols) {
+  if (rows < 256) return 0;
+  const long long tiles = ((rows + 255) / 256) * ((cols + 255) / 256);
+  if (tiles * 2 > 74 || tiles * 8 > kSplitCounters) return 0;
+  long long split = 74 / tiles;
+  if (split > kSplitKMax) split = kSplitKMax;
+  return (size_t)(tiles * split) * kSplitTileBytes;
+}
 cudaError_t launch_tc_gemm(int M, const TcOut* outs, int nout, int* status_word, cudaStream_t st,
-                           const TcWork* wl = nullptr);
+                           const TcWork* wl = nullptr, const TcSplit* split = nullptr);
 // Work lists over the sorted slots (need seg_off of the dispatch step):
 //   rows list : for every tile of `tile_rows` sorted slots and every expert with slots in it, `nout` items that
 //               compute that expert's block of r columns for the tile's rows (all k-blocks);

@@ -9,6 +9,7 @@
 //               overlapped with the main loop of the next tile (two accumulators of 256 columns)
 // Reduction segments are walked back to back into the same accumulator (K-concatenation);
 // several outputs (column blocks with their own B and C) share one launch when they share A.
+// A launch with few tiles and a deep reduction may split each tile's reduction over several CTA pairs (TcParams).
 // Every wait is bounded: when a limit runs out the CTA records MIXLORA_ERR_DEVICE_TIMEOUT in the
 // caller's status word, all roles leave their loops, and TMEM is released before exit.
 #include <cuda.h>
@@ -66,9 +67,17 @@ struct alignas(64) TcParams {
   const int* work;
   const int* work_count;
   int* status;
+  // Split reduction (CTA-pair kernel, mode-0 outputs, no work list): every output tile becomes split_k items, each
+  // over an equal share of the concatenated k-blocks.  An item leaves its fp32 partial in `part`
+  // ([tile][share][CTA of the pair][128 rows][256 columns]); per (tile, CTA, epilogue warp) a counter tells the
+  // warp that arrives last, which adds the shares in index order (the same sum whoever is last), writes the
+  // output and sets the counter back to zero.
+  int split_k, total_kb;
+  float* part;
+  int* counters;
 };
 
-struct TileCoord { int o, m0, n0, kb0, kb1, n_lo, n_hi; };
+struct TileCoord { int o, m0, n0, kb0, kb1, n_lo, n_hi, base, ks; };
 
 __device__ __forceinline__ int tile_total(const TcParams& p) {
   if (!p.work) return p.total_tiles;
@@ -82,9 +91,18 @@ __device__ __forceinline__ TileCoord tile_coord(const TcParams& p, int tile) {
     const int4 a = *reinterpret_cast<const int4*>(p.work + (size_t)tile * 8);
     const int4 b = *reinterpret_cast<const int4*>(p.work + (size_t)tile * 8 + 4);
     t.o = a.x; t.m0 = a.y; t.n0 = a.z; t.kb0 = a.w; t.kb1 = b.x; t.n_lo = b.y; t.n_hi = b.z;
+    t.base = tile; t.ks = 0;
     return t;
   }
   t.kb0 = 0; t.kb1 = -1;                  // all k-blocks of every segment
+  t.base = tile; t.ks = 0;
+  if (p.split_k > 1) {
+    t.base = tile / p.split_k;
+    t.ks = tile - t.base * p.split_k;
+    t.kb0 = (int)((long long)t.ks * p.total_kb / p.split_k);
+    t.kb1 = (int)((long long)(t.ks + 1) * p.total_kb / p.split_k);
+    tile = t.base;
+  }
   if (p.row_group > 0) {
     // Row groups (all outputs have the same rows): inside a group of row_group row tiles, rows fastest, then the
     // column tiles of every output in turn.  The CTAs that run together then cover a near-square patch of the
@@ -220,10 +238,15 @@ __global__ void __launch_bounds__(kThreads, 1) tc_gemm_kernel(const __grid_const
         const TileCoord tc = tile_coord(p, tile);
         const int tn = p.tile_n[tc.o];
         const uint32_t tx = kABytes + (uint32_t)tn * BK * 2;
+        int seg_first = 0;
         for (int sg = 0; sg < p.nseg && ok; ++sg) {
           const CUtensorMap* am = &p.a_map[tc.o * p.nseg + sg];
           const CUtensorMap* bm = &p.b_map[tc.o * p.nseg + sg];
-          const int kb_begin = tc.kb1 < 0 ? 0 : tc.kb0, kb_end = tc.kb1 < 0 ? p.kblocks[sg] : tc.kb1;
+          // an item's k-range counts the 64-deep blocks of all segments back to back
+          const int nk = p.kblocks[sg];
+          const int kb_begin = tc.kb1 < 0 ? 0 : max(tc.kb0 - seg_first, 0);
+          const int kb_end = tc.kb1 < 0 ? nk : min(tc.kb1 - seg_first, nk);
+          seg_first += nk;
           for (int kb = kb_begin; kb < kb_end; ++kb, ++it) {
             const int st = it % kStages;
             const uint32_t ph = (it / kStages) & 1u;
@@ -406,10 +429,15 @@ __global__ void __launch_bounds__(kThreads, 1) tc_gemm_pair_kernel(const __grid_
         const int m0 = tc.m0 + (int)rank * BM;
         const int n0 = tc.n0 + (int)rank * half;
         const uint32_t tx_pair = 2u * (kABytes + (uint32_t)half * BK * 2);
+        int seg_first = 0;
         for (int sg = 0; sg < p.nseg && ok; ++sg) {
           const CUtensorMap* am = &p.a_map[tc.o * p.nseg + sg];
           const CUtensorMap* bm = &p.b_map[tc.o * p.nseg + sg];
-          const int kb_begin = tc.kb1 < 0 ? 0 : tc.kb0, kb_end = tc.kb1 < 0 ? p.kblocks[sg] : tc.kb1;
+          // an item's k-range counts the 64-deep blocks of all segments back to back
+          const int nk = p.kblocks[sg];
+          const int kb_begin = tc.kb1 < 0 ? 0 : max(tc.kb0 - seg_first, 0);
+          const int kb_end = tc.kb1 < 0 ? nk : min(tc.kb1 - seg_first, nk);
+          seg_first += nk;
           for (int kb = kb_begin; kb < kb_end; ++kb, ++it) {
             const int st = it % kStages2;
             const uint32_t ph = (it / kStages2) & 1u;
@@ -492,6 +520,59 @@ __global__ void __launch_bounds__(kThreads, 1) tc_gemm_pair_kernel(const __grid_
       tc_fence_after();
       const int row = tc.m0 + (int)rank * BM + q * 32 + lane;
       const uint32_t t_addr = tmem_base + ((uint32_t)(q * 32) << 16) + buf * BN_MAX;
+      if (p.split_k > 1) {
+        // this item's share of the reduction goes to the partial array; the warp that completes the tile adds up
+        const size_t slab = (size_t)BM * BN_MAX;                       // floats of one CTA's half of a tile
+        float* mine = p.part + ((size_t)(tc.base * p.split_k + tc.ks) * 2 + rank) * slab +
+                      (size_t)(q * 32 + lane) * BN_MAX;
+        for (int c = 0; c < tn; c += 32) {
+          uint32_t v[32];
+          if (empty) {
+#pragma unroll
+            for (int j = 0; j < 32; ++j) v[j] = 0u;
+          } else {
+            tmem_ld32(t_addr + c, v);
+            tmem_ld_wait();
+          }
+#pragma unroll
+          for (int j = 0; j < 32; j += 4)
+            *reinterpret_cast<uint4*>(mine + c + j) = make_uint4(v[j], v[j + 1], v[j + 2], v[j + 3]);
+        }
+        tc_fence_before();
+        __threadfence();                                               // the partial is visible before the count
+        __syncwarp();
+        int* counter = p.counters + (tc.base * 2 + (int)rank) * 4 + q;
+        int seen = 0;
+        if (lane == 0) {
+          mbar_arrive_cluster(map_to_cta(tempty_bar(buf), 0));         // the accumulator is free again
+          seen = atomicAdd(counter, 1);
+        }
+        seen = __shfl_sync(0xffffffffu, seen, 0);
+        if (seen == p.split_k - 1) {
+          __threadfence();
+          const float* first = p.part + ((size_t)(tc.base * p.split_k) * 2 + rank) * slab +
+                               (size_t)(q * 32 + lane) * BN_MAX;
+          for (int c = 0; c < tn; c += 32) {
+            float acc[32];
+#pragma unroll
+            for (int j = 0; j < 32; ++j) acc[j] = 0.f;
+            for (int sidx = 0; sidx < p.split_k; ++sidx) {
+              const float4* src = reinterpret_cast<const float4*>(first + (size_t)sidx * 2 * slab + c);
+#pragma unroll
+              for (int j = 0; j < 8; ++j) {
+                const float4 w = __ldcg(src + j);
+                acc[4 * j] += w.x; acc[4 * j + 1] += w.y; acc[4 * j + 2] += w.z; acc[4 * j + 3] += w.w;
+              }
+            }
+            uint32_t v[32];
+#pragma unroll
+            for (int j = 0; j < 32; ++j) v[j] = __float_as_uint(acc[j]);
+            store_chunk32(p, tc.o, row, tc.n0 + c, tc.n_lo, tc.n_hi, v);
+          }
+          if (lane == 0) *counter = 0;                                 // ready for the next launch
+        }
+        continue;
+      }
       for (int c = 0; c < tn; c += 32) {
         uint32_t v[32];
         if (empty) {
@@ -712,7 +793,8 @@ cudaError_t launch_wait_timeout_selftest(int* status, unsigned limit, cudaStream
 
 int tc_gemm_tile_rows(int M) { return (!tc_force_single() && M >= 2 * BM) ? 2 * BM : BM; }
 
-cudaError_t launch_tc_gemm(int M, const TcOut* outs, int nout, int* status_word, cudaStream_t st, const TcWork* wl) {
+cudaError_t launch_tc_gemm(int M, const TcOut* outs, int nout, int* status_word, cudaStream_t st, const TcWork* wl,
+                           const TcSplit* split) {
   TcParams p;
   memset(&p, 0, sizeof(p));
   const int nseg = outs[0].nseg;
@@ -785,6 +867,22 @@ cudaError_t launch_tc_gemm(int M, const TcOut* outs, int nout, int* status_word,
   int dev = 0, sms = 148;
   cudaGetDevice(&dev);
   cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  for (int s = 0; s < nseg; ++s) p.total_kb += p.kblocks[s];
+  if (split && pair && !wl && split->part && split->counters && tiles > 0) {
+    bool plain = true;
+    for (int o = 0; o < nout; ++o) plain = plain && outs[o].mode == 0;
+    int sk = (sms / 2) / tiles;                                       // pairs that would idle otherwise
+    if (sk > kSplitKMax) sk = kSplitKMax;
+    if (sk > p.total_kb / 16) sk = p.total_kb / 16;                   // every share keeps a deep enough loop
+    if (plain && sk >= 2 && (size_t)tiles * sk * kSplitTileBytes <= split->part_bytes &&
+        tiles * 8 <= split->n_counters) {
+      p.split_k = sk;
+      p.part = split->part;
+      p.counters = split->counters;
+      p.total_tiles = tiles * sk;
+      tiles = p.total_tiles;
+    }
+  }
   if (pair) {
     const int pairs = tiles < sms / 2 ? tiles : sms / 2;
     if (a_mn) return b_kn ? launch_pair_variant<1, 1>(p, 2 * pairs, st) : launch_pair_variant<1, 0>(p, 2 * pairs, st);
