@@ -961,7 +961,7 @@ DoraLayout dora_layout(const mixlora_shape_t& s, const WsLayout& L) {
   D.dO = take(T * k * d * E);
   D.D_s = take(T * k * f * E);
   D.spd_s = take(T * k * N * r * E);
-  D.dmp_g = take(mt * f * 4); D.dmp_u = take(mt * f * 4); D.dmp_d = take(mt * d * 4);
+  D.dmp_g = take(4 * mt * f * 4); D.dmp_u = take(4 * mt * f * 4); D.dmp_d = take(mt * d * 4);
   D.total_bwd = off;
   return D;
 }
@@ -1036,7 +1036,15 @@ mixlora_status_t mixlora_dora_ffn_forward(const mixlora_shape_t* shape, const mi
     MIXLORA_CUDA(launch_dora_scales(c, dc));
   }
   if ((st = fwd_shared_projections(&c, 1)) != MIXLORA_OK) return st;   // W1 x, W3 x once per token, A_g x, A_u x
-  { StageScope ss(ST_LORA_B_SWIGLU, c.st, 1); MIXLORA_CUDA(launch_dora_swiglu_fwd(c, dc)); }
+  {
+    StageScope ss(ST_LORA_B_SWIGLU, c.st, 2);
+    if (grouped_swiglu_supported(c)) {      // the tensor-core kernel of the MixLoRA path with the two scale vectors
+      MIXLORA_CUDA(launch_zcompact(c));
+      MIXLORA_CUDA(launch_grouped_swiglu_dora_fwd(c, dc));
+    } else {
+      MIXLORA_CUDA(launch_dora_swiglu_fwd(c, dc));
+    }
+  }
   {   // zd = A_d h against every expert, then the slot's own block (and gate times it)
     StageScope ss(ST_LORA_A_DOWN, c.st, 2);
     TcOut out = tc_out(c.ws + c.L.zd_all, Nr, Nr);
@@ -1092,12 +1100,20 @@ mixlora_status_t mixlora_dora_ffn_backward(const mixlora_shape_t* shape, const m
     outs[1] = tc_out(dc.spd_s, Nr, Nr);  tc_add(outs[1], dc.dO, d, d, c.ws + c.L.bd_cat, Nr, 1);
     MIXLORA_CUDA(dense_product(c, T * k, outs, 2));
   }
-  { StageScope ss(ST_SWIGLU_BWD, c.st, 2);
-    MIXLORA_CUDA(launch_dora_swiglu_bwd(c, dc));
-    MIXLORA_CUDA(launch_dgate_reduce(c, dora_bwd_col_chunks(f))); }
+  const bool tc_swiglu = grouped_swiglu_supported(c);
+  { StageScope ss(ST_SWIGLU_BWD, c.st, 3);
+    if (tc_swiglu) {
+      MIXLORA_CUDA(launch_dora_pcompact(c, dc));
+      MIXLORA_CUDA(launch_grouped_swiglu_dora_bwd(c, dc));
+      MIXLORA_CUDA(launch_dgate_reduce(c, grouped_swiglu_bwd_col_tiles(f)));
+    } else {
+      MIXLORA_CUDA(launch_dora_swiglu_bwd(c, dc));
+      MIXLORA_CUDA(launch_dgate_reduce(c, dora_bwd_col_chunks(f)));
+    } }
   MIXLORA_CUDA(launch_router_bwd(c, aux_coef, grads->d_router_bias, acc, want_dx));
-  if (mgrads->d_m_gate) MIXLORA_CUDA(launch_dora_dm_reduce(c, dc.dmp_g, dc.inv_g, mgrads->d_m_gate, f, acc));
-  if (mgrads->d_m_up) MIXLORA_CUDA(launch_dora_dm_reduce(c, dc.dmp_u, dc.inv_u, mgrads->d_m_up, f, acc));
+  const int dm_sub = tc_swiglu ? 4 : 1;    // partial rows per tile of the gate / up magnitude shares
+  if (mgrads->d_m_gate) MIXLORA_CUDA(launch_dora_dm_reduce(c, dc.dmp_g, dc.inv_g, mgrads->d_m_gate, f, acc, dm_sub));
+  if (mgrads->d_m_up) MIXLORA_CUDA(launch_dora_dm_reduce(c, dc.dmp_u, dc.inv_u, mgrads->d_m_up, f, acc, dm_sub));
   if (mgrads->d_m_down) MIXLORA_CUDA(launch_dora_dm_reduce(c, dc.dmp_d, dc.inv_d, mgrads->d_m_down, d, acc));
   {   // dzg = da (s B_g), dzu = db (s B_u) with da, db the gradients of the pre-scale activations
     TcOut outs[2];

@@ -241,7 +241,9 @@ struct DoraCtx {
   void *dO;                            // act [T k, d]   c_d * dy per sorted slot
   void *D_s;                           // act [T k, f]   dO W2 per sorted slot
   void *spd_s;                         // act [T k, N r] s B_d^T dO for every expert, per sorted slot
-  float *dmp_g, *dmp_u, *dmp_d;        // [tiles, f], [tiles, f], [tiles, d]  per-tile shares of the magnitude gradients
+  float *dmp_g, *dmp_u, *dmp_d;        // [4 tiles, f], [4 tiles, f], [tiles, d]  per-tile shares of the magnitude
+                                       // gradients (gate / up: per tile and lane quarter from the tensor-core kernel,
+                                       // one row per tile from the SIMT kernel)
 };
 int dora_bwd_col_chunks(int f);
 cudaError_t launch_dora_scales(const Ctx& c, const DoraCtx& dc);
@@ -251,7 +253,10 @@ cudaError_t launch_dora_combine_y(const Ctx& c, const DoraCtx& dc, void* y);
 cudaError_t launch_dora_dout(const Ctx& c, const DoraCtx& dc, const void* dy);
 cudaError_t launch_dora_swiglu_bwd(const Ctx& c, const DoraCtx& dc);
 cudaError_t launch_dora_dm_reduce(const Ctx& c, const float* part, const float* inv_n, float* dm, int width,
-                                  int accumulate);
+                                  int accumulate, int sub = 1);
+cudaError_t launch_dora_pcompact(const Ctx& c, const DoraCtx& dc);
+cudaError_t launch_grouped_swiglu_dora_fwd(const Ctx& c, const DoraCtx& dora);   // grouped_swiglu.cu
+cudaError_t launch_grouped_swiglu_dora_bwd(const Ctx& c, const DoraCtx& dora);
 
 // Dense product (tensor-core kernel in tc_gemm.cu, SIMT kernel otherwise), fp32 accumulation:
 //   C_o[M, N_o] = sum_seg op(A_o,seg) * op(B_o,seg)

@@ -3,6 +3,8 @@
 // of the merged weight, so the per-expert scale c = m / n multiplies output rows: the shared W1 x, W3 x and the
 // dense products stay as they are, and these kernels apply c, build it, and collect the magnitude gradients.
 // Work over the sorted slots is cut by the dispatch step's table of single-expert tiles of up to 128 rows.
+// In bf16 the scaled SwiGLU itself (forward and backward) runs on the grouped tensor-core kernel
+// (grouped_swiglu.cu); the SwiGLU kernels here serve fp32.
 #include "common.cuh"
 
 namespace mixlora {
@@ -336,17 +338,31 @@ dora_swiglu_bwd_kernel(const T* __restrict__ G, const T* __restrict__ U, const T
   }
 }
 
-// d_m[e][o] (+)= inv_n[e][o] * sum over the expert's tiles (in table order) of part[tile][o]
+// p_s[pos][c] = spd_s[pos][e r + c] for c < r (e the slot's expert), zero up to the padded width rp: the rank-r
+// operand s B_d[e]^T dO of the grouped backward kernel, per sorted slot
+template <typename T>
+__global__ void dora_pcompact_kernel(const T* __restrict__ spd_s, const int* __restrict__ pos_expert,
+                                     T* __restrict__ p_s, int slots, int N, int r, int rp) {
+  const long long n = (long long)slots * rp;
+  for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < n; i += (long long)gridDim.x * blockDim.x) {
+    const int pos = (int)(i / rp), cidx = (int)(i % rp);
+    p_s[i] = cidx < r ? spd_s[((size_t)pos * N + pos_expert[pos]) * r + cidx] : from_f<T>(0.f);
+  }
+}
+
+// d_m[e][o] (+)= inv_n[e][o] * sum over the expert's tiles (in table order) of part[tile][o]; with sub > 1 a tile
+// has `sub` partial rows (part[tile * sub + j][o]), added in the order of j
 __global__ void dora_dm_reduce_kernel(const float* __restrict__ part, const float* __restrict__ inv_n,
                                       const int* __restrict__ tile_info, int max_tiles, float* __restrict__ dm,
-                                      int N, int width, int accumulate) {
+                                      int N, int width, int accumulate, int sub) {
   const int e = blockIdx.y;
   const int o = blockIdx.x * blockDim.x + threadIdx.x;
   if (o >= width) return;
   const int ntiles = min(tile_info[max_tiles * 4], max_tiles);
   float s = 0.f;
   for (int t = 0; t < ntiles; ++t)
-    if (tile_info[t * 4 + 0] == e) s += part[(size_t)t * width + o];
+    if (tile_info[t * 4 + 0] == e)
+      for (int j = 0; j < sub; ++j) s += part[((size_t)t * sub + j) * width + o];
   const size_t i = (size_t)e * width + o;
   const float v = inv_n[i] * s;
   dm[i] = accumulate ? dm[i] + v : v;
@@ -447,11 +463,20 @@ cudaError_t launch_dora_swiglu_bwd(const Ctx& c, const DoraCtx& dc) {
   return c.bf16 ? swiglu_bwd_t<bf16>(c, dc) : swiglu_bwd_t<float>(c, dc);
 }
 cudaError_t launch_dora_dm_reduce(const Ctx& c, const float* part, const float* inv_n, float* dm, int width,
-                                  int accumulate) {
+                                  int accumulate, int sub) {
   const int mt = max_seg_tiles(c.s.tokens, c.s.top_k, c.s.n_experts);
   dim3 grid((width + 255) / 256, c.s.n_experts);
   dora_dm_reduce_kernel<<<grid, 256, 0, c.st>>>(part, inv_n, c.at<int>(c.L.tile_info), mt, dm, c.s.n_experts, width,
-                                                accumulate);
+                                                accumulate, sub);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_dora_pcompact(const Ctx& c, const DoraCtx& dc) {
+  const int slots = c.s.tokens * c.s.top_k, r = c.s.rank, rp = pad_rank(r);
+  if (!c.bf16) return cudaErrorInvalidValue;       // only the tensor-core grouped kernel reads the compact form
+  dora_pcompact_kernel<bf16><<<grid_for((long long)slots * rp, 256), 256, 0, c.st>>>(
+      reinterpret_cast<const bf16*>(dc.spd_s), c.at<int>(c.L.pos_expert), c.at<bf16>(c.L.p_s), slots, c.s.n_experts, r,
+      rp);
   return cudaGetLastError();
 }
 

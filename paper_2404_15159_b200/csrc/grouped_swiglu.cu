@@ -79,6 +79,10 @@ struct alignas(64) GsParams {
   float* dz_part;          // [groups, slots, 2, r_true]
   int* groups_used;        // the number of column groups the kernel settled on
   int r_true, cg_min;
+  // DORA only (the weight-decomposed variant: a = c_g[e] (G + da), b = c_u[e] (U + db))
+  const float* cg; const float* cu;   // [N, f] scales of the gate and up projections
+  float* dm_g; float* dm_u;           // backward: [max_tiles * 4, f] per (segment tile, lane quarter) sums over rows of
+                                      // d a * a_pre and d b * b_pre (the magnitude gradients before the division by n)
 };
 
 // The order in which a CTA takes (segment tile, column tile) items; every role of the CTA walks it the same way.
@@ -186,8 +190,26 @@ __device__ __forceinline__ uint64_t sigmoid2(uint64_t a) {
   asm("tanh.approx.f32 %0, %1;" : "=f"(th) : "f"(hi));
   return fma2(pk2(tl, th), kHalf2, kHalf2);
 }
-template <int BWD, int FOLD, int UNITS>
+// Sums over the 32 lanes of a warp of 32 values per lane: on return lane l holds the sum of every lane's v[l].
+// Five exchange steps, each halving the number of values a lane still carries (31 shuffles in all).
+__device__ __forceinline__ float warp_transpose_sum32(float (&v)[32], int lane) {
+#pragma unroll
+  for (int st = 0; st < 5; ++st) {
+    const int off = 16 >> st, n = 32 >> st;
+    const bool up = (lane & off) != 0;
+#pragma unroll
+    for (int i = 0; i < n / 2; ++i) {
+      const float send = up ? v[i] : v[i + n / 2];
+      const float keep = up ? v[i + n / 2] : v[i];
+      v[i] = keep + __shfl_xor_sync(0xffffffffu, send, off);
+    }
+  }
+  return v[0];
+}
+
+template <int BWD, int FOLD, int UNITS, int DORA = 0>
 __global__ void __launch_bounds__(kThreadsOf<BWD>, 1) grouped_swiglu_kernel(const __grid_constant__ GsParams p) {
+  static_assert(!DORA || !FOLD, "the scaled variant runs without the rank-r products");
   constexpr int kSplit = Epi<BWD>::kSplit, NET = Epi<BWD>::NET;
   constexpr int COLS = (BWD || FOLD) ? 64 : 128;
   constexpr int CB = COLS / 64;                        // 64-column blocks per tile
@@ -507,6 +529,13 @@ __global__ void __launch_bounds__(kThreadsOf<BWD>, 1) grouped_swiglu_kernel(cons
       for (int ps = 0; ps < kPasses; ++ps)
         roff[ps] = (typename std::conditional<FOLD != 0, uint32_t, size_t>::type)
                        p.pos_token[p0 + min(g_r0 + kRowsPerPass * ps, rows - 1)] * p.f;
+      // DORA backward: D = dO W2 exists per sorted slot (the output scale differs between a token's experts)
+      uint32_t roff_d[(DORA && BWD) ? kPasses : 1];    // element offsets inside the tile's 128 rows of D
+      if (DORA && BWD) {
+#pragma unroll
+        for (int ps = 0; ps < kPasses; ++ps)
+          roff_d[ps] = (uint32_t)min(g_r0 + kRowsPerPass * ps, rows - 1) * (uint32_t)p.f;
+      }
       float gate0 = 0.f, gate1 = 0.f;                  // gates of rows gt and (fewer than 128 gather threads) gt + NGT
       if (BWD) {
         if (gt < rows) gate0 = p.gates[p.perm[p0 + gt]];
@@ -538,6 +567,7 @@ __global__ void __launch_bounds__(kThreadsOf<BWD>, 1) grouped_swiglu_kernel(cons
         reinterpret_cast<int*>(hdr)[128] = p0;
         reinterpret_cast<int*>(hdr)[129] = rows;
         reinterpret_cast<int*>(hdr)[130] = ct;
+        if (DORA) reinterpret_cast<int*>(hdr)[131] = p.tile_info[tile * 4 + 0] | (tile << 8);   // expert, segment tile
       }
       const uint32_t dst_set = g_dst0 + set * kSetBytes;
 #pragma unroll
@@ -558,7 +588,7 @@ __global__ void __launch_bounds__(kThreadsOf<BWD>, 1) grouped_swiglu_kernel(cons
                            : "memory");
             else
               asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst + ps * kRowsPerPass * 128),
-                           "l"(base + roff[ps]), "r"(d_bytes)
+                           "l"((DORA && BWD) ? base + (size_t)p0 * p.f + roff_d[ps] : base + roff[ps]), "r"(d_bytes)
                            : "memory");
           }
         }
@@ -620,6 +650,7 @@ __global__ void __launch_bounds__(kThreadsOf<BWD>, 1) grouped_swiglu_kernel(cons
         p0 = reinterpret_cast<const int*>(hdr)[128];
         rows = reinterpret_cast<const int*>(hdr)[129];
         ct = reinterpret_cast<const int*>(hdr)[130];
+        const int etile = DORA ? reinterpret_cast<const int*>(hdr)[131] : 0;   // expert | segment tile << 8
         pos = p0 + row;
         if (et == 0) {                                 // for the store warp: the set itself is released earlier
           int* oh = out_hdr + 4 * (wcount & 1u);
@@ -631,27 +662,62 @@ __global__ void __launch_bounds__(kThreadsOf<BWD>, 1) grouped_swiglu_kernel(cons
         uint64_t dg2 = 0;
         const float gate = BWD ? hdr[row] : 0.f;
         const uint64_t gate2 = pk2(gate, gate);
+        // DORA: the expert's scales of this thread's columns, and (backward) this row's weight in the column sums
+        const int dcol0 = ct * COLS + part * WCOLS;
+        const float* cg_row = DORA ? p.cg + (size_t)(etile & 255) * p.f : nullptr;
+        const float* cu_row = DORA ? p.cu + (size_t)(etile & 255) * p.f : nullptr;
+        const float live = row < rows ? 1.f : 0.f;
+        const uint64_t live2 = pk2(live, live);
 #pragma unroll
         for (int c16 = 0; c16 < WCOLS; c16 += 16) {
           uint32_t va[16], vb[16], vd[BWD ? 16 : 1];
-          tmem_ld16(t_addr + c16, va);
-          tmem_ld16(t_addr + COLS + c16, vb);
-          if (BWD) tmem_ld16(t_addr + 2 * COLS + c16, reinterpret_cast<uint32_t(&)[16]>(vd));
-          tmem_ld_wait();
+          uint64_t pg2[(DORA && BWD) ? 8 : 1], pu2[(DORA && BWD) ? 8 : 1];
+          constexpr bool kLoad8 = DORA && BWD;          // 8 accumulator columns at a time: the column sums need the registers
+          if (!kLoad8) {
+            tmem_ld16(t_addr + c16, va);
+            tmem_ld16(t_addr + COLS + c16, vb);
+            if (BWD) tmem_ld16(t_addr + 2 * COLS + c16, reinterpret_cast<uint32_t(&)[16]>(vd));
+            tmem_ld_wait();
+          }
 #pragma unroll
           for (int hh8 = 0; hh8 < 2; ++hh8) {
+            if (kLoad8) {
+              uint32_t ta[8], tb[8], td[8];
+              tmem_ld8(t_addr + c16 + hh8 * 8, ta);
+              tmem_ld8(t_addr + COLS + c16 + hh8 * 8, tb);
+              tmem_ld8(t_addr + 2 * COLS + c16 + hh8 * 8, td);
+              tmem_ld_wait();
+#pragma unroll
+              for (int j = 0; j < 8; ++j) {
+                va[hh8 * 8 + j] = ta[j]; vb[hh8 * 8 + j] = tb[j]; vd[BWD ? hh8 * 8 + j : 0] = td[j];
+              }
+            }
             const int ch = c16 / 8 + hh8;
             const uint32_t off = row_off + (((cb0 + ch) ^ rx) << 4);
             const uint4 rg = *reinterpret_cast<const uint4*>(gset + 0 * CB * kBlockBytes + off);
             const uint4 ru = *reinterpret_cast<const uint4*>(gset + 1 * CB * kBlockBytes + off);
             const uint32_t wg[4] = {rg.x, rg.y, rg.z, rg.w}, wu[4] = {ru.x, ru.y, ru.z, ru.w};
+            uint64_t cg2[DORA ? 4 : 1], cu2[DORA ? 4 : 1];
+            if (DORA) {
+              const int dcol = dcol0 + c16 + hh8 * 8;
+              float4 g0 = make_float4(0.f, 0.f, 0.f, 0.f), g1 = g0, u0 = g0, u1 = g0;
+              if (dcol < p.f) {                        // f is a multiple of 8: the chunk is inside the row or past it
+                g0 = __ldg(reinterpret_cast<const float4*>(cg_row + dcol));
+                g1 = __ldg(reinterpret_cast<const float4*>(cg_row + dcol + 4));
+                u0 = __ldg(reinterpret_cast<const float4*>(cu_row + dcol));
+                u1 = __ldg(reinterpret_cast<const float4*>(cu_row + dcol + 4));
+              }
+              cg2[0] = pk2(g0.x, g0.y); cg2[1] = pk2(g0.z, g0.w); cg2[2] = pk2(g1.x, g1.y); cg2[3] = pk2(g1.z, g1.w);
+              cu2[0] = pk2(u0.x, u0.y); cu2[1] = pk2(u0.z, u0.w); cu2[2] = pk2(u1.x, u1.y); cu2[3] = pk2(u1.z, u1.w);
+            }
             if (!BWD) {
               uint32_t ho[4];
 #pragma unroll
               for (int i = 0; i < 4; ++i) {
                 const int v = hh8 * 8 + 2 * i;
-                const uint64_t a = add2(bf2_to_f2(wg[i]), pk2u(va[v], va[v + 1]));
-                const uint64_t b = add2(bf2_to_f2(wu[i]), pk2u(vb[v], vb[v + 1]));
+                uint64_t a = add2(bf2_to_f2(wg[i]), pk2u(va[v], va[v + 1]));
+                uint64_t b = add2(bf2_to_f2(wu[i]), pk2u(vb[v], vb[v + 1]));
+                if (DORA) { a = mul2(a, cg2[i]); b = mul2(b, cu2[i]); }
                 ho[i] = f2_to_bf2(mul2(mul2(a, sigmoid2(a)), b));
               }
               *reinterpret_cast<uint4*>(oset + off) = make_uint4(ho[0], ho[1], ho[2], ho[3]);
@@ -662,8 +728,10 @@ __global__ void __launch_bounds__(kThreadsOf<BWD>, 1) grouped_swiglu_kernel(cons
 #pragma unroll
               for (int i = 0; i < 4; ++i) {
                 const int v = hh8 * 8 + 2 * i;
-                const uint64_t a = add2(bf2_to_f2(wg[i]), pk2u(va[v], va[v + 1]));
-                const uint64_t b = add2(bf2_to_f2(wu[i]), pk2u(vb[v], vb[v + 1]));
+                const uint64_t a_pre = add2(bf2_to_f2(wg[i]), pk2u(va[v], va[v + 1]));
+                const uint64_t b_pre = add2(bf2_to_f2(wu[i]), pk2u(vb[v], vb[v + 1]));
+                const uint64_t a = DORA ? mul2(a_pre, cg2[DORA ? i : 0]) : a_pre;
+                const uint64_t b = DORA ? mul2(b_pre, cu2[DORA ? i : 0]) : b_pre;
                 const uint64_t Dt = add2(bf2_to_f2(wd[i]), pk2u(vd[BWD ? v : 0], vd[BWD ? v + 1 : 0]));
                 const uint64_t sg = sigmoid2(a);
                 const uint64_t sa = mul2(a, sg);                         // SiLU(a)
@@ -671,12 +739,36 @@ __global__ void __launch_bounds__(kThreadsOf<BWD>, 1) grouped_swiglu_kernel(cons
                 const uint64_t dh = mul2(gate2, Dt);
                 // SiLU'(a) = sg (1 + a (1 - sg))
                 const uint64_t ds = mul2(sg, fma2(a, fma2(sg, kMinusOne2, kOne2), kOne2));
-                ao[i] = f2_to_bf2(mul2(mul2(dh, b), ds));
-                bo[i] = f2_to_bf2(mul2(dh, sa));
+                const uint64_t da = mul2(mul2(dh, b), ds), db = mul2(dh, sa);
+                if (DORA) {
+                  // with respect to the scaled a, b: the magnitude gradient collects d a * a_pre over the tile's own
+                  // rows; what goes downstream is the gradient of the pre-scale value
+                  pg2[(DORA && BWD) ? hh8 * 4 + i : 0] = mul2(mul2(da, a_pre), live2);
+                  pu2[(DORA && BWD) ? hh8 * 4 + i : 0] = mul2(mul2(db, b_pre), live2);
+                  ao[i] = f2_to_bf2(mul2(da, cg2[DORA ? i : 0]));
+                  bo[i] = f2_to_bf2(mul2(db, cu2[DORA ? i : 0]));
+                } else {
+                  ao[i] = f2_to_bf2(da);
+                  bo[i] = f2_to_bf2(db);
+                }
               }
               *reinterpret_cast<uint4*>(oset + 0 * CB * kBlockBytes + off) = make_uint4(ao[0], ao[1], ao[2], ao[3]);
               *reinterpret_cast<uint4*>(oset + 1 * CB * kBlockBytes + off) = make_uint4(bo[0], bo[1], bo[2], bo[3]);
             }
+          }
+          if (DORA && BWD) {
+            // column sums over this warp's 32 rows of the 16 + 16 products: lane l ends up with column l & 15 of
+            // the gate (l < 16) or up (l >= 16) side; one partial row per (segment tile, lane quarter)
+            float pv[32];
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+              upk2(pg2[(DORA && BWD) ? i : 0], pv[2 * i], pv[2 * i + 1]);
+              upk2(pu2[(DORA && BWD) ? i : 0], pv[16 + 2 * i], pv[16 + 2 * i + 1]);
+            }
+            const float csum = warp_transpose_sum32(pv, lane);
+            const int col = dcol0 + c16 + (lane & 15);
+            if (col < p.f)
+              ((lane & 16) ? p.dm_u : p.dm_g)[((size_t)(etile >> 8) * 4 + q) * p.f + col] = csum;
           }
         }
         tc_fence_before();
@@ -736,11 +828,12 @@ __global__ void __launch_bounds__(kThreadsOf<BWD>, 1) grouped_swiglu_kernel(cons
 }
 
 template <int BWD>
-cudaError_t launch_t(const Ctx& c) {
+cudaError_t launch_t(const Ctx& c, const DoraCtx* dora = nullptr) {
   constexpr int NMAT = BWD ? 3 : 2;
   const int slots = c.s.tokens * c.s.top_k, f = c.s.d_ff, r = c.s.rank, N = c.s.n_experts;
   const int rp = pad_rank(r);
-  const bool fold = BWD ? ctx_folds_dz(c) : ctx_folds_zd(c);
+  const bool fold = !dora && (BWD ? ctx_folds_dz(c) : ctx_folds_zd(c));
+  if (dora && N > 256) return cudaErrorInvalidConfiguration;   // the item header packs the expert into 8 bits
   const int COLS = (BWD || fold) ? 64 : 128, CB = COLS / 64;
   GsParams p;
   memset(&p, 0, sizeof(p));
@@ -820,13 +913,22 @@ cudaError_t launch_t(const Ctx& c) {
     p.groups_used = c.at<int>(c.L.work_count) + 4;
     p.r_true = r;
   }
+  if (dora) {
+    p.cg = dora->cg; p.cu = dora->cu;
+    p.dm_g = dora->dmp_g; p.dm_u = dora->dmp_u;
+    if (BWD) p.D = reinterpret_cast<const bf16*>(dora->D_s);
+  }
   p.status = c.at<int>(c.L.status);
   int dev = 0, sms = 148;
   cudaGetDevice(&dev);
   cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
   // the number of segment tiles is only known on the device; every CTA reads it and idles if it has no item
   cudaError_t e;
-  if (fold) {
+  if (dora) {
+    e = cudaFuncSetAttribute(grouped_swiglu_kernel<BWD, 0, 0, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes);
+    if (e != cudaSuccess) return e;
+    grouped_swiglu_kernel<BWD, 0, 0, 1><<<sms, kThreadsOf<BWD>, smem_bytes, c.st>>>(p);
+  } else if (fold) {
     e = cudaFuncSetAttribute(grouped_swiglu_kernel<BWD, 1, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes);
     if (e != cudaSuccess) return e;
     grouped_swiglu_kernel<BWD, 1, 1><<<sms, kThreadsOf<BWD>, smem_bytes, c.st>>>(p);
@@ -848,5 +950,9 @@ bool grouped_swiglu_supported(const Ctx& c) {
 int grouped_swiglu_bwd_col_tiles(int f) { return (f + 63) / 64; }
 cudaError_t launch_grouped_swiglu_fwd(const Ctx& c) { return launch_t<0>(c); }
 cudaError_t launch_grouped_swiglu_bwd(const Ctx& c) { return launch_t<1>(c); }
+// The weight-decomposed variant: scales c_g, c_u per (expert, column), D per sorted slot, and (backward) the
+// per-(tile, lane quarter) shares of the magnitude gradients in dora.dmp_g / dmp_u ([4 * max tiles, f]).
+cudaError_t launch_grouped_swiglu_dora_fwd(const Ctx& c, const DoraCtx& dora) { return launch_t<0>(c, &dora); }
+cudaError_t launch_grouped_swiglu_dora_bwd(const Ctx& c, const DoraCtx& dora) { return launch_t<1>(c, &dora); }
 
 }  // namespace mixlora
