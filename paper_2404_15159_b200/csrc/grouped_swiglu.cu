@@ -27,6 +27,10 @@
 // later kernel adds the groups in a fixed order.  da and db are then not read again for this product.
 // Forward with FOLD: the same for zd = h A_d[e]^T (the input of the LoRA of W2): 64-column tiles like the backward
 // kernel's, which leaves TMEM columns for one accumulator of up to 128; B = the r x 64 block of A_d[e].
+// DORA (the weight-decomposed variant, Section 4.1): a = c_g[e] (G + da), b = c_u[e] (U + db) with one scale per
+// expert and column; the epilogue threads load their columns' scales, the backward kernel gathers D per sorted slot,
+// stores the gradients of the pre-scale values and leaves, per (segment tile, lane quarter), the sums over rows of
+// d a * a_pre and d b * b_pre (formed inside each warp by halving shuffle exchanges).
 #include <algorithm>
 #include <type_traits>
 
