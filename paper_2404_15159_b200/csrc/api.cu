@@ -1015,7 +1015,11 @@ mixlora_status_t mixlora_dora_ffn_forward(const mixlora_shape_t* shape, const mi
   const int Nr = N * r;
   if ((st = fwd_clear_status(c)) != MIXLORA_OK) return st;
   if (T == 0) return MIXLORA_OK;
-  if ((st = fwd_route(c)) != MIXLORA_OK) return st;
+  // the router and the dispatch need only x: on a side stream beside the norms and the shared projections
+  Forked fk;
+  if ((st = for_each_adapter(&c, 1, true, [&](const Ctx& cc, int) { return fwd_route(cc); }, &fk)) != MIXLORA_OK)
+    return st;
+  st = [&]() -> mixlora_status_t {
   // the scales c = m / n of the three projections: |W_o + s B_o A|^2 = |W_o|^2 + 2 s B_o . (W A^T)_o + s^2 B_o (A A^T) B_o^T
   {
     StageScope ss(ST_NORM, c.st, 12);
@@ -1035,7 +1039,12 @@ mixlora_status_t mixlora_dora_ffn_forward(const mixlora_shape_t* shape, const mi
     MIXLORA_CUDA(dense_product(c, Nr, &ad, 1));
     MIXLORA_CUDA(launch_dora_scales(c, dc));
   }
-  if ((st = fwd_shared_projections(&c, 1)) != MIXLORA_OK) return st;   // W1 x, W3 x once per token, A_g x, A_u x
+  return fwd_shared_projections(&c, 1);   // W1 x, W3 x once per token, A_g x, A_u x
+  }();
+  {
+    const mixlora_status_t js = join_adapters(c.st, fk);   // always: no side stream is left dangling after an error
+    if (st != MIXLORA_OK || js != MIXLORA_OK) return st != MIXLORA_OK ? st : js;
+  }
   {
     StageScope ss(ST_LORA_B_SWIGLU, c.st, 2);
     if (grouped_swiglu_supported(c)) {      // the tensor-core kernel of the MixLoRA path with the two scale vectors
