@@ -71,7 +71,8 @@ WsLayout ws_layout(const mixlora_shape_t& s, bool allow_fold) {
   L.hbar = take(T * f * E);
   L.work_count = take(8 * 4);
   L.work_rows1 = take((size_t)rows_worklist_max(s.tokens * s.top_k, s.n_experts, 1) * 32);
-  L.splitk_bytes = s.dtype == MIXLORA_DTYPE_BF16 ? splitk_part_bytes(s.tokens, s.d_model) : 0;
+  // rows of the tallest product (the per-slot ones of the weight-decomposed variant), columns of the widest (gate/up)
+  L.splitk_bytes = s.dtype == MIXLORA_DTYPE_BF16 ? splitk_part_bytes((long long)(T * k), (long long)(2 * f + 2 * N * r)) : 0;
   L.splitk_part = take(L.splitk_bytes);
   L.total_fwd = off;
   L.D = L.hbar;                      // hbar (forward scratch) is dead once y is written; D = dy W_d takes its place
@@ -315,8 +316,9 @@ void add_seg(SGemm& g, const SOperand& A, const SOperand& B, int K) {
 }
 
 // Dense product on the tensor-core kernel when it takes the shape, else on the SIMT kernel.
-// `split`: the launch may share each tile's reduction among idle CTA pairs through the workspace's split scratch
-// (the [T, d] products of a short batch: down projection and dx); one such launch at a time per workspace.
+// `split`: the launch may share the reductions of its last round's tiles among the CTA pairs that round would leave
+// idle, through the workspace's split scratch: the frozen-projection products, which follow each other on the
+// caller's stream (one such launch at a time per workspace).
 cudaError_t dense_product(const Ctx& c, int M, const TcOut* outs, int nout, const TcWork* wl = nullptr,
                           bool split = false) {
   if (nout == 0 || M <= 0) return cudaSuccess;
@@ -426,14 +428,28 @@ static mixlora_status_t fwd_clear_status(const Ctx& c) {
   MIXLORA_CUDA(cudaMemsetAsync(c.ws + c.L.status, 0, 256 + kSplitCounters * 4, c.st));   // status, then the split counters
   return MIXLORA_OK;
 }
-static mixlora_status_t fwd_route(const Ctx& c) {
+static mixlora_status_t fwd_route_only(const Ctx& c) {
   if (c.s.tokens == 0) return MIXLORA_OK;
   { StageScope ss(ST_ROUTER, c.st, 2); MIXLORA_CUDA(launch_router(c)); }
   { StageScope ss(ST_DISPATCH, c.st, 3); MIXLORA_CUDA(launch_dispatch(c)); }
-  // repacks that depend on the parameters only (s B_d, s B_g, s B_u with all experts' blocks side by side); the
-  // backward pass finds them in the workspace
+  return MIXLORA_OK;
+}
+// repacks that depend on the parameters only (s B_d, s B_g, s B_u with all experts' blocks side by side); the
+// backward pass finds them in the workspace
+static mixlora_status_t fwd_repacks(const Ctx& c) {
+  if (c.s.tokens == 0) return MIXLORA_OK;
   { StageScope ss(ST_DISPATCH, c.st, 3); MIXLORA_CUDA(launch_bd_cat(c)); MIXLORA_CUDA(launch_bgu_cat(c)); }
   return MIXLORA_OK;
+}
+static mixlora_status_t fwd_route(const Ctx& c) {
+  const mixlora_status_t st = fwd_route_only(c);
+  return st == MIXLORA_OK ? fwd_repacks(c) : st;
+}
+// One adapter: the routing chain and the repacks do not depend on each other and take a side stream each.
+static mixlora_status_t fwd_route_forked(const Ctx& c, Forked* fk) {
+  const Ctx two[2] = {c, c};
+  return for_each_adapter(two, 2, true, [&](const Ctx& cc, int m) { return m == 0 ? fwd_route_only(cc) : fwd_repacks(cc); },
+                          fk);
 }
 
 // Shared gate / up projections, once per token (Section 3.3 (I)), for one adapter (then the LoRA-A columns of every
@@ -458,12 +474,12 @@ static mixlora_status_t fwd_shared_projections(const Ctx* cs, int n) {
     outs[2] = tc_out(c.ws + c.L.zga, Nr, Nr); tc_add(outs[2], c.p.x, d, d, c.p.a_gate, d, 0);
     outs[3] = tc_out(c.ws + c.L.zua, Nr, Nr); tc_add(outs[3], c.p.x, d, d, c.p.a_up, d, 0);
     StageScope ss(ST_GEMM_GATE_UP, c.st, dense_launches(c, T, outs, 4));
-    MIXLORA_CUDA(dense_product(c, T, outs, 4));
+    MIXLORA_CUDA(dense_product(c, T, outs, 4, nullptr, true));
     return MIXLORA_OK;
   }
   {
     StageScope ss(ST_GEMM_GATE_UP, c0.st, dense_launches(c0, Tmax, outs, no));
-    MIXLORA_CUDA(dense_product(c0, Tmax, outs, no));
+    MIXLORA_CUDA(dense_product(c0, Tmax, outs, no, nullptr, true));
   }
   for (int i = 0; i < n; ++i) {
     const Ctx& c = cs[i];
@@ -531,7 +547,7 @@ mixlora_status_t mixlora_ffn_forward(const mixlora_shape_t* shape, const mixlora
   if ((st = fwd_clear_status(c)) != MIXLORA_OK) return st;
   // the router and the dispatch need only x: they run on a side stream beside the shared projections
   Forked fk;
-  if ((st = for_each_adapter(&c, 1, true, [&](const Ctx& cc, int) { return fwd_route(cc); }, &fk)) != MIXLORA_OK)
+  if ((st = fwd_route_forked(c, &fk)) != MIXLORA_OK)
     return st;
   st = fwd_shared_projections(&c, 1);
   mixlora_status_t js = join_adapters(c.st, fk);
@@ -651,7 +667,7 @@ static mixlora_status_t bwd_shared_dgrad(const Ctx* cs, const void* const* dys, 
     outs[0] = tc_out(c.ws + c.L.D, f, f);      tc_add(outs[0], dys[0], d, d, c.p.w_down, f, 1);
     outs[1] = tc_out(c.ws + c.L.spd, Nr, Nr);  tc_add(outs[1], dys[0], d, d, c.ws + c.L.bd_cat, Nr, 1);
     StageScope ss(ST_GEMM_DGRAD_DOWN, c.st, dense_launches(c, T, outs, 2));
-    MIXLORA_CUDA(dense_product(c, T, outs, 2));   // bd_cat is the forward pass's
+    MIXLORA_CUDA(dense_product(c, T, outs, 2, nullptr, true));   // bd_cat is the forward pass's
     return MIXLORA_OK;
   }
   TcOut outs[2];
@@ -668,7 +684,7 @@ static mixlora_status_t bwd_shared_dgrad(const Ctx* cs, const void* const* dys, 
   {
     const Ctx& c0 = cs[last];
     StageScope ss(ST_GEMM_DGRAD_DOWN, c0.st, dense_launches(c0, Tmax, outs, no));
-    MIXLORA_CUDA(dense_product(c0, Tmax, outs, no));
+    MIXLORA_CUDA(dense_product(c0, Tmax, outs, no, nullptr, true));
   }
   for (int i = 0; i < n; ++i) {
     const Ctx& c = cs[i];
@@ -905,7 +921,7 @@ mixlora_status_t mixlora_layer_forward(const mixlora_shape_t* shape, const mixlo
   }
   if ((st = fwd_clear_status(c)) != MIXLORA_OK) return st;
   Forked fk;
-  if ((st = for_each_adapter(&c, 1, true, [&](const Ctx& cc, int) { return fwd_route(cc); }, &fk)) != MIXLORA_OK)
+  if ((st = fwd_route_forked(c, &fk)) != MIXLORA_OK)
     return st;
   st = fwd_shared_projections(&c, 1);
   mixlora_status_t js = join_adapters(c.st, fk);
@@ -1017,7 +1033,7 @@ mixlora_status_t mixlora_dora_ffn_forward(const mixlora_shape_t* shape, const mi
   if (T == 0) return MIXLORA_OK;
   // the router and the dispatch need only x: on a side stream beside the norms and the shared projections
   Forked fk;
-  if ((st = for_each_adapter(&c, 1, true, [&](const Ctx& cc, int) { return fwd_route(cc); }, &fk)) != MIXLORA_OK)
+  if ((st = fwd_route_forked(c, &fk)) != MIXLORA_OK)
     return st;
   st = [&]() -> mixlora_status_t {
   // the scales c = m / n of the three projections: |W_o + s B_o A|^2 = |W_o|^2 + 2 s B_o . (W A^T)_o + s^2 B_o (A A^T) B_o^T
@@ -1067,7 +1083,7 @@ mixlora_status_t mixlora_dora_ffn_forward(const mixlora_shape_t* shape, const mi
     TcOut out = tc_out(dc.o_pre, d, d);
     tc_add(out, c.ws + c.L.h_sorted, f, f, params->w_down, f, 0);
     tc_add(out, dc.Zd_pos, Nr, Nr, c.ws + c.L.bd_cat, Nr, 0);
-    MIXLORA_CUDA(dense_product(c, T * k, &out, 1));
+    MIXLORA_CUDA(dense_product(c, T * k, &out, 1, nullptr, true));
   }
   { StageScope ss(ST_COMBINE_H, c.st, 1); MIXLORA_CUDA(launch_dora_combine_y(c, dc, y)); }
   return MIXLORA_OK;
@@ -1107,7 +1123,7 @@ mixlora_status_t mixlora_dora_ffn_backward(const mixlora_shape_t* shape, const m
     TcOut outs[2];
     outs[0] = tc_out(dc.D_s, f, f);      tc_add(outs[0], dc.dO, d, d, params->w_down, f, 1);
     outs[1] = tc_out(dc.spd_s, Nr, Nr);  tc_add(outs[1], dc.dO, d, d, c.ws + c.L.bd_cat, Nr, 1);
-    MIXLORA_CUDA(dense_product(c, T * k, outs, 2));
+    MIXLORA_CUDA(dense_product(c, T * k, outs, 2, nullptr, true));
   }
   const bool tc_swiglu = grouped_swiglu_supported(c);
   { StageScope ss(ST_SWIGLU_BWD, c.st, 3);

@@ -291,24 +291,25 @@ bool tc_gemm_supported(int M, const TcOut* outs, int nout);
 void tc_set_force_single(int v);   // 1: single-CTA tensor-core kernel for every shape (measurement switch)
 cudaError_t launch_wait_timeout_selftest(int* status, unsigned limit, cudaStream_t st);
 int tc_gemm_tile_rows(int M);   // rows of the tiles the tensor-core kernel will use for a problem with M rows
-// Optional scratch for a split reduction: when a launch has too few output tiles to occupy the CTA pairs (few rows,
-// deep reduction) and every output is of mode 0, the kernel gives each tile's reduction to 2..kSplitKMax pairs that
-// exchange fp32 partials through `part`; `counters` must be zero at the launch and are zero again after it.
+// Optional scratch for a split reduction: the tiles of a launch's last, partial round of CTA pairs (every tile when
+// the launch has fewer tiles than pairs) are given to 2..kSplitKMax pairs each, which exchange fp32 partials through
+// `part`; `counters` must be zero at the launch and are zero again after it.  One launch at a time per scratch.
 constexpr int kSplitKMax = 4;
-constexpr int kSplitCounters = 512;                          // ints; 8 per output tile
+constexpr int kSplitCounters = 1024;                         // ints; 8 per split tile
 constexpr size_t kSplitTileBytes = 256 * 256 * 4;            // one fp32 partial of a 256 x 256 tile
+constexpr int kSplitMaxItems = 222;                          // shares in flight: three rounds of 74 CTA pairs
 struct TcSplit {
   float* part; size_t part_bytes;
   int* counters; int n_counters;
 };
-// Bytes of `part` that make the split possible for an output of [rows, cols] (0 where it would never be used).
+// Bytes of `part` that serve every launch whose outputs have at most `rows` rows and `cols` columns in total
+// (0 where the CTA-pair kernel is not used).
 static inline size_t splitk_part_bytes(long long rows, long long cols) {
   if (rows < 256) return 0;
-  const long long tiles = ((rows + 255) / 256) * ((cols + 255) / 256);
-  if (tiles * 2 > 74 || tiles * 8 > kSplitCounters) return 0;
-  long long split = 74 / tiles;
-  if (split > kSplitKMax) split = kSplitKMax;
-  return (size_t)(tiles * split) * kSplitTileBytes;
+  long long tiles = ((rows + 255) / 256) * ((cols + 255) / 256 + 4);   // a few narrow outputs beside the wide ones
+  long long items = tiles * kSplitKMax;
+  if (items > kSplitMaxItems) items = kSplitMaxItems;
+  return (size_t)items * kSplitTileBytes;
 }
 cudaError_t launch_tc_gemm(int M, const TcOut* outs, int nout, int* status_word, cudaStream_t st,
                            const TcWork* wl = nullptr, const TcSplit* split = nullptr);

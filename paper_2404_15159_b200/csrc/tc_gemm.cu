@@ -41,6 +41,8 @@ constexpr uint32_t kBBytes = BN_MAX * BK * 2;    // 32 KiB
 constexpr uint32_t kStageBytes = kABytes + kBBytes;
 constexpr uint32_t kSmemBytes = kStages * kStageBytes + 1024 /* alignment slack */ + 256 /* barriers */;
 constexpr uint32_t kTmemCols = 512;
+constexpr int kSplitMinBlocks = 32;     // k-blocks a share of a split reduction keeps at least
+constexpr int kSplitShareCost = 24;     // what a share costs beside its loop, in k-blocks' time
 
 struct alignas(64) TcParams {
   CUtensorMap a_map[kMaxB];        // index o * nseg + seg
@@ -67,11 +69,13 @@ struct alignas(64) TcParams {
   const int* work;
   const int* work_count;
   int* status;
-  // Split reduction (CTA-pair kernel, mode-0 outputs, no work list): every output tile becomes split_k items, each
-  // over an equal share of the concatenated k-blocks.  An item leaves its fp32 partial in `part`
-  // ([tile][share][CTA of the pair][128 rows][256 columns]); per (tile, CTA, epilogue warp) a counter tells the
-  // warp that arrives last, which adds the shares in index order (the same sum whoever is last), writes the
-  // output and sets the counter back to zero.
+  // Split reduction (CTA-pair kernel, no work list): the tiles from split_from on (those of the last, partial round
+  // of CTA pairs; all tiles when there are fewer than pairs) become split_k items each, over equal shares of the
+  // concatenated k-blocks, so that the round's idle pairs take part.  An item leaves its fp32 partial in `part`
+  // ([split tile][share][CTA of the pair][128 rows][256 columns]); per (split tile, CTA, epilogue warp) a counter
+  // tells the warp that arrives last, which adds the shares in index order (the same sum whoever is last), writes
+  // the output and sets the counter back to zero.
+  int split_from;
   int split_k, total_kb;
   float* part;
   int* counters;
@@ -91,17 +95,18 @@ __device__ __forceinline__ TileCoord tile_coord(const TcParams& p, int tile) {
     const int4 a = *reinterpret_cast<const int4*>(p.work + (size_t)tile * 8);
     const int4 b = *reinterpret_cast<const int4*>(p.work + (size_t)tile * 8 + 4);
     t.o = a.x; t.m0 = a.y; t.n0 = a.z; t.kb0 = a.w; t.kb1 = b.x; t.n_lo = b.y; t.n_hi = b.z;
-    t.base = tile; t.ks = 0;
+    t.base = 0; t.ks = -1;
     return t;
   }
   t.kb0 = 0; t.kb1 = -1;                  // all k-blocks of every segment
-  t.base = tile; t.ks = 0;
-  if (p.split_k > 1) {
-    t.base = tile / p.split_k;
-    t.ks = tile - t.base * p.split_k;
+  t.base = 0; t.ks = -1;                  // ks >= 0: a share of a split tile, base = index among the split tiles
+  if (p.split_k > 1 && tile >= p.split_from) {
+    const int j = tile - p.split_from;
+    t.base = j / p.split_k;
+    t.ks = j - t.base * p.split_k;
     t.kb0 = (int)((long long)t.ks * p.total_kb / p.split_k);
     t.kb1 = (int)((long long)(t.ks + 1) * p.total_kb / p.split_k);
-    tile = t.base;
+    tile = p.split_from + t.base;
   }
   if (p.row_group > 0) {
     // Row groups (all outputs have the same rows): inside a group of row_group row tiles, rows fastest, then the
@@ -520,11 +525,13 @@ __global__ void __launch_bounds__(kThreads, 1) tc_gemm_pair_kernel(const __grid_
       tc_fence_after();
       const int row = tc.m0 + (int)rank * BM + q * 32 + lane;
       const uint32_t t_addr = tmem_base + ((uint32_t)(q * 32) << 16) + buf * BN_MAX;
-      if (p.split_k > 1) {
-        // this item's share of the reduction goes to the partial array; the warp that completes the tile adds up
+      if (tc.ks >= 0) {
+        // this item's share of the reduction goes to the partial array; the warp that completes the tile adds up.
+        // A warp's 32 rows x 256 columns of a share are laid out [32-column chunk][4-column group][lane]: every
+        // store and load instruction of the warp covers 512 contiguous bytes.
         const size_t slab = (size_t)BM * BN_MAX;                       // floats of one CTA's half of a tile
-        float* mine = p.part + ((size_t)(tc.base * p.split_k + tc.ks) * 2 + rank) * slab +
-                      (size_t)(q * 32 + lane) * BN_MAX;
+        const size_t wofs = (size_t)q * 32 * BN_MAX + (size_t)lane * 4;   // this warp's region, this lane's float4
+        float* mine = p.part + ((size_t)(tc.base * p.split_k + tc.ks) * 2 + rank) * slab + wofs;
         for (int c = 0; c < tn; c += 32) {
           uint32_t v[32];
           if (empty) {
@@ -535,8 +542,9 @@ __global__ void __launch_bounds__(kThreads, 1) tc_gemm_pair_kernel(const __grid_
             tmem_ld_wait();
           }
 #pragma unroll
-          for (int j = 0; j < 32; j += 4)
-            *reinterpret_cast<uint4*>(mine + c + j) = make_uint4(v[j], v[j + 1], v[j + 2], v[j + 3]);
+          for (int j = 0; j < 8; ++j)
+            *reinterpret_cast<uint4*>(mine + (size_t)(c / 32 * 8 + j) * 128) =
+                make_uint4(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]);
         }
         tc_fence_before();
         __threadfence();                                               // the partial is visible before the count
@@ -550,23 +558,29 @@ __global__ void __launch_bounds__(kThreads, 1) tc_gemm_pair_kernel(const __grid_
         seen = __shfl_sync(0xffffffffu, seen, 0);
         if (seen == p.split_k - 1) {
           __threadfence();
-          const float* first = p.part + ((size_t)(tc.base * p.split_k) * 2 + rank) * slab +
-                               (size_t)(q * 32 + lane) * BN_MAX;
+          const float* first = p.part + ((size_t)(tc.base * p.split_k) * 2 + rank) * slab + wofs;
+          const int nshare = p.split_k;
           for (int c = 0; c < tn; c += 32) {
-            float acc[32];
+            // all shares' loads of the chunk are issued before the first sum (one round trip to L2 per chunk)
+            float4 w[kSplitKMax][8];
 #pragma unroll
-            for (int j = 0; j < 32; ++j) acc[j] = 0.f;
-            for (int sidx = 0; sidx < p.split_k; ++sidx) {
-              const float4* src = reinterpret_cast<const float4*>(first + (size_t)sidx * 2 * slab + c);
+            for (int sidx = 0; sidx < kSplitKMax; ++sidx)
 #pragma unroll
-              for (int j = 0; j < 8; ++j) {
-                const float4 w = __ldcg(src + j);
-                acc[4 * j] += w.x; acc[4 * j + 1] += w.y; acc[4 * j + 2] += w.z; acc[4 * j + 3] += w.w;
-              }
-            }
+              for (int j = 0; j < 8; ++j)
+                w[sidx][j] = sidx < nshare
+                                 ? __ldcg(reinterpret_cast<const float4*>(first + (size_t)sidx * 2 * slab +
+                                                                          (size_t)(c / 32 * 8 + j) * 128))
+                                 : make_float4(0.f, 0.f, 0.f, 0.f);
             uint32_t v[32];
 #pragma unroll
-            for (int j = 0; j < 32; ++j) v[j] = __float_as_uint(acc[j]);
+            for (int j = 0; j < 8; ++j) {
+              float4 a = w[0][j];
+#pragma unroll
+              for (int sidx = 1; sidx < kSplitKMax; ++sidx)
+                if (sidx < nshare) { a.x += w[sidx][j].x; a.y += w[sidx][j].y; a.z += w[sidx][j].z; a.w += w[sidx][j].w; }
+              v[4 * j] = __float_as_uint(a.x); v[4 * j + 1] = __float_as_uint(a.y);
+              v[4 * j + 2] = __float_as_uint(a.z); v[4 * j + 3] = __float_as_uint(a.w);
+            }
             store_chunk32(p, tc.o, row, tc.n0 + c, tc.n_lo, tc.n_hi, v);
           }
           if (lane == 0) *counter = 0;                                 // ready for the next launch
@@ -869,17 +883,29 @@ cudaError_t launch_tc_gemm(int M, const TcOut* outs, int nout, int* status_word,
   cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
   for (int s = 0; s < nseg; ++s) p.total_kb += p.kblocks[s];
   if (split && pair && !wl && split->part && split->counters && tiles > 0) {
-    bool plain = true;
-    for (int o = 0; o < nout; ++o) plain = plain && outs[o].mode == 0;
-    int sk = (sms / 2) / tiles;                                       // pairs that would idle otherwise
-    if (sk > kSplitKMax) sk = kSplitKMax;
-    if (sk > p.total_kb / 16) sk = p.total_kb / 16;                   // every share keeps a deep enough loop
-    if (plain && sk >= 2 && (size_t)tiles * sk * kSplitTileBytes <= split->part_bytes &&
-        tiles * 8 <= split->n_counters) {
-      p.split_k = sk;
+    // the tiles of the last, partial round of CTA pairs (all tiles when there are fewer tiles than pairs) share their
+    // reductions: with `rest` such tiles split `sk` ways the round takes ceil(rest sk / pairs) passes of
+    // total_kb / sk k-blocks plus what a share costs on top (partial out, fence, count, and the adding up: measured
+    // at about 24 k-blocks' time); the split must win a tenth of the round to be taken
+    const int pairs = sms / 2;
+    const int rest = tiles % pairs;
+    int best = 1;
+    if (rest > 0) {
+      long long best_cost = (long long)p.total_kb * 9 / 10;
+      for (int sk = 2; sk <= kSplitKMax; ++sk) {
+        if (sk > p.total_kb / kSplitMinBlocks) break;                 // every share keeps a deep enough loop
+        if ((size_t)rest * sk * kSplitTileBytes > split->part_bytes || rest * 8 > split->n_counters) break;
+        const long long passes = (rest * sk + pairs - 1) / pairs;
+        const long long cost = passes * (p.total_kb / sk + kSplitShareCost);
+        if (cost < best_cost) { best_cost = cost; best = sk; }
+      }
+    }
+    if (best >= 2) {
+      p.split_k = best;
+      p.split_from = tiles - rest;
       p.part = split->part;
       p.counters = split->counters;
-      p.total_tiles = tiles * sk;
+      p.total_tiles = p.split_from + rest * best;
       tiles = p.total_tiles;
     }
   }
