@@ -496,15 +496,30 @@ static mixlora_status_t fwd_shared_projections(const Ctx* cs, int n) {
 
 // everything after the shared projections: per-expert deltas, SwiGLU, down projection, combine
 // `residual` (optional, [T, d] of the activation type) is added to y in the down product's epilogue (Eq. 6).
-static mixlora_status_t fwd_experts(const Ctx& c, void* y, const void* residual = nullptr) {
+static mixlora_status_t fwd_experts_main(const Ctx& c, void* y, const void* residual, bool zpos_here);
+// `zpos_aside`: the scatter of zg, zu into the slots' expert blocks, which only the backward pass reads, goes to a
+// side stream that joins the caller's stream at the end (not for callers that already run on a side stream).
+static mixlora_status_t fwd_experts(const Ctx& c, void* y, const void* residual = nullptr, bool zpos_aside = false) {
+  if (c.s.tokens == 0) return MIXLORA_OK;
+  if (!zpos_aside) return fwd_experts_main(c, y, residual, true);
+  Forked fk;
+  mixlora_status_t st = for_each_adapter(&c, 1, true, [&](const Ctx& cc, int) -> mixlora_status_t {
+    StageScope ss(ST_LORA_B_SWIGLU, cc.st, 1);
+    MIXLORA_CUDA(launch_zpos(cc));
+    return MIXLORA_OK;
+  }, &fk);
+  if (st == MIXLORA_OK) st = fwd_experts_main(c, y, residual, false);
+  const mixlora_status_t js = join_adapters(c.st, fk);
+  return st != MIXLORA_OK ? st : js;
+}
+static mixlora_status_t fwd_experts_main(const Ctx& c, void* y, const void* residual, bool zpos_here) {
   const mixlora_params_t* params = &c.p;
   const int T = c.s.tokens, d = c.s.d_model, f = c.s.d_ff, N = c.s.n_experts, r = c.s.rank, k = c.s.top_k;
   const int Nr = N * r;
-  if (T == 0) return MIXLORA_OK;
   // per-slot LoRA-B expansion + SwiGLU
   {
-    StageScope ss(ST_LORA_B_SWIGLU, c.st, 3);
-    MIXLORA_CUDA(launch_zpos(c));
+    StageScope ss(ST_LORA_B_SWIGLU, c.st, zpos_here ? 3 : 2);
+    if (zpos_here) MIXLORA_CUDA(launch_zpos(c));
     if (grouped_swiglu_supported(c)) {
       MIXLORA_CUDA(launch_zcompact(c));
       MIXLORA_CUDA(launch_grouped_swiglu_fwd(c));
@@ -552,7 +567,7 @@ mixlora_status_t mixlora_ffn_forward(const mixlora_shape_t* shape, const mixlora
   st = fwd_shared_projections(&c, 1);
   mixlora_status_t js = join_adapters(c.st, fk);
   if (st != MIXLORA_OK || js != MIXLORA_OK) return st != MIXLORA_OK ? st : js;
-  return fwd_experts(c, y);
+  return fwd_experts(c, y, nullptr, true);
 }
 
 static bool same_frozen_ffn(const Ctx& a, const Ctx& b) {
@@ -926,7 +941,7 @@ mixlora_status_t mixlora_layer_forward(const mixlora_shape_t* shape, const mixlo
   st = fwd_shared_projections(&c, 1);
   mixlora_status_t js = join_adapters(c.st, fk);
   if (st != MIXLORA_OK || js != MIXLORA_OK) return st != MIXLORA_OK ? st : js;
-  return fwd_experts(c, h, params->x);
+  return fwd_experts(c, h, params->x, true);
 }
 
 mixlora_status_t mixlora_layer_backward(const mixlora_shape_t* shape, const mixlora_params_t* params,
