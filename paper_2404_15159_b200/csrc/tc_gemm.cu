@@ -54,6 +54,7 @@ struct alignas(64) TcParams {
   long long s_n[kMaxOut], s_blk[kMaxOut];
   float alpha[kMaxOut];
   int mode[kMaxOut], nb[kMaxOut], accumulate[kMaxOut];
+  int vec4[kMaxOut];               // mode 1: groups of four columns may go out as one 16-byte store
   int N[kMaxOut];                  // columns stored
   int tile_n[kMaxOut];
   int tile_start[kMaxOut + 1];     // first tile index of each output
@@ -151,15 +152,37 @@ __device__ __forceinline__ void store_chunk32(const TcParams& p, int o, int row,
     const long long sn = p.s_n[o], sb = p.s_blk[o];
     const float alpha = p.alpha[o];
     const int accum = p.accumulate[o];
+    const bool vec = p.vec4[o] != 0;                   // four consecutive columns are 16 contiguous, aligned bytes
+    // block and offset inside the block of the chunk's first column, carried along instead of divided out per column
+    int blk = nb > 0 ? n0c / nb : 0;
+    int rem = nb > 0 ? n0c - blk * nb : n0c;
 #pragma unroll
-    for (int j = 0; j < 32; ++j) {
-      const int n = n0c + j;
-      if (n >= n_lo && n < n_hi) {
-        float* dst = base + (nb > 0 ? (size_t)(n / nb) * sb + (size_t)(n % nb) * sn : (size_t)n * sn);
-        float val = alpha * __uint_as_float(v[j]);
-        if (accum) val += *dst;
+    for (int j4 = 0; j4 < 8; ++j4) {
+      const int n = n0c + 4 * j4;
+      if (vec && n >= n_lo && n + 3 < n_hi) {
+        float4* dst = reinterpret_cast<float4*>(base + (size_t)blk * sb + rem);
+        float4 val = make_float4(alpha * __uint_as_float(v[4 * j4]), alpha * __uint_as_float(v[4 * j4 + 1]),
+                                 alpha * __uint_as_float(v[4 * j4 + 2]), alpha * __uint_as_float(v[4 * j4 + 3]));
+        if (accum) {
+          const float4 old = *dst;
+          val.x += old.x; val.y += old.y; val.z += old.z; val.w += old.w;
+        }
         *dst = val;
+      } else {
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          int bi = blk, ri = rem + i;
+          while (nb > 0 && ri >= nb) { ri -= nb; ++bi; }
+          if (n + i >= n_lo && n + i < n_hi) {
+            float* dst = base + (size_t)bi * sb + (size_t)ri * sn;
+            float val = alpha * __uint_as_float(v[4 * j4 + i]);
+            if (accum) val += *dst;
+            *dst = val;
+          }
+        }
       }
+      rem += 4;
+      while (nb > 0 && rem >= nb) { rem -= nb; ++blk; }
     }
   } else {
     bf16* crow = reinterpret_cast<bf16*>(p.C[o]) + (size_t)row * p.ldc[o];
@@ -840,6 +863,8 @@ cudaError_t launch_tc_gemm(int M, const TcOut* outs, int nout, int* status_word,
     p.ldc[o] = t.mode == 0 ? t.ldc : t.s_m;
     p.R[o] = t.mode == 0 ? t.R : nullptr; p.ldr[o] = t.ldr;
     p.s_n[o] = t.s_n; p.s_blk[o] = t.s_blk; p.nb[o] = t.nb; p.alpha[o] = t.alpha; p.accumulate[o] = t.accumulate;
+    p.vec4[o] = t.mode == 1 && t.s_n == 1 && t.nb % 4 == 0 && t.s_m % 4 == 0 && t.s_blk % 4 == 0 &&
+                (reinterpret_cast<uintptr_t>(t.C) & 15u) == 0;
     p.tile_start[o] = tiles;
     p.n_tiles_o[o] = (t.N + tn - 1) / tn;
     p.nt_total += p.n_tiles_o[o];
