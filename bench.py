@@ -539,7 +539,7 @@ def run_cuda(args):
     roofline["hbm_peak_gbs"] = peaks["hbm_gbs"]
     # DRAM bytes (read + write) of the frozen-projection launches, from one single-pass ncu capture of this command's
     # workload at full size (summary under profiles/); other workloads have no capture
-    measured_dram = {"gemm_gate_up": 856.5e6, "gemm_down": 902.1e6, "gemm_dgrad_down": 455.7e6, "gemm_dx": 1759.3e6}
+    measured_dram = {"gemm_gate_up": 876.4e6, "gemm_down": 901.8e6, "gemm_dgrad_down": 462.8e6, "gemm_dx": 1767.2e6}
     algorithmic_dram = {"gemm_gate_up": (T_ * d_ + 2 * f_ * d_ + 2 * T_ * f_) * E,
                         "gemm_down": (T_ * f_ + f_ * d_ + T_ * d_) * E,
                         "gemm_dgrad_down": (T_ * d_ + f_ * d_ + T_ * f_) * E,
