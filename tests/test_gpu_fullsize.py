@@ -151,9 +151,9 @@ def test_c5_skew_sweep_512_tokens_every_output(N, k, r):
 
 @pytest.mark.parametrize("tokens", [256, 300, 640])
 def test_short_batches_whose_down_and_dx_products_split_their_reduction(tokens):
-    # 16, 32 and 48 output tiles for 74 CTA pairs: the [T, d] products share each tile's reduction between 4, 2
-    # and no pairs; 300 and 640 tokens leave a ragged last row tile.  Two runs give the same bits (the shares are
-    # added in index order whichever pair arrives last).
+    # 16, 32 and 48 output tiles for 74 CTA pairs: the [T, d] products share each tile's reduction between several
+    # pairs (4, 2 and, for the deeper dx product, 3 shares per tile); 300 and 640 tokens leave a ragged last row tile.
+    # Two runs give the same bits (the shares are added in index order whichever pair arrives last).
     w = synth.c5(8, 2, 16, tokens)
     full_check(w, aux_coef=0.01)       # dx comes after the down product on the same counters: it needs them back at zero
     t = synth.generate(w)
