@@ -1046,14 +1046,25 @@ mixlora_status_t mixlora_dora_ffn_forward(const mixlora_shape_t* shape, const mi
   const int Nr = N * r;
   if ((st = fwd_clear_status(c)) != MIXLORA_OK) return st;
   if (T == 0) return MIXLORA_OK;
-  // the router and the dispatch need only x: on a side stream beside the norms and the shared projections
+  // the router and the dispatch need only x, the repacks and the row norms of the frozen weights only parameters:
+  // on a side stream each beside the dense products of the norms and the shared projections
   Forked fk;
-  if ((st = fwd_route_forked(c, &fk)) != MIXLORA_OK)
-    return st;
+  {
+    const Ctx two[2] = {c, c};
+    st = for_each_adapter(two, 2, true, [&](const Ctx& cc, int m) -> mixlora_status_t {
+      if (m == 0) return fwd_route_only(cc);
+      const mixlora_status_t rs = fwd_repacks(cc);
+      if (rs != MIXLORA_OK) return rs;
+      StageScope ss(ST_NORM, cc.st, 3);
+      MIXLORA_CUDA(launch_dora_rowsq(cc, dc));
+      return MIXLORA_OK;
+    }, &fk);
+    if (st != MIXLORA_OK) return st;
+  }
   st = [&]() -> mixlora_status_t {
   // the scales c = m / n of the three projections: |W_o + s B_o A|^2 = |W_o|^2 + 2 s B_o . (W A^T)_o + s^2 B_o (A A^T) B_o^T
   {
-    StageScope ss(ST_NORM, c.st, 12);
+    StageScope ss(ST_NORM, c.st, 6);
     TcOut gu[2];
     gu[0] = tc_out_f32(dc.wa_g, Nr, Nr, 1, 0, 0, 1.f, 0); tc_add(gu[0], params->w_gate, d, d, params->a_gate, d, 0);
     gu[1] = tc_out_f32(dc.wa_u, Nr, Nr, 1, 0, 0, 1.f, 0); tc_add(gu[1], params->w_up, d, d, params->a_up, d, 0);
@@ -1068,7 +1079,6 @@ mixlora_status_t mixlora_dora_ffn_forward(const mixlora_shape_t* shape, const mi
     TcOut ad = tc_out_f32(dc.aat_d, Nr, Nr, 1, 0, 0, 1.f, 0);
     tc_add(ad, params->a_down, f, f, params->a_down, f, 0);
     MIXLORA_CUDA(dense_product(c, Nr, &ad, 1));
-    MIXLORA_CUDA(launch_dora_scales(c, dc));
   }
   return fwd_shared_projections(&c, 1);   // W1 x, W3 x once per token, A_g x, A_u x
   }();
@@ -1076,6 +1086,7 @@ mixlora_status_t mixlora_dora_ffn_forward(const mixlora_shape_t* shape, const mi
     const mixlora_status_t js = join_adapters(c.st, fk);   // always: no side stream is left dangling after an error
     if (st != MIXLORA_OK || js != MIXLORA_OK) return st != MIXLORA_OK ? st : js;
   }
+  { StageScope ss(ST_NORM, c.st, 3); MIXLORA_CUDA(launch_dora_scales(c, dc)); }   // needs the row norms and the products
   {
     StageScope ss(ST_LORA_B_SWIGLU, c.st, 2);
     if (grouped_swiglu_supported(c)) {      // the tensor-core kernel of the MixLoRA path with the two scale vectors

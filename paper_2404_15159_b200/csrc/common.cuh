@@ -246,7 +246,8 @@ struct DoraCtx {
                                        // one row per tile from the SIMT kernel)
 };
 int dora_bwd_col_chunks(int f);
-cudaError_t launch_dora_scales(const Ctx& c, const DoraCtx& dc);
+cudaError_t launch_dora_rowsq(const Ctx& c, const DoraCtx& dc);    // squared row norms of the three frozen weights
+cudaError_t launch_dora_scales(const Ctx& c, const DoraCtx& dc);   // c = m / n from the row norms and the W A^T, A A^T products
 cudaError_t launch_dora_swiglu_fwd(const Ctx& c, const DoraCtx& dc);
 cudaError_t launch_dora_own_block(const Ctx& c, const void* in, void* own, void* gown);
 cudaError_t launch_dora_combine_y(const Ctx& c, const DoraCtx& dc, void* y);

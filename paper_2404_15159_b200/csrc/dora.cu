@@ -374,11 +374,17 @@ inline int grid_for(long long n, int block) {
 }
 
 template <typename T>
-cudaError_t scales_t(const Ctx& c, const DoraCtx& dc) {
-  const int d = c.s.d_model, f = c.s.d_ff, N = c.s.n_experts, r = c.s.rank;
+cudaError_t rowsq_t(const Ctx& c, const DoraCtx& dc) {
+  const int d = c.s.d_model, f = c.s.d_ff;
   rowsq_kernel<T><<<(f + 7) / 8, 256, 0, c.st>>>(reinterpret_cast<const T*>(c.p.w_gate), dc.rowsq_g, f, d);
   rowsq_kernel<T><<<(f + 7) / 8, 256, 0, c.st>>>(reinterpret_cast<const T*>(c.p.w_up), dc.rowsq_u, f, d);
   rowsq_kernel<T><<<(d + 7) / 8, 256, 0, c.st>>>(reinterpret_cast<const T*>(c.p.w_down), dc.rowsq_d, d, f);
+  return cudaGetLastError();
+}
+
+template <typename T>
+cudaError_t scales_t(const Ctx& c, const DoraCtx& dc) {
+  const int d = c.s.d_model, f = c.s.d_ff, N = c.s.n_experts, r = c.s.rank;
   dora_scale_kernel<T><<<grid_for((long long)N * f, 256), 256, 0, c.st>>>(
       dc.rowsq_g, dc.wa_g, dc.aat_g, reinterpret_cast<const T*>(c.p.b_gate), dc.m.m_gate, dc.cg, dc.inv_g, f, N, r, c.scale);
   dora_scale_kernel<T><<<grid_for((long long)N * f, 256), 256, 0, c.st>>>(
@@ -446,6 +452,7 @@ cudaError_t swiglu_bwd_t(const Ctx& c, const DoraCtx& dc) {
 
 int dora_bwd_col_chunks(int f) { return (f + kCols - 1) / kCols; }
 
+cudaError_t launch_dora_rowsq(const Ctx& c, const DoraCtx& dc) { return c.bf16 ? rowsq_t<bf16>(c, dc) : rowsq_t<float>(c, dc); }
 cudaError_t launch_dora_scales(const Ctx& c, const DoraCtx& dc) { return c.bf16 ? scales_t<bf16>(c, dc) : scales_t<float>(c, dc); }
 cudaError_t launch_dora_swiglu_fwd(const Ctx& c, const DoraCtx& dc) {
   return c.bf16 ? swiglu_fwd_t<bf16>(c, dc) : swiglu_fwd_t<float>(c, dc);
